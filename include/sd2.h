@@ -1,0 +1,157 @@
+/*
+ * sd2.h -- C ABI of libsd2: decode-time sparse linears of an SD^2 draft model
+ * on one NVIDIA B200 (sm_100a).
+ *
+ * The operation.  A fine-grained-sparse drafter keeps, for every decoder-block
+ * linear (q, k, v, o, gate, up, down), a weight W of shape (C_out, C_in) =
+ * [M x K] and a fixed binary mask; pruned weights are exactly zero and stay so
+ * (paper, Section "Sparse fine-tuning"; W's shape: Appendix "Non-uniform
+ * layer-wise sparsity distributions").  Turning that sparsity into latency
+ * needs "efficient sparse representations and kernels" (Section "Compressed
+ * sparse drafters"); the paper specifies neither, so both are designed here.
+ * Every entry point below computes, or prepares,
+ *
+ *        Y[n, m] = sum over kept k of  W[m, k] * X[n, k]        (Y = X (W.*mask)^T)
+ *
+ * with bf16 inputs, fp32 accumulation and one rounding at the output.
+ *
+ * Conventions
+ *  - All matrices are row-major and dense in memory: W [M*K], mask [M*K],
+ *    X [N*K], Y [N*M].  bf16 values are passed as their 16-bit patterns.
+ *  - "host" / "device" on a pointer says where the memory must live.
+ *  - Every call returns an sd2_status; nothing throws or aborts.  Output
+ *    arguments are written only on SD2_OK.
+ *  - The caller owns every buffer it passes.  The library owns a handle's
+ *    memory (host and device) from sd2_compress / sd2_load_blob to sd2_free.
+ *  - sd2_spmm, sd2_spmm_fused and sd2_block_step are asynchronous on the given
+ *    stream, allocate nothing, never synchronise, overwrite their outputs
+ *    (beta = 0, no bias) and may run concurrently on different streams.  A launch
+ *    failure is reported as SD2_ERR_CUDA by the call that made it.
+ *  - sd2_compress, sd2_load_blob, sd2_decompress and sd2_free may synchronise.
+ *  - There is no CPU fallback: without a CUDA device the device entry points
+ *    return SD2_ERR_CUDA.  sd2_pack_host / sd2_unpack_host need no device.
+ */
+#ifndef SD2_H
+#define SD2_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sd2_handle_s* sd2_handle; /* opaque; owned by the library */
+
+typedef enum {
+    SD2_OK = 0,
+    SD2_ERR_INVALID_ARG = -1, /* NULL pointer, bad option, dead or unknown handle        */
+    SD2_ERR_SHAPE = -2,       /* non-positive or inconsistent dimensions                 */
+    SD2_ERR_ALLOC = -3,       /* host or device allocation failed                        */
+    SD2_ERR_CUDA = -4,        /* CUDA runtime error (no device, launch failure, ...)     */
+    SD2_ERR_UNSUPPORTED = -5, /* valid request this build cannot serve (e.g. huge K)     */
+    SD2_ERR_CORRUPT = -6,     /* a blob failed validation                                */
+    SD2_ERR_TIMEOUT = -7      /* reserved for bounded device-side waits                  */
+} sd2_status;
+
+/* Compressed formats.  Both are lossless; "compressed bytes" always counts every
+ * byte the kernels must read for W: values, position metadata and row offsets. */
+enum {
+    SD2_FORMAT_AUTO = 0,    /* library picks (currently SD2_FORMAT_GAP4 when it applies)    */
+    SD2_FORMAT_BITMASK = 1, /* 1 bit per dense slot + packed kept values + row offsets    */
+    SD2_FORMAT_GAP4 = 2     /* 4-bit column gaps + packed kept values in 8-entry chunks,  */
+                            /* rows cut into lane-balanced tiles (the fast path)          */
+};
+
+enum { SD2_DTYPE_BF16 = 0, SD2_DTYPE_F32 = 1 };
+
+typedef struct {
+    int32_t format;  /* SD2_FORMAT_*                                  */
+    int32_t y_dtype; /* SD2_DTYPE_*: element type of Y for this weight */
+} sd2_options;
+
+/* ---- format builder on the host (no device needed) ----------------------------------- */
+
+/* Encode W.*mask into a self-describing byte blob (the exact image sd2_compress uploads).
+ *   weight_bf16 : host, [M*K] bf16 patterns.
+ *   mask        : host, [M*K] bytes, non-zero = kept; NULL = keep every weight that is
+ *                 not +0/-0.  The mask is authoritative: a kept weight may be zero, NaN or
+ *                 Inf and survives bit for bit; a masked-out weight never takes part.
+ *   opt         : NULL = {AUTO, BF16}.
+ *   blob, blob_bytes : out; release with sd2_blob_free.
+ * Errors: INVALID_ARG (NULL weight/out, unknown format), SHAPE (M or K < 1, or a size
+ * that overflows the format's 32-bit offsets), ALLOC. */
+sd2_status sd2_pack_host(const void* weight_bf16, const uint8_t* mask, int64_t M, int64_t K,
+                         const sd2_options* opt, void** blob, int64_t* blob_bytes);
+
+/* Validate a blob and decode it.  dense_bf16_out (host, [M*K]) may be NULL to only query;
+ * every other out pointer may be NULL.  Decoding yields W with masked-out entries +0.
+ * Errors: INVALID_ARG, CORRUPT (bad magic, sizes, offsets, checksum or metadata). */
+sd2_status sd2_unpack_host(const void* blob, int64_t blob_bytes, void* dense_bf16_out,
+                           int64_t* M, int64_t* K, int64_t* nnz, int64_t* compressed_bytes,
+                           int32_t* format);
+
+sd2_status sd2_blob_free(void* blob);
+
+/* ---- handles ------------------------------------------------------------------------- */
+
+/* Compress once per weight (the topology is static), copy to the current device.
+ * weight_bf16 and mask may each be host or device memory. */
+sd2_status sd2_compress(const void* weight_bf16, const uint8_t* mask, int64_t M, int64_t K,
+                        const sd2_options* opt, sd2_handle* out);
+
+/* Make a handle from a blob produced by sd2_pack_host (host memory). */
+sd2_status sd2_load_blob(const void* blob, int64_t blob_bytes, sd2_handle* out);
+
+/* Read the device copy back and decode it: dense_bf16_out ([M*K], host or device)
+ * receives W.*mask bit-exactly (masked-out entries +0). */
+sd2_status sd2_decompress(sd2_handle h, void* dense_bf16_out);
+
+/* Any out pointer may be NULL. */
+sd2_status sd2_info(sd2_handle h, int64_t* M, int64_t* K, int64_t* nnz,
+                    int64_t* compressed_bytes, int32_t* format);
+
+/* NULL, unknown or already freed handle -> SD2_ERR_INVALID_ARG (no crash). */
+sd2_status sd2_free(sd2_handle h);
+
+/* ---- the hot path -------------------------------------------------------------------- */
+
+/* Y = X (W.*mask)^T.   X: device bf16 [N*K].   Y: device [N*M], bf16 or fp32 per the
+ * handle's y_dtype.  N = 0 is a no-op; N > 8 is processed in panels of at most 8 rows of X
+ * (the weight is re-read from L2 for each panel).  cuda_stream is a cudaStream_t (NULL =
+ * default stream).  X and Y need only their natural alignment. */
+sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_stream);
+
+/* Same-input fusion (q|k|v, gate|up): count <= 4 weights with equal K share one staged X
+ * and one launch.  Y[i] is device [N*M_i] with handle i's y_dtype. */
+sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, void* const* Y,
+                          int64_t N, void* cuda_stream);
+
+/* One drafter block's seven linears in dependency order, h = {q,k,v,o,gate,up,down}
+ * (a block is a self-attention module followed by a feed-forward module: Section "Layer
+ * pruning").  Only the linears are on this path; the glue between them is a documented
+ * stub, every intermediate rounded to bf16 (round-to-nearest-even):
+ *     q = Wq x, k = Wk x, v = Wv x        (one fused launch; k, v stay in the workspace)
+ *     a = q                                (attention stub: identity)
+ *     hdn = Wo a
+ *     g = Wg hdn, u = Wu hdn               (one fused launch)
+ *     t = bf16(silu(g) * u)                (silu in fp32)
+ *     y = Wd t
+ * x: device bf16 [N*hidden]; y: device [N*M_down] in h[6]'s y_dtype.
+ * workspace: device, sd2_block_workspace_bytes bytes, 256-byte aligned; after the call it
+ * holds, in this order and each [N*dim] bf16, 256-byte aligned: q, k, v, hdn, g, u, t.
+ * Errors: SHAPE if the seven shapes do not chain; N must be in [0, 64]. */
+sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N,
+                          void* workspace, void* cuda_stream);
+
+sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* bytes);
+
+/* Byte offsets of q, k, v, hdn, g, u, t inside the workspace (offsets[7]). */
+sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets);
+
+/* Static string for a status code. */
+const char* sd2_status_string(sd2_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SD2_H */

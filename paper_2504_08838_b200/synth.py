@@ -89,14 +89,53 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+_CHUNK = 1 << 19      # elements per work item: temporaries stay in cache
+_POOL = None
+
+
+def _pool():
+    global _POOL
+    if _POOL is None:
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        _POOL = ThreadPoolExecutor(max_workers=max(1, min(32, len(os.sched_getaffinity(0)))))
+    return _POOL
+
+
+def _chunked(fn, n: int, dtype) -> np.ndarray:
+    """``fn(offset, count)`` over [0, n) in even-sized chunks on a thread pool (numpy drops the GIL).
+    The streams are counter based, so chunking never changes a value."""
+    out = np.empty(n, dtype=dtype)
+    if n <= _CHUNK:
+        out[:] = fn(0, n)
+        return out
+
+    def work(o):
+        c = min(_CHUNK, n - o)
+        out[o:o + c] = fn(o, c)
+
+    list(_pool().map(work, range(0, n, _CHUNK)))
+    return out
+
+
 def normal_bf16(seed: int, shape, sigma: float) -> np.ndarray:
     n = int(np.prod(shape))
-    return f32_to_bf16_bits(normal(seed, n, sigma).astype(np.float32)).reshape(shape)
+
+    def part(o, c):           # o is even: Box-Muller pairs never straddle a chunk
+        pairs = (c + 1) // 2
+        u = uniform(seed, 2 * pairs, offset=o)
+        r = np.sqrt(-2.0 * np.log(1.0 - u[0::2]))
+        z = np.empty(2 * pairs, dtype=np.float64)
+        z[0::2] = r * np.cos(2.0 * np.pi * u[1::2])
+        z[1::2] = r * np.sin(2.0 * np.pi * u[1::2])
+        return f32_to_bf16_bits((z[:c] * sigma).astype(np.float32))
+
+    return _chunked(part, n, np.uint16).reshape(shape)
 
 
 def bernoulli_mask(seed: int, shape, density: float) -> np.ndarray:
     n = int(np.prod(shape))
-    return (uniform(seed, n) < density).astype(np.uint8).reshape(shape)
+    return _chunked(lambda o, c: (uniform(seed, c, offset=o) < density).astype(np.uint8), n, np.uint8).reshape(shape)
 
 
 def beta22(seed: int, n: int) -> np.ndarray:

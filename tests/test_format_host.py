@@ -1,0 +1,162 @@
+"""Host side of the compressed formats: lossless, exact byte counts, validated blobs.
+
+Needs no GPU: ``sd2_pack_host`` / ``sd2_unpack_host`` are the same encoder and decoder
+``sd2_compress`` / ``sd2_decompress`` use.  Expected dense matrices come from the oracle.
+"""
+
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2504_08838_b200 import binding as sd2
+from paper_2504_08838_b200 import synth
+
+FORMATS = [sd2.SD2_FORMAT_BITMASK, sd2.SD2_FORMAT_GAP4]
+
+
+def _case(seed, M, K, d):
+    W = synth.normal_bf16(seed, (M, K), 0.02)
+    mask = synth.bernoulli_mask(seed + 1, (M, K), d)
+    return W, mask
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("M,K,d", [(1, 1, 1.0), (3, 5, 0.5), (7, 130, 0.5), (64, 64, 0.3), (33, 1000, 0.1),
+                                   (5, 4099, 0.5), (17, 257, 0.9), (2, 3000, 0.02), (40, 1536, 0.7)])
+def test_roundtrip_is_bit_exact(fmt, M, K, d):
+    W, mask = _case(1000 + M + K, M, K, d)
+    blob = sd2.sd2_pack_host(W, mask, fmt)
+    dense, info = sd2.sd2_unpack_host(blob)
+    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+    assert info["nnz"] == oracle.nnz(W, mask) == int(mask.sum())
+    assert (info["M"], info["K"], info["format"]) == (M, K, fmt)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_special_bit_patterns_survive(fmt):
+    M, K = 6, 96
+    W, mask = _case(7, M, K, 0.5)
+    mask[0, :4] = 1
+    W[0, 0], W[0, 1], W[0, 2], W[0, 3] = 0x8000, 0x0001, 0x7FC1, 0xFF80   # -0, subnormal, NaN payload, -Inf
+    mask[1, :] = 0                                                        # empty row
+    mask[2, :] = 1                                                        # full row
+    mask[3, :] = 0
+    mask[3, K - 1] = 1                                                    # only the last column
+    W[4, 10] = 0x7F80
+    mask[4, 10] = 0                                                       # masked-out Inf must vanish
+    blob = sd2.sd2_pack_host(W, mask, fmt)
+    dense, info = sd2.sd2_unpack_host(blob)
+    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+    assert info["nnz"] == int(mask.sum())
+    assert dense[0, 0] == 0x8000 and dense[4, 10] == 0
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_zero_and_full_masks(fmt):
+    W = synth.normal_bf16(9, (10, 200), 0.02)
+    zero = np.zeros((10, 200), np.uint8)
+    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, zero, fmt))
+    assert not dense.any() and info["nnz"] == 0
+    if fmt == sd2.SD2_FORMAT_BITMASK:
+        assert info["compressed_bytes"] == 4 * 11 + 4 * 10 * 7      # offsets + mask words, no values
+    else:
+        assert info["compressed_bytes"] == 4 * 11                   # offsets only, no chunks
+    full = np.ones((10, 200), np.uint8)
+    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, full, fmt))
+    assert np.array_equal(dense, W) and info["nnz"] == 2000
+
+
+def test_null_mask_means_nonzero_weights():
+    W = synth.normal_bf16(11, (8, 100), 0.02)
+    W[0, :50] = 0
+    W[1, 7] = 0x8000
+    for fmt in FORMATS:
+        dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, None, fmt))
+        assert np.array_equal(dense, oracle.roundtrip_ref(W, None))
+        assert info["nnz"] == oracle.nnz(W, None)
+
+
+def test_bitmask_byte_count_closed_form():
+    M, K = 37, 1000
+    W, mask = _case(21, M, K, 0.5)
+    _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_BITMASK), want_dense=False)
+    assert info["compressed_bytes"] == 4 * (M + 1) + 4 * M * ((K + 31) // 32) + 2 * int(mask.sum())
+
+
+def _gap4_entries(row_mask):
+    """Entries (kept + fillers) of one row under the 4-bit gap code, from its definition."""
+    cursor, e = 0, 0
+    for k in np.nonzero(row_mask)[0]:
+        while k - cursor > 15:
+            e += 1
+            cursor += 16
+        e += 1
+        cursor = k + 1
+    return e
+
+
+def test_gap4_byte_count_closed_form():
+    M, K = 29, 700
+    for d in (0.5, 0.1, 0.03):
+        W, mask = _case(31, M, K, d)
+        chunks = sum((_gap4_entries(mask[m]) + 7) // 8 for m in range(M))
+        _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
+        assert info["compressed_bytes"] == 4 * (M + 1) + 20 * chunks
+
+
+def test_gap4_long_rows_span_several_tiles():
+    # 11008 columns at 90 % density: ~1240 chunks per row -> 8 tiles of ~155 chunks, J = 5
+    M, K = 3, 11008
+    W, mask = _case(41, M, K, 0.9)
+    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+    # every chunk count from 1 to 400 exercises every (J, L, cnt_last) tile geometry
+    K = 8 * 400
+    mask = np.zeros((400, K), np.uint8)
+    for m in range(400):
+        mask[m, : 8 * (m + 1)] = 1
+    W = synth.normal_bf16(43, (400, K), 0.02)
+    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+    assert info["compressed_bytes"] == 4 * 401 + 20 * sum(range(1, 401))
+
+
+def test_sizes_at_half_density_match_the_format_arithmetic():
+    M, K = 256, 2048
+    W, mask = _case(51, M, K, 0.5)
+    nnz = int(mask.sum())
+    _, bm = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_BITMASK), want_dense=False)
+    _, g4 = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
+    assert abs(bm["compressed_bytes"] / nnz - 2.25) < 0.01       # 2 B value + 2 bits of mask per kept weight
+    assert 2.5 <= g4["compressed_bytes"] / nnz < 2.53            # 2 B value + 4-bit gap + row padding
+    assert g4["compressed_bytes"] < 0.64 * 2 * M * K             # well under the dense bf16 bytes
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_corrupt_blobs_are_rejected(fmt):
+    W, mask = _case(61, 20, 300, 0.5)
+    blob = bytearray(sd2.sd2_pack_host(W, mask, fmt))
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_unpack_host(bytes(blob[:100]))
+    assert e.value.status == sd2.SD2_ERR_CORRUPT
+    bad = bytearray(blob)
+    bad[0] ^= 0xFF                                               # magic
+    with pytest.raises(sd2.Sd2Error):
+        sd2.sd2_unpack_host(bytes(bad))
+    bad = bytearray(blob)
+    bad[len(bad) // 2] ^= 0x10                                   # payload bit flip -> checksum
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_unpack_host(bytes(bad))
+    assert e.value.status == sd2.SD2_ERR_CORRUPT
+    with pytest.raises(sd2.Sd2Error):
+        sd2.sd2_unpack_host(bytes(blob) + b"\0" * 256)           # wrong total size
+
+
+def test_bad_arguments():
+    W, mask = _case(71, 4, 8, 0.5)
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, fmt=99)
+    assert e.value.status == sd2.SD2_ERR_INVALID_ARG
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, y_dtype=5)
+    assert e.value.status == sd2.SD2_ERR_INVALID_ARG

@@ -1,0 +1,297 @@
+"""Parity of the CUDA path with the CPU oracle, element by element, through the C ABI.
+
+Tolerance (stated by the benchmark spec for this path): |y - y_ref| <= 1e-3 * S with
+S = sum_k |w_k x_k| for fp32 outputs; bf16 outputs add their own rounding, 2^-9 |y_ref|.
+Integer-valued inputs must match bit for bit in any summation order.
+"""
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import oracle
+from paper_2504_08838_b200 import binding as sd2
+from paper_2504_08838_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+FORMATS = [sd2.SD2_FORMAT_BITMASK, sd2.SD2_FORMAT_GAP4]
+POISON = 0x7FC0  # bf16 NaN
+
+
+def dev_bf16(bits: np.ndarray):
+    return torch.from_numpy(bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
+
+
+def run_spmm(h, X_bits, f32: bool):
+    """Launch on poisoned output with guard bands; returns Y as fp64 numpy [N, M]."""
+    N = X_bits.shape[0]
+    guard = 64
+    if f32:
+        buf = torch.full((N * h.M + 2 * guard,), float("nan"), dtype=torch.float32, device="cuda")
+    else:
+        buf = torch.full((N * h.M + 2 * guard,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Y = buf[guard:guard + N * h.M].view(N, h.M)
+    sd2.sd2_spmm(h, dev_bf16(X_bits), Y)
+    torch.cuda.synchronize()
+    out = buf.float().cpu().numpy().astype(np.float64)
+    assert np.isnan(out[:guard]).all() and np.isnan(out[-guard:]).all(), "guard band overwritten"
+    y = out[guard:-guard].reshape(N, h.M)
+    assert not np.isnan(y).any(), "output element left unwritten"
+    return y
+
+
+def check(y, Yr, S, f32: bool):
+    tol = 1e-3 * S + (0.0 if f32 else 2.0 ** -9 * np.abs(Yr))
+    bad = np.abs(y - Yr) > tol
+    assert not bad.any(), "max err/S = %g" % np.max(np.abs(y - Yr) / np.maximum(S, 1e-300))
+    assert np.all(y[S == 0] == 0)
+
+
+def case(seed, M, K, d, N, kind="bernoulli"):
+    W = synth.normal_bf16(seed, (M, K), 0.02)
+    mask = synth.bernoulli_mask(seed + 1, (M, K), d) if kind == "bernoulli" else synth.magnitude_mask(W, seed + 1, d)
+    X = synth.normal_bf16(seed + 2, (N, K), 1.0)
+    return W, mask, X
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("M,K,d", [(1, 1, 1.0), (3, 5, 0.5), (7, 130, 0.5), (100, 1000, 0.1), (64, 4099, 0.5)])
+def test_device_roundtrip_is_bit_exact(fmt, M, K, d):
+    W, mask, _ = case(500 + M, M, K, d, 1)
+    h = sd2.sd2_compress(W, mask, fmt)
+    assert np.array_equal(sd2.sd2_decompress(h), oracle.roundtrip_ref(W, mask))
+    assert h.nnz == int(mask.sum())
+    # device-resident inputs give the same handle contents
+    h2 = sd2.sd2_compress(dev_bf16(W), torch.from_numpy(mask).cuda(), fmt)
+    assert np.array_equal(sd2.sd2_decompress(h2), oracle.roundtrip_ref(W, mask))
+    assert h2.compressed_bytes == h.compressed_bytes
+    sd2.sd2_free(h)
+    sd2.sd2_free(h2)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("f32", [True, False])
+@pytest.mark.parametrize("M,K,d,N", [
+    (1, 1, 1.0, 1), (3, 5, 0.5, 1), (7, 130, 0.5, 2), (64, 64, 0.5, 1), (33, 1000, 0.1, 3),
+    (257, 2048, 0.5, 1), (40, 1536, 0.3, 5), (19, 8960, 0.5, 1), (9, 11008, 0.9, 8), (300, 777, 0.02, 4),
+])
+def test_spmm_matches_oracle(fmt, f32, M, K, d, N):
+    W, mask, X = case(900 + M + K + N, M, K, d, N)
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32 if f32 else sd2.SD2_DTYPE_BF16)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(run_spmm(h, X, f32), Yr, S, f32)
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_config1_single_sparse_linear(fmt):
+    # 2048 x 2048, 50 % Bernoulli, N(0, 0.02) weights, one N(0,1) activation row
+    W, mask = synth.make_linear(1, 0, 0, 2048, 2048, 0.5)
+    X = synth.make_activations(1, 0, 0, 1, 2048)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    for f32 in (True, False):
+        h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32 if f32 else sd2.SD2_DTYPE_BF16)
+        check(run_spmm(h, X, f32), Yr, S, f32)
+        sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("N", [1, 2, 3, 4, 7, 8, 9, 16, 33, 64])
+def test_all_panel_widths(fmt, N):
+    W, mask, X = case(1300 + N, 130, 1536, 0.5, N)
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    y = run_spmm(h, X, True)
+    check(y, Yr, S, True)
+    # row n of a panel agrees with the same row run alone (both within tolerance of one oracle row)
+    y0 = run_spmm(h, X[N - 1:N], True)
+    check(y0, Yr[N - 1:N], S[N - 1:N], True)
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_integer_inputs_are_bit_exact(fmt):
+    M, K, N = 96, 4096, 3
+    W = synth.integer_bf16(1, (M, K), -16, 16)
+    X = synth.integer_bf16(2, (N, K), -16, 16)
+    mask = synth.bernoulli_mask(3, (M, K), 0.5)
+    Yr, _ = oracle.masked_linear(W, mask, X)
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+    assert np.array_equal(run_spmm(h, X, True), Yr)
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_degenerate_masks_and_rows(fmt):
+    M, K = 70, 900
+    W = synth.normal_bf16(5, (M, K), 0.02)
+    X = synth.normal_bf16(6, (2, K), 1.0)
+    for mask in (np.zeros((M, K), np.uint8), np.ones((M, K), np.uint8)):
+        h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+        Yr, S = oracle.masked_linear(W, mask, X)
+        y = run_spmm(h, X, True)
+        check(y, Yr, S, True)
+        if not mask.any():
+            assert not y.any() and not np.signbit(y).any()      # empty rows write +0
+        sd2.sd2_free(h)
+    mask = synth.bernoulli_mask(7, (M, K), 0.5)
+    mask[::3, :] = 0                 # empty rows between populated ones
+    mask[1, :] = 0
+    mask[1, K - 1] = 1               # a single entry in the last column
+    mask[4, :] = 0
+    mask[4, 0] = 1                   # a single entry in the first column
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(run_spmm(h, X, True), Yr, S, True)
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_one_hot_activation_decodes_every_column_exactly(fmt):
+    M, K = 40, 1200
+    W, mask, _ = case(77, M, K, 0.5, 1)
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+    cols = [0, 1, 15, 16, 17, 255, 256, 1023, K - 2, K - 1]
+    X = np.zeros((len(cols), K), np.uint16)
+    for i, c in enumerate(cols):
+        X[i, c] = 0x3F80
+    y = run_spmm(h, X, True)
+    Wm = synth.bf16_bits_to_f32(oracle.roundtrip_ref(W, mask)).astype(np.float64)
+    for i, c in enumerate(cols):
+        assert np.array_equal(y[i], Wm[:, c])
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_uneven_rows_magnitude_masks(fmt):
+    # per-row densities spread over (0, 1) at 50 % and (0, 0.6) at 70 % sparsity
+    for d in (0.5, 0.3):
+        W, mask, X = case(2000, 512, 1536, d, 2, kind="magnitude")
+        h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+        Yr, S = oracle.masked_linear(W, mask, X)
+        check(run_spmm(h, X, True), Yr, S, True)
+        sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+def test_linearity_and_scaling(fmt):
+    M, K = 64, 2048
+    W, mask, _ = case(88, M, K, 0.5, 1)
+    X1 = synth.integer_bf16(33, (1, K), -8, 8)
+    X4 = synth.f32_to_bf16_bits(synth.bf16_bits_to_f32(X1) * 4.0)
+    h = sd2.sd2_compress(W, mask, fmt, sd2.SD2_DTYPE_F32)
+    y1 = run_spmm(h, X1, True)
+    y4 = run_spmm(h, X4, True)
+    assert np.array_equal(y4, 4.0 * y1)      # power-of-two scaling commutes with every rounding
+    sd2.sd2_free(h)
+
+
+def test_fused_launch_equals_separate_launches():
+    K, N = 2048, 4
+    X = synth.normal_bf16(3, (N, K), 1.0)
+    hs, refs = [], []
+    for i, M in enumerate((256, 64, 64)):
+        W, mask = synth.make_linear(2, 0, i, M, K, 0.5)
+        hs.append(sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32))
+        refs.append(oracle.masked_linear(W, mask, X))
+    Xd = dev_bf16(X)
+    Ys = [torch.full((N, h.M), float("nan"), dtype=torch.float32, device="cuda") for h in hs]
+    sd2.sd2_spmm_fused(hs, Xd, Ys)
+    torch.cuda.synchronize()
+    for h, Y, (Yr, S) in zip(hs, Ys, refs):
+        y = Y.cpu().numpy().astype(np.float64)
+        check(y, Yr, S, True)
+        Y1 = torch.empty_like(Y)
+        sd2.sd2_spmm(h, Xd, Y1)
+        torch.cuda.synchronize()
+        assert torch.equal(Y, Y1)            # same kernel, same order: identical bits
+    for h in hs:
+        sd2.sd2_free(h)
+
+
+def bf16_ulp_distance(a_bits, b_bits):
+    def key(b):
+        b = b.astype(np.int32)
+        return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    return np.abs(key(a_bits) - key(b_bits))
+
+
+@pytest.mark.parametrize("fmt", FORMATS)
+@pytest.mark.parametrize("N", [1, 3, 8])
+def test_block_step_teacher_forced(fmt, N):
+    # a scaled-down block with the Llama layout: hidden 256, kv 64, inter 1024
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 1)
+    lin = synth.make_block(2, 0, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m, fmt, sd2.SD2_DTYPE_F32 if i == 6 else sd2.SD2_DTYPE_BF16)
+          for i, (W, m) in enumerate(lin)]
+    x = synth.make_activations(2, 0, 0, N, shape.hidden)
+    xd = dev_bf16(x)
+    nbytes = sd2.sd2_block_workspace_bytes(hs, N)
+    off = sd2.sd2_block_workspace_layout(hs, N)
+    ws = torch.full((nbytes // 2,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_block_step(hs, xd, y, ws)
+    torch.cuda.synchronize()
+    wsb = ws.view(torch.int16).cpu().numpy().view(np.uint16)
+    dims = [shape.hidden, shape.kv, shape.kv, shape.hidden, shape.inter, shape.inter, shape.inter]
+    q, k, v, hdn, g, u, t = [wsb[o // 2:o // 2 + N * dm].reshape(N, dm) for o, dm in zip(off, dims)]
+
+    def lin_check(idx, inp_bits, out_bits):
+        Yr, S = oracle.masked_linear(lin[idx][0], lin[idx][1], inp_bits)
+        check(synth.bf16_bits_to_f32(out_bits).astype(np.float64), Yr, S, False)
+
+    lin_check(0, x, q)
+    lin_check(1, x, k)
+    lin_check(2, x, v)
+    lin_check(3, q, hdn)            # attention stub: the o projection reads q as is
+    lin_check(4, hdn, g)
+    lin_check(5, hdn, u)
+    t_ref = oracle.silu_mul(g, u)
+    t_ref_bits = np.array([oracle.f64_to_bf16_rne(float(z)) for z in t_ref], np.uint16).reshape(N, -1)
+    assert bf16_ulp_distance(t, t_ref_bits).max() <= 2
+    Yr, S = oracle.masked_linear(lin[6][0], lin[6][1], t)
+    check(y.cpu().numpy().astype(np.float64), Yr, S, True)
+    for h in hs:
+        sd2.sd2_free(h)
+
+
+def test_block_step_rejects_shapes_that_do_not_chain():
+    shape = synth.DrafterShape("tiny", 128, 32, 256, 1)
+    lin = synth.make_block(2, 1, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m) for W, m in lin]
+    bad = list(hs)
+    bad[6] = hs[3]                  # down must take `inter` inputs
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_block_workspace_bytes(bad, 1)
+    assert e.value.status == sd2.SD2_ERR_SHAPE
+    for h in hs:
+        sd2.sd2_free(h)
+
+
+def test_handle_lifecycle_errors():
+    W, mask, X = case(5, 8, 64, 0.5, 1)
+    h = sd2.sd2_compress(W, mask)
+    raw = h.raw
+    L = sd2.lib()
+    assert L.sd2_free(raw) == sd2.SD2_OK
+    assert L.sd2_free(raw) == sd2.SD2_ERR_INVALID_ARG          # double free is refused, not a crash
+    h.raw = None
+    h2 = sd2.sd2_compress(W, mask)
+    Xd = dev_bf16(X)
+    Y = torch.empty((1, 8), dtype=torch.bfloat16, device="cuda")
+    assert L.sd2_spmm(h2.raw, Xd.data_ptr(), Y.data_ptr(), 0, None) == sd2.SD2_OK       # N = 0: no-op
+    assert L.sd2_spmm(h2.raw, None, Y.data_ptr(), 1, None) == sd2.SD2_ERR_INVALID_ARG
+    assert L.sd2_spmm(h2.raw, Xd.data_ptr(), Y.data_ptr(), -1, None) == sd2.SD2_ERR_SHAPE
+    sd2.sd2_free(h2)
+
+
+def test_blob_made_on_the_host_runs_on_the_device():
+    W, mask, X = case(11, 50, 640, 0.5, 2)
+    for fmt in FORMATS:
+        blob = sd2.sd2_pack_host(W, mask, fmt, sd2.SD2_DTYPE_F32)
+        h = sd2.sd2_load_blob(blob, sd2.SD2_DTYPE_F32)
+        Yr, S = oracle.masked_linear(W, mask, X)
+        check(run_spmm(h, X, True), Yr, S, True)
+        sd2.sd2_free(h)
