@@ -148,6 +148,12 @@ sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* by
 /* Byte offsets of q, k, v, hdn, g, u, t inside the workspace (offsets[7]). */
 sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets);
 
+/* Wait for the stream and report device-side trouble: kernels bound every wait on an
+ * asynchronous copy; one that runs out raises an error word instead of hanging.  Returns
+ * SD2_ERR_TIMEOUT (and clears the word) if that happened since the last check, SD2_ERR_CUDA
+ * if the stream itself failed, SD2_OK otherwise.  Synchronises; not for the hot loop. */
+sd2_status sd2_stream_check(void* cuda_stream);
+
 /* Static string for a status code. */
 const char* sd2_status_string(sd2_status s);
 

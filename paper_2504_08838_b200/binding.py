@@ -24,7 +24,7 @@ SD2_DTYPE_BF16, SD2_DTYPE_F32 = 0, 1
 EXPORTS = [
     "sd2_pack_host", "sd2_unpack_host", "sd2_blob_free", "sd2_compress", "sd2_load_blob",
     "sd2_decompress", "sd2_info", "sd2_free", "sd2_spmm", "sd2_spmm_fused", "sd2_block_step",
-    "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string",
+    "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
 ]
 
 
@@ -68,6 +68,7 @@ def lib():
             "sd2_block_step": [pp, p, p, i64, p, p],
             "sd2_block_workspace_bytes": [pp, i64, pi64],
             "sd2_block_workspace_layout": [pp, i64, pi64],
+            "sd2_stream_check": [p],
         }
         for name, argtypes in sig.items():
             fn = getattr(L, name)
@@ -239,6 +240,11 @@ def sd2_block_workspace_layout(hs, N: int):
     off = (ctypes.c_int64 * 7)()
     _check(lib().sd2_block_workspace_layout(_handle_array(hs), N, off), "sd2_block_workspace_layout")
     return list(off)
+
+
+def sd2_stream_check(stream=None):
+    """Synchronise the stream; raises Sd2Error(TIMEOUT) if a device-side wait ran out."""
+    _check(lib().sd2_stream_check(_stream(stream)), "sd2_stream_check")
 
 
 def sd2_block_step(hs, x, y, workspace, stream=None, handle_array=None):

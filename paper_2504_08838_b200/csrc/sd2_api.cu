@@ -30,7 +30,11 @@ namespace {
 std::mutex g_mu;
 std::unordered_set<sd2_handle> g_live;
 int g_sm_count[64];
+int* g_err_word[64];
 bool g_dev_ready[64];
+int g_ctas_per_sm = 2;     // SD2_CTAS_PER_SM overrides (tuning aid)
+int g_depth_cap = 4;       // SD2_RING_DEPTH overrides (tuning aid)
+int g_use_pdl = 1;         // SD2_PDL=0 disables programmatic dependent launch
 
 bool live(sd2_handle h)
 {
@@ -50,17 +54,31 @@ sd2_status from_pack(int s)
     }
 }
 
-constexpr size_t kSmemBudget = 200 * 1024;  // per CTA, leaves room under the 227 KB limit
+constexpr size_t kSmemBudget = 220 * 1024;  // per CTA, under the 227 KB limit
+constexpr size_t kRingPerStage = (size_t)kWarpsPerCta * (kStageBytes + 16 + 8);
 
-size_t gap4_smem(int K, int NT) { return (size_t)(K + kGap4Slack) * 4 * NT; }
+size_t gap4_x_bytes(int K, int NT) { return (((size_t)(K + kGap4Slack) * 4 * NT) + 15) & ~size_t(15); }
 
-// Largest panel width (1, 2, 4, 8) whose staged activations fit in shared memory; 0 if none.
+// Largest panel width (1, 2, 4, 8) whose staged activations plus a two-stage ring fit; 0 if none.
 int gap4_max_nt(int K)
 {
     for (int nt = 8; nt >= 1; nt >>= 1)
-        if (gap4_smem(K, nt) <= kSmemBudget) return nt;
+        if (gap4_x_bytes(K, nt) + 2 * kRingPerStage <= kSmemBudget) return nt;
     return 0;
 }
+
+// Ring depth: as deep as the cap allows while `ctas_per_sm` CTAs still fit in one SM's shared memory.
+int gap4_depth(int K, int NT, int ctas_per_sm)
+{
+    const size_t per_cta = (227 * 1024) / (size_t)ctas_per_sm - 1024;
+    const size_t xb = gap4_x_bytes(K, NT);
+    int d = xb < per_cta ? (int)((per_cta - xb) / kRingPerStage) : 0;
+    if (d > g_depth_cap) d = g_depth_cap;
+    if (d < 2) d = 2;
+    return d;
+}
+
+size_t gap4_smem(int K, int NT, int depth) { return gap4_x_bytes(K, NT) + (size_t)depth * kRingPerStage; }
 
 template <int NT>
 cudaError_t set_smem_attr()
@@ -83,6 +101,13 @@ sd2_status ensure_device(int* dev_out)
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
+        int* err = nullptr;
+        if (cudaMalloc((void**)&err, 256) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_ALLOC; }
+        if (cudaMemset(err, 0, 256) != cudaSuccess) { cudaGetLastError(); cudaFree(err); return SD2_ERR_CUDA; }
+        if (const char* e = std::getenv("SD2_CTAS_PER_SM")) { int v = std::atoi(e); if (v >= 1 && v <= 8) g_ctas_per_sm = v; }
+        if (const char* e = std::getenv("SD2_RING_DEPTH")) { int v = std::atoi(e); if (v >= 2 && v <= kMaxDepth) g_depth_cap = v; }
+        if (const char* e = std::getenv("SD2_PDL")) g_use_pdl = std::atoi(e) != 0;
+        g_err_word[dev] = err;
         g_sm_count[dev] = sms;
         g_dev_ready[dev] = true;
     }
@@ -159,11 +184,11 @@ bool is_device_ptr(const void* p)
     return a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged;
 }
 
-// CTAs to give a weight of M rows: one row per warp until the device is full.
-int ctas_for(int64_t M, int sms)
+// CTAs of the whole launch: one row per warp until `ctas_per_sm` CTAs sit on every SM.
+int grid_for(int64_t rows_total, int sms)
 {
-    int64_t want = (M + kWarpsPerCta - 1) / kWarpsPerCta;
-    int64_t cap = (int64_t)sms * 4;
+    int64_t want = (rows_total + kWarpsPerCta - 1) / kWarpsPerCta;
+    int64_t cap = (int64_t)sms * g_ctas_per_sm;
     return (int)(want < cap ? want : cap);
 }
 
@@ -171,7 +196,17 @@ template <int NT>
 sd2_status launch_nt(int format, const LaunchGroup& grp, int grid, cudaStream_t s)
 {
     if (format == SD2_FORMAT_GAP4) {
-        gap4_kernel<NT><<<grid, kThreads, gap4_smem(grp.K, NT), s>>>(grp);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = gap4_smem(grp.K, NT, grp.depth);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = g_use_pdl ? 1 : 0;
+        if (cudaLaunchKernelEx(&cfg, gap4_kernel<NT>, grp) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
     } else {
         bitmask_kernel<NT><<<grid, kThreads, 0, s>>>(grp);
     }
@@ -228,6 +263,11 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
     std::memset(&grp, 0, sizeof grp);
     grp.count = count;
     grp.K = (int)K;
+    grp.err = g_err_word[dev];
+    // CTAs are shared out in proportion to the bytes each weight streams
+    int64_t rows_total = 0, bytes_total = 0;
+    for (int i = 0; i < count; ++i) { rows_total += hs[i]->M; bytes_total += hs[i]->compressed_bytes; }
+    const int grid_total = grid_for(rows_total, g_sm_count[dev]);
     int grid = 0;
     for (int i = 0; i < count; ++i) {
         MatDesc& md = grp.mat[i];
@@ -237,12 +277,20 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
         md.M = (int)hs[i]->M;
         md.y_f32 = (!y_force_bf16 && hs[i]->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
         md.cta_begin = grid;
-        md.cta_count = ctas_for(hs[i]->M, g_sm_count[dev]);
+        int64_t share = (int64_t)((double)grid_total * (double)hs[i]->compressed_bytes / (double)bytes_total + 0.5);
+        const int64_t need = (hs[i]->M + kWarpsPerCta - 1) / kWarpsPerCta;
+        if (share > need) share = need;
+        if (share < 1) share = 1;
+        md.cta_count = (int)share;
         grid += md.cta_count;
     }
     for (int64_t n0 = 0; n0 < N; n0 += max_nt) {
         const int n = (int)((N - n0) < max_nt ? (N - n0) : max_nt);
         grp.N = n;
+        if (format == SD2_FORMAT_GAP4) {
+            grp.depth = gap4_depth((int)K, round_nt(n), g_ctas_per_sm);
+            grp.x_bytes = (int)gap4_x_bytes((int)K, round_nt(n));
+        }
         grp.x = x ? x + n0 * K : nullptr;
         grp.g = g ? g + n0 * K : nullptr;
         grp.u = u ? u + n0 * K : nullptr;
@@ -441,6 +489,21 @@ sd2_status sd2_free(sd2_handle h)
     if (cudaFree(h->d_blob) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
     delete h;
     return st;
+}
+
+sd2_status sd2_stream_check(void* cuda_stream)
+{
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    int flag = 0;
+    if (cudaMemcpy(&flag, g_err_word[dev], sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    if (flag) {
+        cudaMemset(g_err_word[dev], 0, sizeof flag);
+        return SD2_ERR_TIMEOUT;
+    }
+    return SD2_OK;
 }
 
 sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_stream)

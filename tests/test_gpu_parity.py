@@ -34,7 +34,7 @@ def run_spmm(h, X_bits, f32: bool):
         buf = torch.full((N * h.M + 2 * guard,), float("nan"), dtype=torch.bfloat16, device="cuda")
     Y = buf[guard:guard + N * h.M].view(N, h.M)
     sd2.sd2_spmm(h, dev_bf16(X_bits), Y)
-    torch.cuda.synchronize()
+    sd2.sd2_stream_check()          # synchronises; raises if a device-side wait ran out
     out = buf.float().cpu().numpy().astype(np.float64)
     assert np.isnan(out[:guard]).all() and np.isnan(out[-guard:]).all(), "guard band overwritten"
     y = out[guard:-guard].reshape(N, h.M)
