@@ -40,7 +40,8 @@
 extern "C" {
 #endif
 
-typedef struct sd2_handle_s* sd2_handle; /* opaque; owned by the library */
+typedef struct sd2_handle_s* sd2_handle;   /* opaque; one compressed weight; owned by the library */
+typedef struct sd2_drafter_s* sd2_drafter; /* opaque; a chain of drafter blocks; owned by the library */
 
 typedef enum {
     SD2_OK = 0,
@@ -59,7 +60,8 @@ enum {
     SD2_FORMAT_AUTO = 0,    /* library picks (currently SD2_FORMAT_GAP4 when it applies)    */
     SD2_FORMAT_BITMASK = 1, /* 1 bit per dense slot + packed kept values + row offsets    */
     SD2_FORMAT_GAP4 = 2     /* 4-bit column gaps + packed kept values in 8-entry chunks,  */
-                            /* rows cut into lane-balanced tiles (the fast path)          */
+                            /* rows cut into column strips, 32 strips to a tile (the fast */
+                            /* path; column strips wider than 496 are not supported)      */
 };
 
 enum { SD2_DTYPE_BF16 = 0, SD2_DTYPE_F32 = 1 };
@@ -116,9 +118,11 @@ sd2_status sd2_free(sd2_handle h);
 /* ---- the hot path -------------------------------------------------------------------- */
 
 /* Y = X (W.*mask)^T.   X: device bf16 [N*K].   Y: device [N*M], bf16 or fp32 per the
- * handle's y_dtype.  N = 0 is a no-op; N > 8 is processed in panels of at most 8 rows of X
- * (the weight is re-read from L2 for each panel).  cuda_stream is a cudaStream_t (NULL =
- * default stream).  X and Y need only their natural alignment. */
+ * handle's y_dtype.  N = 0 is a no-op; N > 4 (GAP4) or N > 8 (BITMASK) is processed in panels
+ * of at most that many rows of X (the weight is re-read for each panel).  cuda_stream is a
+ * cudaStream_t (NULL = default stream).  X and Y need only their natural alignment; all
+ * activations are expected to be finite (a filler entry of the GAP4 format multiplies +0 by
+ * the activation of a masked-out column). */
 sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_stream);
 
 /* Same-input fusion (q|k|v, gate|up): count <= 4 weights with equal K share one staged X
@@ -139,6 +143,10 @@ sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, voi
  * x: device bf16 [N*hidden]; y: device [N*M_down] in h[6]'s y_dtype.
  * workspace: device, sd2_block_workspace_bytes bytes, 256-byte aligned; after the call it
  * holds, in this order and each [N*dim] bf16, 256-byte aligned: q, k, v, hdn, g, u, t.
+ * With seven GAP4 weights the block is ONE launch: a persistent CTA per SM runs the stages
+ * one after another, separated by grid-wide barriers, while a producer warp keeps copying the
+ * coming stages' weights into shared memory.  Such launches take every SM; two of them should
+ * not be put on different streams in the hope of overlap.
  * Errors: SHAPE if the seven shapes do not chain; N must be in [0, 64]. */
 sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N,
                           void* workspace, void* cuda_stream);
@@ -147,6 +155,29 @@ sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* by
 
 /* Byte offsets of q, k, v, hdn, g, u, t inside the workspace (offsets[7]). */
 sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets);
+
+/* ---- a whole drafter: L blocks chained, one launch per panel of activation rows --------- */
+
+/* h: 7 * L live GAP4 handles on the current device, block by block in the order q,k,v,o,gate,
+ * up,down; block b+1 reads block b's output (rounded to bf16), so out(b) must equal
+ * hidden(b+1).  n_max in [1, 64] sizes the intermediate buffers, which the drafter owns.
+ * The handles must outlive the drafter.  May synchronise; allocates device memory.
+ * Errors: INVALID_ARG, SHAPE (shapes do not chain, L or n_max out of range), UNSUPPORTED (a
+ * handle is not GAP4, or a layer is too wide for shared memory), ALLOC. */
+sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2_drafter* out);
+
+/* One token step through all L blocks: x device bf16 [N*hidden], y device [N*out] in the
+ * last down projection's y_dtype, 0 <= N <= n_max.  Same stub glue as sd2_block_step.
+ * Asynchronous on the stream, allocates nothing.  Steps of one drafter must not overlap in
+ * time (they share its buffers): keep them on one stream. */
+sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, void* cuda_stream);
+
+/* Device addresses of block `block`'s buffers after a step, ptrs[8] = q, k, v, hdn, g, u, t and
+ * the block's bf16 output (not written for the last block, whose output goes to y).  Each is
+ * [n_max rows capacity] with row n at n * width. */
+sd2_status sd2_drafter_buffers(sd2_drafter d, int32_t block, void** ptrs);
+
+sd2_status sd2_drafter_free(sd2_drafter d);
 
 /* Wait for the stream and report device-side trouble: kernels bound every wait on an
  * asynchronous copy; one that runs out raises an error word instead of hanging.  Returns

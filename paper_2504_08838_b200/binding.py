@@ -25,6 +25,7 @@ EXPORTS = [
     "sd2_pack_host", "sd2_unpack_host", "sd2_blob_free", "sd2_compress", "sd2_load_blob",
     "sd2_decompress", "sd2_info", "sd2_free", "sd2_spmm", "sd2_spmm_fused", "sd2_block_step",
     "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
+    "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
 ]
 
 
@@ -69,6 +70,10 @@ def lib():
             "sd2_block_workspace_bytes": [pp, i64, pi64],
             "sd2_block_workspace_layout": [pp, i64, pi64],
             "sd2_stream_check": [p],
+            "sd2_drafter_create": [pp, i32, i64, pp],
+            "sd2_drafter_step": [p, p, p, i64, p],
+            "sd2_drafter_buffers": [p, i32, pp],
+            "sd2_drafter_free": [p],
         }
         for name, argtypes in sig.items():
             fn = getattr(L, name)
@@ -251,3 +256,48 @@ def sd2_block_step(hs, x, y, workspace, stream=None, handle_array=None):
     N = x.shape[0] if x.dim() == 2 else 1
     arr = handle_array if handle_array is not None else _handle_array(hs)
     _check(lib().sd2_block_step(arr, _ptr(x), _ptr(y), N, _ptr(workspace), _stream(stream)), "sd2_block_step")
+
+
+# ---- whole drafter ---------------------------------------------------------------------
+
+class Drafter:
+    """Owns one ``sd2_drafter`` (and keeps its handles alive)."""
+
+    def __init__(self, raw: int, blocks):
+        self.raw = ctypes.c_void_p(raw)
+        self.blocks = blocks
+
+    def close(self):
+        if self.raw is not None and self.raw.value:
+            lib().sd2_drafter_free(self.raw)
+            self.raw = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def sd2_drafter_create(blocks, n_max: int = 1) -> Drafter:
+    """``blocks``: list of 7-handle lists (q, k, v, o, gate, up, down), one per drafter block."""
+    flat = [h for hs in blocks for h in hs]
+    out = ctypes.c_void_p()
+    _check(lib().sd2_drafter_create(_handle_array(flat), len(blocks), n_max, ctypes.byref(out)), "sd2_drafter_create")
+    return Drafter(out.value, blocks)
+
+
+def sd2_drafter_step(d: Drafter, x, y, stream=None):
+    N = x.shape[0] if x.dim() == 2 else 1
+    _check(lib().sd2_drafter_step(d.raw, _ptr(x), _ptr(y), N, _stream(stream)), "sd2_drafter_step")
+
+
+def sd2_drafter_buffers(d: Drafter, block: int):
+    """Device addresses of q, k, v, hdn, g, u, t and the block output of one block."""
+    ptrs = (ctypes.c_void_p * 8)()
+    _check(lib().sd2_drafter_buffers(d.raw, block, ptrs), "sd2_drafter_buffers")
+    return [int(p or 0) for p in ptrs]
+
+
+def sd2_drafter_free(d: Drafter):
+    d.close()

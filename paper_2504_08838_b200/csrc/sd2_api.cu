@@ -3,12 +3,14 @@
 
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
 #include <unordered_set>
+#include <vector>
 
 #include "../../include/sd2.h"
 #include "sd2_format.hpp"
@@ -23,18 +25,45 @@ struct sd2_handle_s {
     const uint32_t* d_sec0;
     const uint32_t* d_sec1;
     const void* d_sec2;
+    // GAP4 geometry
+    int S, B, T, max_tile_bytes;
+};
+
+struct sd2_drafter_s {
+    int L, device;
+    int64_t n_max;
+    int n_stages;
+    int y_f32;                 // dtype of the last block's output
+    int64_t hidden, out_dim;
+    std::vector<sd2_handle> handles;
+    std::vector<int64_t> ws_off;        // per block: offsets of q,k,v,hdn,g,u,t and the block output inside d_ws
+    uint8_t* d_ws;
+    SStage* d_stages;
+    unsigned int* d_gbar;
+    int K_max, max_tile;       // what decides the shared-memory split
+    int xs_need[3];            // bytes of staged activations at panel widths 1, 2, 4
 };
 
 namespace {
 
 std::mutex g_mu;
 std::unordered_set<sd2_handle> g_live;
-int g_sm_count[64];
-int* g_err_word[64];
-bool g_dev_ready[64];
-int g_ctas_per_sm = 2;     // SD2_CTAS_PER_SM overrides (tuning aid)
-int g_depth_cap = 4;       // SD2_RING_DEPTH overrides (tuning aid)
-int g_use_pdl = 1;         // SD2_PDL=0 disables programmatic dependent launch
+std::unordered_set<sd2_drafter> g_live_drafters;
+
+constexpr int kMaxDevices = 64;
+constexpr int kBarrierPool = 64;             // grid-barrier word pairs handed out round-robin
+constexpr int kBarrierStrideWords = 64;      // 256 bytes apart
+constexpr int kSmemMax = 227 * 1024;         // dynamic shared memory a CTA may opt in to
+
+struct DeviceState {
+    bool ready;
+    int sms;
+    int clock_khz;
+    int* err_word;
+    unsigned int* barriers;
+};
+DeviceState g_dev[kMaxDevices];
+std::atomic<unsigned> g_next_barrier{0};
 
 bool live(sd2_handle h)
 {
@@ -43,82 +72,72 @@ bool live(sd2_handle h)
     return g_live.count(h) != 0;
 }
 
+bool live(sd2_drafter d)
+{
+    if (!d) return false;
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_live_drafters.count(d) != 0;
+}
+
 sd2_status from_pack(int s)
 {
     switch (s) {
         case 0: return SD2_OK;
         case -2: return SD2_ERR_SHAPE;
         case -3: return SD2_ERR_ALLOC;
+        case -5: return SD2_ERR_UNSUPPORTED;
         case -6: return SD2_ERR_CORRUPT;
         default: return SD2_ERR_INVALID_ARG;
     }
 }
 
-constexpr size_t kSmemBudget = 220 * 1024;  // per CTA, under the 227 KB limit
-constexpr size_t kRingPerStage = (size_t)kWarpsPerCta * (kStageBytes + 16 + 8);
-
-size_t gap4_x_bytes(int K, int NT) { return (((size_t)(K + kGap4Slack) * 4 * NT) + 15) & ~size_t(15); }
-
-// Largest panel width (1, 2, 4, 8) whose staged activations plus a two-stage ring fit; 0 if none.
-int gap4_max_nt(int K)
-{
-    for (int nt = 8; nt >= 1; nt >>= 1)
-        if (gap4_x_bytes(K, nt) + 2 * kRingPerStage <= kSmemBudget) return nt;
-    return 0;
-}
-
-// Ring depth: as deep as the cap allows while `ctas_per_sm` CTAs still fit in one SM's shared memory.
-int gap4_depth(int K, int NT, int ctas_per_sm)
-{
-    const size_t per_cta = (227 * 1024) / (size_t)ctas_per_sm - 1024;
-    const size_t xb = gap4_x_bytes(K, NT);
-    int d = xb < per_cta ? (int)((per_cta - xb) / kRingPerStage) : 0;
-    if (d > g_depth_cap) d = g_depth_cap;
-    if (d < 2) d = 2;
-    return d;
-}
-
-size_t gap4_smem(int K, int NT, int depth) { return gap4_x_bytes(K, NT) + (size_t)depth * kRingPerStage; }
-
 template <int NT>
 cudaError_t set_smem_attr()
 {
-    return cudaFuncSetAttribute(gap4_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+    return cudaFuncSetAttribute(stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
 }
 
-// Once per device: SM count and the shared-memory opt-in of every gap4 instantiation.
+// Once per device: SM count, shared-memory opt-in, the error word and the barrier pool.
 sd2_status ensure_device(int* dev_out)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-    if (dev < 0 || dev >= 64) return SD2_ERR_UNSUPPORTED;
+    if (dev < 0 || dev >= kMaxDevices) return SD2_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lk(g_mu);
-    if (!g_dev_ready[dev]) {
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess ||
-            set_smem_attr<4>() != cudaSuccess || set_smem_attr<8>() != cudaSuccess) {
+    DeviceState& ds = g_dev[dev];
+    if (!ds.ready) {
+        int sms = 0, khz = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess) {
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
         int* err = nullptr;
+        unsigned int* bars = nullptr;
+        const size_t bar_bytes = (size_t)kBarrierPool * kBarrierStrideWords * 4;
         if (cudaMalloc((void**)&err, 256) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_ALLOC; }
-        if (cudaMemset(err, 0, 256) != cudaSuccess) { cudaGetLastError(); cudaFree(err); return SD2_ERR_CUDA; }
-        if (const char* e = std::getenv("SD2_CTAS_PER_SM")) { int v = std::atoi(e); if (v >= 1 && v <= 8) g_ctas_per_sm = v; }
-        if (const char* e = std::getenv("SD2_RING_DEPTH")) { int v = std::atoi(e); if (v >= 2 && v <= kMaxDepth) g_depth_cap = v; }
-        if (const char* e = std::getenv("SD2_PDL")) g_use_pdl = std::atoi(e) != 0;
-        g_err_word[dev] = err;
-        g_sm_count[dev] = sms;
-        g_dev_ready[dev] = true;
+        if (cudaMalloc((void**)&bars, bar_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(err); return SD2_ERR_ALLOC; }
+        if (cudaMemset(err, 0, 256) != cudaSuccess || cudaMemset(bars, 0, bar_bytes) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(err);
+            cudaFree(bars);
+            return SD2_ERR_CUDA;
+        }
+        ds.err_word = err;
+        ds.barriers = bars;
+        ds.sms = sms;
+        ds.clock_khz = khz > 0 ? khz : 2000000;
+        ds.ready = true;
     }
     *dev_out = dev;
     return SD2_OK;
 }
 
-int resolve_format(const sd2_options* opt, int64_t K)
+int resolve_format(const sd2_options* opt, int64_t M, int64_t K)
 {
     int f = opt ? opt->format : SD2_FORMAT_AUTO;
-    if (f == SD2_FORMAT_AUTO) f = gap4_max_nt((int)(K > 1000000 ? 1000000 : K)) > 0 ? SD2_FORMAT_GAP4 : SD2_FORMAT_BITMASK;
+    if (f == SD2_FORMAT_AUTO) f = gap4_geometry(M, K).S > 0 ? SD2_FORMAT_GAP4 : SD2_FORMAT_BITMASK;
     return f;
 }
 
@@ -129,7 +148,7 @@ sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K
     if (M < 1 || K < 1 || M > 0x7FFFFFF0ll || K > 0x7FFFFFF0ll || M * K > (1ll << 40)) return SD2_ERR_SHAPE;
     const int y_dtype = opt ? opt->y_dtype : SD2_DTYPE_BF16;
     if (y_dtype != SD2_DTYPE_BF16 && y_dtype != SD2_DTYPE_F32) return SD2_ERR_INVALID_ARG;
-    const int f = resolve_format(opt, K);
+    const int f = resolve_format(opt, M, K);
     PackResult r;
     try {
         if (f == SD2_FORMAT_BITMASK) r = pack_bitmask(W, mask, M, K, y_dtype);
@@ -169,6 +188,10 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     h->d_sec0 = (const uint32_t*)(h->d_blob + hd.sec_off[0]);
     h->d_sec1 = (const uint32_t*)(h->d_blob + hd.sec_off[1]);
     h->d_sec2 = (const void*)(h->d_blob + hd.sec_off[2]);
+    h->S = (int)hd.strips;
+    h->B = (int)hd.strip_cols;
+    h->T = (int)hd.n_tiles;
+    h->max_tile_bytes = (int)hd.max_tile_bytes;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(h);
@@ -184,90 +207,37 @@ bool is_device_ptr(const void* p)
     return a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged;
 }
 
-// CTAs of the whole launch: one row per warp until `ctas_per_sm` CTAs sit on every SM.
-int grid_for(int64_t rows_total, int sms)
+// ------------------------------------------------------------------ BITMASK launches
+
+int bitmask_grid(int64_t rows_total, int sms)
 {
     int64_t want = (rows_total + kWarpsPerCta - 1) / kWarpsPerCta;
-    int64_t cap = (int64_t)sms * g_ctas_per_sm;
+    int64_t cap = (int64_t)sms * 8;
     return (int)(want < cap ? want : cap);
 }
 
 template <int NT>
-sd2_status launch_nt(int format, const LaunchGroup& grp, int grid, cudaStream_t s)
+sd2_status launch_bitmask_nt(const LaunchGroup& grp, int grid, cudaStream_t s)
 {
-    if (format == SD2_FORMAT_GAP4) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = gap4_smem(grp.K, NT, grp.depth);
-        cfg.stream = s;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = g_use_pdl ? 1 : 0;
-        if (cudaLaunchKernelEx(&cfg, gap4_kernel<NT>, grp) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-    } else {
-        bitmask_kernel<NT><<<grid, kThreads, 0, s>>>(grp);
-    }
+    bitmask_kernel<NT><<<grid, kThreads, 0, s>>>(grp);
     if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
     return SD2_OK;
 }
 
-sd2_status launch(int format, int nt, const LaunchGroup& grp, int grid, cudaStream_t s)
-{
-    switch (nt) {
-        case 1: return launch_nt<1>(format, grp, grid, s);
-        case 2: return launch_nt<2>(format, grp, grid, s);
-        case 4: return launch_nt<4>(format, grp, grid, s);
-        default: return launch_nt<8>(format, grp, grid, s);
-    }
-}
+int round_nt(int n, int cap) { int r = n <= 1 ? 1 : n <= 2 ? 2 : n <= 4 ? 4 : 8; return r > cap ? cap : r; }
 
-int round_nt(int n) { return n <= 1 ? 1 : n <= 2 ? 2 : n <= 4 ? 4 : 8; }
-
-// Shared by sd2_spmm, sd2_spmm_fused and sd2_block_step.  Exactly one of x / (g, u) is set.
-// y_force_bf16: intermediates of a block are bf16 whatever the handle says.
-sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
-                     uint16_t* t_out, void* const* Y, int64_t N, bool y_force_bf16, cudaStream_t s)
+// One launch per panel of at most 8 activation rows.  Exactly one of x / (g, u) is set.
+sd2_status run_bitmask(const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
+                       uint16_t* t_out, void* const* Y, int64_t N, bool y_force_bf16, int dev, cudaStream_t s)
 {
-    if (count < 1 || count > kMaxFused) return SD2_ERR_INVALID_ARG;
-    for (int i = 0; i < count; ++i)
-        if (!live(hs[i]) || !Y[i]) return SD2_ERR_INVALID_ARG;
-    if (N < 0) return SD2_ERR_SHAPE;
-    if (N == 0) return SD2_OK;
     const int64_t K = hs[0]->K;
-    const int format = hs[0]->format;
-    for (int i = 1; i < count; ++i)
-        if (hs[i]->K != K) return SD2_ERR_SHAPE;
-    for (int i = 1; i < count; ++i) {
-        if (hs[i]->format != format) {  // mixed formats cannot share a launch: one launch each
-            for (int j = 0; j < count; ++j) {
-                sd2_status sj = run_group(hs + j, 1, x, g, u, j == 0 ? t_out : nullptr, Y + j, N, y_force_bf16, s);
-                if (sj != SD2_OK) return sj;
-            }
-            return SD2_OK;
-        }
-    }
-    int dev = 0;
-    sd2_status st = ensure_device(&dev);
-    if (st != SD2_OK) return st;
-    for (int i = 0; i < count; ++i)
-        if (hs[i]->device != dev) return SD2_ERR_INVALID_ARG;
-    int max_nt = 8;
-    if (format == SD2_FORMAT_GAP4) {
-        max_nt = gap4_max_nt((int)K);
-        if (max_nt == 0) return SD2_ERR_UNSUPPORTED;
-    }
     LaunchGroup grp;
     std::memset(&grp, 0, sizeof grp);
     grp.count = count;
     grp.K = (int)K;
-    grp.err = g_err_word[dev];
-    // CTAs are shared out in proportion to the bytes each weight streams
     int64_t rows_total = 0, bytes_total = 0;
     for (int i = 0; i < count; ++i) { rows_total += hs[i]->M; bytes_total += hs[i]->compressed_bytes; }
-    const int grid_total = grid_for(rows_total, g_sm_count[dev]);
+    const int grid_total = bitmask_grid(rows_total, g_dev[dev].sms);
     int grid = 0;
     for (int i = 0; i < count; ++i) {
         MatDesc& md = grp.mat[i];
@@ -284,13 +254,9 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
         md.cta_count = (int)share;
         grid += md.cta_count;
     }
-    for (int64_t n0 = 0; n0 < N; n0 += max_nt) {
-        const int n = (int)((N - n0) < max_nt ? (N - n0) : max_nt);
+    for (int64_t n0 = 0; n0 < N; n0 += 8) {
+        const int n = (int)((N - n0) < 8 ? (N - n0) : 8);
         grp.N = n;
-        if (format == SD2_FORMAT_GAP4) {
-            grp.depth = gap4_depth((int)K, round_nt(n), g_ctas_per_sm);
-            grp.x_bytes = (int)gap4_x_bytes((int)K, round_nt(n));
-        }
         grp.x = x ? x + n0 * K : nullptr;
         grp.g = g ? g + n0 * K : nullptr;
         grp.u = u ? u + n0 * K : nullptr;
@@ -299,10 +265,209 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
             const size_t esz = grp.mat[i].y_f32 ? 4 : 2;
             grp.mat[i].y = (char*)Y[i] + (size_t)n0 * (size_t)hs[i]->M * esz;
         }
-        st = launch(format, round_nt(n), grp, grid, s);
+        sd2_status st;
+        switch (round_nt(n, 8)) {
+            case 1: st = launch_bitmask_nt<1>(grp, grid, s); break;
+            case 2: st = launch_bitmask_nt<2>(grp, grid, s); break;
+            case 4: st = launch_bitmask_nt<4>(grp, grid, s); break;
+            default: st = launch_bitmask_nt<8>(grp, grid, s); break;
+        }
         if (st != SD2_OK) return st;
     }
     return SD2_OK;
+}
+
+// ------------------------------------------------------------------ GAP4 programs
+
+// Largest panel width (4, 2, 1) whose staged activations leave room for a ring that holds
+// `max_tile` bytes at least twice; 0 if even one row does not fit.
+struct SmemPlan {
+    int nt, xs_bytes, xlin_bytes, ring_bytes;
+};
+
+int xs_bytes_for(int S, int B, int nt)
+{
+    const int groups = 32 / nt;
+    const int planes = S > groups ? S / groups : 1;
+    return planes * (B + kGap4Slack) * 128;
+}
+
+bool plan_smem(int nt, int xs_max, int K_max, int max_tile, SmemPlan* p)
+{
+    const int fixed = (int)((sizeof(StreamShared) + 127) & ~127);
+    const int xlin = (2 * K_max + 127) & ~127;
+    const int ring = (kSmemMax - fixed - xs_max - xlin) & ~127;
+    if (ring < 2 * max_tile + 256) return false;
+    p->nt = nt;
+    p->xs_bytes = xs_max;
+    p->xlin_bytes = xlin;
+    p->ring_bytes = ring;
+    return true;
+}
+
+template <int NT>
+sd2_status launch_stream_nt(const SArgs& a, int grid, int smem, bool cooperative, cudaStream_t s)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = cooperative ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, stream_kernel<NT>, a) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
+    return SD2_OK;
+}
+
+sd2_status launch_stream(int nt, const SArgs& a, int grid, bool cooperative, cudaStream_t s)
+{
+    const int smem = a.xs_bytes + a.xlin_bytes + (int)((sizeof(StreamShared) + 127) & ~127) + a.ring_bytes;
+    switch (nt) {
+        case 1: return launch_stream_nt<1>(a, grid, smem, cooperative, s);
+        case 2: return launch_stream_nt<2>(a, grid, smem, cooperative, s);
+        default: return launch_stream_nt<4>(a, grid, smem, cooperative, s);
+    }
+}
+
+// Fills one stage from `count` GAP4 handles of equal K and S.
+void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
+                uint16_t* t_out, void* const* Y, bool y_force_bf16)
+{
+    std::memset(&st, 0, sizeof st);
+    st.count = count;
+    st.K = (int)hs[0]->K;
+    st.S = hs[0]->S;
+    st.B = hs[0]->B;
+    st.hdr_bytes = gap4_tile_header_bytes(32 / hs[0]->S);
+    st.x = x;
+    st.g = g;
+    st.u = u;
+    st.t_out = t_out;
+    int T = 0;
+    for (int i = 0; i < count; ++i) {
+        SMat& m = st.mat[i];
+        m.tile_off = hs[i]->d_sec0;
+        m.stream = (const unsigned char*)hs[i]->d_sec1;
+        m.y = Y[i];
+        m.M = (int)hs[i]->M;
+        m.T = hs[i]->T;
+        m.y_f32 = (!y_force_bf16 && hs[i]->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
+        T += hs[i]->T;
+    }
+    st.T_total = T;
+}
+
+long long wait_budget(int dev)
+{
+    // about two seconds of SM clock; SD2_WAIT_MS overrides (tests use a short one)
+    long long ms = 2000;
+    if (const char* e = std::getenv("SD2_WAIT_MS")) { long long v = std::atoll(e); if (v >= 1 && v <= 60000) ms = v; }
+    return ms * (long long)g_dev[dev].clock_khz;
+}
+
+// Tracks what a program needs from shared memory.
+struct ProgramNeeds {
+    int K_max = 0, max_tile = 0, tiles_max = 0;
+    int xs_need[3] = {0, 0, 0};   // staged activations at panel widths 1, 2, 4: the largest over all stages
+    void add(const sd2_handle* hs, int count)
+    {
+        int T = 0;
+        for (int i = 0; i < count; ++i) {
+            if (hs[i]->K > K_max) K_max = (int)hs[i]->K;
+            if (hs[i]->max_tile_bytes > max_tile) max_tile = hs[i]->max_tile_bytes;
+            for (int w = 0; w < 3; ++w) {
+                const int need = xs_bytes_for(hs[i]->S, hs[i]->B, 1 << w);
+                if (need > xs_need[w]) xs_need[w] = need;
+            }
+            T += hs[i]->T;
+        }
+        if (T > tiles_max) tiles_max = T;
+    }
+};
+
+int nt_index(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : 2; }
+
+// Widest panel (4, 2, 1 rows) whose staged activations still leave room for the ring; 0 if none.
+int widest_panel(const int xs_need[3], int K_max, int max_tile)
+{
+    SmemPlan p;
+    for (int nt = 4; nt >= 1; nt >>= 1)
+        if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return nt;
+    return 0;
+}
+
+// Launches a program over all N rows, in panels of at most `nt_cap` rows (rows are independent).
+sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[3], int K_max, int max_tile, int grid, cudaStream_t s)
+{
+    const int nt_cap = widest_panel(xs_need, K_max, max_tile);
+    if (nt_cap == 0) return SD2_ERR_UNSUPPORTED;
+    for (int64_t n0 = 0; n0 < N; n0 += nt_cap) {
+        const int n = (int)((N - n0) < nt_cap ? (N - n0) : nt_cap);
+        const int nt = round_nt(n, nt_cap);
+        SmemPlan p;   // the narrower the panel, the more room for the ring
+        if (!plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return SD2_ERR_UNSUPPORTED;
+        a.N = n;
+        a.n0 = (int)n0;
+        a.xs_bytes = p.xs_bytes;
+        a.xlin_bytes = p.xlin_bytes;
+        a.ring_bytes = p.ring_bytes;
+        sd2_status st = launch_stream(nt, a, grid, a.n_stages > 1, s);
+        if (st != SD2_OK) return st;
+    }
+    return SD2_OK;
+}
+
+// Runs a program of inline stages.
+sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, cudaStream_t s)
+{
+    const bool coop = a.n_stages > 1;
+    int grid = g_dev[dev].sms;
+    if (!coop && needs.tiles_max < grid) grid = needs.tiles_max < 1 ? 1 : needs.tiles_max;
+    a.err = g_dev[dev].err_word;
+    a.wait_cycles = wait_budget(dev);
+    a.gbar = coop ? g_dev[dev].barriers + (size_t)(g_next_barrier.fetch_add(1) % kBarrierPool) * kBarrierStrideWords : nullptr;
+    return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, grid, s);
+}
+
+// Shared by sd2_spmm and sd2_spmm_fused (and by block steps that mix formats).
+sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
+                     uint16_t* t_out, void* const* Y, int64_t N, bool y_force_bf16, cudaStream_t s)
+{
+    if (count < 1 || count > kMaxFused) return SD2_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i)
+        if (!live(hs[i]) || !Y[i]) return SD2_ERR_INVALID_ARG;
+    if (N < 0) return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    const int64_t K = hs[0]->K;
+    for (int i = 1; i < count; ++i)
+        if (hs[i]->K != K) return SD2_ERR_SHAPE;
+    bool same = true;
+    for (int i = 1; i < count; ++i)
+        if (hs[i]->format != hs[0]->format || hs[i]->S != hs[0]->S) same = false;
+    if (!same) {  // weights that cannot share a stage: one launch each
+        for (int j = 0; j < count; ++j) {
+            sd2_status sj = run_group(hs + j, 1, x, g, u, j == 0 ? t_out : nullptr, Y + j, N, y_force_bf16, s);
+            if (sj != SD2_OK) return sj;
+        }
+        return SD2_OK;
+    }
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    for (int i = 0; i < count; ++i)
+        if (hs[i]->device != dev) return SD2_ERR_INVALID_ARG;
+    if (hs[0]->format == SD2_FORMAT_BITMASK) return run_bitmask(hs, count, x, g, u, t_out, Y, N, y_force_bf16, dev, s);
+    SArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.n_stages = 1;
+    fill_stage(a.inl[0], hs, count, x, g, u, t_out, Y, y_force_bf16);
+    ProgramNeeds needs;
+    needs.add(hs, count);
+    return run_program(a, dev, N, needs, s);
 }
 
 struct BlockDims {
@@ -340,6 +505,39 @@ void block_layout(const sd2_handle* h, const BlockDims& d, int64_t N, int64_t of
         o = a256(o + 2 * N * dims[i]);
     }
     off[7] = o;
+}
+
+// Appends the stages of one block (h[0..6] = q,k,v,o,gate,up,down) to `stages`.  Weights of a
+// group that do not share a strip geometry get a stage each.  Returns the number appended.
+int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
+                        uint16_t* hdn, uint16_t* g, uint16_t* u, uint16_t* t, void* y, bool y_force_bf16,
+                        ProgramNeeds* needs)
+{
+    int n = 0;
+    auto group = [&](const sd2_handle* hs, int count, const uint16_t* xin, const uint16_t* gg, const uint16_t* uu,
+                     uint16_t* tt, void* const* Y, bool force) {
+        bool same = true;
+        for (int i = 1; i < count; ++i)
+            if (hs[i]->S != hs[0]->S) same = false;
+        if (same) {
+            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force);
+            needs->add(hs, count);
+        } else {
+            for (int i = 0; i < count; ++i) {
+                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force);
+                needs->add(hs + i, 1);
+            }
+        }
+    };
+    void* y_qkv[3] = {q, k, v};
+    group(h + 0, 3, x, nullptr, nullptr, nullptr, y_qkv, true);
+    void* y_o[1] = {hdn};
+    group(h + 3, 1, q, nullptr, nullptr, nullptr, y_o, true);
+    void* y_gu[2] = {g, u};
+    group(h + 4, 2, hdn, nullptr, nullptr, nullptr, y_gu, true);
+    void* y_d[1] = {y};
+    group(h + 6, 1, nullptr, g, u, t, y_d, y_force_bf16);
+    return n;   // at most 7
 }
 
 }  // namespace
@@ -442,8 +640,13 @@ sd2_status sd2_load_blob(const void* blob, int64_t blob_bytes, sd2_handle* out)
     BlobHeader hd;
     if (check_header((const uint8_t*)blob, blob_bytes, hd, true) != 0) return SD2_ERR_CORRUPT;
     // full structural validation before anything reaches a kernel
-    const int rc = hd.format == (uint32_t)kFormatBitmask ? unpack_bitmask(hd, (const uint8_t*)blob, nullptr)
-                                                         : unpack_gap4(hd, (const uint8_t*)blob, nullptr);
+    int rc;
+    try {
+        rc = hd.format == (uint32_t)kFormatBitmask ? unpack_bitmask(hd, (const uint8_t*)blob, nullptr)
+                                                   : unpack_gap4(hd, (const uint8_t*)blob, nullptr);
+    } catch (const std::bad_alloc&) {
+        return SD2_ERR_ALLOC;
+    }
     if (rc != 0) return SD2_ERR_CORRUPT;
     return upload((const uint8_t*)blob, blob_bytes, hd, out);
 }
@@ -498,9 +701,18 @@ sd2_status sd2_stream_check(void* cuda_stream)
     if (st != SD2_OK) return st;
     if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
     int flag = 0;
-    if (cudaMemcpy(&flag, g_err_word[dev], sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    if (cudaMemcpy(&flag, g_dev[dev].err_word, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
     if (flag) {
-        cudaMemset(g_err_word[dev], 0, sizeof flag);
+        // a kernel that gave up leaves its barrier words behind: wait for the device, clear everything
+        cudaDeviceSynchronize();
+        cudaMemset(g_dev[dev].err_word, 0, sizeof flag);
+        cudaMemset(g_dev[dev].barriers, 0, (size_t)kBarrierPool * kBarrierStrideWords * 4);
+        {
+            std::lock_guard<std::mutex> lk(g_mu);
+            for (sd2_drafter d : g_live_drafters)
+                if (d->device == dev) cudaMemset(d->d_gbar, 0, 256);
+        }
+        cudaGetLastError();
         return SD2_ERR_TIMEOUT;
     }
     return SD2_OK;
@@ -566,6 +778,22 @@ sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N
     uint16_t* u = (uint16_t*)(ws + off[5]);
     uint16_t* t = (uint16_t*)(ws + off[6]);
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    bool all_gap4 = true;
+    for (int i = 0; i < 7; ++i)
+        if (h[i]->format != SD2_FORMAT_GAP4) all_gap4 = false;
+    if (all_gap4) {
+        // one persistent launch: the stages of the block separated by grid barriers
+        int dev = 0;
+        st = ensure_device(&dev);
+        if (st != SD2_OK) return st;
+        for (int i = 0; i < 7; ++i)
+            if (h[i]->device != dev) return SD2_ERR_INVALID_ARG;
+        SArgs a;
+        std::memset(&a, 0, sizeof a);
+        ProgramNeeds needs;
+        a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, q, k, v, hdn, g, u, t, y, false, &needs);
+        return run_program(a, dev, N, needs, s);
+    }
     void* y_qkv[3] = {q, k, v};
     st = run_group(h + 0, 3, (const uint16_t*)x, nullptr, nullptr, nullptr, y_qkv, N, true, s);
     if (st != SD2_OK) return st;
@@ -577,6 +805,137 @@ sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N
     if (st != SD2_OK) return st;
     void* y_d[1] = {y};
     return run_group(h + 6, 1, nullptr, g, u, t, y_d, N, false, s);
+}
+
+// ---- whole drafter ---------------------------------------------------------------------
+
+sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2_drafter* out)
+{
+    if (!h || !out) return SD2_ERR_INVALID_ARG;
+    if (L < 1 || L > 4096 || n_max < 1 || n_max > 64) return SD2_ERR_SHAPE;
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    std::vector<BlockDims> dims((size_t)L);
+    for (int b = 0; b < L; ++b) {
+        st = block_dims(h + 7 * b, &dims[(size_t)b]);
+        if (st != SD2_OK) return st;
+        for (int i = 0; i < 7; ++i) {
+            if (h[7 * b + i]->format != SD2_FORMAT_GAP4) return SD2_ERR_UNSUPPORTED;
+            if (h[7 * b + i]->device != dev) return SD2_ERR_INVALID_ARG;
+        }
+        if (b > 0 && dims[(size_t)b].hidden != dims[(size_t)b - 1].out) return SD2_ERR_SHAPE;
+    }
+    sd2_drafter d = new (std::nothrow) sd2_drafter_s();
+    if (!d) return SD2_ERR_ALLOC;
+    d->L = L;
+    d->device = dev;
+    d->n_max = n_max;
+    d->hidden = dims[0].hidden;
+    d->out_dim = dims[(size_t)L - 1].out;
+    d->y_f32 = h[7 * (L - 1) + 6]->y_dtype == SD2_DTYPE_F32;
+    d->handles.assign(h, h + 7 * (size_t)L);
+    d->d_ws = nullptr;
+    d->d_stages = nullptr;
+    d->d_gbar = nullptr;
+    // workspace: per block q,k,v,hdn,g,u,t and the block's bf16 output (the next block's input)
+    d->ws_off.assign((size_t)L * 8 + 1, 0);
+    int64_t o = 0;
+    for (int b = 0; b < L; ++b) {
+        int64_t off[8];
+        block_layout(h + 7 * b, dims[(size_t)b], n_max, off);
+        for (int i = 0; i < 7; ++i) d->ws_off[(size_t)b * 8 + i] = o + off[i];
+        d->ws_off[(size_t)b * 8 + 7] = o + off[7];
+        o = a256(o + off[7] + 2 * n_max * dims[(size_t)b].out);
+    }
+    d->ws_off[(size_t)L * 8] = o;
+    std::vector<SStage> stages((size_t)L * 7);
+    ProgramNeeds needs;
+    bool ok = cudaMalloc((void**)&d->d_ws, (size_t)o) == cudaSuccess && cudaMemset(d->d_ws, 0, (size_t)o) == cudaSuccess;
+    int n = 0;
+    if (ok) {
+        for (int b = 0; b < L; ++b) {
+            uint8_t* base = d->d_ws;
+            const int64_t* wo = &d->ws_off[(size_t)b * 8];
+            const uint16_t* xin = b == 0 ? nullptr : (const uint16_t*)(base + d->ws_off[(size_t)(b - 1) * 8 + 7]);
+            void* yout = base + wo[7];
+            n += append_block_stages(stages.data() + n, h + 7 * b, xin, (uint16_t*)(base + wo[0]), (uint16_t*)(base + wo[1]),
+                                     (uint16_t*)(base + wo[2]), (uint16_t*)(base + wo[3]), (uint16_t*)(base + wo[4]),
+                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs);
+        }
+        d->n_stages = n;
+        ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
+             cudaMemcpy(d->d_stages, stages.data(), sizeof(SStage) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMalloc((void**)&d->d_gbar, 256) == cudaSuccess && cudaMemset(d->d_gbar, 0, 256) == cudaSuccess;
+    }
+    if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
+        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar);
+        delete d;
+        return SD2_ERR_UNSUPPORTED;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar);
+        cudaGetLastError();
+        delete d;
+        return SD2_ERR_ALLOC;
+    }
+    d->K_max = needs.K_max;
+    d->max_tile = needs.max_tile;
+    for (int w = 0; w < 3; ++w) d->xs_need[w] = needs.xs_need[w];
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_live_drafters.insert(d);
+    }
+    *out = d;
+    return SD2_OK;
+}
+
+sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, void* cuda_stream)
+{
+    if (!live(d) || !x || !y) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || N > d->n_max) return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    if (dev != d->device) return SD2_ERR_INVALID_ARG;
+    SArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.ext = d->d_stages;
+    a.n_stages = d->n_stages;
+    a.x_in = (const uint16_t*)x;
+    a.y_out = y;
+    a.gbar = d->d_gbar;
+    a.err = g_dev[dev].err_word;
+    a.wait_cycles = wait_budget(dev);
+    // Rows of X are independent through the whole drafter: panels run one after another.  Row n
+    // of every buffer starts at n * width, whatever N is.
+    return run_panels(a, N, d->xs_need, d->K_max, d->max_tile, g_dev[dev].sms, (cudaStream_t)cuda_stream);
+}
+
+sd2_status sd2_drafter_buffers(sd2_drafter d, int32_t block, void** ptrs)
+{
+    if (!live(d) || !ptrs) return SD2_ERR_INVALID_ARG;
+    if (block < 0 || block >= d->L) return SD2_ERR_SHAPE;
+    for (int i = 0; i < 8; ++i) ptrs[i] = d->d_ws + d->ws_off[(size_t)block * 8 + i];
+    return SD2_OK;
+}
+
+sd2_status sd2_drafter_free(sd2_drafter d)
+{
+    if (!d) return SD2_ERR_INVALID_ARG;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!g_live_drafters.erase(d)) return SD2_ERR_INVALID_ARG;
+    }
+    sd2_status st = SD2_OK;
+    if (cudaFree(d->d_ws) != cudaSuccess) st = SD2_ERR_CUDA;
+    if (cudaFree(d->d_stages) != cudaSuccess) st = SD2_ERR_CUDA;
+    if (cudaFree(d->d_gbar) != cudaSuccess) st = SD2_ERR_CUDA;
+    cudaGetLastError();
+    delete d;
+    return st;
 }
 
 }  // extern "C"

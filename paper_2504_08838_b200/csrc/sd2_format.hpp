@@ -5,39 +5,51 @@
 // non-contiguous parameters and storing the structure metadata (Introduction).  It gives
 // no format; the two below are this library's own.
 //
-// A blob is a header followed by three sections, each 256-byte aligned:
+// A blob is a 256-byte header followed by sections, each 256-byte aligned:
 //
 //   BITMASK  sec0  row_val_ptr  u32[M+1]      first value of each row, in values
 //            sec1  mask_words   u32[M*K32]    K32 = ceil(K/32); bit b of word w of row m is
 //                                             column 32w+b; bits at columns >= K are 0
 //            sec2  vals         u16[nnz]      kept bf16 patterns, row-major, ascending column
 //
-//   GAP4     sec0  row_chunk_ptr u32[M+1]     first chunk of each row, in chunks
-//            sec1  codes         u32[C]       eight 4-bit column gaps per chunk
-//            sec2  vals          u16[8*C]     eight bf16 patterns per chunk (16 bytes)
+//   GAP4     sec0  tile_off     u32[T+1]      start of each tile record in sec1, in 16-byte units
+//            sec1  tiles        T tile records (see below), each a multiple of 16 bytes
+//            (sec2 is empty)
 //
-// GAP4 in detail.  A row's kept entries, in ascending column order, become a list of
-// (column, value) entries.  A running cursor starts at column 0; an entry at column c is
-// coded as the gap g = c - cursor in [0, 15] and moves the cursor to c + 1.  When the next
-// kept column is more than 15 ahead, a filler entry (value +0) is placed at cursor + 15
-// first.  The list is then filled up to a multiple of 8 with gap-0 fillers (value +0),
-// which may run up to 7 columns past K - 1: kernels give the activation vector 8 zero
-// columns of slack and the decoder drops columns >= K.  Fillers sit on masked-out columns
-// and carry +0, so decoding still yields W.*mask bit for bit; they are not counted in nnz,
-// and their bytes are part of "compressed bytes" but never called useful.
-// Eight consecutive entries form a chunk: 16 bytes of values + one 32-bit code word whose
-// nibble i (bits 4i..4i+3) is entry i's gap.
-// A row with c chunks is cut into n_sc = ceil(c / 160) tiles of near-equal size; a tile of
-// cs <= 160 chunks is shared by L <= 32 lanes, J = ceil(cs/32) <= 5 consecutive chunks per
-// lane (lane L-1 may have fewer), and stored step-major so that step j of all lanes is one
-// contiguous run: see Gap4Tile below.  One warp-wide prefix sum per tile turns the lanes'
-// gap totals into their starting columns.
+// GAP4 in detail.  The K columns are cut into S strips of B columns (S a power of two <= 32,
+// S * B >= K) and a *segment* is one row restricted to one strip.  A segment's kept entries,
+// in ascending column order, become a list of (gap, value) entries: a cursor starts at the
+// strip's first column; an entry at column c is coded as g = c - cursor in [0, 15] and moves
+// the cursor to c + 1.  When the next kept column is more than 15 ahead, a filler entry
+// (value +0) is placed at cursor + 15 first.  The list is then filled up to a multiple of 8
+// with gap-0 fillers (value +0), which may run up to 7 columns past the strip's end: kernels
+// give every strip 8 zero columns of slack and the decoder drops such columns.  Fillers sit
+// on masked-out columns and carry +0, so decoding still yields W.*mask bit for bit; they
+// are not counted in nnz, and their bytes are part of "compressed bytes" but never called
+// useful.  Eight consecutive entries form a chunk: 16 bytes of values + one 32-bit code word
+// whose nibble i (bits 4i..4i+3) is entry i's gap.
+//
+// Rows are ordered by chunk count (most first, ties by row index), so that rows of like
+// density share a tile.  A tile is R = 32 / S consecutive rows of that order: 32 segments,
+// one per lane of a warp; lane l holds strip l % S of the tile's row l / S.  Lanes step
+// through their chunks together; step j of the tile stores chunk j of every lane that has
+// more than j chunks, in lane order, so each step is one contiguous, fully used run.
+//
+//   tile record   u16 cnt[32]          chunks of each lane's segment
+//                 u32 n_chunks         sum of cnt
+//                 u32 row[R]           original row index of each tile row, 0xFFFFFFFF = none
+//                 (pad to 16 bytes)
+//                 u32 code[n_chunks]   step-major as described
+//                 (pad to 16 bytes)
+//                 u16 val[8*n_chunks]  same order, 16 bytes per chunk
 
 #pragma once
 
+#include <algorithm>
 #include <cstdint>
 #include <cstdlib>
 #include <cstring>
+#include <numeric>
 #include <vector>
 
 #if defined(__CUDACC__)
@@ -50,12 +62,13 @@ namespace sd2 {
 
 constexpr int kFormatBitmask = 1;
 constexpr int kFormatGap4 = 2;
-constexpr int kGap4Jmax = 5;                    // chunks per lane per tile, at most
-constexpr int kGap4TileMax = 32 * kGap4Jmax;    // chunks per tile, at most
-constexpr int kGap4Slack = 8;                   // zero columns kernels append to x
+constexpr int kGap4Slack = 8;          // zero columns kernels append to every strip
+constexpr int kGap4MaxStrip = 496;     // widest strip: at most 63 chunks per segment
+constexpr int kGap4MinStrip = 64;      // strips narrower than this pay too much padding
+constexpr int kGap4TileTarget = 2048;  // tiles a matrix should have, if its shape allows
 
 struct BlobHeader {
-    char magic[8];          // "SD2BLOB1"
+    char magic[8];          // "SD2BLOB2"
     uint32_t version;
     uint32_t format;
     uint32_t y_dtype;
@@ -65,39 +78,41 @@ struct BlobHeader {
     int64_t compressed_bytes;   // sum of section sizes: what a kernel reads for W
     uint64_t sec_off[4];
     uint64_t sec_bytes[4];
-    uint64_t n_chunks;          // GAP4: C; BITMASK: 0
+    uint64_t n_chunks;          // GAP4: chunks in all tiles; BITMASK: 0
     uint64_t checksum;          // FNV-1a over bytes [sizeof(BlobHeader), total_bytes)
-    uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16];
+    uint32_t strips;            // GAP4: S
+    uint32_t strip_cols;        // GAP4: B
+    uint32_t n_tiles;           // GAP4: T
+    uint32_t max_tile_bytes;    // GAP4: largest tile record
+    uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16 - 16];
 };
 static_assert(sizeof(BlobHeader) == 256, "header is 256 bytes");
 
-// Geometry of one tile of a GAP4 row (shared by the encoder, the decoder and the kernels).
-struct Gap4Tile {
-    int cs;        // chunks in the tile
-    int J;         // chunks per lane (lanes 0..L-2)
-    int L;         // lanes that hold chunks
-    int cnt_last;  // chunks of lane L-1 (1..J)
-    // memory slot, relative to the tile's first chunk, of chunk j of lane l
-    SD2_HD int slot(int l, int j) const { return j * (L - 1) + (j < cnt_last ? j : cnt_last) + l; }
-    SD2_HD int count(int l) const { return l < L - 1 ? J : (l == L - 1 ? cnt_last : 0); }
+// Strip geometry of a GAP4 matrix.
+struct Gap4Geom {
+    int S;   // strips per row
+    int B;   // columns per strip
+    int R;   // rows per tile
 };
 
-SD2_HD Gap4Tile gap4_tile(int cs)
-{
-    Gap4Tile t;
-    t.cs = cs;
-    t.J = (cs + 31) >> 5;
-    t.L = (cs + t.J - 1) / t.J;
-    t.cnt_last = cs - (t.L - 1) * t.J;
-    return t;
-}
+// Header bytes of a tile record with R rows.
+SD2_HD int gap4_tile_header_bytes(int R) { return (64 + 4 + 4 * R + 15) & ~15; }
 
-// Tiles of a row with c > 0 chunks: n_sc tiles, the first `rem` of size q + 1, the rest q.
-SD2_HD void gap4_row_tiles(int c, int& n_sc, int& q, int& rem)
+// Picks S: enough tiles to spread over every SM's warps, strips neither too narrow (padding)
+// nor wider than the chunk counters allow.  B is odd so that strips start in distinct
+// shared-memory banks when a kernel transposes the activations.  S == 0: K is too large.
+inline Gap4Geom gap4_geometry(int64_t M, int64_t K)
 {
-    n_sc = (c + kGap4TileMax - 1) / kGap4TileMax;
-    q = c / n_sc;
-    rem = c - q * n_sc;
+    int S = 1;
+    while (S < 32 && M * S / 32 < kGap4TileTarget) S <<= 1;
+    while (S > 1 && (K + S - 1) / S < kGap4MinStrip) S >>= 1;
+    while (S < 32 && ((K + S - 1) / S | 1) > kGap4MaxStrip) S <<= 1;
+    Gap4Geom g;
+    g.S = S;
+    g.B = (int)((K + S - 1) / S) | 1;
+    g.R = 32 / S;
+    if (g.B > kGap4MaxStrip) g.S = 0;
+    return g;
 }
 
 inline uint64_t fnv1a(const uint8_t* p, size_t n)
@@ -115,6 +130,7 @@ inline uint64_t fnv1a(const uint8_t* p, size_t n)
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
 
 inline bool is_kept(const uint16_t* W, const uint8_t* mask, int64_t idx)
 {
@@ -124,15 +140,15 @@ inline bool is_kept(const uint16_t* W, const uint8_t* mask, int64_t idx)
 struct PackResult {
     uint8_t* blob = nullptr;
     int64_t bytes = 0;
-    int status = 0;  // 0 ok, -2 shape, -3 alloc
+    int status = 0;  // 0 ok, -2 shape, -3 alloc, -5 unsupported
 };
 
 inline void fill_header(BlobHeader& h, int format, int y_dtype, int64_t M, int64_t K, int64_t nnz,
                         const size_t sec_bytes[3], uint64_t n_chunks)
 {
     std::memset(&h, 0, sizeof h);
-    std::memcpy(h.magic, "SD2BLOB1", 8);
-    h.version = 1;
+    std::memcpy(h.magic, "SD2BLOB2", 8);
+    h.version = 2;
     h.format = (uint32_t)format;
     h.y_dtype = (uint32_t)y_dtype;
     h.n_sections = 3;
@@ -234,89 +250,136 @@ inline int unpack_bitmask(const BlobHeader& h, const uint8_t* blob, uint16_t* de
 
 // ---------------------------------------------------------------- GAP4
 
-// Entries (kept + fillers) a row needs, before rounding up to a multiple of 8.
-inline int64_t gap4_row_entries(const uint16_t* W, const uint8_t* mask, int64_t m, int64_t K, int64_t* kept_out)
+// Entries (kept + far-gap fillers) of the segment [c0, c1) of row m, before rounding up to 8.
+inline int gap4_segment_entries(const uint16_t* W, const uint8_t* mask, int64_t m, int64_t K, int64_t c0, int64_t c1,
+                                int64_t* kept_out)
 {
-    int64_t cursor = 0, e = 0, kept = 0;
-    for (int64_t k = 0; k < K; ++k) {
+    int64_t cursor = c0, e = 0, kept = 0;
+    for (int64_t k = c0; k < c1; ++k) {
         if (!is_kept(W, mask, m * K + k)) continue;
-        int64_t gap = k - cursor;
-        e += gap / 16 + 1;  // one filler per full 16 columns skipped, then the entry
+        e += (k - cursor) / 16 + 1;  // one filler per full 16 columns skipped, then the entry
         cursor = k + 1;
         ++kept;
     }
-    *kept_out = kept;
-    return e;
+    *kept_out += kept;
+    return (int)e;
 }
 
 inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype)
 {
     PackResult r;
-    std::vector<uint32_t> rcp((size_t)M + 1, 0);
-    std::vector<int64_t> chunks((size_t)M, 0), kept((size_t)M, 0);
+    const Gap4Geom g = gap4_geometry(M, K);
+    if (g.S == 0) { r.status = -5; return r; }
+    const int S = g.S, B = g.B, R = g.R;
+    // chunks of every segment, kept entries of every row
+    std::vector<uint16_t> seg_chunks((size_t)M * S);
+    std::vector<int64_t> row_chunks((size_t)M, 0), row_kept((size_t)M, 0);
 #pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m) {
-        int64_t kc;
-        int64_t e = gap4_row_entries(W, mask, m, K, &kc);
-        chunks[(size_t)m] = (e + 7) / 8;
-        kept[(size_t)m] = kc;
+        int64_t tot = 0;
+        for (int s = 0; s < S; ++s) {
+            const int64_t c0 = std::min<int64_t>(K, (int64_t)s * B), c1 = std::min<int64_t>(K, c0 + B);
+            const int e = gap4_segment_entries(W, mask, m, K, c0, c1, &row_kept[(size_t)m]);
+            const int c = (e + 7) / 8;
+            seg_chunks[(size_t)m * S + s] = (uint16_t)c;
+            tot += c;
+        }
+        row_chunks[(size_t)m] = tot;
     }
-    int64_t C = 0, nnz = 0;
-    for (int64_t m = 0; m < M; ++m) {
-        rcp[(size_t)m] = (uint32_t)C;
-        C += chunks[(size_t)m];
-        nnz += kept[(size_t)m];
-        if (C > 0x0FFFFFFFll) { r.status = -2; return r; }
+    // rows by chunk count, most first, ties by index
+    std::vector<uint32_t> order((size_t)M);
+    std::iota(order.begin(), order.end(), 0u);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](uint32_t a, uint32_t b) { return row_chunks[a] > row_chunks[b]; });
+    const int64_t T = (M + R - 1) / R;
+    const int hdr = gap4_tile_header_bytes(R);
+    std::vector<uint32_t> toff((size_t)T + 1, 0);
+    int64_t C = 0, nnz = 0, units = 0;
+    uint32_t max_tile = 0;
+    for (int64_t m = 0; m < M; ++m) nnz += row_kept[(size_t)m];
+    for (int64_t t = 0; t < T; ++t) {
+        int64_t ct = 0;
+        for (int rr = 0; rr < R; ++rr) {
+            const int64_t i = t * R + rr;
+            if (i < M) ct += row_chunks[order[(size_t)i]];
+        }
+        const size_t bytes = (size_t)hdr + align16((size_t)ct * 4) + (size_t)ct * 16;
+        toff[(size_t)t] = (uint32_t)units;
+        units += (int64_t)(bytes / 16);
+        C += ct;
+        if (bytes > max_tile) max_tile = (uint32_t)bytes;
+        if (units > 0xFFFFFFF0ll) { r.status = -2; return r; }
     }
-    rcp[(size_t)M] = (uint32_t)C;
-    size_t sec[3] = {(size_t)(M + 1) * 4, (size_t)C * 4, (size_t)C * 16};
+    toff[(size_t)T] = (uint32_t)units;
+    size_t sec[3] = {(size_t)(T + 1) * 4, (size_t)units * 16, 0};
     BlobHeader h;
     fill_header(h, kFormatGap4, y_dtype, M, K, nnz, sec, (uint64_t)C);
+    h.strips = (uint32_t)S;
+    h.strip_cols = (uint32_t)B;
+    h.n_tiles = (uint32_t)T;
+    h.max_tile_bytes = max_tile;
     uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
     if (!blob) { r.status = -3; return r; }
-    std::memcpy(blob + h.sec_off[0], rcp.data(), sec[0]);
-    uint32_t* codes = (uint32_t*)(blob + h.sec_off[1]);
-    uint16_t* vals = (uint16_t*)(blob + h.sec_off[2]);
-#pragma omp parallel for schedule(dynamic, 16)
-    for (int64_t m = 0; m < M; ++m) {
-        const int c = (int)chunks[(size_t)m];
-        if (c == 0) continue;
-        // logical entry list of the row
-        std::vector<uint16_t> ev((size_t)c * 8, 0);
-        std::vector<uint8_t> eg((size_t)c * 8, 0);
-        int64_t cursor = 0, e = 0;
-        for (int64_t k = 0; k < K; ++k) {
-            if (!is_kept(W, mask, m * K + k)) continue;
-            while (k - cursor > 15) {  // filler 15 columns ahead
-                eg[(size_t)e] = 15;
-                ev[(size_t)e] = 0;
-                ++e;
-                cursor += 16;
-            }
-            eg[(size_t)e] = (uint8_t)(k - cursor);
-            ev[(size_t)e] = W[m * K + k];
-            ++e;
-            cursor = k + 1;
-        }
-        // (entries e .. 8c-1 stay gap 0 / value +0)
-        int n_sc, q, rem;
-        gap4_row_tiles(c, n_sc, q, rem);
-        int64_t tile0 = rcp[(size_t)m];
-        int t_logical = 0;
-        for (int s = 0; s < n_sc; ++s) {
-            const Gap4Tile t = gap4_tile(q + (s < rem ? 1 : 0));
-            for (int l = 0; l < t.L; ++l) {
-                for (int j = 0; j < t.count(l); ++j, ++t_logical) {
-                    const int64_t slot = tile0 + t.slot(l, j);
-                    uint32_t code = 0;
-                    for (int i = 0; i < 8; ++i) {
-                        code |= (uint32_t)eg[(size_t)t_logical * 8 + i] << (4 * i);
-                        vals[slot * 8 + i] = ev[(size_t)t_logical * 8 + i];
-                    }
-                    codes[slot] = code;
+    std::memcpy(blob + h.sec_off[0], toff.data(), sec[0]);
+    uint8_t* tiles = blob + h.sec_off[1];
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t t = 0; t < T; ++t) {
+        uint8_t* rec = tiles + (size_t)toff[(size_t)t] * 16;
+        uint16_t* cnt = (uint16_t*)rec;
+        uint32_t* nch = (uint32_t*)(rec + 64);
+        uint32_t* rows = (uint32_t*)(rec + 68);
+        // logical entry lists of the 32 segments
+        std::vector<uint8_t> eg[32];
+        std::vector<uint16_t> ev[32];
+        uint32_t ct = 0;
+        int maxc = 0;
+        for (int l = 0; l < 32; ++l) {
+            const int rr = l / S, s = l % S;
+            const int64_t i = t * R + rr;
+            if (s == 0) rows[rr] = i < M ? order[(size_t)i] : 0xFFFFFFFFu;
+            cnt[l] = 0;
+            if (i >= M) continue;
+            const int64_t m = order[(size_t)i];
+            const int c = seg_chunks[(size_t)m * S + s];
+            cnt[l] = (uint16_t)c;
+            ct += (uint32_t)c;
+            if (c > maxc) maxc = c;
+            if (c == 0) continue;
+            eg[l].assign((size_t)c * 8, 0);
+            ev[l].assign((size_t)c * 8, 0);
+            const int64_t c0 = std::min<int64_t>(K, (int64_t)s * B), c1 = std::min<int64_t>(K, c0 + B);
+            int64_t cursor = c0;
+            size_t e = 0;
+            for (int64_t k = c0; k < c1; ++k) {
+                if (!is_kept(W, mask, m * K + k)) continue;
+                while (k - cursor > 15) {  // filler 15 columns ahead
+                    eg[l][e] = 15;
+                    ev[l][e] = 0;
+                    ++e;
+                    cursor += 16;
                 }
+                eg[l][e] = (uint8_t)(k - cursor);
+                ev[l][e] = W[m * K + k];
+                ++e;
+                cursor = k + 1;
             }
-            tile0 += t.cs;
+            // entries e .. 8c-1 stay gap 0 / value +0
+        }
+        *nch = ct;
+        uint32_t* codes = (uint32_t*)(rec + hdr);
+        uint16_t* vals = (uint16_t*)(rec + hdr + align16((size_t)ct * 4));
+        size_t slot = 0;
+        for (int j = 0; j < maxc; ++j) {
+            for (int l = 0; l < 32; ++l) {
+                if (cnt[l] <= j) continue;
+                uint32_t code = 0;
+                for (int i = 0; i < 8; ++i) {
+                    code |= (uint32_t)eg[l][(size_t)j * 8 + i] << (4 * i);
+                    vals[slot * 8 + i] = ev[l][(size_t)j * 8 + i];
+                }
+                codes[slot] = code;
+                ++slot;
+            }
         }
     }
     h.checksum = fnv1a(blob + sizeof h, (size_t)h.total_bytes - sizeof h);
@@ -326,50 +389,92 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     return r;
 }
 
+// Validates every tile record (so that a kernel can trust it) and, if `dense` is given, decodes.
 inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense)
 {
     const int64_t M = h.M, K = h.K;
-    const int64_t C = (int64_t)h.n_chunks;
-    if (h.sec_bytes[0] != (uint64_t)(M + 1) * 4 || h.sec_bytes[1] != (uint64_t)C * 4 ||
-        h.sec_bytes[2] != (uint64_t)C * 16)
-        return -6;
-    const uint32_t* rcp = (const uint32_t*)(blob + h.sec_off[0]);
-    const uint32_t* codes = (const uint32_t*)(blob + h.sec_off[1]);
-    const uint16_t* vals = (const uint16_t*)(blob + h.sec_off[2]);
-    if (rcp[0] != 0 || rcp[M] != (uint64_t)C) return -6;
-    for (int64_t m = 0; m < M; ++m)
-        if (rcp[m + 1] < rcp[m]) return -6;
+    const Gap4Geom g = gap4_geometry(M, K);
+    if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B) return -6;
+    const int S = g.S, B = g.B, R = g.R;
+    const int64_t T = (M + R - 1) / R;
+    if (h.n_tiles != (uint64_t)T || h.sec_bytes[0] != (uint64_t)(T + 1) * 4 || h.sec_bytes[2] != 0) return -6;
+    if (h.sec_bytes[1] % 16) return -6;
+    const uint32_t* toff = (const uint32_t*)(blob + h.sec_off[0]);
+    const uint8_t* tiles = blob + h.sec_off[1];
+    const uint64_t units = h.sec_bytes[1] / 16;
+    const int hdr = gap4_tile_header_bytes(R);
+    if (toff[0] != 0 || toff[T] != units) return -6;
+    for (int64_t t = 0; t < T; ++t)
+        if (toff[t + 1] <= toff[t]) return -6;
+    std::vector<uint8_t> seen((size_t)M, 0);
     int bad = 0;
-#pragma omp parallel for schedule(dynamic, 16) reduction(| : bad)
-    for (int64_t m = 0; m < M; ++m) {
-        if (dense) std::memset(dense + m * K, 0, (size_t)K * 2);
-        const int c = (int)(rcp[m + 1] - rcp[m]);
-        if (c == 0) continue;
-        int n_sc, q, rem;
-        gap4_row_tiles(c, n_sc, q, rem);
-        int64_t tile0 = rcp[m];
-        int64_t cursor = 0;
-        for (int s = 0; s < n_sc; ++s) {
-            const Gap4Tile t = gap4_tile(q + (s < rem ? 1 : 0));
-            for (int l = 0; l < t.L; ++l) {
-                for (int j = 0; j < t.count(l); ++j) {
-                    const int64_t slot = tile0 + t.slot(l, j);
-                    const uint32_t code = codes[slot];
-                    for (int i = 0; i < 8; ++i) {
-                        const int64_t col = cursor + ((code >> (4 * i)) & 15);
-                        cursor = col + 1;
-                        const uint16_t v = vals[slot * 8 + i];
-                        if (col < K) {
-                            if (dense) dense[m * K + col] = v;
-                        } else if (v != 0 || col >= K + kGap4Slack) {
-                            bad |= 1;  // only +0 fillers may pass the row end, and only by < 8
-                        }
-                    }
-                }
+    int64_t chunks = 0;
+    for (int64_t t = 0; t < T; ++t) {  // row ids: a permutation of 0..M-1, checked serially
+        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 68);
+        if ((uint64_t)(toff[t + 1] - toff[t]) * 16 < (uint64_t)hdr) return -6;
+        for (int rr = 0; rr < R; ++rr) {
+            const int64_t i = t * R + rr;
+            if (i < M) {
+                if (rows[rr] >= (uint64_t)M || seen[rows[rr]]) return -6;
+                seen[rows[rr]] = 1;
+            } else if (rows[rr] != 0xFFFFFFFFu) {
+                return -6;
             }
-            tile0 += t.cs;
         }
     }
+    if (dense) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < M; ++m) std::memset(dense + m * K, 0, (size_t)K * 2);
+    }
+#pragma omp parallel for schedule(dynamic, 8) reduction(| : bad) reduction(+ : chunks)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint8_t* rec = tiles + (size_t)toff[t] * 16;
+        const size_t rec_bytes = (size_t)(toff[t + 1] - toff[t]) * 16;
+        const uint16_t* cnt = (const uint16_t*)rec;
+        const uint32_t ct = *(const uint32_t*)(rec + 64);
+        const uint32_t* rows = (const uint32_t*)(rec + 68);
+        uint32_t sum = 0;
+        int maxc = 0;
+        for (int l = 0; l < 32; ++l) {
+            if (cnt[l] > (B + kGap4Slack) / 8 + 1) bad |= 1;
+            if (rows[l / S] == 0xFFFFFFFFu && cnt[l] != 0) bad |= 1;
+            sum += cnt[l];
+            if (cnt[l] > maxc) maxc = cnt[l];
+        }
+        if (sum != ct || rec_bytes != (size_t)hdr + align16((size_t)ct * 4) + (size_t)ct * 16 ||
+            rec_bytes > h.max_tile_bytes) {
+            bad |= 1;
+            continue;
+        }
+        if (bad) continue;
+        chunks += ct;
+        const uint32_t* codes = (const uint32_t*)(rec + hdr);
+        const uint16_t* vals = (const uint16_t*)(rec + hdr + align16((size_t)ct * 4));
+        int64_t cursor[32];
+        for (int l = 0; l < 32; ++l) cursor[l] = (int64_t)(l % S) * B;
+        size_t slot = 0;
+        for (int j = 0; j < maxc; ++j) {
+            for (int l = 0; l < 32; ++l) {
+                if (cnt[l] <= j) continue;
+                const int s = l % S;
+                const int64_t m = rows[l / S];
+                const int64_t c1 = std::min<int64_t>(K, (int64_t)(s + 1) * B);  // end of the strip's real columns
+                const uint32_t code = codes[slot];
+                for (int i = 0; i < 8; ++i) {
+                    const int64_t col = cursor[l] + ((code >> (4 * i)) & 15);
+                    cursor[l] = col + 1;
+                    const uint16_t v = vals[slot * 8 + i];
+                    if (col < c1) {
+                        if (dense && v != 0) dense[m * K + col] = v;
+                    } else if (v != 0 || col >= (int64_t)s * B + B + kGap4Slack) {
+                        bad |= 1;  // only +0 fillers may pass the strip's end, and only by < 8 columns
+                    }
+                }
+                ++slot;
+            }
+        }
+    }
+    if (chunks != (int64_t)h.n_chunks) bad |= 1;
     return bad ? -6 : 0;
 }
 
@@ -378,7 +483,7 @@ inline int check_header(const uint8_t* blob, int64_t bytes, BlobHeader& h, bool 
 {
     if (bytes < (int64_t)sizeof(BlobHeader)) return -6;
     std::memcpy(&h, blob, sizeof h);
-    if (std::memcmp(h.magic, "SD2BLOB1", 8) != 0 || h.version != 1) return -6;
+    if (std::memcmp(h.magic, "SD2BLOB2", 8) != 0 || h.version != 2) return -6;
     if (h.format != (uint32_t)kFormatBitmask && h.format != (uint32_t)kFormatGap4) return -6;
     if (h.y_dtype > 1 || h.n_sections != 3) return -6;
     if (h.M < 1 || h.K < 1 || h.nnz < 0 || h.nnz > h.M * h.K) return -6;

@@ -2,15 +2,15 @@
 // Y[n, m] = sum over kept k of W[m, k] X[n, k]  (bf16 in, fp32 accumulate, one rounding).
 //
 // The work is a streaming scan of a compressed matrix, bound by HBM bandwidth at N = 1
-// and by instruction issue from N of about 8 upward; it is not a dense contraction, so
-// there are no tensor-core instructions here.  What matters instead:
-//   - every byte of the compressed weight is read exactly once, by fully coalesced
-//     128-bit (values) and 32-bit (codes) loads, step j of a tile being one contiguous run;
-//   - the activation panel is staged once per CTA in shared memory as fp32 [K+8][NT];
-//   - position decoding costs under one instruction per entry (byte-parallel prefix sums
-//     of eight 4-bit gaps), leaving about six instructions per kept weight at N = 1;
-//   - rows are reduced with warp shuffles; one row's sum order is fixed, so results are
-//     deterministic run to run.
+// and by instruction issue as N grows; it is not a dense contraction, so there are no
+// tensor-core instructions here.  What matters instead:
+//   - every byte of the compressed weight is read from HBM exactly once, by bulk
+//     asynchronous copies (cp.async.bulk, global -> shared) that a producer warp issues tile
+//     by tile into a ring and that run ahead of the arithmetic, across stage boundaries;
+//   - the activations are staged once per stage in shared memory in a layout in which the
+//     32 lanes of a warp always read 32 different banks, whatever columns they gather;
+//   - position decoding is byte-parallel (prefix sums of eight 4-bit gaps in two registers);
+//   - one row's sum order is fixed, so results are deterministic run to run.
 
 #pragma once
 
@@ -21,36 +21,7 @@
 
 namespace sd2 {
 
-constexpr int kWarpsPerCta = 8;
-constexpr int kThreads = kWarpsPerCta * 32;
 constexpr int kMaxFused = 4;
-
-// One weight as a kernel sees it.
-struct MatDesc {
-    const uint32_t* sec0;   // GAP4: row_chunk_ptr   BITMASK: row_val_ptr
-    const uint32_t* sec1;   // GAP4: codes           BITMASK: mask words
-    const void* sec2;       // GAP4: uint4 values    BITMASK: u16 values
-    void* y;                // [N*M]
-    int M;
-    int y_f32;              // 1: fp32 output, 0: bf16
-    int cta_begin;          // first CTA of this weight in a fused launch
-    int cta_count;
-};
-
-struct LaunchGroup {
-    MatDesc mat[kMaxFused];
-    int count;
-    int K;
-    int N;                  // rows of X in this launch, 1..NT
-    // activation source: x (plain) or silu(g)*u rounded to bf16 (feed-forward glue)
-    const uint16_t* x;      // [N*K] bf16, or NULL in glue mode
-    const uint16_t* g;      // glue mode: gate output [N*K]
-    const uint16_t* u;      // glue mode: up output   [N*K]
-    uint16_t* t_out;        // glue mode: optional copy of t = bf16(silu(g)*u), written by CTA 0
-    int* err;               // device error word: set to 1 when a bounded wait ran out
-    int depth;              // GAP4: stages per warp ring
-    int x_bytes;            // GAP4: bytes of the staged activation panel (16-byte multiple)
-};
 
 __device__ __forceinline__ float bf16_lo(uint32_t r) { return __uint_as_float(r << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t r) { return __uint_as_float(r & 0xFFFF0000u); }
@@ -64,98 +35,11 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
     return (uint16_t)(b >> 16);
 }
 
-__device__ __forceinline__ uint4 ld_stream_v4(const uint4* p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ uint32_t ld_stream_u32(const uint32_t* p)
-{
-    uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ float silu_mul_bf16(uint16_t g, uint16_t u, uint16_t* t_bits)
+// t = bf16(silu(g) * u), silu in fp32
+__device__ __forceinline__ uint16_t silu_mul_bits(uint16_t g, uint16_t u)
 {
     const float a = bf16_to_f32(g);
-    const uint16_t t = f32_to_bf16_rne((a / (1.f + expf(-a))) * bf16_to_f32(u));
-    *t_bits = t;
-    return bf16_to_f32(t);
-}
-
-// Stage the activation panel as fp32 xs[(K + slack)][NT]; columns n >= N and rows k >= K are 0.
-// Source: x, or in glue mode t = bf16(silu(g) * u), which CTA 0 also writes to t_out.
-template <int NT>
-__device__ __forceinline__ void stage_x(const LaunchGroup& grp, float* xs, int slack)
-{
-    const int K = grp.K, N = grp.N;
-    const bool glue = grp.x == nullptr;
-    const bool pub = glue && grp.t_out && blockIdx.x == 0;
-    const bool vec = (K % 8 == 0) && (((uintptr_t)grp.x | (uintptr_t)grp.g | (uintptr_t)grp.u | (uintptr_t)grp.t_out) % 16 == 0);
-    if (vec) {
-        const int K8 = K >> 3;
-        for (int i = threadIdx.x; i < K8 * N; i += blockDim.x) {
-            const int n = i / K8, k8 = i - n * K8;
-            uint32_t w[4];
-            if (!glue) {
-                const uint4 v = __ldg((const uint4*)(grp.x + (size_t)n * K) + k8);
-                w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-            } else {
-                const uint4 gv = __ldg((const uint4*)(grp.g + (size_t)n * K) + k8);
-                const uint4 uv = __ldg((const uint4*)(grp.u + (size_t)n * K) + k8);
-                const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w}, uu[4] = {uv.x, uv.y, uv.z, uv.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint16_t lo, hi;
-                    silu_mul_bf16((uint16_t)(gg[q] & 0xFFFFu), (uint16_t)(uu[q] & 0xFFFFu), &lo);
-                    silu_mul_bf16((uint16_t)(gg[q] >> 16), (uint16_t)(uu[q] >> 16), &hi);
-                    w[q] = (uint32_t)lo | ((uint32_t)hi << 16);
-                }
-                if (pub) ((uint4*)(grp.t_out + (size_t)n * K))[k8] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                xs[(size_t)(8 * k8 + 2 * q) * NT + n] = bf16_lo(w[q]);
-                xs[(size_t)(8 * k8 + 2 * q + 1) * NT + n] = bf16_hi(w[q]);
-            }
-        }
-    } else {
-        for (int i = threadIdx.x; i < K * N; i += blockDim.x) {
-            const int n = i / K, k = i - n * K;
-            float v;
-            if (!glue) {
-                v = bf16_to_f32(grp.x[(size_t)n * K + k]);
-            } else {
-                uint16_t t;
-                v = silu_mul_bf16(grp.g[(size_t)n * K + k], grp.u[(size_t)n * K + k], &t);
-                if (pub) grp.t_out[(size_t)n * K + k] = t;
-            }
-            xs[(size_t)k * NT + n] = v;
-        }
-    }
-    if (N < NT)
-        for (int i = threadIdx.x; i < K * (NT - N); i += blockDim.x) {
-            const int k = i / (NT - N), n = N + (i - k * (NT - N));
-            xs[(size_t)k * NT + n] = 0.f;
-        }
-    for (int i = threadIdx.x; i < slack * NT; i += blockDim.x) xs[(size_t)K * NT + i] = 0.f;
-}
-
-template <int NT>
-__device__ __forceinline__ void store_row(const MatDesc& md, int row, const float (&acc)[NT], int N)
-{
-#pragma unroll
-    for (int n = 0; n < NT; ++n) {
-        if (n < N) {
-            if (md.y_f32) ((float*)md.y)[(size_t)n * md.M + row] = acc[n];
-            else ((uint16_t*)md.y)[(size_t)n * md.M + row] = f32_to_bf16_rne(acc[n]);
-        }
-    }
+    return f32_to_bf16_rne((a / (1.f + expf(-a))) * bf16_to_f32(u));
 }
 
 __device__ __forceinline__ float warp_sum(float v)
@@ -165,53 +49,76 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// acc[n] += w * xs[col][n]
-template <int NT>
-__device__ __forceinline__ void fma_entry(float (&acc)[NT], float w, const char* xrow)
-{
-    if (NT == 1) {
-        acc[0] = fmaf(w, *(const float*)xrow, acc[0]);
-    } else if (NT == 2) {
-        const float2 x = *(const float2*)xrow;
-        acc[0] = fmaf(w, x.x, acc[0]);
-        acc[1] = fmaf(w, x.y, acc[1]);
-    } else {
-#pragma unroll
-        for (int q = 0; q < NT / 4; ++q) {
-            const float4 x = *(const float4*)(xrow + 16 * q);
-            acc[4 * q + 0] = fmaf(w, x.x, acc[4 * q + 0]);
-            acc[4 * q + 1] = fmaf(w, x.y, acc[4 * q + 1]);
-            acc[4 * q + 2] = fmaf(w, x.z, acc[4 * q + 2]);
-            acc[4 * q + 3] = fmaf(w, x.w, acc[4 * q + 3]);
-        }
-    }
-}
-
 // ------------------------------------------------------------------------------ GAP4
 //
-// Rows are dealt round-robin to the launch's warps; a warp owns whole rows, so a row's sum
-// is formed in one fixed order by one warp (deterministic, no atomics, no fix-up pass).
+// One persistent CTA per SM runs a *program* of stages.  A stage is one launch's worth of
+// work: up to four weights that read the same activations (q|k|v, gate|up, or one weight).
+// Consecutive stages depend on each other (the next one reads what this one wrote), so they
+// are separated by a grid-wide barrier; the weights, however, never depend on anything, and
+// the producer warp keeps copying the tiles of coming stages into the ring while the
+// consumer warps are still computing, waiting at the barrier or staging activations.
 //
-// Weight streaming.  Every warp runs a private ring of `depth` stages in shared memory.  A
-// stage holds one tile (<= 160 chunks: 2560 B of values + its code words) and is filled by
-// two bulk asynchronous copies (cp.async.bulk, global -> shared) that complete on the
-// stage's mbarrier.  Lane 0 walks the warp's rows ahead of the computation and keeps the
-// ring full, so about depth * 3 KB per warp are in flight whatever the registers hold; the
-// first `depth` tiles are requested before the kernel waits for the previous kernel on the
-// stream (programmatic dependent launch), because weights never depend on it.
-// There is no cross-warp synchronisation after the activation panel is staged.  Every wait
-// on an mbarrier is bounded: on a time-out the warp raises the error word and returns.
+// Tiles of a stage are dealt round-robin to the CTAs (tile v of the stage goes to CTA
+// v % gridDim.x) and, inside a CTA, round-robin to the consumer warps.  A warp owns whole
+// tiles, so a row's sum is formed in one fixed order (deterministic, no atomics).
 //
-// Per tile, lane l owns J consecutive chunks.  Per chunk: E = even nibbles, O = odd nibbles
-// as bytes; S = E + O; P = S * 0x01010100 is the exclusive prefix of the pair sums;
-// PE = P + E and PO = PE + O are the inclusive gap prefixes of the even and odd entries;
-// entry i sits at column base + prefix_i + i.  One warp prefix sum per tile gives `base`.
+// Per tile, lane l owns one segment (strip l % S of tile row l / S) and walks its chunks;
+// per chunk: E = even nibbles, O = odd nibbles as bytes; P = (E + O) * 0x01010100 is the
+// exclusive prefix of the pair sums; PE = P + E and PO = PE + O are the inclusive gap
+// prefixes of the even and odd entries; entry i sits at local column cursor + prefix_i + i.
+// The activations live in shared memory as xs[column][32 / NT groups][NT]: lane l reads
+// group l % (32 / NT), so one warp-wide gather touches every bank once.
+//
+// Every wait (ring barriers, grid barrier) is bounded by a cycle budget: when it runs out
+// the CTA raises the error word and winds down instead of hanging.
 
-constexpr int kStageValBytes = kGap4TileMax * 16;                 // 2560
-constexpr int kStageCodeSlots = kGap4TileMax + 8;                 // tile + alignment slop
-constexpr int kStageBytes = kStageValBytes + kStageCodeSlots * 4; // 3232, a multiple of 16
-constexpr int kMaxDepth = 8;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kConsumerWarps = 16;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
+constexpr int kSlots = 32;                               // tiles in flight per CTA, at most
+constexpr int kMaxStagesInline = 8;
+
+struct SMat {
+    const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
+    const unsigned char* stream;   // tile records
+    void* y;                       // [N * M]
+    int M;
+    int T;
+    int y_f32;                     // 1: fp32 output, 0: bf16
+    int reserved;
+};
+
+struct SStage {
+    SMat mat[kMaxFused];
+    const uint16_t* x;     // [N * K] bf16, or NULL in glue mode
+    const uint16_t* g;     // glue mode: t = bf16(silu(g) * u) is the activation
+    const uint16_t* u;
+    uint16_t* t_out;       // glue mode: CTA 0 also writes t here (may be NULL)
+    int count;             // weights in the stage
+    int K;
+    int S;                 // strips; equal for all weights of a stage
+    int B;                 // strip width
+    int T_total;           // tiles of all weights
+    int hdr_bytes;         // tile header bytes (depends on S)
+    int reserved[2];
+};
+static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
+
+struct SArgs {
+    SStage inl[kMaxStagesInline];   // used when ext == NULL
+    const SStage* ext;              // device array of stages (programs longer than four stages)
+    const uint16_t* x_in;           // replaces stage 0's x when not NULL
+    void* y_out;                    // replaces the last stage's mat[0].y when not NULL
+    unsigned int* gbar;             // grid barrier: [0] arrivals, [32] exits (two cache lines)
+    int* err;                       // device error word
+    long long wait_cycles;          // budget of every bounded wait
+    int n_stages;
+    int N;                          // activation rows of this launch, 1..NT
+    int n0;                         // first activation row: every X / Y pointer is advanced by n0 rows
+    int xs_bytes;                   // shared memory for the transposed activations
+    int xlin_bytes;                 // shared memory for one linear activation row
+    int ring_bytes;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -251,228 +158,463 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  : "memory");
 }
 
-// x / J for J in 1..5 and x <= 200 (exact; checked on the host in the format tests)
-__device__ __forceinline__ int div_small(int x, int J)
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a)
 {
-    const uint32_t magic = J == 1 ? 65536u : J == 2 ? 32768u : J == 3 ? 21846u : J == 4 ? 16384u : 13108u;
-    return (int)(((uint32_t)x * magic) >> 16);
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ float lds_f32_off(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(a), "n"(OFF));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ float2 lds_f32x2_off(uint32_t a)
+{
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(a), "n"(OFF));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ float4 lds_f32x4_off(uint32_t a)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a), "n"(OFF));
+    return v;
 }
 
-// Walks a warp's rows tile by tile (all lanes hold the same state).
-struct TileCursor {
-    int ri;      // ordinal of the current row among this warp's rows of the batch
-    int nrows;   // rows in the batch (<= 32)
-    int s, n_sc, q, rem, tile0;
+__device__ __forceinline__ void named_bar_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Shared-memory bookkeeping of one CTA (placed after xs and xlin).
+struct StreamShared {
+    int4 desc[kSlots];                 // x: ring offset, y: weight index, z: tile index, w: bytes
+    unsigned long long full[kSlots];   // mbarriers: tile landed
+    unsigned long long empty[kSlots];  // mbarriers: tile consumed
+    int abort_flag;                    // any warp: a bounded wait ran out
+    int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
+    int pad[2];
 };
 
+struct WaitCtx {
+    volatile int* abort_flag;
+    long long budget;
+};
+
+// Bounded wait on an mbarrier phase.  false: the budget ran out (or another warp gave up).
+__device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, const WaitCtx& w)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 15u) == 0u) {
+            if (*w.abort_flag) return false;
+            if (clock64() - t0 > w.budget) {
+                *w.abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`
+template <int NT, int OFF>
+__device__ __forceinline__ void fma_at(float (&acc)[NT], float w, uint32_t addr)
+{
+    if (NT == 1) {
+        acc[0] = fmaf(w, lds_f32_off<OFF>(addr), acc[0]);
+    } else if (NT == 2) {
+        const float2 x = lds_f32x2_off<OFF>(addr);
+        acc[0] = fmaf(w, x.x, acc[0]);
+        acc[1] = fmaf(w, x.y, acc[1]);
+    } else {
+        const float4 x = lds_f32x4_off<OFF>(addr);
+        acc[0] = fmaf(w, x.x, acc[0]);
+        acc[1] = fmaf(w, x.y, acc[1]);
+        acc[2] = fmaf(w, x.z, acc[2]);
+        acc[3] = fmaf(w, x.w, acc[3]);
+    }
+}
+
+// One chunk: eight (gap, value) entries against the activations at `xb` (the lane's cursor).
+// Returns the cursor after the chunk.  Two accumulator sets keep two FMA chains in flight.
 template <int NT>
-__global__ void __launch_bounds__(kThreads) gap4_kernel(const __grid_constant__ LaunchGroup grp)
+__device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uint32_t xb, float (&a0)[NT], float (&a1)[NT])
+{
+    const uint32_t E = code & 0x0F0F0F0Fu;
+    const uint32_t O = (code >> 4) & 0x0F0F0F0Fu;
+    const uint32_t PE = (E + O) * 0x01010100u + E;
+    const uint32_t PO = PE + O;
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#define SD2_PAIR(k)                                                              \
+    {                                                                            \
+        const uint32_t ae = xb + (__byte_perm(PE, 0, 0x4440 + (k)) << 7);        \
+        const uint32_t ao = xb + (__byte_perm(PO, 0, 0x4440 + (k)) << 7);        \
+        fma_at<NT, (2 * (k)) * 128>(a0, bf16_lo(w[k]), ae);                      \
+        fma_at<NT, (2 * (k) + 1) * 128>(a1, bf16_hi(w[k]), ao);                  \
+    }
+    SD2_PAIR(0)
+    SD2_PAIR(1)
+    SD2_PAIR(2)
+    SD2_PAIR(3)
+#undef SD2_PAIR
+    return xb + ((PO >> 24) << 7) + 1024u;
+}
+
+// Stage the activations of one stage: xs[plane][column c][group][NT] (fp32) with
+// value = X[n][strip * B + c] where strip = plane * groups + group % S (for S <= groups the
+// strips repeat across the groups), zero for c >= B, strip * B + c >= K or n >= N.
+// Row by row through `xlin` (bf16, linear) so that global memory is read with 128-bit loads.
+// x_src, g, u, t_out already point at the launch's first activation row.
+template <int NT>
+__device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
+                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int ctid)
+{
+    constexpr int kGroups = 32 / NT;
+    const int K = st.K, S = st.S, B = st.B;
+    const bool glue = x_src == nullptr;
+    const int planes = S > kGroups ? S / kGroups : 1;
+    const int rows = B + kGap4Slack;
+    const bool vec = (K % 8 == 0) && ((((uintptr_t)x_src | (uintptr_t)g | (uintptr_t)u | (uintptr_t)t_out) & 15) == 0);
+    const bool pub = glue && t_out && blockIdx.x == 0;
+    for (int n = 0; n < NT; ++n) {
+        if (n < N) {
+            if (vec) {
+                for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
+                    uint4 v;
+                    if (!glue) {
+                        v = __ldcg((const uint4*)(x_src + (size_t)n * K) + i);
+                    } else {
+                        const uint4 gv = __ldcg((const uint4*)(g + (size_t)n * K) + i);
+                        const uint4 uv = __ldcg((const uint4*)(u + (size_t)n * K) + i);
+                        const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w}, uu[4] = {uv.x, uv.y, uv.z, uv.w};
+                        uint32_t w[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const uint32_t lo = silu_mul_bits((uint16_t)(gg[q] & 0xFFFFu), (uint16_t)(uu[q] & 0xFFFFu));
+                            const uint32_t hi = silu_mul_bits((uint16_t)(gg[q] >> 16), (uint16_t)(uu[q] >> 16));
+                            w[q] = lo | (hi << 16);
+                        }
+                        v = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (pub) ((uint4*)(t_out + (size_t)n * K))[i] = v;
+                    }
+                    ((uint4*)xlin)[i] = v;
+                }
+            } else {
+                for (int i = ctid; i < K; i += kConsumerThreads) {
+                    uint16_t v;
+                    if (!glue) {
+                        v = __ldcg(x_src + (size_t)n * K + i);
+                    } else {
+                        v = silu_mul_bits(__ldcg(g + (size_t)n * K + i), __ldcg(u + (size_t)n * K + i));
+                        if (pub) t_out[(size_t)n * K + i] = v;
+                    }
+                    xlin[i] = v;
+                }
+            }
+        }
+        named_bar_sync(1, kConsumerThreads);
+        // scatter row n: consecutive threads take consecutive groups of one column
+        for (int p = 0; p < planes; ++p) {
+            float* xp = xs + (size_t)p * rows * 32;
+            for (int i = ctid; i < rows * kGroups; i += kConsumerThreads) {
+                const int grp = i % kGroups;
+                const int c = i / kGroups;
+                const int strip = S > kGroups ? p * kGroups + grp : grp % S;
+                const int col = strip * B + c;
+                float v = 0.f;
+                if (n < N && c < B && col < K) v = bf16_to_f32(xlin[col]);
+                xp[(size_t)i * NT + n] = v;
+            }
+        }
+        named_bar_sync(1, kConsumerThreads);
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_constant__ SArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    const int lane = threadIdx.x & 31;
-    const int wib = threadIdx.x >> 5;
-    const int depth = grp.depth;
     float* xs = (float*)smem;
-    unsigned char* ring = smem + grp.x_bytes + (size_t)wib * depth * kStageBytes;
-    int4* descq = (int4*)(smem + grp.x_bytes + (size_t)kWarpsPerCta * depth * kStageBytes) + wib * depth;
-    const uint32_t bars = smem_u32(smem + grp.x_bytes + (size_t)kWarpsPerCta * depth * (kStageBytes + 16)) + wib * depth * 8;
+    uint16_t* xlin = (uint16_t*)(smem + a.xs_bytes);
+    StreamShared* sh = (StreamShared*)(smem + a.xs_bytes + a.xlin_bytes);
+    unsigned char* ring = smem + a.xs_bytes + a.xlin_bytes + ((sizeof(StreamShared) + 127) & ~127);
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int cta = blockIdx.x;
+    const int G = gridDim.x;
+    const uint32_t full0 = smem_u32(&sh->full[0]);
+    const uint32_t empty0 = smem_u32(&sh->empty[0]);
+    const uint32_t ring0 = smem_u32(ring);
 
-    int mi = 0;
-#pragma unroll
-    for (int i = 1; i < kMaxFused; ++i)
-        if (i < grp.count && (int)blockIdx.x >= grp.mat[i].cta_begin) mi = i;
-    const MatDesc& md = grp.mat[mi];
-    const int gw = ((int)blockIdx.x - md.cta_begin) * kWarpsPerCta + wib;
-    const int GW = md.cta_count * kWarpsPerCta;
-    const uint32_t* __restrict__ rcp = md.sec0;
-    const uint32_t* __restrict__ codes = md.sec1;
-    const uint4* __restrict__ vals = (const uint4*)md.sec2;
-    constexpr int kRowBytes = 4 * NT;
-
-    if (lane == 0)
-        for (int i = 0; i < depth; ++i) mbar_init(bars + 8 * i, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    __syncwarp();
-
-    // let the next kernel on the stream start its own weight prefetch
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    int fetched = 0, consumed = 0;   // tile ordinals of this warp; stage = ordinal % depth
-    int f_stage = 0, c_stage = 0;
-    uint32_t c_parity = 0;
-    bool staged = false;
-    bool dead = false;
-
-    for (int row_base = gw; row_base < md.M && !dead; row_base += 32 * GW) {
-        // this lane's row of the batch
-        const int my_row = row_base + lane * GW;
-        int my_c0 = 0, my_c1 = 0;
-        if (my_row < md.M) {
-            my_c0 = (int)__ldg(rcp + my_row);
-            my_c1 = (int)__ldg(rcp + my_row + 1);
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, 1);
         }
-        TileCursor cu;
-        cu.ri = -1;
-        cu.nrows = min(32, (md.M - row_base + GW - 1) / GW);
-        cu.s = cu.n_sc = cu.q = cu.rem = cu.tile0 = 0;
-        bool more = true;
+        sh->abort_flag = 0;
+        sh->stage_dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
-        // Request the next tile of the batch into stage f_stage (uniform; lane 0 issues).
-        auto fetch_one = [&]() {
-            int row = 0, a = 0, cs = 0, flags = 0;
-            while (true) {
-                if (cu.s < cu.n_sc) {
-                    cs = cu.q + (cu.s < cu.rem ? 1 : 0);
-                    a = cu.tile0;
-                    cu.tile0 += cs;
-                    flags = (cu.s == 0 ? 1 : 0) | (cu.s == cu.n_sc - 1 ? 2 : 0);
-                    ++cu.s;
-                    row = row_base + cu.ri * GW;
-                    break;
-                }
-                ++cu.ri;
-                if (cu.ri >= cu.nrows) { more = false; return; }
-                const int c0 = __shfl_sync(0xFFFFFFFFu, my_c0, cu.ri);
-                const int c = __shfl_sync(0xFFFFFFFFu, my_c1, cu.ri) - c0;
-                cu.tile0 = c0;
-                cu.s = 0;
-                if (c == 0) {  // empty row: a descriptor without data, so that its +0 is stored in order
-                    cu.n_sc = 0;
-                    row = row_base + cu.ri * GW;
-                    cs = 0;
-                    flags = 3;
-                    break;
-                }
-                if (c <= kGap4TileMax) { cu.n_sc = 1; cu.q = c; cu.rem = 0; }
-                else gap4_row_tiles(c, cu.n_sc, cu.q, cu.rem);
-            }
-            if (lane == 0) {
-                const uint32_t bar = bars + 8 * f_stage;
-                descq[f_stage] = make_int4(a, cs, row, flags);
-                if (cs > 0) {
-                    const int a4 = a & ~3;
-                    const uint32_t vbytes = (uint32_t)cs * 16u;
-                    const uint32_t cbytes = (uint32_t)(((a + cs + 3) & ~3) - a4) * 4u;
-                    unsigned char* st = ring + (size_t)f_stage * kStageBytes;
-                    mbar_expect_tx(bar, vbytes + cbytes);
-                    bulk_g2s(smem_u32(st), vals + a, vbytes, bar);
-                    bulk_g2s(smem_u32(st + kStageValBytes), codes + a4, cbytes, bar);
-                } else {
-                    mbar_arrive(bar);
-                }
-            }
-            ++fetched;
-            if (++f_stage == depth) f_stage = 0;
-            __syncwarp();   // the descriptor is visible to every lane
-        };
+    WaitCtx wc;
+    wc.abort_flag = &sh->abort_flag;
+    wc.budget = a.wait_cycles;
 
-        while (more && fetched - consumed < depth) fetch_one();
-
-        if (!staged) {
-            // weights above never depend on the previous kernel; the activations below do
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            stage_x<NT>(grp, xs, kGap4Slack);
-            __syncthreads();
-            staged = true;
-        }
-
-        float acc[NT];
-#pragma unroll
-        for (int n = 0; n < NT; ++n) acc[n] = 0.f;
-        float acc_b = 0.f;  // second chain at NT == 1 for instruction-level parallelism
-        int cursor = 0;     // column cursor at the start of the tile (warp-uniform)
-
-        while (consumed < fetched) {
-            const uint32_t bar = bars + 8 * c_stage;
-            uint32_t spins = 0;
-            while (!mbar_try_wait(bar, c_parity)) {
-                if (++spins > kSpinLimit) { dead = true; break; }
-            }
-            dead = __any_sync(0xFFFFFFFFu, dead);
-            if (dead) break;
-            const int4 d = descq[c_stage];
-            const int a = d.x, cs = d.y, row = d.z, flags = d.w;
-            const unsigned char* st = ring + (size_t)c_stage * kStageBytes;
-            if (flags & 1) {
-#pragma unroll
-                for (int n = 0; n < NT; ++n) acc[n] = 0.f;
-                acc_b = 0.f;
-                cursor = 0;
-            }
-            if (cs > 0) {
-                const uint4* sv = (const uint4*)st;
-                const uint32_t* sc = (const uint32_t*)(st + kStageValBytes) + (a & 3);
-                Gap4Tile t;
-                t.cs = cs;
-                t.J = (cs + 31) >> 5;
-                t.L = div_small(cs + t.J - 1, t.J);
-                t.cnt_last = cs - (t.L - 1) * t.J;
-                const int my_cnt = t.count(lane);
-                uint32_t code[kGap4Jmax];
-                int tot = 0;
-#pragma unroll
-                for (int j = 0; j < kGap4Jmax; ++j) {
-                    code[j] = 0;
-                    if (j < my_cnt) {
-                        code[j] = sc[t.slot(lane, j)];
-                        const uint32_t S = (code[j] & 0x0F0F0F0Fu) + ((code[j] >> 4) & 0x0F0F0F0Fu);
-                        tot += (int)((S * 0x01010101u) >> 24) + 8;
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer warp
+        uint32_t q = 0, oldest = 0;         // tile sequence numbers of this CTA
+        uint32_t head = 0, tail = 0;        // ring bytes: [tail, head) is in use (mod wrap)
+        const uint32_t ring_bytes = (uint32_t)a.ring_bytes;
+        bool ok = true;
+        for (int s = 0; s < a.n_stages && ok; ++s) {
+            const SStage* st = a.ext ? a.ext + s : &a.inl[s];
+            const int count = st->count;
+            const int T_total = st->T_total;
+            const int n_cta = T_total > cta ? (T_total - cta + G - 1) / G : 0;
+            for (int k0 = 0; k0 < n_cta && ok; k0 += 32) {
+                const int k = k0 + lane;
+                uint32_t bytes = 0;
+                int mi = 0, ti = 0;
+                unsigned long long src = 0;
+                if (k < n_cta) {
+                    int v = cta + k * G;
+                    while (mi + 1 < count && v >= st->mat[mi].T) {
+                        v -= st->mat[mi].T;
+                        ++mi;
                     }
+                    ti = v;
+                    const uint32_t o0 = __ldg(st->mat[mi].tile_off + v);
+                    const uint32_t o1 = __ldg(st->mat[mi].tile_off + v + 1);
+                    bytes = (o1 - o0) * 16u;
+                    src = (unsigned long long)(st->mat[mi].stream + (size_t)o0 * 16);
                 }
-                int inc = tot;
-#pragma unroll
-                for (int dd = 1; dd < 32; dd <<= 1) {
-                    const int up = __shfl_up_sync(0xFFFFFFFFu, inc, dd);
-                    if (lane >= dd) inc += up;
-                }
-                int base = cursor + inc - tot;
-                cursor += __shfl_sync(0xFFFFFFFFu, inc, 31);
-#pragma unroll
-                for (int j = 0; j < kGap4Jmax; ++j) {
-                    if (j < my_cnt) {
-                        const uint4 v = sv[t.slot(lane, j)];
-                        const uint32_t E = code[j] & 0x0F0F0F0Fu;
-                        const uint32_t O = (code[j] >> 4) & 0x0F0F0F0Fu;
-                        const uint32_t PE = (E + O) * 0x01010100u + E;
-                        const uint32_t PO = PE + O;
-                        const char* xb = (const char*)xs + (size_t)base * kRowBytes;
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const uint32_t oe = __byte_perm(PE, 0, 0x4440 + k);
-                            const uint32_t oo = __byte_perm(PO, 0, 0x4440 + k);
-                            const char* xe = xb + oe * kRowBytes + (2 * k) * kRowBytes;
-                            const char* xo = xb + oo * kRowBytes + (2 * k + 1) * kRowBytes;
-                            if (NT == 1) {
-                                acc[0] = fmaf(bf16_lo(w[k]), *(const float*)xe, acc[0]);
-                                acc_b = fmaf(bf16_hi(w[k]), *(const float*)xo, acc_b);
-                            } else {
-                                fma_entry<NT>(acc, bf16_lo(w[k]), xe);
-                                fma_entry<NT>(acc, bf16_hi(w[k]), xo);
-                            }
+                const int cnt = min(32, n_cta - k0);
+                for (int i = 0; i < cnt && ok; ++i) {
+                    const uint32_t b = __shfl_sync(0xFFFFFFFFu, bytes, i);
+                    const unsigned long long sp = __shfl_sync(0xFFFFFFFFu, src, i);
+                    const int m_i = __shfl_sync(0xFFFFFFFFu, mi, i);
+                    const int t_i = __shfl_sync(0xFFFFFFFFu, ti, i);
+                    // find room for b contiguous bytes and a free slot (all lanes run this alike)
+                    while (true) {
+                        const uint32_t outstanding = q - oldest;
+                        bool fits;
+                        if (outstanding == 0) {
+                            head = tail = 0;
+                            fits = true;
+                        } else if (head >= tail) {
+                            if (head + b <= ring_bytes) fits = true;
+                            else if (b < tail) { head = 0; fits = true; }
+                            else fits = false;
+                        } else {
+                            fits = head + b < tail;
                         }
-                        base += (int)(PO >> 24) + 8;
+                        if (fits && outstanding < (uint32_t)kSlots) break;
+                        if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
+                        ++oldest;
+                        tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
+                    }
+                    if (!ok) break;
+                    const uint32_t slot = q % kSlots;
+                    if (lane == 0) {
+                        sh->desc[slot] = make_int4((int)head, m_i, t_i, (int)b);
+                        mbar_expect_tx(full0 + 8 * slot, b);
+                        bulk_g2s(ring0 + head, (const void*)sp, b, full0 + 8 * slot);
+                    }
+                    __syncwarp();
+                    head += b;
+                    ++q;
+                }
+            }
+        }
+        if (!ok) {
+            // give the copies already issued time to land before this CTA's memory is released
+            for (uint32_t t = oldest; t != q; ++t) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(full0 + 8 * (t % kSlots), (t / kSlots) & 1u))
+                    if (clock64() - t0 > wc.budget) break;
+            }
+            if (lane == 0 && a.err) atomicExch(a.err, 1);
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- consumer warps
+    // Consumer threads meet at named barrier 1.  A warp that gave up on a wait keeps meeting
+    // the others there; the decision to stop is taken by all of them together, right after
+    // a barrier, from a word that only thread 0 writes.
+    constexpr int kGroups = 32 / NT;
+    const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
+    const int N = a.N;
+    uint32_t qbase = 0;
+    bool failed = false;
+    int s = 0;
+    for (; s < a.n_stages; ++s) {
+        const SStage& st = a.ext ? a.ext[s] : a.inl[s];
+        if (ctid == 0) {
+            if (s > 0) {
+                // grid barrier: every CTA has written the previous stage's outputs
+                const unsigned int target = (unsigned int)s * (unsigned int)G;
+                const long long t0 = clock64();
+                uint32_t it = 0;
+                while ((int)(ld_acquire_gpu(a.gbar) - target) < 0) {
+                    if ((++it & 15u) == 0u) {
+                        if (sh->abort_flag) break;
+                        if (clock64() - t0 > wc.budget) { sh->abort_flag = 1; break; }
+                    }
+                }
+                __threadfence();
+            }
+            sh->stage_dead = sh->abort_flag;
+        }
+        named_bar_sync(1, kConsumerThreads);
+        if (sh->stage_dead) break;
+
+        const int K = st.K;
+        const uint16_t* x_src = (s == 0 && a.x_in) ? a.x_in : st.x;
+        const size_t xoff = (size_t)a.n0 * K;
+        stage_x<NT>(st, N, x_src ? x_src + xoff : nullptr, st.g ? st.g + xoff : nullptr, st.u ? st.u + xoff : nullptr,
+                    st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid);
+
+        const int S = st.S;
+        const int T_total = st.T_total;
+        const int n_cta = T_total > cta ? (T_total - cta + G - 1) / G : 0;
+        const int hdr_bytes = st.hdr_bytes;
+        const int strip = lane % S;
+        const int plane = S > kGroups ? strip / kGroups : 0;
+        const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)((st.B + kGap4Slack) * 128) +
+                                 (uint32_t)(lane % kGroups) * (4u * NT);
+        const uint32_t lt = (1u << lane) - 1u;
+
+        for (int k = warp; k < n_cta && !failed; k += kConsumerWarps) {
+            const uint32_t q = qbase + (uint32_t)k;
+            const uint32_t slot = q % kSlots;
+            if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
+            const int4 d = sh->desc[slot];
+            const uint32_t tb = ring0 + (uint32_t)d.x;
+            const SMat& md = st.mat[d.y];
+            const uint32_t cnt = lds_u16(tb + 2u * lane);
+            const uint32_t ct = lds_u32(tb + 64u);
+            const uint32_t cb = tb + (uint32_t)hdr_bytes;                 // code words
+            const uint32_t vb = cb + ((ct * 4u + 15u) & ~15u);            // values
+
+            float a0[NT], a1[NT];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) a0[n] = a1[n] = 0.f;
+            uint32_t xb = xs_lane;
+
+            // steps every populated lane takes: addresses advance by a constant
+            const uint32_t bal0 = __ballot_sync(0xFFFFFFFFu, cnt > 0);
+            const uint32_t n0 = __popc(bal0);
+            const uint32_t jmin = __reduce_min_sync(0xFFFFFFFFu, cnt > 0 ? cnt : 0xFFFFu);
+            const uint32_t jmax = __reduce_max_sync(0xFFFFFFFFu, cnt);
+            uint32_t j = 0;
+            if (bal0 != 0u) {
+                if (cnt > 0) {
+                    const uint32_t rank0 = __popc(bal0 & lt);
+                    uint32_t ca = cb + rank0 * 4u, va = vb + rank0 * 16u;
+                    uint32_t code = lds_u32(ca);
+                    uint4 v = lds_v4(va);
+                    for (uint32_t jj = 1; jj < jmin; ++jj) {
+                        ca += n0 * 4u;
+                        va += n0 * 16u;
+                        const uint32_t code_n = lds_u32(ca);
+                        const uint4 v_n = lds_v4(va);
+                        xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                        code = code_n;
+                        v = v_n;
+                    }
+                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                }
+                j = jmin;
+            }
+            // ragged tail: the set of lanes that still have a chunk shrinks step by step
+            uint32_t off = n0 * j;
+            for (; j < jmax; ++j) {
+                const bool act = j < cnt;
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, act);
+                if (act) {
+                    const uint32_t idx = off + __popc(bal & lt);
+                    const uint32_t code = lds_u32(cb + idx * 4u);
+                    const uint4 v = lds_v4(vb + idx * 16u);
+                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                }
+                off += __popc(bal);
+            }
+
+            // the S lanes of a row add up; the lane of strip 0 stores
+            float r[NT];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                r[n] = a0[n] + a1[n];
+                for (int dd = 1; dd < S; dd <<= 1) r[n] += __shfl_xor_sync(0xFFFFFFFFu, r[n], dd);
+            }
+            if (strip == 0) {
+                const uint32_t row = lds_u32(tb + 68u + 4u * (uint32_t)(lane / S));
+                if (row != 0xFFFFFFFFu) {
+                    void* yp = (s == a.n_stages - 1 && a.y_out && d.y == 0) ? a.y_out : md.y;
+                    const size_t M = (size_t)md.M;
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        if (n < N) {
+                            const size_t at = (size_t)(a.n0 + n) * M + row;
+                            if (md.y_f32) ((float*)yp)[at] = r[n];
+                            else ((uint16_t*)yp)[at] = f32_to_bf16_rne(r[n]);
+                        }
                     }
                 }
             }
-            __syncwarp();   // every lane is done with the stage before it is refilled
-            ++consumed;
-            if (++c_stage == depth) { c_stage = 0; c_parity ^= 1u; }
-            if (more) fetch_one();
-            if (flags & 2) {
-                float r[NT];
-#pragma unroll
-                for (int n = 0; n < NT; ++n) r[n] = warp_sum(n == 0 && NT == 1 ? acc[0] + acc_b : acc[n]);
-                if (lane == 0) store_row<NT>(md, row, r, grp.N);
-            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+        }
+        qbase += (uint32_t)n_cta;
+        // everything this CTA wrote in the stage is visible before it arrives at the barrier
+        named_bar_sync(1, kConsumerThreads);
+        if (s + 1 < a.n_stages && ctid == 0) {
+            __threadfence();
+            atomicAdd(a.gbar, 1u);
         }
     }
-    if (!staged) {  // a warp without rows still takes part in the one CTA-wide barrier
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        stage_x<NT>(grp, xs, kGap4Slack);
-        __syncthreads();
+    if (s < a.n_stages || sh->abort_flag) {   // a bounded wait ran out somewhere in this CTA
+        if (ctid == 0 && a.err) atomicExch(a.err, 1);
+        return;
     }
-    if (dead && lane == 0 && grp.err) atomicExch(grp.err, 1);
+    // leave the barrier words as they were found: the last CTA out clears them
+    if (a.n_stages > 1 && ctid == 0) {
+        const unsigned int prev = atomicAdd(a.gbar + 32, 1u);
+        if (prev == (unsigned int)G - 1u) {
+            atomicExch(a.gbar, 0u);
+            atomicExch(a.gbar + 32, 0u);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------ BITMASK
@@ -480,6 +622,45 @@ __global__ void __launch_bounds__(kThreads) gap4_kernel(const __grid_constant__ 
 // General-purpose path (any M, K; activations read through L1 from global memory, so no
 // shared-memory limit on K).  One warp per row; lane l takes mask words l, l+32, ...; a
 // warp prefix sum of the words' popcounts gives each lane its first value.
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kThreads = kWarpsPerCta * 32;
+
+struct MatDesc {
+    const uint32_t* sec0;   // row_val_ptr
+    const uint32_t* sec1;   // mask words
+    const void* sec2;       // u16 values
+    void* y;                // [N*M]
+    int M;
+    int y_f32;              // 1: fp32 output, 0: bf16
+    int cta_begin;          // first CTA of this weight in a fused launch
+    int cta_count;
+};
+
+struct LaunchGroup {
+    MatDesc mat[kMaxFused];
+    int count;
+    int K;
+    int N;                  // rows of X in this launch, 1..NT
+    // activation source: x (plain) or silu(g)*u rounded to bf16 (feed-forward glue)
+    const uint16_t* x;      // [N*K] bf16, or NULL in glue mode
+    const uint16_t* g;      // glue mode: gate output [N*K]
+    const uint16_t* u;      // glue mode: up output   [N*K]
+    uint16_t* t_out;        // glue mode: optional copy of t = bf16(silu(g)*u), written by CTA 0
+};
+
+template <int NT>
+__device__ __forceinline__ void store_row(const MatDesc& md, int row, const float (&acc)[NT], int N)
+{
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+        if (n < N) {
+            if (md.y_f32) ((float*)md.y)[(size_t)n * md.M + row] = acc[n];
+            else ((uint16_t*)md.y)[(size_t)n * md.M + row] = f32_to_bf16_rne(acc[n]);
+        }
+    }
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kThreads) bitmask_kernel(const __grid_constant__ LaunchGroup grp)
 {
@@ -527,9 +708,7 @@ __global__ void __launch_bounds__(kThreads) bitmask_kernel(const __grid_constant
                         if (grp.x) {
                             xv = bf16_to_f32(__ldg(grp.x + (size_t)n * K + col));
                         } else {
-                            const float a = bf16_to_f32(__ldg(grp.g + (size_t)n * K + col));
-                            const float bb = bf16_to_f32(__ldg(grp.u + (size_t)n * K + col));
-                            xv = bf16_to_f32(f32_to_bf16_rne((a / (1.f + expf(-a))) * bb));
+                            xv = bf16_to_f32(silu_mul_bits(__ldg(grp.g + (size_t)n * K + col), __ldg(grp.u + (size_t)n * K + col)));
                         }
                         acc[n] = fmaf(wv, xv, acc[n]);
                     }
@@ -542,11 +721,7 @@ __global__ void __launch_bounds__(kThreads) bitmask_kernel(const __grid_constant
     }
     // glue mode: CTA 0 also publishes t = bf16(silu(g) * u)
     if (!grp.x && grp.t_out && blockIdx.x == 0) {
-        for (int i = threadIdx.x; i < K * N; i += blockDim.x) {
-            const float a = bf16_to_f32(grp.g[i]);
-            const float bb = bf16_to_f32(grp.u[i]);
-            grp.t_out[i] = f32_to_bf16_rne((a / (1.f + expf(-a))) * bb);
-        }
+        for (int i = threadIdx.x; i < K * N; i += blockDim.x) grp.t_out[i] = silu_mul_bits(grp.g[i], grp.u[i]);
     }
 }
 

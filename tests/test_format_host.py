@@ -60,7 +60,7 @@ def test_zero_and_full_masks(fmt):
     if fmt == sd2.SD2_FORMAT_BITMASK:
         assert info["compressed_bytes"] == 4 * 11 + 4 * 10 * 7      # offsets + mask words, no values
     else:
-        assert info["compressed_bytes"] == 4 * 11                   # offsets only, no chunks
+        assert info["compressed_bytes"] == _gap4_bytes(zero)       # tile offsets and tile headers, no chunks
     full = np.ones((10, 200), np.uint8)
     dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, full, fmt))
     assert np.array_equal(dense, W) and info["nnz"] == 2000
@@ -83,10 +83,22 @@ def test_bitmask_byte_count_closed_form():
     assert info["compressed_bytes"] == 4 * (M + 1) + 4 * M * ((K + 31) // 32) + 2 * int(mask.sum())
 
 
-def _gap4_entries(row_mask):
-    """Entries (kept + fillers) of one row under the 4-bit gap code, from its definition."""
+def _gap4_geometry(M, K):
+    """Strip geometry (S strips of B columns, R rows per tile) from the format's definition."""
+    S = 1
+    while S < 32 and M * S // 32 < 2048:
+        S *= 2
+    while S > 1 and (K + S - 1) // S < 64:
+        S //= 2
+    while S < 32 and ((K + S - 1) // S | 1) > 496:
+        S *= 2
+    return S, (K + S - 1) // S | 1, 32 // S
+
+
+def _gap4_entries(seg_mask):
+    """Entries (kept + fillers) of one segment under the 4-bit gap code, from its definition."""
     cursor, e = 0, 0
-    for k in np.nonzero(row_mask)[0]:
+    for k in np.nonzero(seg_mask)[0]:
         while k - cursor > 15:
             e += 1
             cursor += 16
@@ -95,41 +107,67 @@ def _gap4_entries(row_mask):
     return e
 
 
+def _gap4_bytes(mask):
+    """Compressed bytes of a mask: tile offsets + per tile (header, code words, values)."""
+    M, K = mask.shape
+    S, B, R = _gap4_geometry(M, K)
+    row_chunks = np.array([sum((_gap4_entries(mask[m, s * B:(s + 1) * B]) + 7) // 8 for s in range(S)) for m in range(M)])
+    order = np.argsort(-row_chunks, kind="stable")
+    T = (M + R - 1) // R
+    hdr = (64 + 4 + 4 * R + 15) // 16 * 16
+    total = 4 * (T + 1)
+    for t in range(T):
+        ct = int(row_chunks[order[t * R:(t + 1) * R]].sum())
+        total += hdr + (4 * ct + 15) // 16 * 16 + 16 * ct
+    return total
+
+
 def test_gap4_byte_count_closed_form():
-    M, K = 29, 700
-    for d in (0.5, 0.1, 0.03):
-        W, mask = _case(31, M, K, d)
-        chunks = sum((_gap4_entries(mask[m]) + 7) // 8 for m in range(M))
-        _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
-        assert info["compressed_bytes"] == 4 * (M + 1) + 20 * chunks
+    for M, K in ((29, 700), (70, 2048), (5, 11008)):
+        for d in (0.5, 0.1, 0.03):
+            W, mask = _case(31, M, K, d)
+            _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
+            assert info["compressed_bytes"] == _gap4_bytes(mask)
 
 
-def test_gap4_long_rows_span_several_tiles():
-    # 11008 columns at 90 % density: ~1240 chunks per row -> 8 tiles of ~155 chunks, J = 5
-    M, K = 3, 11008
-    W, mask = _case(41, M, K, 0.9)
+def test_gap4_geometries_and_ragged_tiles():
+    # every strip count, tiles with missing rows, rows of very different lengths
+    for M, K in ((3, 11008), (100, 64), (2500, 100), (5000, 70), (33, 2048), (9000, 130), (70000, 3)):
+        W, mask = _case(41 + M, M, K, 0.5)
+        if M >= 33:
+            mask[::7, :] = 0                     # empty rows between populated ones
+            mask[1::11, :] = 1                   # full rows
+        dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+        assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+        assert info["compressed_bytes"] == _gap4_bytes(mask)
+    # every segment length from 0 to a full strip
+    K = 257
+    mask = np.zeros((K + 1, K), np.uint8)
+    for m in range(K + 1):
+        mask[m, :m] = 1
+    W = synth.normal_bf16(43, (K + 1, K), 0.02)
     dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
     assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
-    # every chunk count from 1 to 400 exercises every (J, L, cnt_last) tile geometry
-    K = 8 * 400
-    mask = np.zeros((400, K), np.uint8)
-    for m in range(400):
-        mask[m, : 8 * (m + 1)] = 1
-    W = synth.normal_bf16(43, (400, K), 0.02)
-    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
-    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
-    assert info["compressed_bytes"] == 4 * 401 + 20 * sum(range(1, 401))
+
+
+def test_gap4_is_unsupported_for_very_wide_matrices():
+    W = np.zeros((2, 32 * 496 + 1), np.uint16)
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, None, sd2.SD2_FORMAT_GAP4)
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+    _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, None, sd2.SD2_FORMAT_AUTO), want_dense=False)
+    assert info["format"] == sd2.SD2_FORMAT_BITMASK
 
 
 def test_sizes_at_half_density_match_the_format_arithmetic():
-    M, K = 256, 2048
+    M, K = 8192, 2048                                            # a gate / up projection: strips of 257 columns
     W, mask = _case(51, M, K, 0.5)
     nnz = int(mask.sum())
     _, bm = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_BITMASK), want_dense=False)
     _, g4 = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
     assert abs(bm["compressed_bytes"] / nnz - 2.25) < 0.01       # 2 B value + 2 bits of mask per kept weight
-    assert 2.5 <= g4["compressed_bytes"] / nnz < 2.53            # 2 B value + 4-bit gap + row padding
-    assert g4["compressed_bytes"] < 0.64 * 2 * M * K             # well under the dense bf16 bytes
+    assert 2.5 <= g4["compressed_bytes"] / nnz < 2.62            # 2 B value + 4-bit gap + segment padding + headers
+    assert g4["compressed_bytes"] < 0.66 * 2 * M * K             # well under the dense bf16 bytes
 
 
 @pytest.mark.parametrize("fmt", FORMATS)

@@ -257,6 +257,75 @@ def test_block_step_teacher_forced(fmt, N):
         sd2.sd2_free(h)
 
 
+_cudart = None
+
+
+def _read_u16(ptr, count):
+    """Copy `count` bf16 patterns from a raw device address (through the CUDA runtime torch loaded)."""
+    import ctypes
+    global _cudart
+    if _cudart is None:
+        _cudart = ctypes.CDLL("libcudart.so.12")
+        _cudart.cudaMemcpy.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int]
+        _cudart.cudaMemcpy.restype = ctypes.c_int
+    buf = np.empty(count, np.uint16)
+    rc = _cudart.cudaMemcpy(buf.ctypes.data, ptr, count * 2, 2)               # 2 = device to host
+    assert rc == 0
+    return buf
+
+
+@pytest.mark.parametrize("N", [1, 3, 6])
+def test_drafter_step_teacher_forced(N):
+    # three chained blocks in one persistent launch per panel: every linear is checked against
+    # the oracle on the input the device actually gave it
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 3)
+    L = 3
+    lins, blocks = [], []
+    for b in range(L):
+        lin = synth.make_block(2, b, shape, 0.5)
+        lins.append(lin)
+        blocks.append([sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4,
+                                        sd2.SD2_DTYPE_F32 if (b == L - 1 and i == 6) else sd2.SD2_DTYPE_BF16)
+                       for i, (W, m) in enumerate(lin)])
+    d = sd2.sd2_drafter_create(blocks, n_max=8)
+    x = synth.make_activations(2, 0, 0, N, shape.hidden)
+    xd = dev_bf16(x)
+    y = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):                       # twice: the barrier words must come back clean
+        y.fill_(float("nan"))
+        sd2.sd2_drafter_step(d, xd, y)
+        sd2.sd2_stream_check()
+    dims = [shape.hidden, shape.kv, shape.kv, shape.hidden, shape.inter, shape.inter, shape.inter, shape.hidden]
+
+    def lin_check(W, m, inp_bits, out, f32=False):
+        Yr, S = oracle.masked_linear(W, m, inp_bits)
+        check(out if f32 else synth.bf16_bits_to_f32(out).astype(np.float64), Yr, S, f32)
+
+    inp = x
+    for b in range(L):
+        ptrs = sd2.sd2_drafter_buffers(d, b)
+        q, k, v, hdn, g, u, t, out = [_read_u16(p, N * dm).reshape(N, dm) for p, dm in zip(ptrs, dims)]
+        lin = lins[b]
+        lin_check(*lin[0], inp, q)
+        lin_check(*lin[1], inp, k)
+        lin_check(*lin[2], inp, v)
+        lin_check(*lin[3], q, hdn)
+        lin_check(*lin[4], hdn, g)
+        lin_check(*lin[5], hdn, u)
+        t_ref = oracle.silu_mul(g, u)
+        t_ref_bits = np.array([oracle.f64_to_bf16_rne(float(z)) for z in t_ref], np.uint16).reshape(N, -1)
+        assert bf16_ulp_distance(t, t_ref_bits).max() <= 2
+        if b < L - 1:
+            lin_check(*lin[6], t, out)
+            inp = out
+        else:
+            lin_check(*lin[6], t, y.cpu().numpy().astype(np.float64), f32=True)
+    sd2.sd2_drafter_free(d)
+    for hs in blocks:
+        for h in hs:
+            sd2.sd2_free(h)
+
+
 def test_block_step_rejects_shapes_that_do_not_chain():
     shape = synth.DrafterShape("tiny", 128, 32, 256, 1)
     lin = synth.make_block(2, 1, shape, 0.5)
