@@ -333,9 +333,15 @@ sd2_status launch_stream(int nt, const SArgs& a, int grid, bool cooperative, cud
     }
 }
 
-// Fills one stage from `count` GAP4 handles of equal K and S.
+void set_stage_grid(SStage& st, int grid)
+{
+    st.tiles_div = st.T_total / grid;
+    st.tiles_rem = st.T_total % grid;
+}
+
+// Fills one stage from `count` GAP4 handles of equal K and S, to be run by `grid` CTAs.
 void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
-                uint16_t* t_out, void* const* Y, bool y_force_bf16)
+                uint16_t* t_out, void* const* Y, bool y_force_bf16, int grid)
 {
     std::memset(&st, 0, sizeof st);
     st.count = count;
@@ -343,6 +349,8 @@ void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, 
     st.S = hs[0]->S;
     st.B = hs[0]->B;
     st.hdr_bytes = gap4_tile_header_bytes(32 / hs[0]->S);
+    st.log2S = 0;
+    while ((1 << st.log2S) < hs[0]->S) ++st.log2S;
     st.x = x;
     st.g = g;
     st.u = u;
@@ -359,7 +367,12 @@ void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, 
         T += hs[i]->T;
     }
     st.T_total = T;
+    set_stage_grid(st, grid);
 }
+
+#ifdef SD2_TRACE
+long long* g_trace = nullptr;   // set through sd2_debug_set_trace (trace builds only)
+#endif
 
 long long wait_budget(int dev)
 {
@@ -415,6 +428,9 @@ sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[3], int K_max, int 
         a.xs_bytes = p.xs_bytes;
         a.xlin_bytes = p.xlin_bytes;
         a.ring_bytes = p.ring_bytes;
+#ifdef SD2_TRACE
+        a.trace = g_trace;
+#endif
         sd2_status st = launch_stream(nt, a, grid, a.n_stages > 1, s);
         if (st != SD2_OK) return st;
     }
@@ -427,6 +443,7 @@ sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, 
     const bool coop = a.n_stages > 1;
     int grid = g_dev[dev].sms;
     if (!coop && needs.tiles_max < grid) grid = needs.tiles_max < 1 ? 1 : needs.tiles_max;
+    if (!coop) set_stage_grid(a.inl[0], grid);
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
     a.gbar = coop ? g_dev[dev].barriers + (size_t)(g_next_barrier.fetch_add(1) % kBarrierPool) * kBarrierStrideWords : nullptr;
@@ -464,7 +481,7 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
     SArgs a;
     std::memset(&a, 0, sizeof a);
     a.n_stages = 1;
-    fill_stage(a.inl[0], hs, count, x, g, u, t_out, Y, y_force_bf16);
+    fill_stage(a.inl[0], hs, count, x, g, u, t_out, Y, y_force_bf16, g_dev[dev].sms);
     ProgramNeeds needs;
     needs.add(hs, count);
     return run_program(a, dev, N, needs, s);
@@ -511,7 +528,7 @@ void block_layout(const sd2_handle* h, const BlockDims& d, int64_t N, int64_t of
 // group that do not share a strip geometry get a stage each.  Returns the number appended.
 int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
                         uint16_t* hdn, uint16_t* g, uint16_t* u, uint16_t* t, void* y, bool y_force_bf16,
-                        ProgramNeeds* needs)
+                        ProgramNeeds* needs, int grid)
 {
     int n = 0;
     auto group = [&](const sd2_handle* hs, int count, const uint16_t* xin, const uint16_t* gg, const uint16_t* uu,
@@ -520,11 +537,11 @@ int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, 
         for (int i = 1; i < count; ++i)
             if (hs[i]->S != hs[0]->S) same = false;
         if (same) {
-            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force);
+            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force, grid);
             needs->add(hs, count);
         } else {
             for (int i = 0; i < count; ++i) {
-                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force);
+                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force, grid);
                 needs->add(hs + i, 1);
             }
         }
@@ -791,7 +808,7 @@ sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N
         SArgs a;
         std::memset(&a, 0, sizeof a);
         ProgramNeeds needs;
-        a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, q, k, v, hdn, g, u, t, y, false, &needs);
+        a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, q, k, v, hdn, g, u, t, y, false, &needs, g_dev[dev].sms);
         return run_program(a, dev, N, needs, s);
     }
     void* y_qkv[3] = {q, k, v};
@@ -861,7 +878,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
             void* yout = base + wo[7];
             n += append_block_stages(stages.data() + n, h + 7 * b, xin, (uint16_t*)(base + wo[0]), (uint16_t*)(base + wo[1]),
                                      (uint16_t*)(base + wo[2]), (uint16_t*)(base + wo[3]), (uint16_t*)(base + wo[4]),
-                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs);
+                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs, g_dev[dev].sms);
         }
         d->n_stages = n;
         ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
@@ -937,5 +954,9 @@ sd2_status sd2_drafter_free(sd2_drafter d)
     delete d;
     return st;
 }
+
+#ifdef SD2_TRACE
+void sd2_debug_set_trace(long long* device_buffer) { g_trace = device_buffer; }
+#endif
 
 }  // extern "C"

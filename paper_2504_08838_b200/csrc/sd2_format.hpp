@@ -37,6 +37,9 @@
 //
 //   tile record   u16 cnt[32]          chunks of each lane's segment
 //                 u32 n_chunks         sum of cnt
+//                 u32 cnt_range        smallest non-zero cnt | largest cnt << 16 (0 if all are zero)
+//                 u32 lane_mask        bit l set iff cnt[l] > 0
+//                 u32 reserved         0
 //                 u32 row[R]           original row index of each tile row, 0xFFFFFFFF = none
 //                 (pad to 16 bytes)
 //                 u32 code[n_chunks]   step-major as described
@@ -96,7 +99,7 @@ struct Gap4Geom {
 };
 
 // Header bytes of a tile record with R rows.
-SD2_HD int gap4_tile_header_bytes(int R) { return (64 + 4 + 4 * R + 15) & ~15; }
+SD2_HD int gap4_tile_header_bytes(int R) { return (80 + 4 * R + 15) & ~15; }
 
 // Picks S: enough tiles to spread over every SM's warps, strips neither too narrow (padding)
 // nor wider than the chunk counters allow.  B is odd so that strips start in distinct
@@ -327,12 +330,12 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
         uint8_t* rec = tiles + (size_t)toff[(size_t)t] * 16;
         uint16_t* cnt = (uint16_t*)rec;
         uint32_t* nch = (uint32_t*)(rec + 64);
-        uint32_t* rows = (uint32_t*)(rec + 68);
+        uint32_t* rows = (uint32_t*)(rec + 80);
         // logical entry lists of the 32 segments
         std::vector<uint8_t> eg[32];
         std::vector<uint16_t> ev[32];
-        uint32_t ct = 0;
-        int maxc = 0;
+        uint32_t ct = 0, lane_mask = 0;
+        int maxc = 0, minc = 0xFFFF;
         for (int l = 0; l < 32; ++l) {
             const int rr = l / S, s = l % S;
             const int64_t i = t * R + rr;
@@ -345,6 +348,8 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
             ct += (uint32_t)c;
             if (c > maxc) maxc = c;
             if (c == 0) continue;
+            if (c < minc) minc = c;
+            lane_mask |= 1u << l;
             eg[l].assign((size_t)c * 8, 0);
             ev[l].assign((size_t)c * 8, 0);
             const int64_t c0 = std::min<int64_t>(K, (int64_t)s * B), c1 = std::min<int64_t>(K, c0 + B);
@@ -365,7 +370,10 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
             }
             // entries e .. 8c-1 stay gap 0 / value +0
         }
-        *nch = ct;
+        nch[0] = ct;
+        nch[1] = lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u;
+        nch[2] = lane_mask;
+        nch[3] = 0;
         uint32_t* codes = (uint32_t*)(rec + hdr);
         uint16_t* vals = (uint16_t*)(rec + hdr + align16((size_t)ct * 4));
         size_t slot = 0;
@@ -410,7 +418,7 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
     int bad = 0;
     int64_t chunks = 0;
     for (int64_t t = 0; t < T; ++t) {  // row ids: a permutation of 0..M-1, checked serially
-        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 68);
+        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 80);
         if ((uint64_t)(toff[t + 1] - toff[t]) * 16 < (uint64_t)hdr) return -6;
         for (int rr = 0; rr < R; ++rr) {
             const int64_t i = t * R + rr;
@@ -431,16 +439,23 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
         const uint8_t* rec = tiles + (size_t)toff[t] * 16;
         const size_t rec_bytes = (size_t)(toff[t + 1] - toff[t]) * 16;
         const uint16_t* cnt = (const uint16_t*)rec;
-        const uint32_t ct = *(const uint32_t*)(rec + 64);
-        const uint32_t* rows = (const uint32_t*)(rec + 68);
-        uint32_t sum = 0;
-        int maxc = 0;
+        const uint32_t* meta = (const uint32_t*)(rec + 64);
+        const uint32_t ct = meta[0];
+        const uint32_t* rows = (const uint32_t*)(rec + 80);
+        uint32_t sum = 0, lane_mask = 0;
+        int maxc = 0, minc = 0xFFFF;
         for (int l = 0; l < 32; ++l) {
             if (cnt[l] > (B + kGap4Slack) / 8 + 1) bad |= 1;
             if (rows[l / S] == 0xFFFFFFFFu && cnt[l] != 0) bad |= 1;
             sum += cnt[l];
             if (cnt[l] > maxc) maxc = cnt[l];
+            if (cnt[l] > 0) {
+                lane_mask |= 1u << l;
+                if (cnt[l] < minc) minc = cnt[l];
+            }
         }
+        if (meta[1] != (lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u) || meta[2] != lane_mask || meta[3] != 0)
+            bad |= 1;
         if (sum != ct || rec_bytes != (size_t)hdr + align16((size_t)ct * 4) + (size_t)ct * 16 ||
             rec_bytes > h.max_tile_bytes) {
             bad |= 1;

@@ -39,7 +39,7 @@ __device__ __forceinline__ uint16_t f32_to_bf16_rne(float f)
 __device__ __forceinline__ uint16_t silu_mul_bits(uint16_t g, uint16_t u)
 {
     const float a = bf16_to_f32(g);
-    return f32_to_bf16_rne((a / (1.f + expf(-a))) * bf16_to_f32(u));
+    return f32_to_bf16_rne(__fdividef(a, 1.f + __expf(-a)) * bf16_to_f32(u));
 }
 
 __device__ __forceinline__ float warp_sum(float v)
@@ -100,7 +100,10 @@ struct SStage {
     int B;                 // strip width
     int T_total;           // tiles of all weights
     int hdr_bytes;         // tile header bytes (depends on S)
-    int reserved[2];
+    int log2S;
+    int tiles_div;         // T_total / grid size: CTA c runs tiles_div + (c < tiles_rem) tiles
+    int tiles_rem;         // T_total % grid size
+    int reserved[3];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
@@ -118,7 +121,14 @@ struct SArgs {
     int xs_bytes;                   // shared memory for the transposed activations
     int xlin_bytes;                 // shared memory for one linear activation row
     int ring_bytes;
+    long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
 };
+
+#ifdef SD2_TRACE
+#define SD2_STAMP(slot) do { if (a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define SD2_STAMP(slot) do { } while (0)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -177,25 +187,56 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t a)
     return v;
 }
 template <int OFF>
-__device__ __forceinline__ float lds_f32_off(uint32_t a)
+__device__ __forceinline__ uint32_t lds_u32_off(uint32_t a)
 {
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(a), "n"(OFF));
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF));
     return v;
 }
 template <int OFF>
-__device__ __forceinline__ float2 lds_f32x2_off(uint32_t a)
+__device__ __forceinline__ uint2 lds_u32x2_off(uint32_t a)
 {
-    float2 v;
-    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(a), "n"(OFF));
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(a), "n"(OFF));
     return v;
 }
 template <int OFF>
-__device__ __forceinline__ float4 lds_f32x4_off(uint32_t a)
+__device__ __forceinline__ uint4 lds_u32x4_off(uint32_t a)
 {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a), "n"(OFF));
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a), "n"(OFF));
     return v;
+}
+
+// c + w * x for bf16 w and x with an fp32 sum (the product of two bf16 values is exact in
+// fp32, so this equals an fp32 fused multiply-add of the widened values).  w is the low or the
+// high half of `wpair`; x is the high half of `xword`, an fp32 whose low 16 bits are zero.
+__device__ __forceinline__ float fma_bf16_lo(uint32_t wpair, uint32_t xword, float c)
+{
+    float d;
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, wl, xh, %3;\n\t}"
+        : "=f"(d)
+        : "r"(wpair), "r"(xword), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float fma_bf16_hi(uint32_t wpair, uint32_t xword, float c)
+{
+    float d;
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, wh, xh, %3;\n\t}"
+        : "=f"(d)
+        : "r"(wpair), "r"(xword), "f"(c));
+    return d;
+}
+
+// c + 128 * byte K8 of p (one integer dot-product instruction with a one-hot operand)
+template <int K8>
+__device__ __forceinline__ uint32_t byte_times_128_plus(uint32_t p, uint32_t c)
+{
+    uint32_t d;
+    asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(p), "r"(0x80u << (8 * K8)), "r"(c));
+    return d;
 }
 
 __device__ __forceinline__ void named_bar_sync(int id, int threads)
@@ -212,6 +253,7 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p)
 
 // Shared-memory bookkeeping of one CTA (placed after xs and xlin).
 struct StreamShared {
+    SStage stage[2];                   // descriptors of the current and the next stage
     int4 desc[kSlots];                 // x: ring offset, y: weight index, z: tile index, w: bytes
     unsigned long long full[kSlots];   // mbarriers: tile landed
     unsigned long long empty[kSlots];  // mbarriers: tile consumed
@@ -243,23 +285,27 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, const 
     return true;
 }
 
-// acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`
-template <int NT, int OFF>
-__device__ __forceinline__ void fma_at(float (&acc)[NT], float w, uint32_t addr)
+// acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`;
+// w is the low (HI = 0) or high (HI = 1) bf16 of `wpair`.
+template <int NT, int OFF, int HI>
+__device__ __forceinline__ void fma_at(float (&acc)[NT], uint32_t wpair, uint32_t addr)
 {
+    uint32_t x[NT];
     if (NT == 1) {
-        acc[0] = fmaf(w, lds_f32_off<OFF>(addr), acc[0]);
+        x[0] = lds_u32_off<OFF>(addr);
     } else if (NT == 2) {
-        const float2 x = lds_f32x2_off<OFF>(addr);
-        acc[0] = fmaf(w, x.x, acc[0]);
-        acc[1] = fmaf(w, x.y, acc[1]);
+        const uint2 t = lds_u32x2_off<OFF>(addr);
+        x[0] = t.x;
+        x[NT - 1] = t.y;
     } else {
-        const float4 x = lds_f32x4_off<OFF>(addr);
-        acc[0] = fmaf(w, x.x, acc[0]);
-        acc[1] = fmaf(w, x.y, acc[1]);
-        acc[2] = fmaf(w, x.z, acc[2]);
-        acc[3] = fmaf(w, x.w, acc[3]);
+        const uint4 t = lds_u32x4_off<OFF>(addr);
+        x[0] = t.x;
+        x[1 % NT] = t.y;
+        x[2 % NT] = t.z;
+        x[3 % NT] = t.w;
     }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) acc[n] = HI ? fma_bf16_hi(wpair, x[n], acc[n]) : fma_bf16_lo(wpair, x[n], acc[n]);
 }
 
 // One chunk: eight (gap, value) entries against the activations at `xb` (the lane's cursor).
@@ -274,17 +320,17 @@ __device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uin
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #define SD2_PAIR(k)                                                              \
     {                                                                            \
-        const uint32_t ae = xb + (__byte_perm(PE, 0, 0x4440 + (k)) << 7);        \
-        const uint32_t ao = xb + (__byte_perm(PO, 0, 0x4440 + (k)) << 7);        \
-        fma_at<NT, (2 * (k)) * 128>(a0, bf16_lo(w[k]), ae);                      \
-        fma_at<NT, (2 * (k) + 1) * 128>(a1, bf16_hi(w[k]), ao);                  \
+        const uint32_t ae = byte_times_128_plus<k>(PE, xb);                      \
+        const uint32_t ao = byte_times_128_plus<k>(PO, xb);                      \
+        fma_at<NT, (2 * (k)) * 128, 0>(a0, w[k], ae);                            \
+        fma_at<NT, (2 * (k) + 1) * 128, 1>(a1, w[k], ao);                        \
     }
     SD2_PAIR(0)
     SD2_PAIR(1)
     SD2_PAIR(2)
     SD2_PAIR(3)
 #undef SD2_PAIR
-    return xb + ((PO >> 24) << 7) + 1024u;
+    return byte_times_128_plus<3>(PO, xb + 1024u);
 }
 
 // Stage the activations of one stage: xs[plane][column c][group][NT] (fp32) with
@@ -341,13 +387,15 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
         }
         named_bar_sync(1, kConsumerThreads);
         // scatter row n: consecutive threads take consecutive groups of one column
+        const int per_plane = rows * kGroups;
         for (int p = 0; p < planes; ++p) {
             float* xp = xs + (size_t)p * rows * 32;
-            for (int i = ctid; i < rows * kGroups; i += kConsumerThreads) {
-                const int grp = i % kGroups;
+            const int strip = S > kGroups ? p * kGroups + (ctid % kGroups) : (ctid % kGroups) & (S - 1);   // fixed per thread
+            const int col0 = strip * B;
+#pragma unroll 4
+            for (int i = ctid; i < per_plane; i += kConsumerThreads) {
                 const int c = i / kGroups;
-                const int strip = S > kGroups ? p * kGroups + grp : grp % S;
-                const int col = strip * B + c;
+                const int col = col0 + c;
                 float v = 0.f;
                 if (n < N && c < B && col < K) v = bf16_to_f32(xlin[col]);
                 xp[(size_t)i * NT + n] = v;
@@ -398,8 +446,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         for (int s = 0; s < a.n_stages && ok; ++s) {
             const SStage* st = a.ext ? a.ext + s : &a.inl[s];
             const int count = st->count;
-            const int T_total = st->T_total;
-            const int n_cta = T_total > cta ? (T_total - cta + G - 1) / G : 0;
+            const int n_cta = st->tiles_div + (cta < st->tiles_rem ? 1 : 0);
             for (int k0 = 0; k0 < n_cta && ok; k0 += 32) {
                 const int k = k0 + lane;
                 uint32_t bytes = 0;
@@ -454,6 +501,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     ++q;
                 }
             }
+            if (lane == 0) SD2_STAMP(6);
         }
         if (!ok) {
             // give the copies already issued time to land before this CTA's memory is released
@@ -471,15 +519,22 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     // Consumer threads meet at named barrier 1.  A warp that gave up on a wait keeps meeting
     // the others there; the decision to stop is taken by all of them together, right after
     // a barrier, from a word that only thread 0 writes.
+    // The descriptor of stage s sits in sh->stage[s & 1]: warp 1 fetches the next stage's while
+    // the current one is computed; the barrier at the end of the stage makes it visible.
     constexpr int kGroups = 32 / NT;
+    constexpr int kStageWords = (int)(sizeof(SStage) / 4);
     const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
     const int N = a.N;
     uint32_t qbase = 0;
     bool failed = false;
+    if (warp == 1) {
+        const uint32_t* src = (const uint32_t*)(a.ext ? a.ext : &a.inl[0]);
+        for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[0])[i] = src[i];
+    }
     int s = 0;
     for (; s < a.n_stages; ++s) {
-        const SStage& st = a.ext ? a.ext[s] : a.inl[s];
         if (ctid == 0) {
+            SD2_STAMP(0);
             if (s > 0) {
                 // grid barrier: every CTA has written the previous stage's outputs
                 const unsigned int target = (unsigned int)s * (unsigned int)G;
@@ -494,37 +549,53 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 __threadfence();
             }
             sh->stage_dead = sh->abort_flag;
+            SD2_STAMP(1);
         }
         named_bar_sync(1, kConsumerThreads);
         if (sh->stage_dead) break;
+        const SStage& st = sh->stage[s & 1];
 
         const int K = st.K;
         const uint16_t* x_src = (s == 0 && a.x_in) ? a.x_in : st.x;
         const size_t xoff = (size_t)a.n0 * K;
         stage_x<NT>(st, N, x_src ? x_src + xoff : nullptr, st.g ? st.g + xoff : nullptr, st.u ? st.u + xoff : nullptr,
                     st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid);
+        if (ctid == 0) SD2_STAMP(2);
+        if (warp == 1 && s + 1 < a.n_stages) {
+            const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);
+            for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[(s + 1) & 1])[i] = src[i];
+        }
 
         const int S = st.S;
-        const int T_total = st.T_total;
-        const int n_cta = T_total > cta ? (T_total - cta + G - 1) / G : 0;
-        const int hdr_bytes = st.hdr_bytes;
-        const int strip = lane % S;
+        const int n_cta = st.tiles_div + (cta < st.tiles_rem ? 1 : 0);
+        const uint32_t hdr_bytes = (uint32_t)st.hdr_bytes;
+        const int strip = lane & (S - 1);
         const int plane = S > kGroups ? strip / kGroups : 0;
         const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)((st.B + kGap4Slack) * 128) +
                                  (uint32_t)(lane % kGroups) * (4u * NT);
         const uint32_t lt = (1u << lane) - 1u;
+        const bool last_stage = s == a.n_stages - 1;
 
         for (int k = warp; k < n_cta && !failed; k += kConsumerWarps) {
             const uint32_t q = qbase + (uint32_t)k;
             const uint32_t slot = q % kSlots;
+#ifdef SD2_TRACE
+            const long long tw0 = clock64();
+#endif
             if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
+#ifdef SD2_TRACE
+            if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] += clock64() - tw0;
+#endif
+            if (ctid == 0 && k == 0) SD2_STAMP(3);
             const int4 d = sh->desc[slot];
             const uint32_t tb = ring0 + (uint32_t)d.x;
-            const SMat& md = st.mat[d.y];
             const uint32_t cnt = lds_u16(tb + 2u * lane);
-            const uint32_t ct = lds_u32(tb + 64u);
-            const uint32_t cb = tb + (uint32_t)hdr_bytes;                 // code words
-            const uint32_t vb = cb + ((ct * 4u + 15u) & ~15u);            // values
+            const uint4 meta = lds_v4(tb + 64u);                           // n_chunks, min | max << 16, lane mask
+            const uint32_t cb = tb + hdr_bytes;                           // code words
+            const uint32_t vb = cb + ((meta.x * 4u + 15u) & ~15u);        // values
+            const uint32_t jmin = meta.y & 0xFFFFu, jmax = meta.y >> 16;
+            const uint32_t bal0 = meta.z;
+            const uint32_t n0 = __popc(bal0);
 
             float a0[NT], a1[NT];
 #pragma unroll
@@ -532,33 +603,26 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             uint32_t xb = xs_lane;
 
             // steps every populated lane takes: addresses advance by a constant
-            const uint32_t bal0 = __ballot_sync(0xFFFFFFFFu, cnt > 0);
-            const uint32_t n0 = __popc(bal0);
-            const uint32_t jmin = __reduce_min_sync(0xFFFFFFFFu, cnt > 0 ? cnt : 0xFFFFu);
-            const uint32_t jmax = __reduce_max_sync(0xFFFFFFFFu, cnt);
-            uint32_t j = 0;
-            if (bal0 != 0u) {
-                if (cnt > 0) {
-                    const uint32_t rank0 = __popc(bal0 & lt);
-                    uint32_t ca = cb + rank0 * 4u, va = vb + rank0 * 16u;
-                    uint32_t code = lds_u32(ca);
-                    uint4 v = lds_v4(va);
-                    for (uint32_t jj = 1; jj < jmin; ++jj) {
-                        ca += n0 * 4u;
-                        va += n0 * 16u;
-                        const uint32_t code_n = lds_u32(ca);
-                        const uint4 v_n = lds_v4(va);
-                        xb = chunk_fma<NT>(code, v, xb, a0, a1);
-                        code = code_n;
-                        v = v_n;
-                    }
+            if (cnt > 0) {
+                const uint32_t rank0 = __popc(bal0 & lt);
+                uint32_t ca = cb + rank0 * 4u, va = vb + rank0 * 16u;
+                uint32_t code = lds_u32(ca);
+                uint4 v = lds_v4(va);
+                for (uint32_t jj = 1; jj < jmin; ++jj) {
+                    ca += n0 * 4u;
+                    va += n0 * 16u;
+                    const uint32_t code_n = lds_u32(ca);
+                    const uint4 v_n = lds_v4(va);
                     xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                    code = code_n;
+                    v = v_n;
                 }
-                j = jmin;
+                xb = chunk_fma<NT>(code, v, xb, a0, a1);
             }
+            __syncwarp();
             // ragged tail: the set of lanes that still have a chunk shrinks step by step
-            uint32_t off = n0 * j;
-            for (; j < jmax; ++j) {
+            uint32_t off = n0 * jmin;
+            for (uint32_t j = jmin; j < jmax; ++j) {
                 const bool act = j < cnt;
                 const uint32_t bal = __ballot_sync(0xFFFFFFFFu, act);
                 if (act) {
@@ -578,15 +642,17 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 for (int dd = 1; dd < S; dd <<= 1) r[n] += __shfl_xor_sync(0xFFFFFFFFu, r[n], dd);
             }
             if (strip == 0) {
-                const uint32_t row = lds_u32(tb + 68u + 4u * (uint32_t)(lane / S));
+                const uint32_t row = lds_u32(tb + 80u + 4u * (uint32_t)(lane >> st.log2S));
                 if (row != 0xFFFFFFFFu) {
-                    void* yp = (s == a.n_stages - 1 && a.y_out && d.y == 0) ? a.y_out : md.y;
+                    const SMat& md = st.mat[d.y];
+                    void* yp = (last_stage && a.y_out && d.y == 0) ? a.y_out : md.y;
                     const size_t M = (size_t)md.M;
+                    const bool f32 = md.y_f32 != 0;
 #pragma unroll
                     for (int n = 0; n < NT; ++n) {
                         if (n < N) {
                             const size_t at = (size_t)(a.n0 + n) * M + row;
-                            if (md.y_f32) ((float*)yp)[at] = r[n];
+                            if (f32) ((float*)yp)[at] = r[n];
                             else ((uint16_t*)yp)[at] = f32_to_bf16_rne(r[n]);
                         }
                     }
@@ -596,8 +662,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             if (lane == 0) mbar_arrive(empty0 + 8 * slot);
         }
         qbase += (uint32_t)n_cta;
+        if (ctid == 0) SD2_STAMP(4);
         // everything this CTA wrote in the stage is visible before it arrives at the barrier
         named_bar_sync(1, kConsumerThreads);
+        if (ctid == 0) SD2_STAMP(5);
         if (s + 1 < a.n_stages && ctid == 0) {
             __threadfence();
             atomicAdd(a.gbar, 1u);

@@ -114,7 +114,7 @@ def _gap4_bytes(mask):
     row_chunks = np.array([sum((_gap4_entries(mask[m, s * B:(s + 1) * B]) + 7) // 8 for s in range(S)) for m in range(M)])
     order = np.argsort(-row_chunks, kind="stable")
     T = (M + R - 1) // R
-    hdr = (64 + 4 + 4 * R + 15) // 16 * 16
+    hdr = (80 + 4 * R + 15) // 16 * 16
     total = 4 * (T + 1)
     for t in range(T):
         ct = int(row_chunks[order[t * R:(t + 1) * R]].sum())
