@@ -156,6 +156,27 @@ sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* by
 /* Byte offsets of q, k, v, hdn, g, u, t inside the workspace (offsets[7]). */
 sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets);
 
+/* sd2_block_step for callers that must not allocate device memory and have no workspace
+ * to hand over.  (No counterpart in the paper: it exists for hosts such as a serving loop
+ * that runs under a fixed memory plan, a plugin inside another runtime's allocator, or code
+ * on a path where cudaMalloc's implicit device synchronisation is not acceptable.)  The
+ * block's intermediates (q, k, v, hdn, g, u, t) and the grid-barrier words live in an array
+ * built into the library image: 1 MiB + 256 bytes that every GPU which loads the library
+ * keeps until the process exits.  Same result as sd2_block_step, same stub glue; x: device
+ * bf16 [N*hidden], y: device [N*M_down] in h[6]'s y_dtype, 0 <= N <= 64.
+ *  - all seven weights must be GAP4 (SD2_ERR_UNSUPPORTED otherwise), live on the current device;
+ *  - sd2_block_workspace_bytes(h, N) must not exceed 1 MiB, else SD2_ERR_UNSUPPORTED and
+ *    nothing is launched (e.g. a Llama-3.2-3B block fits up to N = 16);
+ *  - the first call on each device looks up the array's device address; make that call
+ *    before any stream capture;
+ *  - the call itself enqueues a 256-byte clear of the barrier words and then the launches;
+ *    it calls no allocation routine;
+ *  - every call uses the same array, and the intermediates of the previous call stay in it
+ *    until overwritten: two calls that overlap on the GPU (different streams, no ordering)
+ *    race on it.  Keep calls on one stream or order them with events.  The intermediates
+ *    cannot be read back through this entry point. */
+sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, int64_t N, void* cuda_stream);
+
 /* ---- a whole drafter: L blocks chained, one launch per panel of activation rows --------- */
 
 /* h: 7 * L live GAP4 handles on the current device, block by block in the order q,k,v,o,gate,

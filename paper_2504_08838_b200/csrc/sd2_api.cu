@@ -824,6 +824,62 @@ sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N
     return run_group(h + 6, 1, nullptr, g, u, t, y_d, N, false, s);
 }
 
+// ---- block step without allocation -----------------------------------------------------
+
+// Scratch of sd2_block_step_static: grid-barrier words (first 256 bytes), then the block's
+// intermediates.  It lives in the library image, so every GPU that loads the library holds
+// it until the process exits.
+constexpr int64_t kStaticWorkspaceMax = 1 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[256 + kStaticWorkspaceMax];
+
+namespace {
+unsigned char* g_static_ptr[kMaxDevices];   // device address of g_static_scratch, per device
+}
+
+sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, int64_t N, void* cuda_stream)
+{
+    if (!x || !y) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
+    BlockDims d;
+    sd2_status st = block_dims(h, &d);
+    if (st != SD2_OK) return st;
+    if (N == 0) return SD2_OK;
+    for (int i = 0; i < 7; ++i)
+        if (h[i]->format != SD2_FORMAT_GAP4) return SD2_ERR_UNSUPPORTED;
+    int64_t off[8];
+    block_layout(h, d, N, off);
+    if (off[7] > kStaticWorkspaceMax) return SD2_ERR_UNSUPPORTED;   // intermediates do not fit the built-in scratch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices || !g_dev[dev].ready) return SD2_ERR_INVALID_ARG;   // live handles imply a ready device
+    for (int i = 0; i < 7; ++i)
+        if (h[i]->device != dev) return SD2_ERR_INVALID_ARG;
+    {
+        // once per device, with that device current: the array's name is only a host-side stand-in
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!g_static_ptr[dev]) {
+            unsigned char* p = nullptr;
+            if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return SD2_ERR_CUDA; }
+            g_static_ptr[dev] = p;
+        }
+    }
+    unsigned char* base = g_static_ptr[dev];
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // the barrier words must start at zero whatever the last call left behind
+    if (cudaMemsetAsync(base, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    char* ws = (char*)base + 256;
+    SArgs a;
+    std::memset(&a, 0, sizeof a);
+    ProgramNeeds needs;
+    a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, (uint16_t*)(ws + off[0]), (uint16_t*)(ws + off[1]),
+                                     (uint16_t*)(ws + off[2]), (uint16_t*)(ws + off[3]), (uint16_t*)(ws + off[4]),
+                                     (uint16_t*)(ws + off[5]), (uint16_t*)(ws + off[6]), y, false, &needs, g_dev[dev].sms);
+    a.err = g_dev[dev].err_word;
+    a.wait_cycles = wait_budget(dev);
+    a.gbar = (unsigned int*)base;
+    return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, g_dev[dev].sms, s);
+}
+
 // ---- whole drafter ---------------------------------------------------------------------
 
 sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2_drafter* out)
