@@ -195,8 +195,12 @@ def measured_peak():
 
 def ncu_traffic_ratio():
     """DRAM bytes per algorithmic byte of the dominant kernel, from the committed ncu summary."""
+    import re
+    name = "stream_kernel_nt1_llama1b_2blocks.md"
     try:
-        return json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json")))
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+        m = re.search(r"dram_bytes_per_algorithmic_byte = ([0-9.]+)", text)
+        return {"dram_bytes_per_algorithmic_byte": float(m.group(1)), "source": "profiles/" + name}
     except Exception:
         return None
 
