@@ -42,6 +42,17 @@ __device__ __forceinline__ uint16_t silu_mul_bits(uint16_t g, uint16_t u)
     return f32_to_bf16_rne(__fdividef(a, 1.f + __expf(-a)) * bf16_to_f32(u));
 }
 
+// bf16 pair {lo, hi} of silu(g) * u for a pair of gates and ups, one rounding instruction for both
+__device__ __forceinline__ uint32_t silu_mul_pair(uint32_t gpair, uint32_t upair)
+{
+    const float g0 = bf16_lo(gpair), g1 = bf16_hi(gpair);
+    const float t0 = __fdividef(g0, 1.f + __expf(-g0)) * bf16_lo(upair);
+    const float t1 = __fdividef(g1, 1.f + __expf(-g1)) * bf16_hi(upair);
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(t1), "f"(t0));
+    return d;
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll
@@ -72,11 +83,18 @@ __device__ __forceinline__ float warp_sum(float v)
 // Every wait (ring barriers, grid barrier) is bounded by a cycle budget: when it runs out
 // the CTA raises the error word and winds down instead of hanging.
 
-constexpr int kConsumerWarps = 16;
+#ifndef SD2_CONSUMER_WARPS
+#define SD2_CONSUMER_WARPS 16
+#endif
+constexpr int kConsumerWarps = SD2_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
 constexpr int kSlots = 32;                               // tiles in flight per CTA, at most
 constexpr int kMaxStagesInline = 8;
+#ifndef SD2_RELEASE_BATCH
+#define SD2_RELEASE_BATCH 1
+#endif
+constexpr int kReleaseBatch = SD2_RELEASE_BATCH;   // tiles the producer waits for when the ring is full
 
 struct SMat {
     const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
@@ -153,6 +171,20 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// non-blocking: has the phase of this parity completed?
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
@@ -362,11 +394,7 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                         const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w}, uu[4] = {uv.x, uv.y, uv.z, uv.w};
                         uint32_t w[4];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const uint32_t lo = silu_mul_bits((uint16_t)(gg[q] & 0xFFFFu), (uint16_t)(uu[q] & 0xFFFFu));
-                            const uint32_t hi = silu_mul_bits((uint16_t)(gg[q] >> 16), (uint16_t)(uu[q] >> 16));
-                            w[q] = lo | (hi << 16);
-                        }
+                        for (int q = 0; q < 4; ++q) w[q] = silu_mul_pair(gg[q], uu[q]);
                         v = make_uint4(w[0], w[1], w[2], w[3]);
                         if (pub) ((uint4*)(t_out + (size_t)n * K))[i] = v;
                     }
@@ -465,40 +493,58 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     src = (unsigned long long)(st->mat[mi].stream + (size_t)o0 * 16);
                 }
                 const int cnt = min(32, n_cta - k0);
-                for (int i = 0; i < cnt && ok; ++i) {
-                    const uint32_t b = __shfl_sync(0xFFFFFFFFu, bytes, i);
-                    const unsigned long long sp = __shfl_sync(0xFFFFFFFFu, src, i);
-                    const int m_i = __shfl_sync(0xFFFFFFFFu, mi, i);
-                    const int t_i = __shfl_sync(0xFFFFFFFFu, ti, i);
-                    // find room for b contiguous bytes and a free slot (all lanes run this alike)
-                    while (true) {
+                // One thread can start only about three bulk copies per microsecond, whatever
+                // their size, so tiles are issued in groups: room is found for as many of the
+                // batch's tiles as fit right now (alike in all lanes), then every lane that
+                // got a place issues its own tile's copy in the same instruction.
+                int i = 0;
+                while (i < cnt && ok) {
+                    const int first = i;
+                    uint32_t my_head = 0, my_slot = 0;
+                    bool mine = false;
+                    while (i < cnt) {
+                        const uint32_t b = __shfl_sync(0xFFFFFFFFu, bytes, i);
                         const uint32_t outstanding = q - oldest;
+                        uint32_t start;
                         bool fits;
                         if (outstanding == 0) {
                             head = tail = 0;
+                            start = 0;
                             fits = true;
                         } else if (head >= tail) {
-                            if (head + b <= ring_bytes) fits = true;
-                            else if (b < tail) { head = 0; fits = true; }
-                            else fits = false;
+                            if (head + b <= ring_bytes) { start = head; fits = true; }
+                            else if (b < tail) { start = 0; fits = true; }
+                            else { start = 0; fits = false; }
                         } else {
+                            start = head;
                             fits = head + b < tail;
                         }
-                        if (fits && outstanding < (uint32_t)kSlots) break;
+                        if (!fits || outstanding >= (uint32_t)kSlots) break;
+                        if (lane == i) { my_head = start; my_slot = q % kSlots; mine = true; }
+                        head = start + b;
+                        ++q;
+                        ++i;
+                    }
+                    if (i > first) {
+                        if (mine) {
+                            sh->desc[my_slot] = make_int4((int)my_head, mi, ti, (int)bytes);
+                            mbar_expect_tx(full0 + 8 * my_slot, bytes);
+                            bulk_g2s(ring0 + my_head, (const void*)src, bytes, full0 + 8 * my_slot);
+                        }
+                        __syncwarp();
+                    } else {
+                        // no room: wait until the oldest tile in the ring has been consumed
                         if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
                         ++oldest;
+                        // wait for a few more when the ring is far from empty, and take along every
+                        // further tile that is already done: the more room, the more copies start together
+                        for (int r = 1; r < kReleaseBatch && ok && q - oldest > (uint32_t)kConsumerWarps / 2; ++r) {
+                            if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
+                            ++oldest;
+                        }
+                        while (oldest != q && mbar_test_wait(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u)) ++oldest;
                         tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
                     }
-                    if (!ok) break;
-                    const uint32_t slot = q % kSlots;
-                    if (lane == 0) {
-                        sh->desc[slot] = make_int4((int)head, m_i, t_i, (int)b);
-                        mbar_expect_tx(full0 + 8 * slot, b);
-                        bulk_g2s(ring0 + head, (const void*)sp, b, full0 + 8 * slot);
-                    }
-                    __syncwarp();
-                    head += b;
-                    ++q;
                 }
             }
             if (lane == 0) SD2_STAMP(6);
