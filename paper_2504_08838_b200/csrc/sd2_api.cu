@@ -40,6 +40,9 @@ struct sd2_drafter_s {
     uint8_t* d_ws;
     SStage* d_stages;
     unsigned int* d_gbar;
+    uint32_t* d_tags;          // tagged copies of q, hdn, g, u and the block output of every block (or NULL)
+    int64_t tags_bytes;
+    int64_t last_n;            // rows of the previous step: a change clears d_tags (stale tags of other rows)
     int K_max, max_tile;       // what decides the shared-memory split
     int xs_need[3];            // bytes of staged activations at panel widths 1, 2, 4
 };
@@ -341,7 +344,8 @@ void set_stage_grid(SStage& st, int grid)
 
 // Fills one stage from `count` GAP4 handles of equal K and S, to be run by `grid` CTAs.
 void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
-                uint16_t* t_out, void* const* Y, bool y_force_bf16, int grid)
+                uint16_t* t_out, void* const* Y, bool y_force_bf16, int grid, uint32_t* const* YT = nullptr,
+                int tagged_in = 0)
 {
     std::memset(&st, 0, sizeof st);
     st.count = count;
@@ -361,12 +365,14 @@ void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, 
         m.tile_off = hs[i]->d_sec0;
         m.stream = (const unsigned char*)hs[i]->d_sec1;
         m.y = Y[i];
+        m.yt = YT ? YT[i] : nullptr;
         m.M = (int)hs[i]->M;
         m.T = hs[i]->T;
         m.y_f32 = (!y_force_bf16 && hs[i]->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
         T += hs[i]->T;
     }
     st.T_total = T;
+    st.tagged_in = tagged_in;
     set_stage_grid(st, grid);
 }
 
@@ -524,36 +530,57 @@ void block_layout(const sd2_handle* h, const BlockDims& d, int64_t N, int64_t of
     off[7] = o;
 }
 
+// Tagged 32-bit copies of a block's activations (value << 16 | stage tag) through which the
+// stages of a tagged program hand their outputs to the next stage without a grid barrier.
+struct BlockTags {
+    const uint32_t* x_t;   // the block's input as tagged words, or NULL (plain bf16 input)
+    uint32_t *q_t, *hdn_t, *g_t, *u_t, *out_t;   // out_t NULL: the block's output is not handed on
+    uint32_t* t_t;                               // tagged t = silu(g) * u, one slice per CTA
+};
+
 // Appends the stages of one block (h[0..6] = q,k,v,o,gate,up,down) to `stages`.  Weights of a
 // group that do not share a strip geometry get a stage each.  Returns the number appended.
 int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
                         uint16_t* hdn, uint16_t* g, uint16_t* u, uint16_t* t, void* y, bool y_force_bf16,
-                        ProgramNeeds* needs, int grid)
+                        ProgramNeeds* needs, int grid, const BlockTags* tg = nullptr)
 {
     int n = 0;
     auto group = [&](const sd2_handle* hs, int count, const uint16_t* xin, const uint16_t* gg, const uint16_t* uu,
-                     uint16_t* tt, void* const* Y, bool force) {
+                     uint16_t* tt, void* const* Y, bool force, uint32_t* const* YT, int tin) {
         bool same = true;
         for (int i = 1; i < count; ++i)
             if (hs[i]->S != hs[0]->S) same = false;
         if (same) {
-            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force, grid);
+            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force, grid, YT, tin);
             needs->add(hs, count);
         } else {
             for (int i = 0; i < count; ++i) {
-                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force, grid);
+                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force, grid, YT ? YT + i : nullptr, tin);
                 needs->add(hs + i, 1);
             }
         }
     };
     void* y_qkv[3] = {q, k, v};
-    group(h + 0, 3, x, nullptr, nullptr, nullptr, y_qkv, true);
     void* y_o[1] = {hdn};
-    group(h + 3, 1, q, nullptr, nullptr, nullptr, y_o, true);
     void* y_gu[2] = {g, u};
-    group(h + 4, 2, hdn, nullptr, nullptr, nullptr, y_gu, true);
     void* y_d[1] = {y};
-    group(h + 6, 1, nullptr, g, u, t, y_d, y_force_bf16);
+    if (!tg) {
+        group(h + 0, 3, x, nullptr, nullptr, nullptr, y_qkv, true, nullptr, 0);
+        group(h + 3, 1, q, nullptr, nullptr, nullptr, y_o, true, nullptr, 0);
+        group(h + 4, 2, hdn, nullptr, nullptr, nullptr, y_gu, true, nullptr, 0);
+        group(h + 6, 1, nullptr, g, u, t, y_d, y_force_bf16, nullptr, 0);
+    } else {
+        uint32_t* t_qkv[3] = {tg->q_t, nullptr, nullptr};
+        uint32_t* t_o[1] = {tg->hdn_t};
+        uint32_t* t_gu[2] = {tg->g_t, tg->u_t};
+        uint32_t* t_d[1] = {tg->out_t};
+        group(h + 0, 3, tg->x_t ? (const uint16_t*)tg->x_t : x, nullptr, nullptr, nullptr, y_qkv, true, t_qkv, tg->x_t ? 1 : 0);
+        group(h + 3, 1, (const uint16_t*)tg->q_t, nullptr, nullptr, nullptr, y_o, true, t_o, 1);
+        group(h + 4, 2, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_gu, true, t_gu, 1);
+        const int before = n;
+        group(h + 6, 1, nullptr, (const uint16_t*)tg->g_t, (const uint16_t*)tg->u_t, t, y_d, y_force_bf16, t_d, 1);
+        for (int i = before; i < n; ++i) stages[i].tt = tg->t_t;
+    }
     return n;   // at most 7
 }
 
@@ -727,7 +754,7 @@ sd2_status sd2_stream_check(void* cuda_stream)
         {
             std::lock_guard<std::mutex> lk(g_mu);
             for (sd2_drafter d : g_live_drafters)
-                if (d->device == dev) cudaMemset(d->d_gbar, 0, 256);
+                if (d->device == dev) { cudaMemset(d->d_gbar, 0, 256); d->last_n = -1; }
         }
         cudaGetLastError();
         return SD2_ERR_TIMEOUT;
@@ -925,6 +952,25 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
     std::vector<SStage> stages((size_t)L * 7);
     ProgramNeeds needs;
     bool ok = cudaMalloc((void**)&d->d_ws, (size_t)o) == cudaSuccess && cudaMemset(d->d_ws, 0, (size_t)o) == cudaSuccess;
+    // Tagged hand-off (stage tags are 8 bits wide): per block q, hdn, g, u, out as 32-bit words
+    const bool tagged = 7 * L <= 254;
+    std::vector<int64_t> tag_off((size_t)L * 6 + 1, 0);
+    d->d_tags = nullptr;
+    d->tags_bytes = 0;
+    d->last_n = -1;
+    if (tagged) {
+        int64_t to = 0;
+        for (int b = 0; b < L; ++b) {
+            const BlockDims& bd = dims[(size_t)b];
+            const int64_t w[6] = {bd.q_out, h[7 * b + 3]->M, bd.inter, bd.inter, bd.out, bd.inter};
+            for (int i = 0; i < 6; ++i) {
+                tag_off[(size_t)b * 6 + i] = to;
+                to = a256(to + 4 * n_max * w[i]);
+            }
+        }
+        d->tags_bytes = to;
+        ok = ok && cudaMalloc((void**)&d->d_tags, (size_t)to) == cudaSuccess && cudaMemset(d->d_tags, 0, (size_t)to) == cudaSuccess;
+    }
     int n = 0;
     if (ok) {
         for (int b = 0; b < L; ++b) {
@@ -932,9 +978,22 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
             const int64_t* wo = &d->ws_off[(size_t)b * 8];
             const uint16_t* xin = b == 0 ? nullptr : (const uint16_t*)(base + d->ws_off[(size_t)(b - 1) * 8 + 7]);
             void* yout = base + wo[7];
+            BlockTags tg;
+            if (tagged) {
+                uint8_t* tb = (uint8_t*)d->d_tags;
+                const int64_t* to = &tag_off[(size_t)b * 6];
+                tg.x_t = b == 0 ? nullptr : (const uint32_t*)(tb + tag_off[(size_t)(b - 1) * 6 + 4]);
+                tg.q_t = (uint32_t*)(tb + to[0]);
+                tg.hdn_t = (uint32_t*)(tb + to[1]);
+                tg.g_t = (uint32_t*)(tb + to[2]);
+                tg.u_t = (uint32_t*)(tb + to[3]);
+                tg.out_t = b + 1 < L ? (uint32_t*)(tb + to[4]) : nullptr;
+                tg.t_t = (uint32_t*)(tb + to[5]);
+            }
             n += append_block_stages(stages.data() + n, h + 7 * b, xin, (uint16_t*)(base + wo[0]), (uint16_t*)(base + wo[1]),
                                      (uint16_t*)(base + wo[2]), (uint16_t*)(base + wo[3]), (uint16_t*)(base + wo[4]),
-                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs, g_dev[dev].sms);
+                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs, g_dev[dev].sms,
+                                     tagged ? &tg : nullptr);
         }
         d->n_stages = n;
         ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
@@ -942,13 +1001,13 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
              cudaMalloc((void**)&d->d_gbar, 256) == cudaSuccess && cudaMemset(d->d_gbar, 0, 256) == cudaSuccess;
     }
     if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
-        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar);
+        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar); cudaFree(d->d_tags);
         delete d;
         return SD2_ERR_UNSUPPORTED;
     }
     if (!ok) {
         cudaGetLastError();
-        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar);
+        cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar); cudaFree(d->d_tags);
         cudaGetLastError();
         delete d;
         return SD2_ERR_ALLOC;
@@ -982,6 +1041,16 @@ sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, vo
     a.gbar = d->d_gbar;
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
+    if (d->d_tags) {
+        a.tagged = 1;
+        a.seq = d->d_gbar + 48;   // third cache-line-sized slot of the 256-byte block
+        // Only rows [0, N) are written and polled in a step.  When N changes, rows written long ago
+        // could carry a tag that comes round again (tags are 16 bits): start from clean words.
+        if (d->last_n != N) {
+            if (cudaMemsetAsync(d->d_tags, 0, (size_t)d->tags_bytes, (cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+            d->last_n = N;
+        }
+    }
     // Rows of X are independent through the whole drafter: panels run one after another.  Row n
     // of every buffer starts at n * width, whatever N is.
     return run_panels(a, N, d->xs_need, d->K_max, d->max_tile, g_dev[dev].sms, (cudaStream_t)cuda_stream);
@@ -1006,6 +1075,7 @@ sd2_status sd2_drafter_free(sd2_drafter d)
     if (cudaFree(d->d_ws) != cudaSuccess) st = SD2_ERR_CUDA;
     if (cudaFree(d->d_stages) != cudaSuccess) st = SD2_ERR_CUDA;
     if (cudaFree(d->d_gbar) != cudaSuccess) st = SD2_ERR_CUDA;
+    if (d->d_tags && cudaFree(d->d_tags) != cudaSuccess) st = SD2_ERR_CUDA;
     cudaGetLastError();
     delete d;
     return st;

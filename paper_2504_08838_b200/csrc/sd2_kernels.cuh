@@ -99,7 +99,8 @@ constexpr int kReleaseBatch = SD2_RELEASE_BATCH;   // tiles the producer waits f
 struct SMat {
     const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
     const unsigned char* stream;   // tile records
-    void* y;                       // [N * M]
+    void* y;                       // [N * M], may be NULL when yt is set
+    uint32_t* yt;                  // [N * M] tagged words (bf16 << 16 | stage tag) for the next stage, or NULL
     int M;
     int T;
     int y_f32;                     // 1: fp32 output, 0: bf16
@@ -111,7 +112,8 @@ struct SStage {
     const uint16_t* x;     // [N * K] bf16, or NULL in glue mode
     const uint16_t* g;     // glue mode: t = bf16(silu(g) * u) is the activation
     const uint16_t* u;
-    uint16_t* t_out;       // glue mode: CTA 0 also writes t here (may be NULL)
+    uint16_t* t_out;       // glue mode: t is also written here as plain bf16 (may be NULL)
+    uint32_t* tt;          // tagged glue mode: tagged copy of t, computed once, a slice per CTA (or NULL)
     int count;             // weights in the stage
     int K;
     int S;                 // strips; equal for all weights of a stage
@@ -121,7 +123,8 @@ struct SStage {
     int log2S;
     int tiles_div;         // T_total / grid size: CTA c runs tiles_div + (c < tiles_rem) tiles
     int tiles_rem;         // T_total % grid size
-    int reserved[3];
+    int tagged_in;         // x / g / u point at tagged 32-bit words written by the previous stage
+    int reserved[4];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
@@ -139,6 +142,8 @@ struct SArgs {
     int xs_bytes;                   // shared memory for the transposed activations
     int xlin_bytes;                 // shared memory for one linear activation row
     int ring_bytes;
+    int tagged;                     // 1: stages hand activations over as tagged words, no grid barrier
+    unsigned int* seq;              // tagged programs: launch counter (device word), bumped by the last CTA out
     long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
 };
 
@@ -291,7 +296,8 @@ struct StreamShared {
     unsigned long long empty[kSlots];  // mbarriers: tile consumed
     int abort_flag;                    // any warp: a bounded wait ran out
     int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
-    int pad[2];
+    unsigned int tag_base;             // tagged programs: (launch counter & 0xFF) << 8
+    int pad[1];
 };
 
 struct WaitCtx {
@@ -370,9 +376,118 @@ __device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uin
 // strips repeat across the groups), zero for c >= B, strip * B + c >= K or n >= N.
 // Row by row through `xlin` (bf16, linear) so that global memory is read with 128-bit loads.
 // x_src, g, u, t_out already point at the launch's first activation row.
+// One 128-bit load of four tagged words, repeated until all four carry `tag` (their producers,
+// on other SMs, have stored them) or the wait budget runs out.  Value and tag share a 32-bit
+// word, so a word that shows the tag also shows its value: no fence is needed.
+__device__ __forceinline__ uint4 poll_tagged(const uint32_t* p, uint32_t tag, const WaitCtx& w)
+{
+    uint4 v;
+    long long t0 = 0;
+    uint32_t it = 0;
+    while (true) {
+        asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+        if (((v.x ^ tag) & 0xFFFFu) == 0 && ((v.y ^ tag) & 0xFFFFu) == 0 && ((v.z ^ tag) & 0xFFFFu) == 0 && ((v.w ^ tag) & 0xFFFFu) == 0) break;
+        if (it == 0) t0 = clock64();
+        if ((++it & 7u) == 0u) {
+            if (*w.abort_flag) break;
+            if (clock64() - t0 > w.budget) { *w.abort_flag = 1; break; }
+        }
+    }
+    return v;
+}
+__device__ __forceinline__ uint32_t poll_tagged1(const uint32_t* p, uint32_t tag, const WaitCtx& w)
+{
+    uint32_t v;
+    long long t0 = 0;
+    uint32_t it = 0;
+    while (true) {
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (((v ^ tag) & 0xFFFFu) == 0) break;
+        if (it == 0) t0 = clock64();
+        if ((++it & 7u) == 0u) {
+            if (*w.abort_flag) break;
+            if (clock64() - t0 > w.budget) { *w.abort_flag = 1; break; }
+        }
+    }
+    return v;
+}
+
+// Linear phase of the staging for tagged inputs: xlin[k] = bf16 of word k of row n (or of
+// silu(g) * u in glue mode), waiting for each word's tag.
+__device__ __forceinline__ void stage_linear_tagged(int K, const uint32_t* x, const uint32_t* g, const uint32_t* u,
+                                                    uint16_t* t_out, bool pub, uint16_t* xlin, uint32_t tag, const WaitCtx& w, int ctid)
+{
+    const bool glue = x == nullptr;
+    const bool vec = (K % 4 == 0) && ((((uintptr_t)x | (uintptr_t)g | (uintptr_t)u) & 15) == 0) && ((((uintptr_t)t_out) & 7) == 0);
+    if (vec) {
+        for (int i = ctid; i < (K >> 2); i += kConsumerThreads) {
+            uint32_t lo, hi;
+            if (!glue) {
+                const uint4 v = poll_tagged(x + 4 * i, tag, w);
+                lo = __byte_perm(v.x, v.y, 0x7632);
+                hi = __byte_perm(v.z, v.w, 0x7632);
+            } else {
+                const uint4 gv = poll_tagged(g + 4 * i, tag, w);
+                const uint4 uv = poll_tagged(u + 4 * i, tag, w);
+                lo = silu_mul_pair(__byte_perm(gv.x, gv.y, 0x7632), __byte_perm(uv.x, uv.y, 0x7632));
+                hi = silu_mul_pair(__byte_perm(gv.z, gv.w, 0x7632), __byte_perm(uv.z, uv.w, 0x7632));
+                if (pub) ((uint2*)t_out)[i] = make_uint2(lo, hi);
+            }
+            ((uint2*)xlin)[i] = make_uint2(lo, hi);
+        }
+    } else {
+        for (int i = ctid; i < K; i += kConsumerThreads) {
+            uint16_t v;
+            if (!glue) {
+                v = (uint16_t)(poll_tagged1(x + i, tag, w) >> 16);
+            } else {
+                v = silu_mul_bits((uint16_t)(poll_tagged1(g + i, tag, w) >> 16), (uint16_t)(poll_tagged1(u + i, tag, w) >> 16));
+                if (pub) t_out[i] = v;
+            }
+            xlin[i] = v;
+        }
+    }
+}
+
+// Tagged glue, first half: t = bf16(silu(g) * u) is computed once per launch instead of once
+// per CTA.  CTA c takes the c-th slice of every row, waits for exactly the g and u words it
+// needs, and publishes its slice of t as tagged words (and as plain bf16 if asked); every CTA
+// then stages the whole of t like any tagged activation.
+__device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g, const uint32_t* u, uint32_t* tt,
+                                                uint16_t* t_out, uint32_t tag, const WaitCtx& w, int ctid)
+{
+    const int G = gridDim.x;
+    const int slice = ((K + G - 1) / G + 3) & ~3;
+    const int k0 = (int)blockIdx.x * slice;
+    const bool vec = (K % 4 == 0) && ((((uintptr_t)g | (uintptr_t)u | (uintptr_t)tt) & 15) == 0);
+    for (int i = ctid; i < N * slice; i += kConsumerThreads) {
+        const int n = i / slice, k = k0 + (i - n * slice);
+        if (k >= K) continue;
+        const size_t at = (size_t)n * K + k;
+        if (vec) {
+            if (k & 3) continue;   // one thread per group of four
+            const uint4 gv = poll_tagged(g + at, tag, w);
+            const uint4 uv = poll_tagged(u + at, tag, w);
+            const uint32_t lo = silu_mul_pair(__byte_perm(gv.x, gv.y, 0x7632), __byte_perm(uv.x, uv.y, 0x7632));
+            const uint32_t hi = silu_mul_pair(__byte_perm(gv.z, gv.w, 0x7632), __byte_perm(uv.z, uv.w, 0x7632));
+            *(uint4*)(tt + at) = make_uint4((lo << 16) | tag, (lo & 0xFFFF0000u) | tag, (hi << 16) | tag, (hi & 0xFFFF0000u) | tag);
+            if (t_out) {
+                t_out[at] = (uint16_t)lo; t_out[at + 1] = (uint16_t)(lo >> 16);
+                t_out[at + 2] = (uint16_t)hi; t_out[at + 3] = (uint16_t)(hi >> 16);
+            }
+        } else {
+            const uint16_t v = silu_mul_bits((uint16_t)(poll_tagged1(g + at, tag, w) >> 16), (uint16_t)(poll_tagged1(u + at, tag, w) >> 16));
+            tt[at] = ((uint32_t)v << 16) | tag;
+            if (t_out) t_out[at] = v;
+        }
+    }
+}
+
+// `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged).
 template <int NT>
 __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
-                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int ctid)
+                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int ctid,
+                                        uint32_t tag, const WaitCtx& wc)
 {
     constexpr int kGroups = 32 / NT;
     const int K = st.K, S = st.S, B = st.B;
@@ -382,7 +497,11 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
     const bool vec = (K % 8 == 0) && ((((uintptr_t)x_src | (uintptr_t)g | (uintptr_t)u | (uintptr_t)t_out) & 15) == 0);
     const bool pub = glue && t_out && blockIdx.x == 0;
     for (int n = 0; n < NT; ++n) {
-        if (n < N) {
+        if (n < N && tag != 0u) {
+            stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
+                                g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
+                                t_out ? t_out + (size_t)n * K : nullptr, pub, xlin, tag, wc, ctid);
+        } else if (n < N) {
             if (vec) {
                 for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
                     uint4 v;
@@ -577,11 +696,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const uint32_t* src = (const uint32_t*)(a.ext ? a.ext : &a.inl[0]);
         for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[0])[i] = src[i];
     }
+    if (ctid == 0) sh->tag_base = a.tagged ? ((*(volatile unsigned int*)a.seq) & 0xFFu) << 8 : 0u;
     int s = 0;
     for (; s < a.n_stages; ++s) {
         if (ctid == 0) {
             SD2_STAMP(0);
-            if (s > 0) {
+            if (s > 0 && !a.tagged) {
                 // grid barrier: every CTA has written the previous stage's outputs
                 const unsigned int target = (unsigned int)s * (unsigned int)G;
                 const long long t0 = clock64();
@@ -604,8 +724,20 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const int K = st.K;
         const uint16_t* x_src = (s == 0 && a.x_in) ? a.x_in : st.x;
         const size_t xoff = (size_t)a.n0 * K;
-        stage_x<NT>(st, N, x_src ? x_src + xoff : nullptr, st.g ? st.g + xoff : nullptr, st.u ? st.u + xoff : nullptr,
-                    st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid);
+        // tagged inputs are 32-bit words: twice the stride of bf16; stage s reads what stage s - 1 tagged
+        const bool tin = a.tagged && st.tagged_in && !(s == 0 && a.x_in);
+        const size_t xw = tin ? 2 * xoff : xoff;
+        const uint32_t tag_in = tin ? (sh->tag_base | (uint32_t)s) : 0u;
+        const uint32_t tag_out = sh->tag_base | (uint32_t)(s + 1);
+        if (tin && !x_src && st.tt) {
+            // glue: this CTA's share of t first, then all of t like any tagged activation
+            publish_t_slice(K, N, (const uint32_t*)st.g + xoff, (const uint32_t*)st.u + xoff, st.tt + xoff,
+                            st.t_out ? st.t_out + xoff : nullptr, tag_in, wc, ctid);
+            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, ctid, tag_in, wc);
+        } else {
+            stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
+                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid, tag_in, wc);
+        }
         if (ctid == 0) SD2_STAMP(2);
         if (warp == 1 && s + 1 < a.n_stages) {
             const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);
@@ -694,12 +826,20 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     void* yp = (last_stage && a.y_out && d.y == 0) ? a.y_out : md.y;
                     const size_t M = (size_t)md.M;
                     const bool f32 = md.y_f32 != 0;
+                    uint32_t* yt = a.tagged ? md.yt : nullptr;
 #pragma unroll
                     for (int n = 0; n < NT; ++n) {
                         if (n < N) {
                             const size_t at = (size_t)(a.n0 + n) * M + row;
-                            if (f32) ((float*)yp)[at] = r[n];
-                            else ((uint16_t*)yp)[at] = f32_to_bf16_rne(r[n]);
+                            if (yt) {   // value and tag in one word: the next stage polls it
+                                const uint32_t bits = f32_to_bf16_rne(r[n]);
+                                yt[at] = (bits << 16) | tag_out;
+                                if (yp) ((uint16_t*)yp)[at] = (uint16_t)bits;
+                            } else if (f32) {
+                                ((float*)yp)[at] = r[n];
+                            } else {
+                                ((uint16_t*)yp)[at] = f32_to_bf16_rne(r[n]);
+                            }
                         }
                     }
                 }
@@ -712,7 +852,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         // everything this CTA wrote in the stage is visible before it arrives at the barrier
         named_bar_sync(1, kConsumerThreads);
         if (ctid == 0) SD2_STAMP(5);
-        if (s + 1 < a.n_stages && ctid == 0) {
+        if (s + 1 < a.n_stages && ctid == 0 && !a.tagged) {
             __threadfence();
             atomicAdd(a.gbar, 1u);
         }
@@ -727,6 +867,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         if (prev == (unsigned int)G - 1u) {
             atomicExch(a.gbar, 0u);
             atomicExch(a.gbar + 32, 0u);
+            if (a.tagged) atomicAdd(a.seq, 1u);   // the next launch tags its words differently
         }
     }
 }
