@@ -89,7 +89,7 @@ __device__ __forceinline__ float warp_sum(float v)
 constexpr int kConsumerWarps = SD2_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
-constexpr int kSlots = 32;                               // tiles in flight per CTA, at most
+constexpr int kSlots = 64;                               // tiles in flight per CTA, at most
 constexpr int kMaxStagesInline = 8;
 #ifndef SD2_RELEASE_BATCH
 #define SD2_RELEASE_BATCH 1
@@ -148,9 +148,12 @@ struct SArgs {
 };
 
 #ifdef SD2_TRACE
+// per-tile stamps of CTA 0 (issue, wait begin, start, end), after the per-stage stamps
+#define SD2_TILE_STAMP(q, slot) do { if (a.trace && cta == 0 && (q) < 4096u) a.trace[(size_t)gridDim.x * a.n_stages * 8 + (size_t)(q) * 4 + (slot)] = clock64(); } while (0)
 #define SD2_STAMP(slot) do { if (a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + (slot)] = clock64(); } while (0)
 #else
 #define SD2_STAMP(slot) do { } while (0)
+#define SD2_TILE_STAMP(q, slot) do { } while (0)
 #endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -639,7 +642,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                             fits = head + b < tail;
                         }
                         if (!fits || outstanding >= (uint32_t)kSlots) break;
-                        if (lane == i) { my_head = start; my_slot = q % kSlots; mine = true; }
+                        if (lane == i) { my_head = start; my_slot = q % kSlots; mine = true; SD2_TILE_STAMP(q, 0); }
                         head = start + b;
                         ++q;
                         ++i;
@@ -759,12 +762,14 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             const uint32_t slot = q % kSlots;
 #ifdef SD2_TRACE
             const long long tw0 = clock64();
+            if (lane == 0) SD2_TILE_STAMP(q, 1);
 #endif
             if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
 #ifdef SD2_TRACE
             if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] += clock64() - tw0;
 #endif
             if (ctid == 0 && k == 0) SD2_STAMP(3);
+            if (lane == 0) SD2_TILE_STAMP(q, 2);
             const int4 d = sh->desc[slot];
             const uint32_t tb = ring0 + (uint32_t)d.x;
             const uint32_t cnt = lds_u16(tb + 2u * lane);
@@ -845,6 +850,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 }
             }
             __syncwarp();
+            if (lane == 0) SD2_TILE_STAMP(q, 3);
             if (lane == 0) mbar_arrive(empty0 + 8 * slot);
         }
         qbase += (uint32_t)n_cta;
