@@ -91,10 +91,6 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
 constexpr int kSlots = 64;                               // tiles in flight per CTA, at most
 constexpr int kMaxStagesInline = 8;
-#ifndef SD2_RELEASE_BATCH
-#define SD2_RELEASE_BATCH 1
-#endif
-constexpr int kReleaseBatch = SD2_RELEASE_BATCH;   // tiles the producer waits for when the ring is full
 
 struct SMat {
     const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
@@ -589,87 +585,131 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------------------ producer warp
+        // Walks this CTA's tiles of all stages in order, one batch of up to 32 tiles (one per
+        // lane) at a time.  Everything it needs is fetched ahead: the descriptor fields of
+        // stage s + 2 and the tile offsets of stage s + 1 are loaded while the copies of stage
+        // s are issued, so its own global-memory latencies stay off the ring's critical path.
+        // Room in the ring is found for a whole run of tiles at once (a warp prefix sum of
+        // their sizes against the free stretch), and every lane that got a place issues its
+        // own copy in the same instruction: one thread can start only about three bulk copies
+        // per microsecond, whatever their size.
+        struct PStage {          // what the producer needs of a stage (the same in every lane)
+            int count, n_cta;
+            int T[kMaxFused];
+            const uint32_t* toff[kMaxFused];
+            const unsigned char* strm[kMaxFused];
+        };
+        struct PBatch {          // one tile per lane
+            uint32_t bytes;
+            unsigned long long src;
+            int mi, ti;
+        };
+        auto load_stage = [&](int s) {
+            PStage p;
+            const SStage* st = a.ext ? a.ext + s : &a.inl[s];
+            p.count = st->count;
+            p.n_cta = st->tiles_div + (cta < st->tiles_rem ? 1 : 0);
+#pragma unroll
+            for (int m = 0; m < kMaxFused; ++m) {
+                p.T[m] = st->mat[m].T;
+                p.toff[m] = st->mat[m].tile_off;
+                p.strm[m] = st->mat[m].stream;
+            }
+            return p;
+        };
+        auto load_batch = [&](const PStage& p, int k0) {
+            PBatch b;
+            b.bytes = 0; b.src = 0; b.mi = 0; b.ti = 0;
+            const int k = k0 + lane;
+            if (k < p.n_cta) {
+                int v = cta + k * G;
+                int mi = 0;
+#pragma unroll
+                for (int m = 0; m + 1 < kMaxFused; ++m)
+                    if (mi == m && m + 1 < p.count && v >= p.T[m]) { v -= p.T[m]; mi = m + 1; }
+                const uint32_t* toff = p.toff[0];
+                const unsigned char* strm = p.strm[0];
+#pragma unroll
+                for (int m = 1; m < kMaxFused; ++m)
+                    if (mi == m) { toff = p.toff[m]; strm = p.strm[m]; }
+                const uint32_t o0 = __ldg(toff + v);
+                const uint32_t o1 = __ldg(toff + v + 1);
+                b.bytes = (o1 - o0) * 16u;
+                b.src = (unsigned long long)(strm + (size_t)o0 * 16);
+                b.mi = mi;
+                b.ti = v;
+            }
+            return b;
+        };
+
         uint32_t q = 0, oldest = 0;         // tile sequence numbers of this CTA
         uint32_t head = 0, tail = 0;        // ring bytes: [tail, head) is in use (mod wrap)
         const uint32_t ring_bytes = (uint32_t)a.ring_bytes;
         bool ok = true;
+        PStage ps_cur = load_stage(0);
+        PStage ps_next = a.n_stages > 1 ? load_stage(1) : ps_cur;
+        PBatch pb_cur = load_batch(ps_cur, 0);
         for (int s = 0; s < a.n_stages && ok; ++s) {
-            const SStage* st = a.ext ? a.ext + s : &a.inl[s];
-            const int count = st->count;
-            const int n_cta = st->tiles_div + (cta < st->tiles_rem ? 1 : 0);
+            // fetch ahead: first batch of stage s + 1, fields of stage s + 2
+            PBatch pb_next = pb_cur;
+            PStage ps_next2 = ps_next;
+            if (s + 1 < a.n_stages) pb_next = load_batch(ps_next, 0);
+            if (s + 2 < a.n_stages) ps_next2 = load_stage(s + 2);
+            const int n_cta = ps_cur.n_cta;
             for (int k0 = 0; k0 < n_cta && ok; k0 += 32) {
-                const int k = k0 + lane;
-                uint32_t bytes = 0;
-                int mi = 0, ti = 0;
-                unsigned long long src = 0;
-                if (k < n_cta) {
-                    int v = cta + k * G;
-                    while (mi + 1 < count && v >= st->mat[mi].T) {
-                        v -= st->mat[mi].T;
-                        ++mi;
-                    }
-                    ti = v;
-                    const uint32_t o0 = __ldg(st->mat[mi].tile_off + v);
-                    const uint32_t o1 = __ldg(st->mat[mi].tile_off + v + 1);
-                    bytes = (o1 - o0) * 16u;
-                    src = (unsigned long long)(st->mat[mi].stream + (size_t)o0 * 16);
-                }
+                if (k0 > 0) pb_cur = load_batch(ps_cur, k0);   // stages of more than 32 tiles per CTA: not fetched ahead
+                const uint32_t bytes = pb_cur.bytes;
                 const int cnt = min(32, n_cta - k0);
-                // One thread can start only about three bulk copies per microsecond, whatever
-                // their size, so tiles are issued in groups: room is found for as many of the
-                // batch's tiles as fit right now (alike in all lanes), then every lane that
-                // got a place issues its own tile's copy in the same instruction.
-                int i = 0;
-                while (i < cnt && ok) {
-                    const int first = i;
-                    uint32_t my_head = 0, my_slot = 0;
-                    bool mine = false;
-                    while (i < cnt) {
-                        const uint32_t b = __shfl_sync(0xFFFFFFFFu, bytes, i);
-                        const uint32_t outstanding = q - oldest;
-                        uint32_t start;
-                        bool fits;
-                        if (outstanding == 0) {
-                            head = tail = 0;
-                            start = 0;
-                            fits = true;
-                        } else if (head >= tail) {
-                            if (head + b <= ring_bytes) { start = head; fits = true; }
-                            else if (b < tail) { start = 0; fits = true; }
-                            else { start = 0; fits = false; }
-                        } else {
-                            start = head;
-                            fits = head + b < tail;
-                        }
-                        if (!fits || outstanding >= (uint32_t)kSlots) break;
-                        if (lane == i) { my_head = start; my_slot = q % kSlots; mine = true; SD2_TILE_STAMP(q, 0); }
-                        head = start + b;
-                        ++q;
-                        ++i;
+                int i0 = 0;
+                while (i0 < cnt && ok) {
+                    const uint32_t outstanding = q - oldest;
+                    if (outstanding == 0) head = tail = 0;
+                    // free stretch that starts at head: up to the ring's end, or up to just before tail
+                    const uint32_t limit = head >= tail ? ring_bytes : tail - 1u;
+                    const bool cand = lane >= i0 && lane < cnt;
+                    uint32_t incl = cand ? bytes : 0u;
+#pragma unroll
+                    for (int dd = 1; dd < 32; dd <<= 1) {
+                        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, dd);
+                        if (lane >= dd) incl += up;
                     }
-                    if (i > first) {
-                        if (mine) {
-                            sh->desc[my_slot] = make_int4((int)my_head, mi, ti, (int)bytes);
+                    const uint32_t fit_mask = __ballot_sync(0xFFFFFFFFu, cand && head + incl <= limit);
+                    int nfit = __popc(fit_mask);                       // a run of lanes starting at i0
+                    const int slots_free = kSlots - (int)outstanding;
+                    if (nfit > slots_free) nfit = slots_free;
+                    if (nfit > 0) {
+                        if (cand && lane < i0 + nfit) {
+                            const uint32_t my_head = head + incl - bytes;
+                            const uint32_t my_q = q + (uint32_t)(lane - i0);
+                            const uint32_t my_slot = my_q % kSlots;
+                            SD2_TILE_STAMP(my_q, 0);
+                            sh->desc[my_slot] = make_int4((int)my_head, pb_cur.mi, pb_cur.ti, (int)bytes);
                             mbar_expect_tx(full0 + 8 * my_slot, bytes);
-                            bulk_g2s(ring0 + my_head, (const void*)src, bytes, full0 + 8 * my_slot);
+                            bulk_g2s(ring0 + my_head, (const void*)pb_cur.src, bytes, full0 + 8 * my_slot);
                         }
                         __syncwarp();
-                    } else {
-                        // no room: wait until the oldest tile in the ring has been consumed
-                        if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
-                        ++oldest;
-                        // wait for a few more when the ring is far from empty, and take along every
-                        // further tile that is already done: the more room, the more copies start together
-                        for (int r = 1; r < kReleaseBatch && ok && q - oldest > (uint32_t)kConsumerWarps / 2; ++r) {
-                            if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
-                            ++oldest;
-                        }
-                        while (oldest != q && mbar_test_wait(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u)) ++oldest;
-                        tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
+                        head += __shfl_sync(0xFFFFFFFFu, incl, i0 + nfit - 1);
+                        q += (uint32_t)nfit;
+                        i0 += nfit;
+                        continue;
                     }
+                    const uint32_t b_next = __shfl_sync(0xFFFFFFFFu, bytes, i0);
+                    if (slots_free > 0 && head >= tail && b_next < tail) {   // nothing fits at the end: start over at the front
+                        head = 0;
+                        continue;
+                    }
+                    // no room: wait until the oldest tile in the ring has been consumed, and take
+                    // along every further tile that is already done
+                    if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
+                    ++oldest;
+                    while (oldest != q && mbar_test_wait(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u)) ++oldest;
+                    tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
                 }
             }
             if (lane == 0) SD2_STAMP(6);
+            ps_cur = ps_next;
+            ps_next = ps_next2;
+            pb_cur = pb_next;
         }
         if (!ok) {
             // give the copies already issued time to land before this CTA's memory is released
