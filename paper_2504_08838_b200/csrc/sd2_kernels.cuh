@@ -144,8 +144,8 @@ struct SArgs {
 };
 
 #ifdef SD2_TRACE
-// per-tile stamps of CTA 0 (issue, wait begin, start, end), after the per-stage stamps
-#define SD2_TILE_STAMP(q, slot) do { if (a.trace && cta == 0 && (q) < 4096u) a.trace[(size_t)gridDim.x * a.n_stages * 8 + (size_t)(q) * 4 + (slot)] = clock64(); } while (0)
+// per-tile stamps of CTA 0 (issue, wait begin, start, end, producer waits for its release: begin, end)
+#define SD2_TILE_STAMP(q, slot) do { if (a.trace && cta == 0 && (q) < 4096u) a.trace[(size_t)gridDim.x * a.n_stages * 8 + (size_t)(q) * 8 + (slot)] = clock64(); } while (0)
 #define SD2_STAMP(slot) do { if (a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + (slot)] = clock64(); } while (0)
 #else
 #define SD2_STAMP(slot) do { } while (0)
@@ -169,15 +169,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// A waiting thread is parked by the hardware until the phase completes or this many
+// nanoseconds pass, instead of spinning through the shared-memory pipe that working warps need.
+constexpr uint32_t kSuspendHintNs = 20000;
+
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok;
 }
@@ -700,9 +704,17 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     }
                     // no room: wait until the oldest tile in the ring has been consumed, and take
                     // along every further tile that is already done
+                    if (lane == 0) SD2_TILE_STAMP(oldest, 4);
                     if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
+                    if (lane == 0) SD2_TILE_STAMP(oldest, 5);
                     ++oldest;
-                    while (oldest != q && mbar_test_wait(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u)) ++oldest;
+                    while (oldest != q) {   // each lane looks at one of the next 32 tiles; the leading run of done ones goes
+                        const uint32_t t = oldest + (uint32_t)lane;
+                        const bool done = (int)(q - t) > 0 && mbar_test_wait(empty0 + 8 * (t % kSlots), (t / kSlots) & 1u);
+                        const uint32_t run = __ffs(~__ballot_sync(0xFFFFFFFFu, done)) - 1;   // 32 if all are done
+                        oldest += run > 32u ? 32u : run;
+                        if (run < 32u) break;
+                    }
                     tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
                 }
             }
