@@ -26,7 +26,7 @@ struct sd2_handle_s {
     const uint32_t* d_sec1;
     const void* d_sec2;
     // GAP4 geometry
-    int S, B, T, max_tile_bytes;
+    int S, B, T, max_tile_bytes, V;
 };
 
 struct sd2_drafter_s {
@@ -195,6 +195,7 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     h->B = (int)hd.strip_cols;
     h->T = (int)hd.n_tiles;
     h->max_tile_bytes = (int)hd.max_tile_bytes;
+    h->V = (int)hd.overlap;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(h);
@@ -288,11 +289,11 @@ struct SmemPlan {
     int nt, xs_bytes, xlin_bytes, ring_bytes;
 };
 
-int xs_bytes_for(int S, int B, int nt)
+int xs_bytes_for(int S, int B, int V, int nt)
 {
     const int groups = 32 / nt;
     const int planes = S > groups ? S / groups : 1;
-    return planes * (B + kGap4Slack) * 128;
+    return planes * ((B + 2 * V + kGap4Slack + 3) & ~3) * 128;
 }
 
 bool plan_smem(int nt, int xs_max, int K_max, int max_tile, SmemPlan* p)
@@ -352,6 +353,7 @@ void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, 
     st.K = (int)hs[0]->K;
     st.S = hs[0]->S;
     st.B = hs[0]->B;
+    st.V = hs[0]->V;
     st.hdr_bytes = gap4_tile_header_bytes(32 / hs[0]->S);
     st.log2S = 0;
     while ((1 << st.log2S) < hs[0]->S) ++st.log2S;
@@ -396,10 +398,12 @@ struct ProgramNeeds {
     {
         int T = 0;
         for (int i = 0; i < count; ++i) {
-            if (hs[i]->K > K_max) K_max = (int)hs[i]->K;
+            // elements of the linear staging row: the strips, the zero pads on both sides, read-ahead
+            const int lin = hs[i]->S * hs[i]->B + 2 * hs[i]->V + 64;
+            if (lin > K_max) K_max = lin;
             if (hs[i]->max_tile_bytes > max_tile) max_tile = hs[i]->max_tile_bytes;
             for (int w = 0; w < 3; ++w) {
-                const int need = xs_bytes_for(hs[i]->S, hs[i]->B, 1 << w);
+                const int need = xs_bytes_for(hs[i]->S, hs[i]->B, hs[i]->V, 1 << w);
                 if (need > xs_need[w]) xs_need[w] = need;
             }
             T += hs[i]->T;

@@ -65,7 +65,8 @@ namespace sd2 {
 
 constexpr int kFormatBitmask = 1;
 constexpr int kFormatGap4 = 2;
-constexpr int kGap4Slack = 8;          // zero columns kernels append to every strip
+constexpr int kGap4Slack = 8;          // zero columns kernels append to every lane's window
+constexpr int kGap4Overlap = 64;       // columns a lane's window reaches into the strips on either side
 constexpr int kGap4MaxStrip = 496;     // widest strip: at most 63 chunks per segment
 constexpr int kGap4MinStrip = 64;      // strips narrower than this pay too much padding
 constexpr int kGap4TileTarget = 2048;  // tiles a matrix should have, if its shape allows
@@ -87,7 +88,9 @@ struct BlobHeader {
     uint32_t strip_cols;        // GAP4: B
     uint32_t n_tiles;           // GAP4: T
     uint32_t max_tile_bytes;    // GAP4: largest tile record
-    uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16 - 16];
+    uint32_t overlap;           // GAP4: V, columns a lane's window reaches into its neighbours' strips
+    uint32_t reserved[3];
+    uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16 - 16 - 16];
 };
 static_assert(sizeof(BlobHeader) == 256, "header is 256 bytes");
 
@@ -96,10 +99,11 @@ struct Gap4Geom {
     int S;   // strips per row
     int B;   // columns per strip
     int R;   // rows per tile
+    int V;   // overlap: a lane's window is its strip widened by V columns on both sides
 };
 
 // Header bytes of a tile record with R rows.
-SD2_HD int gap4_tile_header_bytes(int R) { return (80 + 4 * R + 15) & ~15; }
+SD2_HD int gap4_tile_header_bytes(int R) { return (144 + 4 * R + 15) & ~15; }
 
 // Picks S: enough tiles to spread over every SM's warps, strips neither too narrow (padding)
 // nor wider than the chunk counters allow.  B is odd so that strips start in distinct
@@ -114,6 +118,7 @@ inline Gap4Geom gap4_geometry(int64_t M, int64_t K)
     g.S = S;
     g.B = (int)((K + S - 1) / S) | 1;
     g.R = 32 / S;
+    g.V = kGap4Overlap;
     if (g.B > kGap4MaxStrip) g.S = 0;
     return g;
 }
@@ -253,19 +258,55 @@ inline int unpack_bitmask(const BlobHeader& h, const uint8_t* blob, uint16_t* de
 
 // ---------------------------------------------------------------- GAP4
 
-// Entries (kept + far-gap fillers) of the segment [c0, c1) of row m, before rounding up to 8.
-inline int gap4_segment_entries(const uint16_t* W, const uint8_t* mask, int64_t m, int64_t K, int64_t c0, int64_t c1,
-                                int64_t* kept_out)
+// Deals the kept columns of one row (ascending, `E` of them) to the S lanes: lane l gets the run
+// cols[first[l] .. first[l+1]).  The aim is the same number of whole chunks in every lane (the
+// warp walks the lanes' chunks in lock step, so the longest lane sets the time, and only a lane
+// whose count is not a multiple of 8 pays padding), under the rule that a lane's columns lie in
+// its window [l*B - V, (l+1)*B + V): a lane must take what the next one cannot reach and cannot
+// take what lies beyond its own window.
+inline void gap4_deal_row(const int32_t* cols, int E, int S, int B, int V, int* first)
 {
-    int64_t cursor = c0, e = 0, kept = 0;
-    for (int64_t k = c0; k < c1; ++k) {
-        if (!is_kept(W, mask, m * K + k)) continue;
-        e += (k - cursor) / 16 + 1;  // one filler per full 16 columns skipped, then the entry
-        cursor = k + 1;
-        ++kept;
+    const int full = E / 8;
+    const int base = full / S, extra = full % S;
+    int e = 0;
+    first[0] = 0;
+    for (int l = 0; l < S; ++l) {
+        int n;
+        if (l == S - 1) {
+            n = E - e;
+        } else {
+            const int64_t must_below = (int64_t)(l + 1) * B - V;   // the next lane's window starts here
+            const int64_t can_below = (int64_t)(l + 1) * B + V;    // this lane's window ends here
+            int lo = 0, hi = 0;
+            while (e + lo < E && cols[e + lo] < must_below) ++lo;
+            hi = lo;
+            while (e + hi < E && cols[e + hi] < can_below) ++hi;
+            const int want = 8 * (base + (l < extra ? 1 : 0));
+            n = want < lo ? lo : want > hi ? hi : want;
+            if (n % 8) {   // whole chunks if the limits allow: up first, then down
+                const int up = (n + 7) / 8 * 8, down = n / 8 * 8;
+                if (up <= hi) n = up;
+                else if (down >= lo) n = down;
+            }
+        }
+        e += n;
+        first[l + 1] = e;
     }
-    *kept_out += kept;
-    return (int)e;
+}
+
+// Entries (kept + far-gap fillers) of a lane's run, before rounding up to 8.
+inline int gap4_run_entries(const int32_t* cols, int n)
+{
+    int e = 0;
+    for (int i = 0; i < n; ++i) e += (i == 0 ? 0 : (cols[i] - cols[i - 1] - 1) / 16) + 1;
+    return e;
+}
+
+inline void gap4_row_cols(const uint16_t* W, const uint8_t* mask, int64_t m, int64_t K, std::vector<int32_t>& cols)
+{
+    cols.clear();
+    for (int64_t k = 0; k < K; ++k)
+        if (is_kept(W, mask, m * K + k)) cols.push_back((int32_t)k);
 }
 
 inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype)
@@ -273,21 +314,30 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     PackResult r;
     const Gap4Geom g = gap4_geometry(M, K);
     if (g.S == 0) { r.status = -5; return r; }
-    const int S = g.S, B = g.B, R = g.R;
-    // chunks of every segment, kept entries of every row
+    const int S = g.S, B = g.B, R = g.R, V = g.V;
+    // per row: where each lane's run starts, chunks of each lane
+    std::vector<int32_t> first((size_t)M * (S + 1));
     std::vector<uint16_t> seg_chunks((size_t)M * S);
     std::vector<int64_t> row_chunks((size_t)M, 0), row_kept((size_t)M, 0);
-#pragma omp parallel for schedule(static)
-    for (int64_t m = 0; m < M; ++m) {
-        int64_t tot = 0;
-        for (int s = 0; s < S; ++s) {
-            const int64_t c0 = std::min<int64_t>(K, (int64_t)s * B), c1 = std::min<int64_t>(K, c0 + B);
-            const int e = gap4_segment_entries(W, mask, m, K, c0, c1, &row_kept[(size_t)m]);
-            const int c = (e + 7) / 8;
-            seg_chunks[(size_t)m * S + s] = (uint16_t)c;
-            tot += c;
+#pragma omp parallel
+    {
+        std::vector<int32_t> cols;
+        std::vector<int> f((size_t)S + 1);
+#pragma omp for schedule(static)
+        for (int64_t m = 0; m < M; ++m) {
+            gap4_row_cols(W, mask, m, K, cols);
+            gap4_deal_row(cols.data(), (int)cols.size(), S, B, V, f.data());
+            int64_t tot = 0;
+            for (int l = 0; l < S; ++l) {
+                first[(size_t)m * (S + 1) + l] = f[(size_t)l];
+                const int c = (gap4_run_entries(cols.data() + f[(size_t)l], f[(size_t)l + 1] - f[(size_t)l]) + 7) / 8;
+                seg_chunks[(size_t)m * S + l] = (uint16_t)c;
+                tot += c;
+            }
+            first[(size_t)m * (S + 1) + S] = f[(size_t)S];
+            row_chunks[(size_t)m] = tot;
+            row_kept[(size_t)m] = (int64_t)cols.size();
         }
-        row_chunks[(size_t)m] = tot;
     }
     // rows by chunk count, most first, ties by index
     std::vector<uint32_t> order((size_t)M);
@@ -321,72 +371,85 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     h.strip_cols = (uint32_t)B;
     h.n_tiles = (uint32_t)T;
     h.max_tile_bytes = max_tile;
+    h.overlap = (uint32_t)V;
     uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
     if (!blob) { r.status = -3; return r; }
     std::memcpy(blob + h.sec_off[0], toff.data(), sec[0]);
     uint8_t* tiles = blob + h.sec_off[1];
-#pragma omp parallel for schedule(dynamic, 8)
-    for (int64_t t = 0; t < T; ++t) {
-        uint8_t* rec = tiles + (size_t)toff[(size_t)t] * 16;
-        uint16_t* cnt = (uint16_t*)rec;
-        uint32_t* nch = (uint32_t*)(rec + 64);
-        uint32_t* rows = (uint32_t*)(rec + 80);
-        // logical entry lists of the 32 segments
+#pragma omp parallel
+    {
+        std::vector<int32_t> cols;
         std::vector<uint8_t> eg[32];
         std::vector<uint16_t> ev[32];
-        uint32_t ct = 0, lane_mask = 0;
-        int maxc = 0, minc = 0xFFFF;
-        for (int l = 0; l < 32; ++l) {
-            const int rr = l / S, s = l % S;
-            const int64_t i = t * R + rr;
-            if (s == 0) rows[rr] = i < M ? order[(size_t)i] : 0xFFFFFFFFu;
-            cnt[l] = 0;
-            if (i >= M) continue;
-            const int64_t m = order[(size_t)i];
-            const int c = seg_chunks[(size_t)m * S + s];
-            cnt[l] = (uint16_t)c;
-            ct += (uint32_t)c;
-            if (c > maxc) maxc = c;
-            if (c == 0) continue;
-            if (c < minc) minc = c;
-            lane_mask |= 1u << l;
-            eg[l].assign((size_t)c * 8, 0);
-            ev[l].assign((size_t)c * 8, 0);
-            const int64_t c0 = std::min<int64_t>(K, (int64_t)s * B), c1 = std::min<int64_t>(K, c0 + B);
-            int64_t cursor = c0;
-            size_t e = 0;
-            for (int64_t k = c0; k < c1; ++k) {
-                if (!is_kept(W, mask, m * K + k)) continue;
-                while (k - cursor > 15) {  // filler 15 columns ahead
-                    eg[l][e] = 15;
-                    ev[l][e] = 0;
-                    ++e;
-                    cursor += 16;
+#pragma omp for schedule(dynamic, 8)
+        for (int64_t t = 0; t < T; ++t) {
+            uint8_t* rec = tiles + (size_t)toff[(size_t)t] * 16;
+            uint16_t* cnt = (uint16_t*)rec;
+            uint32_t* nch = (uint32_t*)(rec + 64);
+            uint16_t* start = (uint16_t*)(rec + 80);
+            uint32_t* rows = (uint32_t*)(rec + 144);
+            uint32_t ct = 0, lane_mask = 0;
+            int maxc = 0, minc = 0xFFFF;
+            for (int rr = 0; rr < R; ++rr) {
+                const int64_t i = t * R + rr;
+                rows[rr] = i < M ? order[(size_t)i] : 0xFFFFFFFFu;
+                if (i >= M) {
+                    for (int s = 0; s < S; ++s) { cnt[rr * S + s] = 0; start[rr * S + s] = 0; }
+                    continue;
                 }
-                eg[l][e] = (uint8_t)(k - cursor);
-                ev[l][e] = W[m * K + k];
-                ++e;
-                cursor = k + 1;
+                const int64_t m = order[(size_t)i];
+                gap4_row_cols(W, mask, m, K, cols);
+                for (int s = 0; s < S; ++s) {
+                    const int l = rr * S + s;
+                    const int e0 = first[(size_t)m * (S + 1) + s], e1 = first[(size_t)m * (S + 1) + s + 1];
+                    const int c = seg_chunks[(size_t)m * S + s];
+                    cnt[l] = (uint16_t)c;
+                    start[l] = 0;
+                    ct += (uint32_t)c;
+                    if (c > maxc) maxc = c;
+                    if (c == 0) continue;
+                    if (c < minc) minc = c;
+                    lane_mask |= 1u << l;
+                    eg[l].assign((size_t)c * 8, 0);
+                    ev[l].assign((size_t)c * 8, 0);
+                    // the cursor starts on the run's first column, given relative to the lane's window
+                    start[l] = (uint16_t)(cols[(size_t)e0] - ((int64_t)s * B - V));
+                    int64_t cursor = cols[(size_t)e0];
+                    size_t e = 0;
+                    for (int x = e0; x < e1; ++x) {
+                        const int64_t k = cols[(size_t)x];
+                        while (k - cursor > 15) {  // filler 15 columns ahead
+                            eg[l][e] = 15;
+                            ev[l][e] = 0;
+                            ++e;
+                            cursor += 16;
+                        }
+                        eg[l][e] = (uint8_t)(k - cursor);
+                        ev[l][e] = W[m * K + k];
+                        ++e;
+                        cursor = k + 1;
+                    }
+                    // entries e .. 8c-1 stay gap 0 / value +0
+                }
             }
-            // entries e .. 8c-1 stay gap 0 / value +0
-        }
-        nch[0] = ct;
-        nch[1] = lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u;
-        nch[2] = lane_mask;
-        nch[3] = 0;
-        uint32_t* codes = (uint32_t*)(rec + hdr);
-        uint16_t* vals = (uint16_t*)(rec + hdr + align16((size_t)ct * 4));
-        size_t slot = 0;
-        for (int j = 0; j < maxc; ++j) {
-            for (int l = 0; l < 32; ++l) {
-                if (cnt[l] <= j) continue;
-                uint32_t code = 0;
-                for (int i = 0; i < 8; ++i) {
-                    code |= (uint32_t)eg[l][(size_t)j * 8 + i] << (4 * i);
-                    vals[slot * 8 + i] = ev[l][(size_t)j * 8 + i];
+            nch[0] = ct;
+            nch[1] = lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u;
+            nch[2] = lane_mask;
+            nch[3] = 0;
+            uint32_t* codes = (uint32_t*)(rec + hdr);
+            uint16_t* vals = (uint16_t*)(rec + hdr + align16((size_t)ct * 4));
+            size_t slot = 0;
+            for (int j = 0; j < maxc; ++j) {
+                for (int l = 0; l < 32; ++l) {
+                    if (cnt[l] <= j) continue;
+                    uint32_t code = 0;
+                    for (int i = 0; i < 8; ++i) {
+                        code |= (uint32_t)eg[l][(size_t)j * 8 + i] << (4 * i);
+                        vals[slot * 8 + i] = ev[l][(size_t)j * 8 + i];
+                    }
+                    codes[slot] = code;
+                    ++slot;
                 }
-                codes[slot] = code;
-                ++slot;
             }
         }
     }
@@ -402,8 +465,8 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
 {
     const int64_t M = h.M, K = h.K;
     const Gap4Geom g = gap4_geometry(M, K);
-    if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B) return -6;
-    const int S = g.S, B = g.B, R = g.R;
+    if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B || h.overlap != (uint32_t)g.V) return -6;
+    const int S = g.S, B = g.B, R = g.R, V = g.V;
     const int64_t T = (M + R - 1) / R;
     if (h.n_tiles != (uint64_t)T || h.sec_bytes[0] != (uint64_t)(T + 1) * 4 || h.sec_bytes[2] != 0) return -6;
     if (h.sec_bytes[1] % 16) return -6;
@@ -411,6 +474,7 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
     const uint8_t* tiles = blob + h.sec_off[1];
     const uint64_t units = h.sec_bytes[1] / 16;
     const int hdr = gap4_tile_header_bytes(R);
+    const int window = B + 2 * V;   // columns a lane may touch, before the slack
     if (toff[0] != 0 || toff[T] != units) return -6;
     for (int64_t t = 0; t < T; ++t)
         if (toff[t + 1] <= toff[t]) return -6;
@@ -418,8 +482,8 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
     int bad = 0;
     int64_t chunks = 0;
     for (int64_t t = 0; t < T; ++t) {  // row ids: a permutation of 0..M-1, checked serially
-        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 80);
         if ((uint64_t)(toff[t + 1] - toff[t]) * 16 < (uint64_t)hdr) return -6;
+        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 144);
         for (int rr = 0; rr < R; ++rr) {
             const int64_t i = t * R + rr;
             if (i < M) {
@@ -440,13 +504,15 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
         const size_t rec_bytes = (size_t)(toff[t + 1] - toff[t]) * 16;
         const uint16_t* cnt = (const uint16_t*)rec;
         const uint32_t* meta = (const uint32_t*)(rec + 64);
+        const uint16_t* start = (const uint16_t*)(rec + 80);
         const uint32_t ct = meta[0];
-        const uint32_t* rows = (const uint32_t*)(rec + 80);
+        const uint32_t* rows = (const uint32_t*)(rec + 144);
         uint32_t sum = 0, lane_mask = 0;
         int maxc = 0, minc = 0xFFFF;
         for (int l = 0; l < 32; ++l) {
-            if (cnt[l] > (B + kGap4Slack) / 8 + 1) bad |= 1;
+            if (cnt[l] > (window + kGap4Slack) / 8 + 1) bad |= 1;
             if (rows[l / S] == 0xFFFFFFFFu && cnt[l] != 0) bad |= 1;
+            if (start[l] >= window + kGap4Slack) bad |= 1;
             sum += cnt[l];
             if (cnt[l] > maxc) maxc = cnt[l];
             if (cnt[l] > 0) {
@@ -465,24 +531,30 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
         chunks += ct;
         const uint32_t* codes = (const uint32_t*)(rec + hdr);
         const uint16_t* vals = (const uint16_t*)(rec + hdr + align16((size_t)ct * 4));
-        int64_t cursor[32];
-        for (int l = 0; l < 32; ++l) cursor[l] = (int64_t)(l % S) * B;
+        int64_t cursor[32], wbase[32];
+        for (int l = 0; l < 32; ++l) {
+            wbase[l] = (int64_t)(l % S) * B - V;          // first column of the lane's window (may be negative)
+            cursor[l] = wbase[l] + start[l];
+        }
         size_t slot = 0;
         for (int j = 0; j < maxc; ++j) {
             for (int l = 0; l < 32; ++l) {
                 if (cnt[l] <= j) continue;
-                const int s = l % S;
                 const int64_t m = rows[l / S];
-                const int64_t c1 = std::min<int64_t>(K, (int64_t)(s + 1) * B);  // end of the strip's real columns
                 const uint32_t code = codes[slot];
                 for (int i = 0; i < 8; ++i) {
                     const int64_t col = cursor[l] + ((code >> (4 * i)) & 15);
                     cursor[l] = col + 1;
                     const uint16_t v = vals[slot * 8 + i];
-                    if (col < c1) {
-                        if (dense && v != 0) dense[m * K + col] = v;
-                    } else if (v != 0 || col >= (int64_t)s * B + B + kGap4Slack) {
-                        bad |= 1;  // only +0 fillers may pass the strip's end, and only by < 8 columns
+                    // a kernel reads window row col - wbase: it must exist (window + slack rows)
+                    if (col - wbase[l] >= window + kGap4Slack) { bad |= 1; continue; }
+                    if (col >= 0 && col < K) {
+                        if (dense && v != 0) {
+                            if (dense[m * K + col] != 0) bad |= 1;   // two lanes claim one column
+                            dense[m * K + col] = v;
+                        }
+                    } else if (v != 0) {
+                        bad |= 1;  // only +0 fillers may lie outside the matrix
                     }
                 }
                 ++slot;

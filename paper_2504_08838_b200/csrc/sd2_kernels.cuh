@@ -120,7 +120,8 @@ struct SStage {
     int tiles_div;         // T_total / grid size: CTA c runs tiles_div + (c < tiles_rem) tiles
     int tiles_rem;         // T_total % grid size
     int tagged_in;         // x / g / u point at tagged 32-bit words written by the previous stage
-    int reserved[4];
+    int V;                 // overlap: lane windows are strips widened by V columns on both sides
+    int reserved[3];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
@@ -374,9 +375,9 @@ __device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uin
     return byte_times_128_plus<3>(PO, xb + 1024u);
 }
 
-// Stage the activations of one stage: xs[plane][column c][group][NT] (fp32) with
-// value = X[n][strip * B + c] where strip = plane * groups + group % S (for S <= groups the
-// strips repeat across the groups), zero for c >= B, strip * B + c >= K or n >= N.
+// Stage the activations of one stage: xs[plane][window row c][group][NT] (fp32) with
+// value = X[n][strip * B - V + c] where strip = plane * groups + group % S (for S <= groups the
+// strips repeat across the groups), zero outside the matrix, in the slack rows and for n >= N.
 // Row by row through `xlin` (bf16, linear) so that global memory is read with 128-bit loads.
 // x_src, g, u, t_out already point at the launch's first activation row.
 // One 128-bit load of four tagged words, repeated until all four carry `tag` (their producers,
@@ -496,14 +497,21 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
     const int K = st.K, S = st.S, B = st.B;
     const bool glue = x_src == nullptr;
     const int planes = S > kGroups ? S / kGroups : 1;
-    const int rows = B + kGap4Slack;
+    const int rows = B + 2 * st.V + kGap4Slack;     // a lane's window and the slack
+    const int rows4 = (rows + 3) & ~3;              // the scatter works on four rows at a time
+    // the linear row sits V elements into xlin, with zeros before it and behind it, so that
+    // the scatter can read any window without bounds checks
+    uint16_t* xl = xlin + st.V;
+    const int tail_pad = S * B - K + st.V + 48;
     const bool vec = (K % 8 == 0) && ((((uintptr_t)x_src | (uintptr_t)g | (uintptr_t)u | (uintptr_t)t_out) & 15) == 0);
     const bool pub = glue && t_out && blockIdx.x == 0;
     for (int n = 0; n < NT; ++n) {
+        for (int i = ctid; i < st.V; i += kConsumerThreads) xlin[i] = 0;
+        for (int i = ctid; i < tail_pad; i += kConsumerThreads) xl[K + i] = 0;
         if (n < N && tag != 0u) {
             stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
                                 g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
-                                t_out ? t_out + (size_t)n * K : nullptr, pub, xlin, tag, wc, ctid);
+                                t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag, wc, ctid);
         } else if (n < N) {
             if (vec) {
                 for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
@@ -520,7 +528,7 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                         v = make_uint4(w[0], w[1], w[2], w[3]);
                         if (pub) ((uint4*)(t_out + (size_t)n * K))[i] = v;
                     }
-                    ((uint4*)xlin)[i] = v;
+                    ((uint4*)xl)[i] = v;
                 }
             } else {
                 for (int i = ctid; i < K; i += kConsumerThreads) {
@@ -531,24 +539,33 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                         v = silu_mul_bits(__ldcg(g + (size_t)n * K + i), __ldcg(u + (size_t)n * K + i));
                         if (pub) t_out[(size_t)n * K + i] = v;
                     }
-                    xlin[i] = v;
+                    xl[i] = v;
                 }
             }
         }
         named_bar_sync(1, kConsumerThreads);
-        // scatter row n: consecutive threads take consecutive groups of one column
-        const int per_plane = rows * kGroups;
+        // scatter row n: consecutive threads take consecutive groups; each takes four window rows
+        // of its group from three aligned 32-bit reads (window row c of strip s is element
+        // s * B + c of xlin)
+        const int per_plane = (rows4 >> 2) * kGroups;
+        const uint32_t* xl32 = (const uint32_t*)xlin;
         for (int p = 0; p < planes; ++p) {
-            float* xp = xs + (size_t)p * rows * 32;
-            const int strip = S > kGroups ? p * kGroups + (ctid % kGroups) : (ctid % kGroups) & (S - 1);   // fixed per thread
-            const int col0 = strip * B;
-#pragma unroll 4
+            float* xp = xs + (size_t)p * rows4 * 32;
+            const int grp = ctid % kGroups;
+            const int strip = S > kGroups ? p * kGroups + grp : grp & (S - 1);   // fixed per thread
+#pragma unroll 2
             for (int i = ctid; i < per_plane; i += kConsumerThreads) {
-                const int c = i / kGroups;
-                const int col = col0 + c;
-                float v = 0.f;
-                if (n < N && c < B && col < K) v = bf16_to_f32(xlin[col]);
-                xp[(size_t)i * NT + n] = v;
+                const int c = (i / kGroups) << 2;
+                const int e = strip * B + c;
+                const uint32_t w0 = xl32[e >> 1], w1 = xl32[(e >> 1) + 1], w2 = xl32[(e >> 1) + 2];
+                const uint32_t sh = (uint32_t)(e & 1) << 4;
+                uint32_t t0 = __funnelshift_r(w0, w1, sh), t1 = __funnelshift_r(w1, w2, sh);
+                if (n >= N) t0 = t1 = 0u;
+                float* dst = xp + ((size_t)c * kGroups + grp) * NT + n;
+                dst[0] = bf16_lo(t0);
+                dst[32] = bf16_hi(t0);
+                dst[64] = bf16_lo(t1);
+                dst[96] = bf16_hi(t1);
             }
         }
         named_bar_sync(1, kConsumerThreads);
@@ -804,7 +821,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const uint32_t hdr_bytes = (uint32_t)st.hdr_bytes;
         const int strip = lane & (S - 1);
         const int plane = S > kGroups ? strip / kGroups : 0;
-        const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)((st.B + kGap4Slack) * 128) +
+        const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)(((st.B + 2 * st.V + kGap4Slack + 3) & ~3) * 128) +
                                  (uint32_t)(lane % kGroups) * (4u * NT);
         const uint32_t lt = (1u << lane) - 1u;
         const bool last_stage = s == a.n_stages - 1;
@@ -835,7 +852,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             float a0[NT], a1[NT];
 #pragma unroll
             for (int n = 0; n < NT; ++n) a0[n] = a1[n] = 0.f;
-            uint32_t xb = xs_lane;
+            uint32_t xb = xs_lane + 128u * lds_u16(tb + 80u + 2u * lane);   // the cursor starts inside the window
 
             // steps every populated lane takes: addresses advance by a constant
             if (cnt > 0) {
@@ -877,7 +894,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 for (int dd = 1; dd < S; dd <<= 1) r[n] += __shfl_xor_sync(0xFFFFFFFFu, r[n], dd);
             }
             if (strip == 0) {
-                const uint32_t row = lds_u32(tb + 80u + 4u * (uint32_t)(lane >> st.log2S));
+                const uint32_t row = lds_u32(tb + 144u + 4u * (uint32_t)(lane >> st.log2S));
                 if (row != 0xFFFFFFFFu) {
                     const SMat& md = st.mat[d.y];
                     void* yp = (last_stage && a.y_out && d.y == 0) ? a.y_out : md.y;
