@@ -66,7 +66,7 @@ namespace sd2 {
 constexpr int kFormatBitmask = 1;
 constexpr int kFormatGap4 = 2;
 constexpr int kGap4Slack = 8;          // zero columns kernels append to every lane's window
-constexpr int kGap4Overlap = 64;       // columns a lane's window reaches into the strips on either side
+constexpr int kGap4Overlap = 32;       // columns a lane's window reaches into the strips on either side
 constexpr int kGap4MaxStrip = 496;     // widest strip: at most 63 chunks per segment
 constexpr int kGap4MinStrip = 64;      // strips narrower than this pay too much padding
 constexpr int kGap4TileTarget = 2048;  // tiles a matrix should have, if its shape allows

@@ -83,7 +83,7 @@ def test_bitmask_byte_count_closed_form():
     assert info["compressed_bytes"] == 4 * (M + 1) + 4 * M * ((K + 31) // 32) + 2 * int(mask.sum())
 
 
-GAP4_OVERLAP = 64
+GAP4_OVERLAP = 32
 
 
 def _gap4_geometry(M, K):
