@@ -17,29 +17,34 @@
 //            (sec2 is empty)
 //
 // GAP4 in detail.  The K columns are cut into S strips of B columns (S a power of two <= 32,
-// S * B >= K) and a *segment* is one row restricted to one strip.  A segment's kept entries,
-// in ascending column order, become a list of (gap, value) entries: a cursor starts at the
-// strip's first column; an entry at column c is coded as g = c - cursor in [0, 15] and moves
-// the cursor to c + 1.  When the next kept column is more than 15 ahead, a filler entry
-// (value +0) is placed at cursor + 15 first.  The list is then filled up to a multiple of 8
-// with gap-0 fillers (value +0), which may run up to 7 columns past the strip's end: kernels
-// give every strip 8 zero columns of slack and the decoder drops such columns.  Fillers sit
-// on masked-out columns and carry +0, so decoding still yields W.*mask bit for bit; they
-// are not counted in nnz, and their bytes are part of "compressed bytes" but never called
-// useful.  Eight consecutive entries form a chunk: 16 bytes of values + one 32-bit code word
-// whose nibble i (bits 4i..4i+3) is entry i's gap.
+// S * B >= K, B odd) and every strip, widened by V columns on both sides, is the *window* of
+// one lane.  A row's kept entries, in ascending column order, are dealt to the S lanes in
+// consecutive runs: every lane gets the same number of whole 8-entry chunks where the windows
+// allow it (a lane must take what the next lane's window cannot reach and cannot take what lies
+// beyond its own), the last lane takes the rest.  So the lanes of a row finish together and
+// only the last one pays padding.  A lane's run becomes a list of (gap, value) entries: a
+// cursor starts on the run's first column; an entry at column c is coded as g = c - cursor in
+// [0, 15] and moves the cursor to c + 1.  When the next kept column is more than 15 ahead, a
+// filler entry (value +0) is placed at cursor + 15 first.  The list is then filled up to a
+// multiple of 8 with gap-0 fillers (value +0), which may run up to 7 columns past the window's
+// end: kernels give every window 8 more rows and the decoder drops such columns.  Fillers sit
+// on masked-out columns (or outside the matrix) and carry +0, so decoding still yields
+// W.*mask bit for bit; they are not counted in nnz, and their bytes are part of "compressed
+// bytes" but never called useful.  Eight consecutive entries form a chunk: 16 bytes of values
+// + one 32-bit code word whose nibble i (bits 4i..4i+3) is entry i's gap.
 //
 // Rows are ordered by chunk count (most first, ties by row index), so that rows of like
-// density share a tile.  A tile is R = 32 / S consecutive rows of that order: 32 segments,
-// one per lane of a warp; lane l holds strip l % S of the tile's row l / S.  Lanes step
+// density share a tile.  A tile is R = 32 / S consecutive rows of that order: 32 runs, one per
+// lane of a warp; lane l holds the run of window l % S of the tile's row l / S.  Lanes step
 // through their chunks together; step j of the tile stores chunk j of every lane that has
 // more than j chunks, in lane order, so each step is one contiguous, fully used run.
 //
-//   tile record   u16 cnt[32]          chunks of each lane's segment
+//   tile record   u16 cnt[32]          chunks of each lane's run
 //                 u32 n_chunks         sum of cnt
 //                 u32 cnt_range        smallest non-zero cnt | largest cnt << 16 (0 if all are zero)
 //                 u32 lane_mask        bit l set iff cnt[l] > 0
 //                 u32 reserved         0
+//                 u16 start[32]        first column of each lane's run, counted from its window's start
 //                 u32 row[R]           original row index of each tile row, 0xFFFFFFFF = none
 //                 (pad to 16 bytes)
 //                 u32 code[n_chunks]   step-major as described
