@@ -417,7 +417,11 @@ int nt_index(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : 2; }
 // Widest panel (4, 2, 1 rows) whose staged activations still leave room for the ring; 0 if none.
 int widest_panel(const int xs_need[3], int K_max, int max_tile)
 {
+    // a wide panel whose activations crowd out the ring cannot stream: ask for a ring of at
+    // least 96 KB first, and settle for whatever fits only if no width leaves that much
     SmemPlan p;
+    for (int nt = 4; nt >= 1; nt >>= 1)
+        if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p) && p.ring_bytes >= 96 * 1024) return nt;
     for (int nt = 4; nt >= 1; nt >>= 1)
         if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return nt;
     return 0;
