@@ -205,6 +205,19 @@ def ncu_traffic_ratio():
         return None
 
 
+def aggregate_replicas(t_step, world, dist, device):
+    """Replicas only: every rank runs its own drafter, nothing is exchanged on the data path.
+    The step time of the job is the slowest rank's (MAX over ranks); in that time `world` tokens are
+    finished, so the time per token of the whole job is max / world.  Returns (max over ranks of
+    t_step, 1e3 * that / world): with t_step in ms the second value is microseconds per token."""
+    if world > 1:
+        import torch
+        t = torch.tensor([t_step], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_step = float(t.item())
+    return t_step, t_step * 1e3 / world
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -359,15 +372,9 @@ def run_ours(args):
             dense_us = e0.elapsed_time(e1) / dsteps * 1e3
 
     ms_step = ms_total / args.steps
-    if world > 1:
-        t = torch.tensor([ms_step], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    us_token = ms_step * 1e3 / world            # aggregate: `world` replicas finish `world` tokens per step
-    e2e_us = e2e_s * 1e6 / world
+    ms_step, us_token = aggregate_replicas(ms_step, world, dist, "cuda")
+    e2e_s, e2e_us = aggregate_replicas(e2e_s, world, dist, "cuda")
+    e2e_us *= 1e3                                # seconds -> the helper's "x 1e3" gives ms; us needs another 1e3
 
     if rank == 0:
         peak, peak_src = measured_peak()
