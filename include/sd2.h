@@ -206,6 +206,12 @@ sd2_status sd2_drafter_free(sd2_drafter d);
  * if the stream itself failed, SD2_OK otherwise.  Synchronises; not for the hot loop. */
 sd2_status sd2_stream_check(void* cuda_stream);
 
+/* Diagnostic for the bounded waits (the paper has no counterpart): launches one warp that waits
+ * on a barrier nothing ever signals, with the budget every device-side wait of this library has
+ * (2 s of SM clock, or SD2_WAIT_MS milliseconds from the environment).  The wait runs out, the
+ * kernel ends normally and the next sd2_stream_check returns SD2_ERR_TIMEOUT once.  Asynchronous. */
+sd2_status sd2_selftest_timeout(void* cuda_stream);
+
 /* Static string for a status code. */
 const char* sd2_status_string(sd2_status s);
 

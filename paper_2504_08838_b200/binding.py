@@ -26,7 +26,7 @@ EXPORTS = [
     "sd2_decompress", "sd2_info", "sd2_free", "sd2_spmm", "sd2_spmm_fused", "sd2_block_step",
     "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
     "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
-    "sd2_block_step_static",
+    "sd2_block_step_static", "sd2_selftest_timeout",
 ]
 
 
@@ -76,6 +76,7 @@ def lib():
             "sd2_drafter_buffers": [p, i32, pp],
             "sd2_drafter_free": [p],
             "sd2_block_step_static": [pp, p, p, i64, p],
+            "sd2_selftest_timeout": [p],
         }
         for name, argtypes in sig.items():
             fn = getattr(L, name)
@@ -310,3 +311,8 @@ def sd2_block_step_static(hs, x, y, stream=None):
     that may not allocate device memory.  Calls must not overlap on the GPU (they share the array)."""
     N = x.shape[0] if x.dim() == 2 else 1
     _check(lib().sd2_block_step_static(_handle_array(hs), _ptr(x), _ptr(y), N, _stream(stream)), "sd2_block_step_static")
+
+
+def sd2_selftest_timeout(stream=None):
+    """Launch the diagnostic whose device-side wait must run out (see ``sd2_stream_check``)."""
+    _check(lib().sd2_selftest_timeout(_stream(stream)), "sd2_selftest_timeout")

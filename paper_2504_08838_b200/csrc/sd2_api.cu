@@ -770,6 +770,16 @@ sd2_status sd2_stream_check(void* cuda_stream)
     return SD2_OK;
 }
 
+sd2_status sd2_selftest_timeout(void* cuda_stream)
+{
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(g_dev[dev].err_word, wait_budget(dev));
+    if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
+    return SD2_OK;
+}
+
 sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_stream)
 {
     if (!X || !Y) return SD2_ERR_INVALID_ARG;

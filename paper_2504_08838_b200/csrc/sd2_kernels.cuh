@@ -947,6 +947,27 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     }
 }
 
+// Diagnostic: one warp waits, with the same bounded wait the stream kernel uses, on an mbarrier
+// that nothing ever arrives at.  The wait must run out, raise the error word and let the kernel
+// end normally (no trap, no hang).
+__global__ void __launch_bounds__(32, 1) wait_selftest_kernel(int* err, long long budget)
+{
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    WaitCtx wc;
+    wc.abort_flag = &abort_flag;
+    wc.budget = budget;
+    const bool ok = wait_phase(b, 0u, wc);
+    if (!ok && threadIdx.x == 0 && err) atomicExch(err, 1);
+}
+
 // ------------------------------------------------------------------------------ BITMASK
 //
 // General-purpose path (any M, K; activations read through L1 from global memory, so no

@@ -365,3 +365,21 @@ def test_blob_made_on_the_host_runs_on_the_device():
         Yr, S = oracle.masked_linear(W, mask, X)
         check(run_spmm(h, X, True), Yr, S, True)
         sd2.sd2_free(h)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_library_carries_on(monkeypatch):
+    # nothing faults or hangs: the diagnostic's wait is bounded (here 20 ms), raises the error word,
+    # the kernel ends normally, and ordinary calls work afterwards
+    monkeypatch.setenv("SD2_WAIT_MS", "20")
+    sd2.sd2_stream_check()                                   # start from a clean error word
+    sd2.sd2_selftest_timeout()
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_stream_check()
+    assert e.value.status == sd2.SD2_ERR_TIMEOUT
+    sd2.sd2_stream_check()                                   # reported once, then clear again
+    monkeypatch.delenv("SD2_WAIT_MS")
+    W, mask, X = case(4242, 70, 900, 0.5, 2)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(run_spmm(h, X, True), Yr, S, True)
+    sd2.sd2_free(h)
