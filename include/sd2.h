@@ -59,9 +59,14 @@ typedef enum {
 enum {
     SD2_FORMAT_AUTO = 0,    /* library picks (currently SD2_FORMAT_GAP4 when it applies)    */
     SD2_FORMAT_BITMASK = 1, /* 1 bit per dense slot + packed kept values + row offsets    */
-    SD2_FORMAT_GAP4 = 2     /* 4-bit column gaps + packed kept values in 8-entry chunks,  */
+    SD2_FORMAT_GAP4 = 2,    /* 4-bit column gaps + packed kept values in 8-entry chunks,  */
                             /* rows cut into column strips, 32 strips to a tile (the fast */
                             /* path; column strips wider than 496 are not supported)      */
+    SD2_FORMAT_GAP4_PAIRED = 3 /* as an option of sd2_pack_host / sd2_compress only: GAP4 */
+                            /* whose rows 2i and 2i+1 stay next to each other in a tile   */
+                            /* (for a stack that interleaves gate row i and up row i; M   */
+                            /* even and at least two rows per tile, else UNSUPPORTED).    */
+                            /* The blob and the handle report SD2_FORMAT_GAP4.            */
 };
 
 enum { SD2_DTYPE_BF16 = 0, SD2_DTYPE_F32 = 1 };
@@ -183,6 +188,10 @@ sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, in
  * up,down; block b+1 reads block b's output (rounded to bf16), so out(b) must equal
  * hidden(b+1).  n_max in [1, 64] sizes the intermediate buffers, which the drafter owns.
  * The handles must outlive the drafter.  May synchronise; allocates device memory.
+ * Where the shapes allow it the drafter keeps its own paired copy of every block's gate and up
+ * (one stacked GAP4 matrix, gate row i and up row i side by side, as large as the two
+ * together), built here on the host from the handles' decoded contents, so that a step forms
+ * t = silu(g) * u where g and u are produced.
  * Errors: INVALID_ARG, SHAPE (shapes do not chain, L or n_max out of range), UNSUPPORTED (a
  * handle is not GAP4, or a layer is too wide for shared memory), ALLOC. */
 sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2_drafter* out);

@@ -27,6 +27,7 @@ struct sd2_handle_s {
     const void* d_sec2;
     // GAP4 geometry
     int S, B, T, max_tile_bytes, V;
+    int paired;   // GAP4: rows 2i, 2i+1 share a tile (header field `pairing`)
 };
 
 struct sd2_drafter_s {
@@ -36,6 +37,7 @@ struct sd2_drafter_s {
     int y_f32;                 // dtype of the last block's output
     int64_t hidden, out_dim;
     std::vector<sd2_handle> handles;
+    std::vector<sd2_handle> owned;      // paired gate|up stacks the drafter built for itself
     std::vector<int64_t> ws_off;        // per block: offsets of q,k,v,hdn,g,u,t and the block output inside d_ws
     uint8_t* d_ws;
     SStage* d_stages;
@@ -141,7 +143,7 @@ int resolve_format(const sd2_options* opt, int64_t M, int64_t K)
 {
     int f = opt ? opt->format : SD2_FORMAT_AUTO;
     if (f == SD2_FORMAT_AUTO) f = gap4_geometry(M, K).S > 0 ? SD2_FORMAT_GAP4 : SD2_FORMAT_BITMASK;
-    return f;
+    return f;   // SD2_FORMAT_GAP4_PAIRED stays as asked: only the packer tells it from GAP4
 }
 
 sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, const sd2_options* opt,
@@ -156,6 +158,7 @@ sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K
     try {
         if (f == SD2_FORMAT_BITMASK) r = pack_bitmask(W, mask, M, K, y_dtype);
         else if (f == SD2_FORMAT_GAP4) r = pack_gap4(W, mask, M, K, y_dtype);
+        else if (f == SD2_FORMAT_GAP4_PAIRED) r = pack_gap4(W, mask, M, K, y_dtype, true);
         else return SD2_ERR_INVALID_ARG;
     } catch (const std::bad_alloc&) {
         return SD2_ERR_ALLOC;
@@ -196,6 +199,7 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     h->T = (int)hd.n_tiles;
     h->max_tile_bytes = (int)hd.max_tile_bytes;
     h->V = (int)hd.overlap;
+    h->paired = (int)hd.pairing;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(h);
@@ -550,7 +554,7 @@ struct BlockTags {
 // group that do not share a strip geometry get a stage each.  Returns the number appended.
 int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
                         uint16_t* hdn, uint16_t* g, uint16_t* u, uint16_t* t, void* y, bool y_force_bf16,
-                        ProgramNeeds* needs, int grid, const BlockTags* tg = nullptr)
+                        ProgramNeeds* needs, int grid, const BlockTags* tg = nullptr, sd2_handle gu_pair = nullptr)
 {
     int n = 0;
     auto group = [&](const sd2_handle* hs, int count, const uint16_t* xin, const uint16_t* gg, const uint16_t* uu,
@@ -584,12 +588,63 @@ int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, 
         uint32_t* t_d[1] = {tg->out_t};
         group(h + 0, 3, tg->x_t ? (const uint16_t*)tg->x_t : x, nullptr, nullptr, nullptr, y_qkv, true, t_qkv, tg->x_t ? 1 : 0);
         group(h + 3, 1, (const uint16_t*)tg->q_t, nullptr, nullptr, nullptr, y_o, true, t_o, 1);
-        group(h + 4, 2, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_gu, true, t_gu, 1);
-        const int before = n;
-        group(h + 6, 1, nullptr, (const uint16_t*)tg->g_t, (const uint16_t*)tg->u_t, t, y_d, y_force_bf16, t_d, 1);
-        for (int i = before; i < n; ++i) stages[i].tt = tg->t_t;
+        if (gu_pair) {
+            // one stacked matrix, gate row i and up row i in one tile: the stage writes g, u and t
+            // as plain bf16 and t as tagged words, and the down stage reads t like any activation
+            void* y_none[1] = {nullptr};
+            SStage& st = stages[n++];
+            fill_stage(st, &gu_pair, 1, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_none, true, grid, nullptr, 1);
+            needs->add(&gu_pair, 1);
+            st.paired = 1;
+            st.g = g;
+            st.u = u;
+            st.t_out = t;
+            st.tt = tg->t_t;
+            group(h + 6, 1, (const uint16_t*)tg->t_t, nullptr, nullptr, nullptr, y_d, y_force_bf16, t_d, 1);
+        } else {
+            group(h + 4, 2, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_gu, true, t_gu, 1);
+            const int before = n;
+            group(h + 6, 1, nullptr, (const uint16_t*)tg->g_t, (const uint16_t*)tg->u_t, t, y_d, y_force_bf16, t_d, 1);
+            for (int i = before; i < n; ++i) stages[i].tt = tg->t_t;
+        }
     }
     return n;   // at most 7
+}
+
+// Builds the paired stack of a block's gate and up (row 2i = gate row i, row 2i+1 = up row i)
+// from the decoded contents of the two handles.  *out stays NULL where the shape has no paired
+// form (fewer than two rows per tile); the caller then keeps the two weights apart.
+sd2_status build_gate_up_pair(sd2_handle gate, sd2_handle up, sd2_handle* out)
+{
+    *out = nullptr;
+    const int64_t I = gate->M, K = gate->K;
+    if (up->M != I || up->K != K) return SD2_OK;
+    const Gap4Geom g = gap4_geometry(2 * I, K);
+    if (g.S == 0 || g.R < 2) return SD2_OK;
+    uint16_t* dense = (uint16_t*)std::malloc((size_t)(2 * I * K) * 2);
+    uint16_t* one = (uint16_t*)std::malloc((size_t)(I * K) * 2);
+    sd2_status st = (dense && one) ? SD2_OK : SD2_ERR_ALLOC;
+    for (int w = 0; w < 2 && st == SD2_OK; ++w) {
+        st = sd2_decompress(w == 0 ? gate : up, one);
+        if (st != SD2_OK) break;
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < I; ++i) std::memcpy(dense + (size_t)(2 * i + w) * K, one + (size_t)i * K, (size_t)K * 2);
+    }
+    std::free(one);
+    uint8_t* blob = nullptr;
+    int64_t bytes = 0;
+    if (st == SD2_OK) {
+        // no mask: what decoded to +0 was masked out (or was a kept zero, which adds nothing)
+        sd2_options opt = {SD2_FORMAT_GAP4_PAIRED, SD2_DTYPE_BF16};
+        st = pack_any(dense, nullptr, 2 * I, K, &opt, &blob, &bytes);
+    }
+    std::free(dense);
+    if (st != SD2_OK) return st;
+    BlobHeader hd;
+    std::memcpy(&hd, blob, sizeof hd);
+    st = upload(blob, bytes, hd, out);
+    std::free(blob);
+    return st;
 }
 
 }  // namespace
@@ -990,6 +1045,20 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         ok = ok && cudaMalloc((void**)&d->d_tags, (size_t)to) == cudaSuccess && cudaMemset(d->d_tags, 0, (size_t)to) == cudaSuccess;
     }
     int n = 0;
+    std::vector<sd2_handle> pairs((size_t)L, nullptr);
+    if (ok && tagged) {
+        for (int b = 0; b < L && st == SD2_OK; ++b) {
+            st = build_gate_up_pair(h[7 * b + 4], h[7 * b + 5], &pairs[(size_t)b]);
+            if (pairs[(size_t)b]) d->owned.push_back(pairs[(size_t)b]);
+        }
+        if (st != SD2_OK) {
+            for (sd2_handle p : d->owned) sd2_free(p);
+            cudaFree(d->d_ws); cudaFree(d->d_tags);
+            cudaGetLastError();
+            delete d;
+            return st;
+        }
+    }
     if (ok) {
         for (int b = 0; b < L; ++b) {
             uint8_t* base = d->d_ws;
@@ -1011,7 +1080,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
             n += append_block_stages(stages.data() + n, h + 7 * b, xin, (uint16_t*)(base + wo[0]), (uint16_t*)(base + wo[1]),
                                      (uint16_t*)(base + wo[2]), (uint16_t*)(base + wo[3]), (uint16_t*)(base + wo[4]),
                                      (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs, g_dev[dev].sms,
-                                     tagged ? &tg : nullptr);
+                                     tagged ? &tg : nullptr, pairs[(size_t)b]);
         }
         d->n_stages = n;
         ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
@@ -1019,12 +1088,14 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
              cudaMalloc((void**)&d->d_gbar, 256) == cudaSuccess && cudaMemset(d->d_gbar, 0, 256) == cudaSuccess;
     }
     if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
+        for (sd2_handle p : d->owned) sd2_free(p);
         cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar); cudaFree(d->d_tags);
         delete d;
         return SD2_ERR_UNSUPPORTED;
     }
     if (!ok) {
         cudaGetLastError();
+        for (sd2_handle p : d->owned) sd2_free(p);
         cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar); cudaFree(d->d_tags);
         cudaGetLastError();
         delete d;
@@ -1094,6 +1165,8 @@ sd2_status sd2_drafter_free(sd2_drafter d)
     if (cudaFree(d->d_stages) != cudaSuccess) st = SD2_ERR_CUDA;
     if (cudaFree(d->d_gbar) != cudaSuccess) st = SD2_ERR_CUDA;
     if (d->d_tags && cudaFree(d->d_tags) != cudaSuccess) st = SD2_ERR_CUDA;
+    for (sd2_handle p : d->owned)
+        if (sd2_free(p) != SD2_OK) st = SD2_ERR_CUDA;
     cudaGetLastError();
     delete d;
     return st;

@@ -34,7 +34,10 @@
 // + one 32-bit code word whose nibble i (bits 4i..4i+3) is entry i's gap.
 //
 // Rows are ordered by chunk count (most first, ties by row index), so that rows of like
-// density share a tile.  A tile is R = 32 / S consecutive rows of that order: 32 runs, one per
+// density share a tile.  A *paired* blob (header field `pairing` = 1; M even, S <= 16) orders
+// the row pairs (2i, 2i+1) instead, by the chunks of both rows together, and keeps each pair
+// in tile rows 2j and 2j+1: a kernel that holds gate row i as row 2i and up row i as row 2i+1
+// of one stacked matrix then finds both results of a pair in the same warp.  A tile is R = 32 / S consecutive rows of that order: 32 runs, one per
 // lane of a warp; lane l holds the run of window l % S of the tile's row l / S.  Lanes step
 // through their chunks together; step j of the tile stores chunk j of every lane that has
 // more than j chunks, in lane order, so each step is one contiguous, fully used run.
@@ -94,7 +97,8 @@ struct BlobHeader {
     uint32_t n_tiles;           // GAP4: T
     uint32_t max_tile_bytes;    // GAP4: largest tile record
     uint32_t overlap;           // GAP4: V, columns a lane's window reaches into its neighbours' strips
-    uint32_t reserved[3];
+    uint32_t pairing;           // GAP4: 1 = rows 2i and 2i+1 sit in tile rows 2j and 2j+1, else 0
+    uint32_t reserved[2];
     uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16 - 16 - 16];
 };
 static_assert(sizeof(BlobHeader) == 256, "header is 256 bytes");
@@ -314,11 +318,12 @@ inline void gap4_row_cols(const uint16_t* W, const uint8_t* mask, int64_t m, int
         if (is_kept(W, mask, m * K + k)) cols.push_back((int32_t)k);
 }
 
-inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype)
+inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype, bool pair_rows = false)
 {
     PackResult r;
     const Gap4Geom g = gap4_geometry(M, K);
     if (g.S == 0) { r.status = -5; return r; }
+    if (pair_rows && ((M & 1) || g.R < 2)) { r.status = -5; return r; }
     const int S = g.S, B = g.B, R = g.R, V = g.V;
     // per row: where each lane's run starts, chunks of each lane
     std::vector<int32_t> first((size_t)M * (S + 1));
@@ -347,8 +352,20 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     // rows by chunk count, most first, ties by index
     std::vector<uint32_t> order((size_t)M);
     std::iota(order.begin(), order.end(), 0u);
-    std::stable_sort(order.begin(), order.end(),
-                     [&](uint32_t a, uint32_t b) { return row_chunks[a] > row_chunks[b]; });
+    if (!pair_rows) {
+        std::stable_sort(order.begin(), order.end(),
+                         [&](uint32_t a, uint32_t b) { return row_chunks[a] > row_chunks[b]; });
+    } else {   // the same for pairs (2i, 2i+1), by the chunks of both rows
+        std::vector<uint32_t> pairs((size_t)(M / 2));
+        std::iota(pairs.begin(), pairs.end(), 0u);
+        std::stable_sort(pairs.begin(), pairs.end(), [&](uint32_t a, uint32_t b) {
+            return row_chunks[2 * (size_t)a] + row_chunks[2 * (size_t)a + 1] > row_chunks[2 * (size_t)b] + row_chunks[2 * (size_t)b + 1];
+        });
+        for (size_t i = 0; i < pairs.size(); ++i) {
+            order[2 * i] = 2 * pairs[i];
+            order[2 * i + 1] = 2 * pairs[i] + 1;
+        }
+    }
     const int64_t T = (M + R - 1) / R;
     const int hdr = gap4_tile_header_bytes(R);
     std::vector<uint32_t> toff((size_t)T + 1, 0);
@@ -377,6 +394,7 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     h.n_tiles = (uint32_t)T;
     h.max_tile_bytes = max_tile;
     h.overlap = (uint32_t)V;
+    h.pairing = pair_rows ? 1u : 0u;
     uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
     if (!blob) { r.status = -3; return r; }
     std::memcpy(blob + h.sec_off[0], toff.data(), sec[0]);
@@ -473,6 +491,7 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
     if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B || h.overlap != (uint32_t)g.V) return -6;
     const int S = g.S, B = g.B, R = g.R, V = g.V;
     const int64_t T = (M + R - 1) / R;
+    if (h.pairing > 1 || (h.pairing == 1 && ((M & 1) || R < 2))) return -6;
     if (h.n_tiles != (uint64_t)T || h.sec_bytes[0] != (uint64_t)(T + 1) * 4 || h.sec_bytes[2] != 0) return -6;
     if (h.sec_bytes[1] % 16) return -6;
     const uint32_t* toff = (const uint32_t*)(blob + h.sec_off[0]);
@@ -498,6 +517,11 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
                 return -6;
             }
         }
+        if (h.pairing == 1)
+            for (int rr = 0; rr + 1 < R; rr += 2) {
+                const bool none = rows[rr] == 0xFFFFFFFFu && rows[rr + 1] == 0xFFFFFFFFu;
+                if (!none && ((rows[rr] & 1u) || rows[rr + 1] != rows[rr] + 1u)) return -6;
+            }
     }
     if (dense) {
 #pragma omp parallel for schedule(static)

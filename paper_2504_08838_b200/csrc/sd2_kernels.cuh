@@ -121,7 +121,9 @@ struct SStage {
     int tiles_rem;         // T_total % grid size
     int tagged_in;         // x / g / u point at tagged 32-bit words written by the previous stage
     int V;                 // overlap: lane windows are strips widened by V columns on both sides
-    int reserved[3];
+    int paired;            // mat[0] stacks gate row i (row 2i) and up row i (row 2i+1), pairs share a tile:
+                           // the stage stores g, u, t_out (plain bf16, each may be NULL) and tt (tagged t)
+    int reserved[2];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
@@ -806,6 +808,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             publish_t_slice(K, N, (const uint32_t*)st.g + xoff, (const uint32_t*)st.u + xoff, st.tt + xoff,
                             st.t_out ? st.t_out + xoff : nullptr, tag_in, wc, ctid);
             stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, ctid, tag_in, wc);
+        } else if (st.paired) {   // g, u, t_out are this stage's outputs
+            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, ctid, tag_in, wc);
         } else {
             stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
                         st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid, tag_in, wc);
@@ -893,7 +897,34 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 r[n] = a0[n] + a1[n];
                 for (int dd = 1; dd < S; dd <<= 1) r[n] += __shfl_xor_sync(0xFFFFFFFFu, r[n], dd);
             }
-            if (strip == 0) {
+            if (st.paired) {
+                // tile rows 2j and 2j+1 are gate row i and up row i: the up result comes over from
+                // S lanes further on, and t = bf16(silu(bf16 g) * bf16 u) is formed right here
+                float ru[NT];
+#pragma unroll
+                for (int n = 0; n < NT; ++n) ru[n] = __shfl_down_sync(0xFFFFFFFFu, r[n], (unsigned)S);
+                const uint32_t trow = (uint32_t)(lane >> st.log2S);
+                if (strip == 0 && !(trow & 1u)) {
+                    const uint32_t row = lds_u32(tb + 144u + 4u * trow);
+                    if (row != 0xFFFFFFFFu) {
+                        const size_t I = (size_t)st.mat[0].M >> 1;
+                        uint16_t* gp = (uint16_t*)st.g;
+                        uint16_t* up = (uint16_t*)st.u;
+#pragma unroll
+                        for (int n = 0; n < NT; ++n) {
+                            if (n < N) {
+                                const size_t at = (size_t)(a.n0 + n) * I + (row >> 1);
+                                const uint16_t gb = f32_to_bf16_rne(r[n]), ub = f32_to_bf16_rne(ru[n]);
+                                const uint16_t tv = silu_mul_bits(gb, ub);
+                                st.tt[at] = ((uint32_t)tv << 16) | tag_out;
+                                if (gp) gp[at] = gb;
+                                if (up) up[at] = ub;
+                                if (st.t_out) st.t_out[at] = tv;
+                            }
+                        }
+                    }
+                }
+            } else if (strip == 0) {
                 const uint32_t row = lds_u32(tb + 144u + 4u * (uint32_t)(lane >> st.log2S));
                 if (row != 0xFFFFFFFFu) {
                     const SMat& md = st.mat[d.y];

@@ -4,6 +4,8 @@ Needs no GPU: ``sd2_pack_host`` / ``sd2_unpack_host`` are the same encoder and d
 ``sd2_compress`` / ``sd2_decompress`` use.  Expected dense matrices come from the oracle.
 """
 
+import struct
+
 import numpy as np
 import pytest
 
@@ -135,7 +137,7 @@ def _gap4_run_chunks(cols):
     return (e + 7) // 8
 
 
-def _gap4_bytes(mask):
+def _gap4_bytes(mask, paired=False):
     """Compressed bytes of a mask: tile offsets + per tile (header, code words, values)."""
     M, K = mask.shape
     S, B, R = _gap4_geometry(M, K)
@@ -145,7 +147,11 @@ def _gap4_bytes(mask):
         first = _gap4_deal_row(cols, S, B, GAP4_OVERLAP)
         row_chunks.append(sum(_gap4_run_chunks(cols[first[l]:first[l + 1]]) for l in range(S)))
     row_chunks = np.array(row_chunks)
-    order = np.argsort(-row_chunks, kind="stable")
+    if paired:      # pairs (2i, 2i+1) ordered by the chunks of both rows, each pair kept together
+        pair_order = np.argsort(-(row_chunks[0::2] + row_chunks[1::2]), kind="stable")
+        order = np.stack([2 * pair_order, 2 * pair_order + 1], axis=1).reshape(-1)
+    else:
+        order = np.argsort(-row_chunks, kind="stable")
     T = (M + R - 1) // R
     hdr = (144 + 4 * R + 15) // 16 * 16
     total = 4 * (T + 1)
@@ -182,6 +188,61 @@ def test_gap4_geometries_and_ragged_tiles():
     W = synth.normal_bf16(43, (K + 1, K), 0.02)
     dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
     assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+
+
+def _tile_rows(blob):
+    """Row ids of every tile, read from the records (header layout as documented with the format)."""
+    M, K = struct.unpack_from("<qq", blob, 24)
+    sec_off = struct.unpack_from("<4Q", blob, 64)
+    S, B, T = struct.unpack_from("<3I", blob, 144)
+    R = 32 // S
+    toff = np.frombuffer(blob, np.uint32, T + 1, sec_off[0])
+    return [np.frombuffer(blob, np.uint32, R, sec_off[1] + 16 * int(toff[t]) + 144) for t in range(T)], M
+
+
+def test_paired_blobs_keep_row_pairs_in_one_tile():
+    for M, K, d in ((64, 300, 0.5), (1000, 1024, 0.5), (4098, 130, 0.3), (2, 300, 0.5)):
+        W, mask = _case(91 + M, M, K, d)
+        mask[4::10, :] = 0                                        # some pairs of very different rows
+        blob = sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)
+        dense, info = sd2.sd2_unpack_host(blob)
+        assert info["format"] == sd2.SD2_FORMAT_GAP4              # an ordering of GAP4, not another format
+        assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+        assert info["compressed_bytes"] == _gap4_bytes(mask, paired=True)
+        tiles, M_hdr = _tile_rows(blob)
+        assert M_hdr == M
+        seen = []
+        for rows in tiles:
+            for j in range(0, len(rows), 2):
+                a, b = int(rows[j]), int(rows[j + 1])
+                if a == 0xFFFFFFFF:
+                    assert b == 0xFFFFFFFF
+                else:
+                    assert a % 2 == 0 and b == a + 1
+                    seen.append(a)
+        assert sorted(seen) == list(range(0, M, 2))
+
+
+def test_paired_needs_even_rows_and_two_rows_per_tile():
+    W, mask = _case(95, 7, 300, 0.5)
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)    # odd M
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+    W, mask = _case(96, 2048, 4096, 0.05)                         # 32 strips: one row per tile
+    assert _gap4_geometry(2048, 4096)[2] == 1
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+
+
+def test_a_blob_that_claims_pairing_without_it_is_rejected():
+    W, mask = _case(97, 64, 300, 0.5)
+    mask[::3, :] = 0                                              # the plain order splits pairs
+    blob = bytearray(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+    struct.pack_into("<I", blob, 164, 1)                          # header field `pairing`
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_unpack_host(bytes(blob))
+    assert e.value.status == sd2.SD2_ERR_CORRUPT
 
 
 def test_gap4_is_unsupported_for_very_wide_matrices():
