@@ -123,8 +123,9 @@ sd2_status sd2_free(sd2_handle h);
 /* ---- the hot path -------------------------------------------------------------------- */
 
 /* Y = X (W.*mask)^T.   X: device bf16 [N*K].   Y: device [N*M], bf16 or fp32 per the
- * handle's y_dtype.  N = 0 is a no-op; N > 4 (GAP4) or N > 8 (BITMASK) is processed in panels
- * of at most that many rows of X (the weight is re-read for each panel).  cuda_stream is a
+ * handle's y_dtype.  N = 0 is a no-op; more than 8 rows (GAP4: fewer where the staged rows of a
+ * wide layer would crowd the weight ring out of shared memory, e.g. 4 for K = 8192) are processed
+ * in panels of at most that many rows of X (the weight is re-read for each panel).  cuda_stream is a
  * cudaStream_t (NULL = default stream).  X and Y need only their natural alignment; all
  * activations are expected to be finite (a filler entry of the GAP4 format multiplies +0 by
  * the activation of a masked-out column). */

@@ -46,7 +46,7 @@ struct sd2_drafter_s {
     int64_t tags_bytes;
     int64_t last_n;            // rows of the previous step: a change clears d_tags (stale tags of other rows)
     int K_max, max_tile;       // what decides the shared-memory split
-    int xs_need[3];            // bytes of staged activations at panel widths 1, 2, 4
+    int xs_need[4];            // bytes of staged activations at panel widths 1, 2, 4, 8
 };
 
 namespace {
@@ -114,7 +114,8 @@ sd2_status ensure_device(int* dev_out)
         int sms = 0, khz = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess) {
+        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess ||
+            set_smem_attr<8>() != cudaSuccess) {
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
@@ -287,7 +288,7 @@ sd2_status run_bitmask(const sd2_handle* hs, int count, const uint16_t* x, const
 
 // ------------------------------------------------------------------ GAP4 programs
 
-// Largest panel width (4, 2, 1) whose staged activations leave room for a ring that holds
+// Largest panel width (8, 4, 2, 1) whose staged activations leave room for a ring that holds
 // `max_tile` bytes at least twice; 0 if even one row does not fit.
 struct SmemPlan {
     int nt, xs_bytes, xlin_bytes, ring_bytes;
@@ -295,7 +296,7 @@ struct SmemPlan {
 
 int xs_bytes_for(int S, int B, int V, int nt)
 {
-    const int groups = 32 / nt;
+    const int groups = 32 / xs_words(nt);
     const int planes = S > groups ? S / groups : 1;
     return planes * ((B + 2 * V + kGap4Slack + 3) & ~3) * 128;
 }
@@ -337,7 +338,8 @@ sd2_status launch_stream(int nt, const SArgs& a, int grid, bool cooperative, cud
     switch (nt) {
         case 1: return launch_stream_nt<1>(a, grid, smem, cooperative, s);
         case 2: return launch_stream_nt<2>(a, grid, smem, cooperative, s);
-        default: return launch_stream_nt<4>(a, grid, smem, cooperative, s);
+        case 4: return launch_stream_nt<4>(a, grid, smem, cooperative, s);
+        default: return launch_stream_nt<8>(a, grid, smem, cooperative, s);
     }
 }
 
@@ -397,7 +399,7 @@ long long wait_budget(int dev)
 // Tracks what a program needs from shared memory.
 struct ProgramNeeds {
     int K_max = 0, max_tile = 0, tiles_max = 0;
-    int xs_need[3] = {0, 0, 0};   // staged activations at panel widths 1, 2, 4: the largest over all stages
+    int xs_need[4] = {0, 0, 0, 0};   // staged activations at panel widths 1, 2, 4, 8: the largest over all stages
     void add(const sd2_handle* hs, int count)
     {
         int T = 0;
@@ -406,7 +408,7 @@ struct ProgramNeeds {
             const int lin = hs[i]->S * hs[i]->B + 2 * hs[i]->V + 64;
             if (lin > K_max) K_max = lin;
             if (hs[i]->max_tile_bytes > max_tile) max_tile = hs[i]->max_tile_bytes;
-            for (int w = 0; w < 3; ++w) {
+            for (int w = 0; w < 4; ++w) {
                 const int need = xs_bytes_for(hs[i]->S, hs[i]->B, hs[i]->V, 1 << w);
                 if (need > xs_need[w]) xs_need[w] = need;
             }
@@ -416,23 +418,23 @@ struct ProgramNeeds {
     }
 };
 
-int nt_index(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : 2; }
+int nt_index(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : nt == 4 ? 2 : 3; }
 
-// Widest panel (4, 2, 1 rows) whose staged activations still leave room for the ring; 0 if none.
-int widest_panel(const int xs_need[3], int K_max, int max_tile)
+// Widest panel (8, 4, 2, 1 rows) whose staged activations still leave room for the ring; 0 if none.
+int widest_panel(const int xs_need[4], int K_max, int max_tile)
 {
     // a wide panel whose activations crowd out the ring cannot stream: ask for a ring of at
     // least 96 KB first, and settle for whatever fits only if no width leaves that much
     SmemPlan p;
-    for (int nt = 4; nt >= 1; nt >>= 1)
+    for (int nt = 8; nt >= 1; nt >>= 1)
         if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p) && p.ring_bytes >= 96 * 1024) return nt;
-    for (int nt = 4; nt >= 1; nt >>= 1)
+    for (int nt = 8; nt >= 1; nt >>= 1)
         if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return nt;
     return 0;
 }
 
 // Launches a program over all N rows, in panels of at most `nt_cap` rows (rows are independent).
-sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[3], int K_max, int max_tile, int grid, cudaStream_t s)
+sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[4], int K_max, int max_tile, int grid, cudaStream_t s)
 {
     const int nt_cap = widest_panel(xs_need, K_max, max_tile);
     if (nt_cap == 0) return SD2_ERR_UNSUPPORTED;
@@ -1103,7 +1105,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
     }
     d->K_max = needs.K_max;
     d->max_tile = needs.max_tile;
-    for (int w = 0; w < 3; ++w) d->xs_need[w] = needs.xs_need[w];
+    for (int w = 0; w < 4; ++w) d->xs_need[w] = needs.xs_need[w];
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live_drafters.insert(d);

@@ -77,8 +77,10 @@ __device__ __forceinline__ float warp_sum(float v)
 // per chunk: E = even nibbles, O = odd nibbles as bytes; P = (E + O) * 0x01010100 is the
 // exclusive prefix of the pair sums; PE = P + E and PO = PE + O are the inclusive gap
 // prefixes of the even and odd entries; entry i sits at local column cursor + prefix_i + i.
-// The activations live in shared memory as xs[column][32 / NT groups][NT]: lane l reads
-// group l % (32 / NT), so one warp-wide gather touches every bank once.
+// The activations live in shared memory as xs[column][groups][W words], 32 words per column: a
+// word holds one bf16 (NT = 1, in the high half) or the bf16 values of two activation rows
+// (row 2j in the low half, row 2j+1 in the high half of word j), W = max(1, NT / 2), groups =
+// 32 / W.  Lane l reads group l % groups, so one warp-wide gather touches every bank W times.
 //
 // Every wait (ring barriers, grid barrier) is bounded by a cycle budget: when it runs out
 // the CTA raises the error word and winds down instead of hanging.
@@ -87,6 +89,8 @@ __device__ __forceinline__ float warp_sum(float v)
 #define SD2_CONSUMER_WARPS 16
 #endif
 constexpr int kConsumerWarps = SD2_CONSUMER_WARPS;
+// words of staged activations a lane reads per gathered column, at a panel width of nt rows
+__host__ __device__ constexpr int xs_words(int nt) { return nt <= 2 ? 1 : nt / 2; }
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
 constexpr int kSlots = 64;                               // tiles in flight per CTA, at most
@@ -251,28 +255,6 @@ __device__ __forceinline__ uint4 lds_u32x4_off(uint32_t a)
     return v;
 }
 
-// c + w * x for bf16 w and x with an fp32 sum (the product of two bf16 values is exact in
-// fp32, so this equals an fp32 fused multiply-add of the widened values).  w is the low or the
-// high half of `wpair`; x is the high half of `xword`, an fp32 whose low 16 bits are zero.
-__device__ __forceinline__ float fma_bf16_lo(uint32_t wpair, uint32_t xword, float c)
-{
-    float d;
-    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\t"
-        "fma.rn.f32.bf16 %0, wl, xh, %3;\n\t}"
-        : "=f"(d)
-        : "r"(wpair), "r"(xword), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float fma_bf16_hi(uint32_t wpair, uint32_t xword, float c)
-{
-    float d;
-    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\t"
-        "fma.rn.f32.bf16 %0, wh, xh, %3;\n\t}"
-        : "=f"(d)
-        : "r"(wpair), "r"(xword), "f"(c));
-    return d;
-}
-
 // c + 128 * byte K8 of p (one integer dot-product instruction with a one-hot operand)
 template <int K8>
 __device__ __forceinline__ uint32_t byte_times_128_plus(uint32_t p, uint32_t c)
@@ -331,25 +313,53 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, const 
 
 // acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`;
 // w is the low (HI = 0) or high (HI = 1) bf16 of `wpair`.
+// c + w * x for bf16 w and x with an fp32 sum (the product of two bf16 values is exact in fp32,
+// so this equals an fp32 fused multiply-add of the widened values): w = half WH of wpair,
+// x = half XH of xword (0: low, 1: high)
+template <int WH, int XH>
+__device__ __forceinline__ float fma_bf16_sel(uint32_t wpair, uint32_t xword, float c)
+{
+    float d;
+    if (WH == 0 && XH == 0)
+        asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\tfma.rn.f32.bf16 %0, wl, xl, %3;\n\t}" : "=f"(d) : "r"(wpair), "r"(xword), "f"(c));
+    else if (WH == 0)
+        asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\tfma.rn.f32.bf16 %0, wl, xh, %3;\n\t}" : "=f"(d) : "r"(wpair), "r"(xword), "f"(c));
+    else if (XH == 0)
+        asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\tfma.rn.f32.bf16 %0, wh, xl, %3;\n\t}" : "=f"(d) : "r"(wpair), "r"(xword), "f"(c));
+    else
+        asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\tmov.b32 {wl, wh}, %1;\n\tmov.b32 {xl, xh}, %2;\n\tfma.rn.f32.bf16 %0, wh, xh, %3;\n\t}" : "=f"(d) : "r"(wpair), "r"(xword), "f"(c));
+    return d;
+}
+
+// acc[n] += w * x[n] for the NT activation rows packed in the words at `addr + OFF`;
+// w is the low (HI = 0) or high (HI = 1) bf16 of `wpair`.
 template <int NT, int OFF, int HI>
 __device__ __forceinline__ void fma_at(float (&acc)[NT], uint32_t wpair, uint32_t addr)
 {
-    uint32_t x[NT];
-    if (NT == 1) {
+    constexpr int W = xs_words(NT);
+    uint32_t x[W];
+    if (W == 1) {
         x[0] = lds_u32_off<OFF>(addr);
-    } else if (NT == 2) {
+    } else if (W == 2) {
         const uint2 t = lds_u32x2_off<OFF>(addr);
         x[0] = t.x;
-        x[NT - 1] = t.y;
+        x[W - 1] = t.y;
     } else {
         const uint4 t = lds_u32x4_off<OFF>(addr);
         x[0] = t.x;
-        x[1 % NT] = t.y;
-        x[2 % NT] = t.z;
-        x[3 % NT] = t.w;
+        x[1 % W] = t.y;
+        x[2 % W] = t.z;
+        x[3 % W] = t.w;
     }
+    if (NT == 1) {
+        acc[0] = fma_bf16_sel<HI, 1>(wpair, x[0], acc[0]);
+    } else {
 #pragma unroll
-    for (int n = 0; n < NT; ++n) acc[n] = HI ? fma_bf16_hi(wpair, x[n], acc[n]) : fma_bf16_lo(wpair, x[n], acc[n]);
+        for (int n = 0; n < NT; n += 2) {
+            acc[n] = fma_bf16_sel<HI, 0>(wpair, x[n / 2], acc[n]);
+            acc[n + 1 < NT ? n + 1 : n] = fma_bf16_sel<HI, 1>(wpair, x[n / 2], acc[n + 1 < NT ? n + 1 : n]);
+        }
+    }
 }
 
 // One chunk: eight (gap, value) entries against the activations at `xb` (the lane's cursor).
@@ -495,7 +505,8 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                                         const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int ctid,
                                         uint32_t tag, const WaitCtx& wc)
 {
-    constexpr int kGroups = 32 / NT;
+    constexpr int W = xs_words(NT);
+    constexpr int kGroups = 32 / W;
     const int K = st.K, S = st.S, B = st.B;
     const bool glue = x_src == nullptr;
     const int planes = S > kGroups ? S / kGroups : 1;
@@ -563,11 +574,19 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                 const uint32_t sh = (uint32_t)(e & 1) << 4;
                 uint32_t t0 = __funnelshift_r(w0, w1, sh), t1 = __funnelshift_r(w1, w2, sh);
                 if (n >= N) t0 = t1 = 0u;
-                float* dst = xp + ((size_t)c * kGroups + grp) * NT + n;
-                dst[0] = bf16_lo(t0);
-                dst[32] = bf16_hi(t0);
-                dst[64] = bf16_lo(t1);
-                dst[96] = bf16_hi(t1);
+                if (NT == 1) {   // one word per column, the value in its high half
+                    float* dst = xp + (size_t)c * 32 + grp;
+                    dst[0] = bf16_lo(t0);
+                    dst[32] = bf16_hi(t0);
+                    dst[64] = bf16_lo(t1);
+                    dst[96] = bf16_hi(t1);
+                } else {         // row n is half n % 2 of word n / 2
+                    uint16_t* dst = (uint16_t*)xp + ((size_t)c * 32 + grp * W) * 2 + n;
+                    dst[0] = (uint16_t)t0;
+                    dst[64] = (uint16_t)(t0 >> 16);
+                    dst[128] = (uint16_t)t1;
+                    dst[192] = (uint16_t)(t1 >> 16);
+                }
             }
         }
         named_bar_sync(1, kConsumerThreads);
@@ -760,7 +779,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     // a barrier, from a word that only thread 0 writes.
     // The descriptor of stage s sits in sh->stage[s & 1]: warp 1 fetches the next stage's while
     // the current one is computed; the barrier at the end of the stage makes it visible.
-    constexpr int kGroups = 32 / NT;
+    constexpr int kGroups = 32 / xs_words(NT);
     constexpr int kStageWords = (int)(sizeof(SStage) / 4);
     const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
     const int N = a.N;
@@ -826,7 +845,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const int strip = lane & (S - 1);
         const int plane = S > kGroups ? strip / kGroups : 0;
         const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)(((st.B + 2 * st.V + kGap4Slack + 3) & ~3) * 128) +
-                                 (uint32_t)(lane % kGroups) * (4u * NT);
+                                 (uint32_t)(lane % kGroups) * (4u * xs_words(NT));
         const uint32_t lt = (1u << lane) - 1u;
         const bool last_stage = s == a.n_stages - 1;
 
