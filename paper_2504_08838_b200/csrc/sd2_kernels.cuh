@@ -285,7 +285,7 @@ struct StreamShared {
     int abort_flag;                    // any warp: a bounded wait ran out
     int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
     unsigned int tag_base;             // tagged programs: (launch counter & 0xFF) << 8
-    int pad[1];
+    unsigned int next_q;               // next tile (sequence number) no consumer warp has taken yet
 };
 
 struct WaitCtx {
@@ -617,6 +617,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         }
         sh->abort_flag = 0;
         sh->stage_dead = 0;
+        sh->next_q = (unsigned int)kConsumerWarps;   // warp w starts on tile w
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -783,7 +784,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     constexpr int kStageWords = (int)(sizeof(SStage) / 4);
     const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
     const int N = a.N;
+    // Tiles go to whichever consumer warp is free next: a warp holds one sequence number and draws
+    // the next from a shared counter when it is done.  Numbers run on across stages, so a number
+    // drawn past the end of a stage is simply the warp's first tile of the next one.
     uint32_t qbase = 0;
+    uint32_t q_mine = (uint32_t)warp;
     bool failed = false;
     if (warp == 1) {
         const uint32_t* src = (const uint32_t*)(a.ext ? a.ext : &a.inl[0]);
@@ -849,8 +854,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const uint32_t lt = (1u << lane) - 1u;
         const bool last_stage = s == a.n_stages - 1;
 
-        for (int k = warp; k < n_cta && !failed; k += kConsumerWarps) {
-            const uint32_t q = qbase + (uint32_t)k;
+#ifdef SD2_TRACE
+        long long trace_wait = 0;   // cycles this warp waited for tiles to land, stored once per stage
+#endif
+        while ((int)(q_mine - (qbase + (uint32_t)n_cta)) < 0 && !failed) {
+            const uint32_t q = q_mine;
             const uint32_t slot = q % kSlots;
 #ifdef SD2_TRACE
             const long long tw0 = clock64();
@@ -858,9 +866,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
 #endif
             if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
 #ifdef SD2_TRACE
-            if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] += clock64() - tw0;
+            trace_wait += clock64() - tw0;
 #endif
-            if (ctid == 0 && k == 0) SD2_STAMP(3);
+            if (ctid == 0 && q == qbase) SD2_STAMP(3);
             if (lane == 0) SD2_TILE_STAMP(q, 2);
             const int4 d = sh->desc[slot];
             const uint32_t tb = ring0 + (uint32_t)d.x;
@@ -970,10 +978,18 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             }
             __syncwarp();
             if (lane == 0) SD2_TILE_STAMP(q, 3);
-            if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+            uint32_t q_next = 0;
+            if (lane == 0) {
+                mbar_arrive(empty0 + 8 * slot);
+                q_next = atomicAdd(&sh->next_q, 1u);
+            }
+            q_mine = __shfl_sync(0xFFFFFFFFu, q_next, 0);
         }
         qbase += (uint32_t)n_cta;
         if (ctid == 0) SD2_STAMP(4);
+#ifdef SD2_TRACE
+        if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] = trace_wait;
+#endif
         // everything this CTA wrote in the stage is visible before it arrives at the barrier
         named_bar_sync(1, kConsumerThreads);
         if (ctid == 0) SD2_STAMP(5);
