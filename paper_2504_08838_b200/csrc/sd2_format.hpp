@@ -17,7 +17,7 @@
 //            (sec2 is empty)
 //
 // GAP4 in detail.  The K columns are cut into S strips of B columns (S a power of two <= 32,
-// S * B >= K, B odd) and every strip, widened by V columns on both sides, is the *window* of
+// S * B >= K, B = 2 mod 4) and every strip, widened by V columns on both sides, is the *window* of
 // one lane.  A row's kept entries, in ascending column order, are dealt to the S lanes in
 // consecutive runs: every lane gets the same number of whole 8-entry chunks where the windows
 // allow it (a lane must take what the next lane's window cannot reach and cannot take what lies
@@ -115,17 +115,26 @@ struct Gap4Geom {
 SD2_HD int gap4_tile_header_bytes(int R) { return (144 + 4 * R + 15) & ~15; }
 
 // Picks S: enough tiles to spread over every SM's warps, strips neither too narrow (padding)
-// nor wider than the chunk counters allow.  B is odd so that strips start in distinct
-// shared-memory banks when a kernel transposes the activations.  S == 0: K is too large.
+// nor wider than the chunk counters allow.  B is twice an odd number: in a linear row of bf16
+// activations the strips then start on 32-bit words in distinct shared-memory banks, and so does
+// every fourth column of them, which is how a kernel spreads the row over the lanes' windows.
+// S == 0: K is too large.
+// Columns per strip: the smallest B >= K / S with B = 2 (mod 4).
+inline int64_t gap4_strip_cols(int64_t K, int S)
+{
+    const int64_t b = (K + S - 1) / S;
+    return b + ((6 - (b & 3)) & 3);
+}
+
 inline Gap4Geom gap4_geometry(int64_t M, int64_t K)
 {
     int S = 1;
     while (S < 32 && M * S / 32 < kGap4TileTarget) S <<= 1;
     while (S > 1 && (K + S - 1) / S < kGap4MinStrip) S >>= 1;
-    while (S < 32 && ((K + S - 1) / S | 1) > kGap4MaxStrip) S <<= 1;
+    while (S < 32 && gap4_strip_cols(K, S) > kGap4MaxStrip) S <<= 1;
     Gap4Geom g;
     g.S = S;
-    g.B = (int)((K + S - 1) / S) | 1;
+    g.B = (int)gap4_strip_cols(K, S);
     g.R = 32 / S;
     g.V = kGap4Overlap;
     if (g.B > kGap4MaxStrip) g.S = 0;

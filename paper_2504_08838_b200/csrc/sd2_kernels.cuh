@@ -558,8 +558,9 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
         }
         named_bar_sync(1, kConsumerThreads);
         // scatter row n: consecutive threads take consecutive groups; each takes four window rows
-        // of its group from three aligned 32-bit reads (window row c of strip s is element
-        // s * B + c of xlin)
+        // of its group from two aligned 32-bit reads (window row c of strip s is element
+        // s * B + c of xlin; B is even and c a multiple of 4, and B / 2 is odd, so the threads of
+        // a warp read 32 different banks)
         const int per_plane = (rows4 >> 2) * kGroups;
         const uint32_t* xl32 = (const uint32_t*)xlin;
         for (int p = 0; p < planes; ++p) {
@@ -569,10 +570,8 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
 #pragma unroll 2
             for (int i = ctid; i < per_plane; i += kConsumerThreads) {
                 const int c = (i / kGroups) << 2;
-                const int e = strip * B + c;
-                const uint32_t w0 = xl32[e >> 1], w1 = xl32[(e >> 1) + 1], w2 = xl32[(e >> 1) + 2];
-                const uint32_t sh = (uint32_t)(e & 1) << 4;
-                uint32_t t0 = __funnelshift_r(w0, w1, sh), t1 = __funnelshift_r(w1, w2, sh);
+                const int e = (strip * B + c) >> 1;
+                uint32_t t0 = xl32[e], t1 = xl32[e + 1];
                 if (n >= N) t0 = t1 = 0u;
                 if (NT == 1) {   // one word per column, the value in its high half
                     float* dst = xp + (size_t)c * 32 + grp;

@@ -95,9 +95,14 @@ def _gap4_geometry(M, K):
         S *= 2
     while S > 1 and (K + S - 1) // S < 64:
         S //= 2
-    while S < 32 and ((K + S - 1) // S | 1) > 496:
+    def strip_cols(S):                      # the smallest B >= K / S that is twice an odd number
+        b = (K + S - 1) // S
+        while b % 4 != 2:
+            b += 1
+        return b
+    while S < 32 and strip_cols(S) > 496:
         S *= 2
-    return S, (K + S - 1) // S | 1, 32 // S
+    return S, strip_cols(S), 32 // S
 
 
 def _gap4_deal_row(cols, S, B, V):
