@@ -304,7 +304,7 @@ int xs_bytes_for(int S, int B, int V, int nt)
 bool plan_smem(int nt, int xs_max, int K_max, int max_tile, SmemPlan* p)
 {
     const int fixed = (int)((sizeof(StreamShared) + 127) & ~127);
-    const int xlin = (2 * K_max + 127) & ~127;
+    const int xlin = ((2 * K_max + 127) & ~127) * (nt > 2 ? 2 : 1);   // panels of 4 and 8 go two rows at a time
     const int ring = (kSmemMax - fixed - xs_max - xlin) & ~127;
     if (ring < 2 * max_tile + 256) return false;
     p->nt = nt;

@@ -500,33 +500,42 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
 }
 
 // `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged).
+// Panels of four and eight rows go two rows at a time: both rows are fetched into their own linear
+// buffer (xlin holds two, `xlin_row` elements apart), then one scatter writes the packed words.
+// (Panels of two keep one buffer and take a pass per row: the second buffer would come out of the
+// weight ring, which costs them more than the extra pass.)
 template <int NT>
 __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
-                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int ctid,
+                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int xlin_row, int ctid,
                                         uint32_t tag, const WaitCtx& wc)
 {
     constexpr int W = xs_words(NT);
     constexpr int kGroups = 32 / W;
+    constexpr int kRowsPerPass = NT <= 2 ? 1 : 2;
     const int K = st.K, S = st.S, B = st.B;
     const bool glue = x_src == nullptr;
     const int planes = S > kGroups ? S / kGroups : 1;
     const int rows = B + 2 * st.V + kGap4Slack;     // a lane's window and the slack
     const int rows4 = (rows + 3) & ~3;              // the scatter works on four rows at a time
-    // the linear row sits V elements into xlin, with zeros before it and behind it, so that
-    // the scatter can read any window without bounds checks
-    uint16_t* xl = xlin + st.V;
     const int tail_pad = S * B - K + st.V + 48;
     const bool vec = (K % 8 == 0) && ((((uintptr_t)x_src | (uintptr_t)g | (uintptr_t)u | (uintptr_t)t_out) & 15) == 0);
     const bool pub = glue && t_out && blockIdx.x == 0;
-    for (int n = 0; n < NT; ++n) {
-        for (int i = ctid; i < st.V; i += kConsumerThreads) xlin[i] = 0;
-        for (int i = ctid; i < tail_pad; i += kConsumerThreads) xl[K + i] = 0;
-        if (n < N && tag != 0u) {
-            stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
-                                g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
-                                t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag, wc, ctid);
-        } else if (n < N) {
-            if (vec) {
+    for (int n0 = 0; n0 < NT; n0 += kRowsPerPass) {
+#pragma unroll
+        for (int r = 0; r < kRowsPerPass; ++r) {
+            const int n = n0 + r;
+            if (n >= N) continue;   // the scatter writes zeros for this row
+            // the linear row sits V elements into its buffer, with zeros before it and behind it, so
+            // that the scatter can read any window without bounds checks
+            uint16_t* xb = xlin + (size_t)r * xlin_row;
+            uint16_t* xl = xb + st.V;
+            for (int i = ctid; i < st.V; i += kConsumerThreads) xb[i] = 0;
+            for (int i = ctid; i < tail_pad; i += kConsumerThreads) xl[K + i] = 0;
+            if (tag != 0u) {
+                stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
+                                    g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
+                                    t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag, wc, ctid);
+            } else if (vec) {
                 for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
                     uint4 v;
                     if (!glue) {
@@ -557,12 +566,14 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
             }
         }
         named_bar_sync(1, kConsumerThreads);
-        // scatter row n: consecutive threads take consecutive groups; each takes four window rows
-        // of its group from two aligned 32-bit reads (window row c of strip s is element
-        // s * B + c of xlin; B is even and c a multiple of 4, and B / 2 is odd, so the threads of
-        // a warp read 32 different banks)
+        // scatter: consecutive threads take consecutive groups; each takes four window rows of its
+        // group from two aligned 32-bit reads per activation row (window row c of strip s is element
+        // s * B + c of the linear buffer; B is even and c a multiple of 4, and B / 2 is odd, so the
+        // threads of a warp read 32 different banks)
         const int per_plane = (rows4 >> 2) * kGroups;
-        const uint32_t* xl32 = (const uint32_t*)xlin;
+        const uint32_t* xa32 = (const uint32_t*)xlin;
+        const uint32_t* xb32 = (const uint32_t*)(xlin + xlin_row);
+        const bool have_a = n0 < N, have_b = n0 + 1 < N;
         for (int p = 0; p < planes; ++p) {
             float* xp = xs + (size_t)p * rows4 * 32;
             const int grp = ctid % kGroups;
@@ -571,20 +582,28 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
             for (int i = ctid; i < per_plane; i += kConsumerThreads) {
                 const int c = (i / kGroups) << 2;
                 const int e = (strip * B + c) >> 1;
-                uint32_t t0 = xl32[e], t1 = xl32[e + 1];
-                if (n >= N) t0 = t1 = 0u;
+                uint32_t t0 = 0u, t1 = 0u;
+                if (have_a) { t0 = xa32[e]; t1 = xa32[e + 1]; }
                 if (NT == 1) {   // one word per column, the value in its high half
                     float* dst = xp + (size_t)c * 32 + grp;
                     dst[0] = bf16_lo(t0);
                     dst[32] = bf16_hi(t0);
                     dst[64] = bf16_lo(t1);
                     dst[96] = bf16_hi(t1);
-                } else {         // row n is half n % 2 of word n / 2
-                    uint16_t* dst = (uint16_t*)xp + ((size_t)c * 32 + grp * W) * 2 + n;
+                } else if (kRowsPerPass == 1) {   // row n0 is half n0 % 2 of word n0 / 2
+                    uint16_t* dst = (uint16_t*)xp + ((size_t)c * 32 + grp * W) * 2 + n0;
                     dst[0] = (uint16_t)t0;
                     dst[64] = (uint16_t)(t0 >> 16);
                     dst[128] = (uint16_t)t1;
                     dst[192] = (uint16_t)(t1 >> 16);
+                } else {         // rows n0 and n0 + 1 are the two halves of word n0 / 2
+                    uint32_t u0 = 0u, u1 = 0u;
+                    if (have_b) { u0 = xb32[e]; u1 = xb32[e + 1]; }
+                    uint32_t* dst = (uint32_t*)xp + (size_t)c * 32 + grp * W + (n0 >> 1);
+                    dst[0] = __byte_perm(t0, u0, 0x5410);
+                    dst[32] = __byte_perm(t0, u0, 0x7632);
+                    dst[64] = __byte_perm(t1, u1, 0x5410);
+                    dst[96] = __byte_perm(t1, u1, 0x7632);
                 }
             }
         }
@@ -783,6 +802,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     constexpr int kStageWords = (int)(sizeof(SStage) / 4);
     const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
     const int N = a.N;
+    const int xlin_row = NT <= 2 ? 0 : a.xlin_bytes >> 2;   // elements between the two linear buffers of a pass
     // Tiles go to whichever consumer warp is free next: a warp holds one sequence number and draws
     // the next from a shared counter when it is done.  Numbers run on across stages, so a number
     // drawn past the end of a stage is simply the warp's first tile of the next one.
@@ -830,12 +850,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             // glue: this CTA's share of t first, then all of t like any tagged activation
             publish_t_slice(K, N, (const uint32_t*)st.g + xoff, (const uint32_t*)st.u + xoff, st.tt + xoff,
                             st.t_out ? st.t_out + xoff : nullptr, tag_in, wc, ctid);
-            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, ctid, tag_in, wc);
+            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
         } else if (st.paired) {   // g, u, t_out are this stage's outputs
-            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, ctid, tag_in, wc);
+            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
         } else {
             stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
-                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, ctid, tag_in, wc);
+                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
         }
         if (ctid == 0) SD2_STAMP(2);
         if (warp == 1 && s + 1 < a.n_stages) {
