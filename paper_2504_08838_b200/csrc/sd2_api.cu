@@ -46,6 +46,7 @@ struct sd2_drafter_s {
     int64_t tags_bytes;
     int64_t last_n;            // rows of the previous step: a change clears d_tags (stale tags of other rows)
     int K_max, max_tile;       // what decides the shared-memory split
+    int free_tiles;            // every stage has enough tiles per CTA for free tile assignment
     int xs_need[4];            // bytes of staged activations at panel widths 1, 2, 4, 8
 };
 
@@ -399,7 +400,11 @@ long long wait_budget(int dev)
 // Tracks what a program needs from shared memory.
 struct ProgramNeeds {
     int K_max = 0, max_tile = 0, tiles_max = 0;
+    int tiles_min = 0x7FFFFFFF;   // fewest tiles of any stage
     int xs_need[4] = {0, 0, 0, 0};   // staged activations at panel widths 1, 2, 4, 8: the largest over all stages
+    // Free tile assignment pays where every stage gives a CTA about as many tiles as it has consumer
+    // warps, or more; with fewer, the fixed deal is faster (see the consumer loop of stream_kernel).
+    int free_tiles(int grid) const { return tiles_min >= 12 * grid ? 1 : 0; }
     void add(const sd2_handle* hs, int count)
     {
         int T = 0;
@@ -415,6 +420,7 @@ struct ProgramNeeds {
             T += hs[i]->T;
         }
         if (T > tiles_max) tiles_max = T;
+        if (T < tiles_min) tiles_min = T;
     }
 };
 
@@ -466,6 +472,7 @@ sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, 
     if (!coop) set_stage_grid(a.inl[0], grid);
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
+    a.free_tiles = needs.free_tiles(grid);
     a.gbar = coop ? g_dev[dev].barriers + (size_t)(g_next_barrier.fetch_add(1) % kBarrierPool) * kBarrierStrideWords : nullptr;
     return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, grid, s);
 }
@@ -621,7 +628,7 @@ sd2_status build_gate_up_pair(sd2_handle gate, sd2_handle up, sd2_handle* out)
     *out = nullptr;
     const int64_t I = gate->M, K = gate->K;
     if (up->M != I || up->K != K) return SD2_OK;
-    const Gap4Geom g = gap4_geometry(2 * I, K);
+    const Gap4Geom g = gap4_geometry(2 * I, K, true);
     if (g.S == 0 || g.R < 2) return SD2_OK;
     uint16_t* dense = (uint16_t*)std::malloc((size_t)(2 * I * K) * 2);
     uint16_t* one = (uint16_t*)std::malloc((size_t)(I * K) * 2);
@@ -1104,6 +1111,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         return SD2_ERR_ALLOC;
     }
     d->K_max = needs.K_max;
+    d->free_tiles = needs.free_tiles(g_dev[dev].sms);
     d->max_tile = needs.max_tile;
     for (int w = 0; w < 4; ++w) d->xs_need[w] = needs.xs_need[w];
     {
@@ -1130,6 +1138,7 @@ sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, vo
     a.x_in = (const uint16_t*)x;
     a.y_out = y;
     a.gbar = d->d_gbar;
+    a.free_tiles = d->free_tiles;
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
     if (d->d_tags) {

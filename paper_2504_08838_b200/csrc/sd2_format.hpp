@@ -126,10 +126,12 @@ inline int64_t gap4_strip_cols(int64_t K, int S)
     return b + ((6 - (b & 3)) & 3);
 }
 
-inline Gap4Geom gap4_geometry(int64_t M, int64_t K)
+// A paired stack counts as one of its two halves, so that it is cut like they are.
+inline Gap4Geom gap4_geometry(int64_t M, int64_t K, bool paired = false)
 {
+    const int64_t Mt = paired ? M / 2 : M;
     int S = 1;
-    while (S < 32 && M * S / 32 < kGap4TileTarget) S <<= 1;
+    while (S < 32 && Mt * S / 32 < kGap4TileTarget) S <<= 1;
     while (S > 1 && (K + S - 1) / S < kGap4MinStrip) S >>= 1;
     while (S < 32 && gap4_strip_cols(K, S) > kGap4MaxStrip) S <<= 1;
     Gap4Geom g;
@@ -330,7 +332,7 @@ inline void gap4_row_cols(const uint16_t* W, const uint8_t* mask, int64_t m, int
 inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype, bool pair_rows = false)
 {
     PackResult r;
-    const Gap4Geom g = gap4_geometry(M, K);
+    const Gap4Geom g = gap4_geometry(M, K, pair_rows);
     if (g.S == 0) { r.status = -5; return r; }
     if (pair_rows && ((M & 1) || g.R < 2)) { r.status = -5; return r; }
     const int S = g.S, B = g.B, R = g.R, V = g.V;
@@ -496,7 +498,8 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
 inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense)
 {
     const int64_t M = h.M, K = h.K;
-    const Gap4Geom g = gap4_geometry(M, K);
+    if (h.pairing > 1) return -6;
+    const Gap4Geom g = gap4_geometry(M, K, h.pairing == 1);
     if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B || h.overlap != (uint32_t)g.V) return -6;
     const int S = g.S, B = g.B, R = g.R, V = g.V;
     const int64_t T = (M + R - 1) / R;

@@ -147,6 +147,8 @@ struct SArgs {
     int ring_bytes;
     int tagged;                     // 1: stages hand activations over as tagged words, no grid barrier
     unsigned int* seq;              // tagged programs: launch counter (device word), bumped by the last CTA out
+    int free_tiles;                 // 1: a consumer warp that is done draws the next tile from a shared counter;
+                                    // 0: tile k of a stage goes to warp k % 16 (see the consumer loop)
     long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
 };
 
@@ -803,9 +805,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
     const int N = a.N;
     const int xlin_row = NT <= 2 ? 0 : a.xlin_bytes >> 2;   // elements between the two linear buffers of a pass
-    // Tiles go to whichever consumer warp is free next: a warp holds one sequence number and draws
-    // the next from a shared counter when it is done.  Numbers run on across stages, so a number
-    // drawn past the end of a stage is simply the warp's first tile of the next one.
+    // With free_tiles, tiles go to whichever consumer warp is free next: a warp holds one sequence
+    // number and draws the next from a shared counter when it is done.  Numbers run on across
+    // stages, so a number drawn past the end of a stage is simply the warp's first tile of the next
+    // one.  That evens out the warps' loads where stages have more tiles than warps; where they have
+    // fewer, the fixed deal (tile k to warp k % 16) keeps the busy warps spread over the SM's four
+    // schedulers, and measures faster.
     uint32_t qbase = 0;
     uint32_t q_mine = (uint32_t)warp;
     bool failed = false;
@@ -876,6 +881,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
 #ifdef SD2_TRACE
         long long trace_wait = 0;   // cycles this warp waited for tiles to land, stored once per stage
 #endif
+        if (!a.free_tiles) q_mine = qbase + (uint32_t)warp;
         while ((int)(q_mine - (qbase + (uint32_t)n_cta)) < 0 && !failed) {
             const uint32_t q = q_mine;
             const uint32_t slot = q % kSlots;
@@ -997,10 +1003,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             }
             __syncwarp();
             if (lane == 0) SD2_TILE_STAMP(q, 3);
-            uint32_t q_next = 0;
+            uint32_t q_next = q + (uint32_t)kConsumerWarps;
             if (lane == 0) {
                 mbar_arrive(empty0 + 8 * slot);
-                q_next = atomicAdd(&sh->next_q, 1u);
+                if (a.free_tiles) q_next = atomicAdd(&sh->next_q, 1u);
             }
             q_mine = __shfl_sync(0xFFFFFFFFu, q_next, 0);
         }

@@ -88,10 +88,11 @@ def test_bitmask_byte_count_closed_form():
 GAP4_OVERLAP = 32
 
 
-def _gap4_geometry(M, K):
+def _gap4_geometry(M, K, paired=False):
     """Strip geometry (S strips of B columns, R rows per tile) from the format's definition."""
+    Mt = M // 2 if paired else M            # a paired stack is cut like one of its halves
     S = 1
-    while S < 32 and M * S // 32 < 2048:
+    while S < 32 and Mt * S // 32 < 2048:
         S *= 2
     while S > 1 and (K + S - 1) // S < 64:
         S //= 2
@@ -145,7 +146,7 @@ def _gap4_run_chunks(cols):
 def _gap4_bytes(mask, paired=False):
     """Compressed bytes of a mask: tile offsets + per tile (header, code words, values)."""
     M, K = mask.shape
-    S, B, R = _gap4_geometry(M, K)
+    S, B, R = _gap4_geometry(M, K, paired)
     row_chunks = []
     for m in range(M):
         cols = np.nonzero(mask[m])[0].tolist()
@@ -234,7 +235,7 @@ def test_paired_needs_even_rows_and_two_rows_per_tile():
         sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)    # odd M
     assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
     W, mask = _case(96, 2048, 4096, 0.05)                         # 32 strips: one row per tile
-    assert _gap4_geometry(2048, 4096)[2] == 1
+    assert _gap4_geometry(2048, 4096, paired=True)[2] == 1
     with pytest.raises(sd2.Sd2Error) as e:
         sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)
     assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
