@@ -51,19 +51,34 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama-3.2-1b", choices=sorted(WORKLOADS))
     ap.add_argument("--sparsity", type=float, default=0.5)
+    ap.add_argument("--mask", default="bernoulli", choices=["bernoulli", "magnitude", "2:4"],
+                    help="mask recipe; 2:4 keeps two of every four columns (sparsity is then 0.5)")
     ap.add_argument("--n", type=int, default=1, help="activation rows per step")
     ap.add_argument("--format", default="auto", choices=["auto", "bitmask", "gap4"])
     ap.add_argument("--blocks", type=int, default=0, help="override the block count (0 = the drafter's)")
     ap.add_argument("--no-dense", action="store_true", help="skip the cuBLAS dense comparison")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
-    return ap.parse_args()
+    args = ap.parse_args()
+    if args.mask == "2:4":
+        args.sparsity = 0.5
+    return args
+
+
+MASK_TEXT = {
+    "bernoulli": "%d%% unstructured Bernoulli sparsity",
+    "magnitude": "%d%% unstructured sparsity by magnitude, per-row densities spread by Beta(2,2)",
+    "2:4": "2:4 sparsity by magnitude (two of every four columns kept)",
+}
 
 
 def config_dict(args, shape, blocks, extra=None):
     cfg = {
-        "workload": "%s-shaped drafter, %d blocks x 7 linears (q,k,v,o,gate,up,down), %d%% unstructured "
-                    "Bernoulli sparsity, bf16 weights N(0,0.02), N=%d activation rows N(0,1)"
-                    % (shape.name, blocks, round(100 * args.sparsity), args.n),
+        "workload": "%s-shaped drafter, %d blocks x 7 linears (q,k,v,o,gate,up,down), %s, "
+                    "bf16 weights N(0,0.02), N=%d activation rows N(0,1)"
+                    % (shape.name, blocks,
+                       MASK_TEXT[args.mask] % round(100 * args.sparsity) if "%d" in MASK_TEXT[args.mask] else MASK_TEXT[args.mask],
+                       args.n),
+        "mask": args.mask,
         "blocks": blocks,
         "sparsity": args.sparsity,
         "n_rows": args.n,
@@ -138,12 +153,12 @@ class ClockSampler:
 # the CPU oracle as a timed baseline (the only place bench.py executes oracle/)
 # ------------------------------------------------------------------------------------------
 
-def time_oracle(shape, cfg_id, density, n_rows, blocks_sample):
+def time_oracle(shape, cfg_id, density, n_rows, blocks_sample, mask_kind="bernoulli"):
     """Seconds the oracle needs for `blocks_sample` blocks' seven linears (single thread)."""
     from oracle import oracle
     total = 0.0
     for b in range(blocks_sample):
-        lin = synth.make_block(cfg_id, b, shape, density)
+        lin = synth.make_block(cfg_id, b, shape, density, mask_kind)
         for i, (W, m) in enumerate(lin):
             X = synth.make_activations(cfg_id, b, i, n_rows, W.shape[1])
             t0 = time.perf_counter()
@@ -163,11 +178,11 @@ def run_reference(args):
     from oracle import oracle
     oracle.build()
     for _ in range(min(args.warmup, 1)):
-        time_oracle(shape, cfg_id, 1.0 - args.sparsity, args.n, 1)
+        time_oracle(shape, cfg_id, 1.0 - args.sparsity, args.n, 1, args.mask)
     steps = max(1, min(args.steps, 5))
     per_step = []
     for _ in range(steps):
-        per_step.append(time_oracle(shape, cfg_id, 1.0 - args.sparsity, args.n, sample) * blocks / sample)
+        per_step.append(time_oracle(shape, cfg_id, 1.0 - args.sparsity, args.n, sample, args.mask) * blocks / sample)
     us = float(np.mean(per_step)) * 1e6
     sample_txt = "%d of %d blocks (all 7 linears, N=%d) per step, scaled by %d/%d" % (sample, blocks, args.n, blocks, sample)
     line = {
@@ -244,7 +259,7 @@ def run_ours(args):
     handles, dense = [], []
     comp_bytes = nnz = dense_elems = 0
     for b in range(blocks):
-        lin = synth.make_block(cfg_id, b, shape, density)
+        lin = synth.make_block(cfg_id, b, shape, density, args.mask)
         hs = []
         for i, (W, m) in enumerate(lin):
             hs.append(sd2.sd2_compress(W, m, fmt, sd2.SD2_DTYPE_BF16))
@@ -394,7 +409,7 @@ def run_ours(args):
             from oracle import oracle
             oracle.build()
             sample = min(blocks, 8)
-            sec = time_oracle(shape, cfg_id, density, N, sample)
+            sec = time_oracle(shape, cfg_id, density, N, sample, args.mask)
             cpu = {"value": sec * blocks / sample * 1e6, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": "%d of %d blocks (all 7 linears, N=1), one pass, scaled by %d/%d" % (sample, blocks, blocks, sample)}
         line = {

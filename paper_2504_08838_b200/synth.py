@@ -161,6 +161,20 @@ def magnitude_mask(w_bits: np.ndarray, seed: int, density: float) -> np.ndarray:
     return (rank < keep[:, None]).astype(np.uint8)
 
 
+def two_four_mask(w_bits: np.ndarray) -> np.ndarray:
+    """2:4 pattern: of every four consecutive columns keep the two largest |w| (ties: lower column).
+
+    The paper's second fine-grained setting; always 50 % dense.  K must be a multiple of 4."""
+    M, K = w_bits.shape
+    if K % 4:
+        raise ValueError("2:4 masks need K to be a multiple of 4")
+    key = (w_bits & np.uint16(0x7FFF)).astype(np.int32).reshape(M, K // 4, 4)
+    order = np.argsort(-key, axis=2, kind="stable")
+    rank = np.empty_like(order)
+    np.put_along_axis(rank, order, np.broadcast_to(np.arange(4), order.shape), axis=2)
+    return (rank < 2).astype(np.uint8).reshape(M, K)
+
+
 def integer_bf16(seed: int, shape, lo: int, hi: int) -> np.ndarray:
     """Small integers in [lo, hi] as bf16 patterns (exact for |v| <= 256)."""
     n = int(np.prod(shape))
@@ -208,6 +222,8 @@ def make_linear(config: int, block: int, linear: int, M: int, K: int, density: f
         mask = bernoulli_mask(ms, (M, K), density)
     elif mask_kind == "magnitude":
         mask = magnitude_mask(w, ms, density)
+    elif mask_kind == "2:4":
+        mask = two_four_mask(w)          # `density` is not used: the pattern fixes it at one half
     else:
         raise ValueError(mask_kind)
     return w, mask

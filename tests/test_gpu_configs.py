@@ -94,6 +94,12 @@ def test_config3_qwen_uneven_rows(sparsity, N):
     run_drafter_and_check(3, synth.QWEN_1P5B, 1.0 - sparsity, "magnitude", N, L=1)
 
 
+@pytest.mark.parametrize("N", [1, 4])
+def test_two_four_masks_llama_1b_block(N):
+    # the paper's 2:4 setting: two kept weights in every four columns, chosen by magnitude
+    run_drafter_and_check(2, synth.LLAMA_1B, 0.5, "2:4", N, L=1)
+
+
 @pytest.mark.parametrize("N", [1, 16])
 def test_config4_llama_3b_block(N):
     run_drafter_and_check(4, synth.LLAMA_3B, 0.5, "bernoulli", N, L=1)

@@ -1,6 +1,7 @@
 """The seeded generator: reproducible, right distributions, right shapes."""
 
 import numpy as np
+import pytest
 
 from paper_2504_08838_b200 import synth
 
@@ -49,6 +50,25 @@ def test_magnitude_mask_keeps_largest_per_row():
     # 70 % sparsity: densities spread over (0, 0.6)
     d7 = synth.row_densities(12, 4096, 0.3)
     assert d7.min() > 0 and d7.max() < 0.6 and abs(d7.mean() - 0.3) < 0.01
+
+
+def test_two_four_mask_keeps_two_largest_of_every_four():
+    w = synth.normal_bf16(77, (37, 64), 0.02)
+    m = synth.two_four_mask(w)
+    assert m.shape == w.shape and m.dtype == np.uint8
+    g = m.reshape(37, 16, 4)
+    assert (g.sum(axis=2) == 2).all()
+    mag = (w & np.uint16(0x7FFF)).astype(np.int32).reshape(37, 16, 4)
+    kept_min = np.where(g == 1, mag, 1 << 20).min(axis=2)
+    dropped_max = np.where(g == 0, mag, -1).max(axis=2)
+    assert (kept_min >= dropped_max).all()
+    # ties go to the lower column
+    t = np.full((1, 4), 0x3C00, np.uint16)
+    assert synth.two_four_mask(t).tolist() == [[1, 1, 0, 0]]
+    with pytest.raises(ValueError):
+        synth.two_four_mask(np.zeros((2, 6), np.uint16))
+    w2, m2 = synth.make_linear(2, 0, 4, 8, 32, 0.5, "2:4")
+    assert np.array_equal(m2, synth.two_four_mask(w2))
 
 
 def test_drafter_shapes():
