@@ -345,6 +345,44 @@ def test_drafter_step_teacher_forced(N, dims3):
             sd2.sd2_free(h)
 
 
+def test_drafter_steps_repeat_bit_for_bit_across_tag_wraparound():
+    # the launch counter that tags the hand-off words is 8 bits wide: 600 steps wrap it twice; every
+    # step must give the first step's result, bit for bit (one row's sum order is fixed)
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 2)
+    blocks = []
+    for b in range(2):
+        lin = synth.make_block(2, b, shape, 0.5)
+        blocks.append([sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32 if (b == 1 and i == 6) else sd2.SD2_DTYPE_BF16)
+                       for i, (W, m) in enumerate(lin)])
+    d = sd2.sd2_drafter_create(blocks, n_max=4)
+    N = 3
+    xd = dev_bf16(synth.make_activations(2, 0, 0, N, shape.hidden))
+    y0 = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_drafter_step(d, xd, y0)
+    sd2.sd2_stream_check()
+    assert not torch.isnan(y0).any()
+    y = torch.empty_like(y0)
+    for k in range(600):
+        if k % 97 == 0:
+            y.fill_(float("nan"))
+        sd2.sd2_drafter_step(d, xd, y)
+        if k % 97 == 0 or k == 599:
+            sd2.sd2_stream_check()
+            assert torch.equal(y, y0), "step %d differs" % k
+    # a different number of rows in between, then back
+    y1 = torch.full((1, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_drafter_step(d, xd[:1], y1)
+    sd2.sd2_stream_check()
+    assert torch.equal(y1[0], y0[0])
+    sd2.sd2_drafter_step(d, xd, y)
+    sd2.sd2_stream_check()
+    assert torch.equal(y, y0)
+    sd2.sd2_drafter_free(d)
+    for hs in blocks:
+        for h in hs:
+            sd2.sd2_free(h)
+
+
 def test_block_step_rejects_shapes_that_do_not_chain():
     shape = synth.DrafterShape("tiny", 128, 32, 256, 1)
     lin = synth.make_block(2, 1, shape, 0.5)
