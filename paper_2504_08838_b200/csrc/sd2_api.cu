@@ -25,7 +25,9 @@ struct sd2_handle_s {
     const uint32_t* d_sec0;
     const uint32_t* d_sec1;
     const void* d_sec2;
-    int B, V;   // GAP4 geometry: strip width, window overlap
+    // GAP4 geometry
+    int S, B, T, max_tile_bytes, V;
+    int paired;   // GAP4: rows 2i, 2i+1 share a tile (header field `pairing`)
 };
 
 struct sd2_drafter_s {
@@ -40,9 +42,12 @@ struct sd2_drafter_s {
     uint8_t* d_ws;
     SStage* d_stages;
     unsigned int* d_gbar;
-    uint32_t* d_tags;          // tagged copies of q, hdn, t and the block output of every block (or NULL)
+    uint32_t* d_tags;          // tagged copies of q, hdn, g, u and the block output of every block (or NULL)
     int64_t tags_bytes;
-    int wrows_even, wrows_odd; // most window rows of the even / odd stages: decides the shared-memory plan
+    int64_t last_n;            // rows of the previous step: a change clears d_tags (stale tags of other rows)
+    int K_max, max_tile;       // what decides the shared-memory split
+    int free_tiles;            // every stage has enough tiles per CTA for free tile assignment
+    int xs_need[4];            // bytes of staged activations at panel widths 1, 2, 4, 8
 };
 
 namespace {
@@ -55,8 +60,6 @@ constexpr int kMaxDevices = 64;
 constexpr int kBarrierPool = 64;             // grid-barrier word pairs handed out round-robin
 constexpr int kBarrierStrideWords = 64;      // 256 bytes apart
 constexpr int kSmemMax = 227 * 1024;         // dynamic shared memory a CTA may opt in to
-constexpr int kMaxBlockRows = 1 << 16;       // activation rows a block step accepts
-constexpr int kDrafterWordsBytes = 512;      // a drafter's device words: barrier (two lines), then 64 production counts
 
 struct DeviceState {
     bool ready;
@@ -112,7 +115,8 @@ sd2_status ensure_device(int* dev_out)
         int sms = 0, khz = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess) {
+        if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess ||
+            set_smem_attr<8>() != cudaSuccess) {
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
@@ -140,8 +144,8 @@ sd2_status ensure_device(int* dev_out)
 int resolve_format(const sd2_options* opt, int64_t M, int64_t K)
 {
     int f = opt ? opt->format : SD2_FORMAT_AUTO;
-    if (f == SD2_FORMAT_AUTO) f = (gap4_strip_cols(K) <= kGap4MaxStrip && M < (1ll << 28)) ? SD2_FORMAT_GAP4 : SD2_FORMAT_BITMASK;
-    return f;
+    if (f == SD2_FORMAT_AUTO) f = gap4_geometry(M, K).S > 0 ? SD2_FORMAT_GAP4 : SD2_FORMAT_BITMASK;
+    return f;   // SD2_FORMAT_GAP4_PAIRED stays as asked: only the packer tells it from GAP4
 }
 
 sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, const sd2_options* opt,
@@ -155,10 +159,9 @@ sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K
     PackResult r;
     try {
         if (f == SD2_FORMAT_BITMASK) r = pack_bitmask(W, mask, M, K, y_dtype);
-        else if (f == SD2_FORMAT_GAP4) {
-            if (M >= (1ll << 28)) return SD2_ERR_UNSUPPORTED;   // kernels keep a row index in 28 bits
-            r = pack_gap4(W, mask, M, K, y_dtype);
-        } else return SD2_ERR_INVALID_ARG;
+        else if (f == SD2_FORMAT_GAP4) r = pack_gap4(W, mask, M, K, y_dtype);
+        else if (f == SD2_FORMAT_GAP4_PAIRED) r = pack_gap4(W, mask, M, K, y_dtype, true);
+        else return SD2_ERR_INVALID_ARG;
     } catch (const std::bad_alloc&) {
         return SD2_ERR_ALLOC;
     }
@@ -193,8 +196,12 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     h->d_sec0 = (const uint32_t*)(h->d_blob + hd.sec_off[0]);
     h->d_sec1 = (const uint32_t*)(h->d_blob + hd.sec_off[1]);
     h->d_sec2 = (const void*)(h->d_blob + hd.sec_off[2]);
+    h->S = (int)hd.strips;
     h->B = (int)hd.strip_cols;
+    h->T = (int)hd.n_tiles;
+    h->max_tile_bytes = (int)hd.max_tile_bytes;
     h->V = (int)hd.overlap;
+    h->paired = (int)hd.pairing;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(h);
@@ -228,7 +235,6 @@ sd2_status launch_bitmask_nt(const LaunchGroup& grp, int grid, cudaStream_t s)
 }
 
 int round_nt(int n, int cap) { int r = n <= 1 ? 1 : n <= 2 ? 2 : n <= 4 ? 4 : 8; return r > cap ? cap : r; }
-int round_nt4(int n, int cap) { int r = n <= 1 ? 1 : n <= 2 ? 2 : 4; return r > cap ? cap : r; }
 
 // One launch per panel of at most 8 activation rows.  Exactly one of x / (g, u) is set.
 sd2_status run_bitmask(const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
@@ -283,47 +289,30 @@ sd2_status run_bitmask(const sd2_handle* hs, int count, const uint16_t* x, const
 
 // ------------------------------------------------------------------ GAP4 programs
 
-// Shared memory of a launch: the control block, the warps' rings, then the staged activations.
-// Consecutive stages stage into different places where there is room for that (even stages at
-// offset 0, odd stages behind the largest even one), so that a CTA can stage the next stage while
-// its slower warps still gather from this one; else into one place, at the price of one more CTA
-// barrier per stage.  What is left decides how many slots a warp's ring has.
+// Largest panel width (8, 4, 2, 1) whose staged activations leave room for a ring that holds
+// `max_tile` bytes at least twice; 0 if even one row does not fit.
 struct SmemPlan {
-    int nt, xs_odd, xs_total, xs_single, nslot;
+    int nt, xs_bytes, xlin_bytes, ring_bytes;
 };
 
-bool plan_smem(int nt, int wrows_even, int wrows_odd, SmemPlan* p)
+int xs_bytes_for(int S, int B, int V, int nt)
 {
-    const int unit = 128 * xs_words(nt);
-    const int ring1 = kConsumerWarps * kSlotBytes;   // one slot for every warp
-    p->nt = nt;
-    int xs_e = wrows_even * unit, xs_o = wrows_odd * unit;
-    int left = kSmemMax - kCtrlBytes - (xs_e + xs_o);
-    if (xs_o > 0 && left >= 2 * ring1) {
-        p->xs_odd = xs_e;
-        p->xs_total = xs_e + xs_o;
-        p->xs_single = 0;
-    } else {
-        const int xs = xs_e > xs_o ? xs_e : xs_o;
-        left = kSmemMax - kCtrlBytes - xs;
-        if (left < 2 * ring1) return false;
-        p->xs_odd = 0;
-        p->xs_total = xs;
-        p->xs_single = 1;
-    }
-    p->nslot = left / ring1 > kMaxSlots ? kMaxSlots : left / ring1;
-    return true;
+    const int groups = 32 / xs_words(nt);
+    const int planes = S > groups ? S / groups : 1;
+    return planes * ((B + 2 * V + kGap4Slack + 3) & ~3) * 128;
 }
 
-// Widest panel (4, 2, 1 rows) that fits; 0 if none.
-int widest_panel(int wrows_even, int wrows_odd)
+bool plan_smem(int nt, int xs_max, int K_max, int max_tile, SmemPlan* p)
 {
-    SmemPlan p;
-    for (int nt = 4; nt >= 1; nt >>= 1)
-        if (plan_smem(nt, wrows_even, wrows_odd, &p) && !p.xs_single) return nt;
-    for (int nt = 4; nt >= 1; nt >>= 1)
-        if (plan_smem(nt, wrows_even, wrows_odd, &p)) return nt;
-    return 0;
+    const int fixed = (int)((sizeof(StreamShared) + 127) & ~127);
+    const int xlin = ((2 * K_max + 127) & ~127) * (nt > 2 ? 2 : 1);   // panels of 4 and 8 go two rows at a time
+    const int ring = (kSmemMax - fixed - xs_max - xlin) & ~127;
+    if (ring < 2 * max_tile + 256) return false;
+    p->nt = nt;
+    p->xs_bytes = xs_max;
+    p->xlin_bytes = xlin;
+    p->ring_bytes = ring;
+    return true;
 }
 
 template <int NT>
@@ -346,51 +335,59 @@ sd2_status launch_stream_nt(const SArgs& a, int grid, int smem, bool cooperative
 
 sd2_status launch_stream(int nt, const SArgs& a, int grid, bool cooperative, cudaStream_t s)
 {
-    const int smem = kCtrlBytes + kConsumerWarps * a.nslot * kSlotBytes + a.xs_total;
+    const int smem = a.xs_bytes + a.xlin_bytes + (int)((sizeof(StreamShared) + 127) & ~127) + a.ring_bytes;
     switch (nt) {
         case 1: return launch_stream_nt<1>(a, grid, smem, cooperative, s);
         case 2: return launch_stream_nt<2>(a, grid, smem, cooperative, s);
-        default: return launch_stream_nt<4>(a, grid, smem, cooperative, s);
+        case 4: return launch_stream_nt<4>(a, grid, smem, cooperative, s);
+        default: return launch_stream_nt<8>(a, grid, smem, cooperative, s);
     }
 }
 
-// Fills one stage from `count` GAP4 handles of equal K.  `paired`: hs[0] is a stack of gate row i
-// (row 2i) and up row i (row 2i+1); a unit is then such a pair of rows.
+void set_stage_grid(SStage& st, int grid)
+{
+    st.tiles_div = st.T_total / grid;
+    st.tiles_rem = st.T_total % grid;
+}
+
+// Fills one stage from `count` GAP4 handles of equal K and S, to be run by `grid` CTAs.
 void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
-                uint16_t* t_out, void* const* Y, bool y_force_bf16, uint32_t* const* YT = nullptr, int tagged_in = 0,
-                bool paired = false)
+                uint16_t* t_out, void* const* Y, bool y_force_bf16, int grid, uint32_t* const* YT = nullptr,
+                int tagged_in = 0)
 {
     std::memset(&st, 0, sizeof st);
     st.count = count;
     st.K = (int)hs[0]->K;
+    st.S = hs[0]->S;
     st.B = hs[0]->B;
-    st.upr = paired ? 2 : 1;
-    st.paired = paired ? 1 : 0;
-    int V = 0;
-    for (int i = 0; i < count; ++i)
-        if (hs[i]->V > V) V = hs[i]->V;
-    st.V = V;
-    st.wrows = gap4_window_rows(st.B, V);
+    st.V = hs[0]->V;
+    st.hdr_bytes = gap4_tile_header_bytes(32 / hs[0]->S);
+    st.log2S = 0;
+    while ((1 << st.log2S) < hs[0]->S) ++st.log2S;
     st.x = x;
     st.g = g;
     st.u = u;
     st.t_out = t_out;
-    int units = 0;
+    int T = 0;
     for (int i = 0; i < count; ++i) {
         SMat& m = st.mat[i];
-        m.rowdir = (const uint4*)hs[i]->d_sec0;
+        m.tile_off = hs[i]->d_sec0;
         m.stream = (const unsigned char*)hs[i]->d_sec1;
         m.y = Y[i];
         m.yt = YT ? YT[i] : nullptr;
         m.M = (int)hs[i]->M;
+        m.T = hs[i]->T;
         m.y_f32 = (!y_force_bf16 && hs[i]->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
-        m.unit0 = units;
-        m.voff = V - hs[i]->V;
-        units += (int)(hs[i]->M / st.upr);
+        T += hs[i]->T;
     }
-    st.units = units;
+    st.T_total = T;
     st.tagged_in = tagged_in;
+    set_stage_grid(st, grid);
 }
+
+#ifdef SD2_TRACE
+long long* g_trace = nullptr;   // set through sd2_debug_set_trace (trace builds only)
+#endif
 
 long long wait_budget(int dev)
 {
@@ -402,34 +399,64 @@ long long wait_budget(int dev)
 
 // Tracks what a program needs from shared memory.
 struct ProgramNeeds {
-    int wrows_even = 0, wrows_odd = 0;   // most window rows of the stages with an even / odd index
-    int units_max = 0;
-    int n = 0;
-    void add(const SStage& st)
+    int K_max = 0, max_tile = 0, tiles_max = 0;
+    int tiles_min = 0x7FFFFFFF;   // fewest tiles of any stage
+    int xs_need[4] = {0, 0, 0, 0};   // staged activations at panel widths 1, 2, 4, 8: the largest over all stages
+    // Free tile assignment pays where every stage gives a CTA about as many tiles as it has consumer
+    // warps, or more; with fewer, the fixed deal is faster (see the consumer loop of stream_kernel).
+    int free_tiles(int grid) const { return tiles_min >= 12 * grid ? 1 : 0; }
+    void add(const sd2_handle* hs, int count)
     {
-        int& w = (n & 1) ? wrows_odd : wrows_even;
-        if (st.wrows > w) w = st.wrows;
-        if (st.units > units_max) units_max = st.units;
-        ++n;
+        int T = 0;
+        for (int i = 0; i < count; ++i) {
+            // elements of the linear staging row: the strips, the zero pads on both sides, read-ahead
+            const int lin = hs[i]->S * hs[i]->B + 2 * hs[i]->V + 64;
+            if (lin > K_max) K_max = lin;
+            if (hs[i]->max_tile_bytes > max_tile) max_tile = hs[i]->max_tile_bytes;
+            for (int w = 0; w < 4; ++w) {
+                const int need = xs_bytes_for(hs[i]->S, hs[i]->B, hs[i]->V, 1 << w);
+                if (need > xs_need[w]) xs_need[w] = need;
+            }
+            T += hs[i]->T;
+        }
+        if (T > tiles_max) tiles_max = T;
+        if (T < tiles_min) tiles_min = T;
     }
 };
 
-// Launches a program over all N rows, in panels of at most `nt_cap` rows (rows are independent).
-sd2_status run_panels(SArgs& a, int64_t N, int wrows_even, int wrows_odd, int grid, cudaStream_t s)
+int nt_index(int nt) { return nt == 1 ? 0 : nt == 2 ? 1 : nt == 4 ? 2 : 3; }
+
+// Widest panel (8, 4, 2, 1 rows) whose staged activations still leave room for the ring; 0 if none.
+int widest_panel(const int xs_need[4], int K_max, int max_tile)
 {
-    const int nt_cap = widest_panel(wrows_even, wrows_odd);
+    // a wide panel whose activations crowd out the ring cannot stream: ask for a ring of at
+    // least 96 KB first, and settle for whatever fits only if no width leaves that much
+    SmemPlan p;
+    for (int nt = 8; nt >= 1; nt >>= 1)
+        if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p) && p.ring_bytes >= 96 * 1024) return nt;
+    for (int nt = 8; nt >= 1; nt >>= 1)
+        if (plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return nt;
+    return 0;
+}
+
+// Launches a program over all N rows, in panels of at most `nt_cap` rows (rows are independent).
+sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[4], int K_max, int max_tile, int grid, cudaStream_t s)
+{
+    const int nt_cap = widest_panel(xs_need, K_max, max_tile);
     if (nt_cap == 0) return SD2_ERR_UNSUPPORTED;
     for (int64_t n0 = 0; n0 < N; n0 += nt_cap) {
         const int n = (int)((N - n0) < nt_cap ? (N - n0) : nt_cap);
-        const int nt = round_nt4(n, nt_cap);
-        SmemPlan p;   // the narrower the panel, the more room for the rings
-        if (!plan_smem(nt, wrows_even, wrows_odd, &p)) return SD2_ERR_UNSUPPORTED;
+        const int nt = round_nt(n, nt_cap);
+        SmemPlan p;   // the narrower the panel, the more room for the ring
+        if (!plan_smem(nt, xs_need[nt_index(nt)], K_max, max_tile, &p)) return SD2_ERR_UNSUPPORTED;
         a.N = n;
         a.n0 = (int)n0;
-        a.xs_odd = p.xs_odd;
-        a.xs_total = p.xs_total;
-        a.xs_single = p.xs_single;
-        a.nslot = p.nslot;
+        a.xs_bytes = p.xs_bytes;
+        a.xlin_bytes = p.xlin_bytes;
+        a.ring_bytes = p.ring_bytes;
+#ifdef SD2_TRACE
+        a.trace = g_trace;
+#endif
         sd2_status st = launch_stream(nt, a, grid, a.n_stages > 1, s);
         if (st != SD2_OK) return st;
     }
@@ -441,12 +468,13 @@ sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, 
 {
     const bool coop = a.n_stages > 1;
     int grid = g_dev[dev].sms;
-    if (!coop && needs.units_max < grid) grid = needs.units_max < 1 ? 1 : needs.units_max;
+    if (!coop && needs.tiles_max < grid) grid = needs.tiles_max < 1 ? 1 : needs.tiles_max;
+    if (!coop) set_stage_grid(a.inl[0], grid);
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
-    a.hinted = coop ? 1 : 0;
+    a.free_tiles = needs.free_tiles(grid);
     a.gbar = coop ? g_dev[dev].barriers + (size_t)(g_next_barrier.fetch_add(1) % kBarrierPool) * kBarrierStrideWords : nullptr;
-    return run_panels(a, N, needs.wrows_even, needs.wrows_odd, grid, s);
+    return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, grid, s);
 }
 
 // Shared by sd2_spmm and sd2_spmm_fused (and by block steps that mix formats).
@@ -463,7 +491,7 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
         if (hs[i]->K != K) return SD2_ERR_SHAPE;
     bool same = true;
     for (int i = 1; i < count; ++i)
-        if (hs[i]->format != hs[0]->format) same = false;
+        if (hs[i]->format != hs[0]->format || hs[i]->S != hs[0]->S) same = false;
     if (!same) {  // weights that cannot share a stage: one launch each
         for (int j = 0; j < count; ++j) {
             sd2_status sj = run_group(hs + j, 1, x, g, u, j == 0 ? t_out : nullptr, Y + j, N, y_force_bf16, s);
@@ -480,9 +508,9 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
     SArgs a;
     std::memset(&a, 0, sizeof a);
     a.n_stages = 1;
-    fill_stage(a.inl[0], hs, count, x, g, u, t_out, Y, y_force_bf16);
+    fill_stage(a.inl[0], hs, count, x, g, u, t_out, Y, y_force_bf16, g_dev[dev].sms);
     ProgramNeeds needs;
-    needs.add(a.inl[0]);
+    needs.add(hs, count);
     return run_program(a, dev, N, needs, s);
 }
 
@@ -523,55 +551,85 @@ void block_layout(const sd2_handle* h, const BlockDims& d, int64_t N, int64_t of
     off[7] = o;
 }
 
-// Tagged 32-bit copies of a block's activations (value << 16 | tag) through which the
+// Tagged 32-bit copies of a block's activations (value << 16 | stage tag) through which the
 // stages of a tagged program hand their outputs to the next stage without a grid barrier.
 struct BlockTags {
     const uint32_t* x_t;   // the block's input as tagged words, or NULL (plain bf16 input)
-    uint32_t *q_t, *hdn_t, *t_t, *out_t;   // out_t NULL: the block's output is not handed on
+    uint32_t *q_t, *hdn_t, *g_t, *u_t, *out_t;   // out_t NULL: the block's output is not handed on
+    uint32_t* t_t;                               // tagged t = silu(g) * u, one slice per CTA
 };
 
-// Appends the four stages of one block (h[0..6] = q,k,v,o,gate,up,down) to `stages`: q|k|v, o,
-// gate|up, down.  Without tags the down stage forms t = silu(g) * u while it stages its
-// activations; with tags (`tg` and the paired stack `gu_pair` of gate and up) the gate|up stage
-// forms t where g and u are produced and hands it on as tagged words.
+// Appends the stages of one block (h[0..6] = q,k,v,o,gate,up,down) to `stages`.  Weights of a
+// group that do not share a strip geometry get a stage each.  Returns the number appended.
 int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
                         uint16_t* hdn, uint16_t* g, uint16_t* u, uint16_t* t, void* y, bool y_force_bf16,
-                        ProgramNeeds* needs, const BlockTags* tg = nullptr, sd2_handle gu_pair = nullptr)
+                        ProgramNeeds* needs, int grid, const BlockTags* tg = nullptr, sd2_handle gu_pair = nullptr)
 {
+    int n = 0;
+    auto group = [&](const sd2_handle* hs, int count, const uint16_t* xin, const uint16_t* gg, const uint16_t* uu,
+                     uint16_t* tt, void* const* Y, bool force, uint32_t* const* YT, int tin) {
+        bool same = true;
+        for (int i = 1; i < count; ++i)
+            if (hs[i]->S != hs[0]->S) same = false;
+        if (same) {
+            fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force, grid, YT, tin);
+            needs->add(hs, count);
+        } else {
+            for (int i = 0; i < count; ++i) {
+                fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force, grid, YT ? YT + i : nullptr, tin);
+                needs->add(hs + i, 1);
+            }
+        }
+    };
     void* y_qkv[3] = {q, k, v};
     void* y_o[1] = {hdn};
     void* y_gu[2] = {g, u};
     void* y_d[1] = {y};
     if (!tg) {
-        fill_stage(stages[0], h + 0, 3, x, nullptr, nullptr, nullptr, y_qkv, true);
-        fill_stage(stages[1], h + 3, 1, q, nullptr, nullptr, nullptr, y_o, true);
-        fill_stage(stages[2], h + 4, 2, hdn, nullptr, nullptr, nullptr, y_gu, true);
-        fill_stage(stages[3], h + 6, 1, nullptr, g, u, t, y_d, y_force_bf16);
+        group(h + 0, 3, x, nullptr, nullptr, nullptr, y_qkv, true, nullptr, 0);
+        group(h + 3, 1, q, nullptr, nullptr, nullptr, y_o, true, nullptr, 0);
+        group(h + 4, 2, hdn, nullptr, nullptr, nullptr, y_gu, true, nullptr, 0);
+        group(h + 6, 1, nullptr, g, u, t, y_d, y_force_bf16, nullptr, 0);
     } else {
         uint32_t* t_qkv[3] = {tg->q_t, nullptr, nullptr};
         uint32_t* t_o[1] = {tg->hdn_t};
+        uint32_t* t_gu[2] = {tg->g_t, tg->u_t};
         uint32_t* t_d[1] = {tg->out_t};
-        void* y_none[1] = {nullptr};
-        fill_stage(stages[0], h + 0, 3, tg->x_t ? (const uint16_t*)tg->x_t : x, nullptr, nullptr, nullptr, y_qkv, true, t_qkv, tg->x_t ? 1 : 0);
-        fill_stage(stages[1], h + 3, 1, (const uint16_t*)tg->q_t, nullptr, nullptr, nullptr, y_o, true, t_o, 1);
-        // one stacked matrix, gate row i and up row i worked on by the same warp: the stage writes g,
-        // u and t as plain bf16 and t as tagged words, and the down stage reads t like any activation
-        fill_stage(stages[2], &gu_pair, 1, (const uint16_t*)tg->hdn_t, g, u, t, y_none, true, nullptr, 1, true);
-        stages[2].tt = tg->t_t;
-        fill_stage(stages[3], h + 6, 1, (const uint16_t*)tg->t_t, nullptr, nullptr, nullptr, y_d, y_force_bf16, t_d, 1);
+        group(h + 0, 3, tg->x_t ? (const uint16_t*)tg->x_t : x, nullptr, nullptr, nullptr, y_qkv, true, t_qkv, tg->x_t ? 1 : 0);
+        group(h + 3, 1, (const uint16_t*)tg->q_t, nullptr, nullptr, nullptr, y_o, true, t_o, 1);
+        if (gu_pair) {
+            // one stacked matrix, gate row i and up row i in one tile: the stage writes g, u and t
+            // as plain bf16 and t as tagged words, and the down stage reads t like any activation
+            void* y_none[1] = {nullptr};
+            SStage& st = stages[n++];
+            fill_stage(st, &gu_pair, 1, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_none, true, grid, nullptr, 1);
+            needs->add(&gu_pair, 1);
+            st.paired = 1;
+            st.g = g;
+            st.u = u;
+            st.t_out = t;
+            st.tt = tg->t_t;
+            group(h + 6, 1, (const uint16_t*)tg->t_t, nullptr, nullptr, nullptr, y_d, y_force_bf16, t_d, 1);
+        } else {
+            group(h + 4, 2, (const uint16_t*)tg->hdn_t, nullptr, nullptr, nullptr, y_gu, true, t_gu, 1);
+            const int before = n;
+            group(h + 6, 1, nullptr, (const uint16_t*)tg->g_t, (const uint16_t*)tg->u_t, t, y_d, y_force_bf16, t_d, 1);
+            for (int i = before; i < n; ++i) stages[i].tt = tg->t_t;
+        }
     }
-    for (int i = 0; i < 4; ++i) needs->add(stages[i]);
-    return 4;
+    return n;   // at most 7
 }
 
 // Builds the paired stack of a block's gate and up (row 2i = gate row i, row 2i+1 = up row i)
-// from the decoded contents of the two handles.
+// from the decoded contents of the two handles.  *out stays NULL where the shape has no paired
+// form (fewer than two rows per tile); the caller then keeps the two weights apart.
 sd2_status build_gate_up_pair(sd2_handle gate, sd2_handle up, sd2_handle* out)
 {
     *out = nullptr;
     const int64_t I = gate->M, K = gate->K;
-    if (up->M != I || up->K != K) return SD2_ERR_SHAPE;
-    if (2 * I >= (1ll << 28)) return SD2_ERR_UNSUPPORTED;
+    if (up->M != I || up->K != K) return SD2_OK;
+    const Gap4Geom g = gap4_geometry(2 * I, K, true);
+    if (g.S == 0 || g.R < 2) return SD2_OK;
     uint16_t* dense = (uint16_t*)std::malloc((size_t)(2 * I * K) * 2);
     uint16_t* one = (uint16_t*)std::malloc((size_t)(I * K) * 2);
     sd2_status st = (dense && one) ? SD2_OK : SD2_ERR_ALLOC;
@@ -586,7 +644,7 @@ sd2_status build_gate_up_pair(sd2_handle gate, sd2_handle up, sd2_handle* out)
     int64_t bytes = 0;
     if (st == SD2_OK) {
         // no mask: what decoded to +0 was masked out (or was a kept zero, which adds nothing)
-        sd2_options opt = {SD2_FORMAT_GAP4, SD2_DTYPE_BF16};
+        sd2_options opt = {SD2_FORMAT_GAP4_PAIRED, SD2_DTYPE_BF16};
         st = pack_any(dense, nullptr, 2 * I, K, &opt, &blob, &bytes);
     }
     std::free(dense);
@@ -768,10 +826,7 @@ sd2_status sd2_stream_check(void* cuda_stream)
         {
             std::lock_guard<std::mutex> lk(g_mu);
             for (sd2_drafter d : g_live_drafters)
-                if (d->device == dev) {   // barrier words, production counts and every tagged word start over
-                    cudaMemset(d->d_gbar, 0, kDrafterWordsBytes);
-                    if (d->d_tags) cudaMemset(d->d_tags, 0, (size_t)d->tags_bytes);
-                }
+                if (d->device == dev) { cudaMemset(d->d_gbar, 0, 256); d->last_n = -1; }
         }
         cudaGetLastError();
         return SD2_ERR_TIMEOUT;
@@ -806,7 +861,7 @@ sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, voi
 sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* bytes)
 {
     if (!bytes) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -819,7 +874,7 @@ sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* by
 sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets)
 {
     if (!offsets) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -832,7 +887,7 @@ sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* o
 sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N, void* workspace, void* cuda_stream)
 {
     if (!x || !y || !workspace) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -862,7 +917,7 @@ sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N
         SArgs a;
         std::memset(&a, 0, sizeof a);
         ProgramNeeds needs;
-        a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, q, k, v, hdn, g, u, t, y, false, &needs);
+        a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, q, k, v, hdn, g, u, t, y, false, &needs, g_dev[dev].sms);
         return run_program(a, dev, N, needs, s);
     }
     void* y_qkv[3] = {q, k, v};
@@ -893,7 +948,7 @@ unsigned char* g_static_ptr[kMaxDevices];   // device address of g_static_scratc
 sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, int64_t N, void* cuda_stream)
 {
     if (!x || !y) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -927,12 +982,11 @@ sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, in
     ProgramNeeds needs;
     a.n_stages = append_block_stages(a.inl, h, (const uint16_t*)x, (uint16_t*)(ws + off[0]), (uint16_t*)(ws + off[1]),
                                      (uint16_t*)(ws + off[2]), (uint16_t*)(ws + off[3]), (uint16_t*)(ws + off[4]),
-                                     (uint16_t*)(ws + off[5]), (uint16_t*)(ws + off[6]), y, false, &needs);
+                                     (uint16_t*)(ws + off[5]), (uint16_t*)(ws + off[6]), y, false, &needs, g_dev[dev].sms);
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
-    a.hinted = 1;
     a.gbar = (unsigned int*)base;
-    return run_panels(a, N, needs.wrows_even, needs.wrows_odd, g_dev[dev].sms, s);
+    return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, g_dev[dev].sms, s);
 }
 
 // ---- whole drafter ---------------------------------------------------------------------
@@ -977,21 +1031,22 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         o = a256(o + off[7] + 2 * n_max * dims[(size_t)b].out);
     }
     d->ws_off[(size_t)L * 8] = o;
-    std::vector<SStage> stages((size_t)L * 4);
+    std::vector<SStage> stages((size_t)L * 7);
     ProgramNeeds needs;
     bool ok = cudaMalloc((void**)&d->d_ws, (size_t)o) == cudaSuccess && cudaMemset(d->d_ws, 0, (size_t)o) == cudaSuccess;
-    // Tagged hand-off (stage tags are 8 bits wide): per block q, hdn, t, out as 32-bit words
-    const bool tagged = 4 * L <= 254;
-    std::vector<int64_t> tag_off((size_t)L * 4 + 1, 0);
+    // Tagged hand-off (stage tags are 8 bits wide): per block q, hdn, g, u, out as 32-bit words
+    const bool tagged = 7 * L <= 254;
+    std::vector<int64_t> tag_off((size_t)L * 6 + 1, 0);
     d->d_tags = nullptr;
     d->tags_bytes = 0;
+    d->last_n = -1;
     if (tagged) {
         int64_t to = 0;
         for (int b = 0; b < L; ++b) {
             const BlockDims& bd = dims[(size_t)b];
-            const int64_t w[4] = {bd.q_out, h[7 * b + 3]->M, bd.inter, bd.out};
-            for (int i = 0; i < 4; ++i) {
-                tag_off[(size_t)b * 4 + i] = to;
+            const int64_t w[6] = {bd.q_out, h[7 * b + 3]->M, bd.inter, bd.inter, bd.out, bd.inter};
+            for (int i = 0; i < 6; ++i) {
+                tag_off[(size_t)b * 6 + i] = to;
                 to = a256(to + 4 * n_max * w[i]);
             }
         }
@@ -1022,24 +1077,26 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
             BlockTags tg;
             if (tagged) {
                 uint8_t* tb = (uint8_t*)d->d_tags;
-                const int64_t* to = &tag_off[(size_t)b * 4];
-                tg.x_t = b == 0 ? nullptr : (const uint32_t*)(tb + tag_off[(size_t)(b - 1) * 4 + 3]);
+                const int64_t* to = &tag_off[(size_t)b * 6];
+                tg.x_t = b == 0 ? nullptr : (const uint32_t*)(tb + tag_off[(size_t)(b - 1) * 6 + 4]);
                 tg.q_t = (uint32_t*)(tb + to[0]);
                 tg.hdn_t = (uint32_t*)(tb + to[1]);
-                tg.t_t = (uint32_t*)(tb + to[2]);
-                tg.out_t = b + 1 < L ? (uint32_t*)(tb + to[3]) : nullptr;
+                tg.g_t = (uint32_t*)(tb + to[2]);
+                tg.u_t = (uint32_t*)(tb + to[3]);
+                tg.out_t = b + 1 < L ? (uint32_t*)(tb + to[4]) : nullptr;
+                tg.t_t = (uint32_t*)(tb + to[5]);
             }
             n += append_block_stages(stages.data() + n, h + 7 * b, xin, (uint16_t*)(base + wo[0]), (uint16_t*)(base + wo[1]),
                                      (uint16_t*)(base + wo[2]), (uint16_t*)(base + wo[3]), (uint16_t*)(base + wo[4]),
-                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs,
+                                     (uint16_t*)(base + wo[5]), (uint16_t*)(base + wo[6]), yout, b + 1 < L, &needs, g_dev[dev].sms,
                                      tagged ? &tg : nullptr, pairs[(size_t)b]);
         }
         d->n_stages = n;
         ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
              cudaMemcpy(d->d_stages, stages.data(), sizeof(SStage) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMalloc((void**)&d->d_gbar, kDrafterWordsBytes) == cudaSuccess && cudaMemset(d->d_gbar, 0, kDrafterWordsBytes) == cudaSuccess;
+             cudaMalloc((void**)&d->d_gbar, 256) == cudaSuccess && cudaMemset(d->d_gbar, 0, 256) == cudaSuccess;
     }
-    if (ok && widest_panel(needs.wrows_even, needs.wrows_odd) == 0) {
+    if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
         for (sd2_handle p : d->owned) sd2_free(p);
         cudaFree(d->d_ws); cudaFree(d->d_stages); cudaFree(d->d_gbar); cudaFree(d->d_tags);
         delete d;
@@ -1053,8 +1110,10 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         delete d;
         return SD2_ERR_ALLOC;
     }
-    d->wrows_even = needs.wrows_even;
-    d->wrows_odd = needs.wrows_odd;
+    d->K_max = needs.K_max;
+    d->free_tiles = needs.free_tiles(g_dev[dev].sms);
+    d->max_tile = needs.max_tile;
+    for (int w = 0; w < 4; ++w) d->xs_need[w] = needs.xs_need[w];
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live_drafters.insert(d);
@@ -1079,19 +1138,22 @@ sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, vo
     a.x_in = (const uint16_t*)x;
     a.y_out = y;
     a.gbar = d->d_gbar;
+    a.free_tiles = d->free_tiles;
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
-    a.hinted = 1;
     if (d->d_tags) {
         a.tagged = 1;
-        // how often each activation row has been produced: the first half of every tag.  A word left
-        // by an earlier launch (or by a launch that covered other rows) can never show the tag that this
-        // launch waits for, so steps of any N, eager or replayed from a CUDA graph, can follow each other.
-        a.rowseq = d->d_gbar + 64;
+        a.seq = d->d_gbar + 48;   // third cache-line-sized slot of the 256-byte block
+        // Only rows [0, N) are written and polled in a step.  When N changes, rows written long ago
+        // could carry a tag that comes round again (tags are 16 bits): start from clean words.
+        if (d->last_n != N) {
+            if (cudaMemsetAsync(d->d_tags, 0, (size_t)d->tags_bytes, (cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+            d->last_n = N;
+        }
     }
     // Rows of X are independent through the whole drafter: panels run one after another.  Row n
     // of every buffer starts at n * width, whatever N is.
-    return run_panels(a, N, d->wrows_even, d->wrows_odd, g_dev[dev].sms, (cudaStream_t)cuda_stream);
+    return run_panels(a, N, d->xs_need, d->K_max, d->max_tile, g_dev[dev].sms, (cudaStream_t)cuda_stream);
 }
 
 sd2_status sd2_drafter_buffers(sd2_drafter d, int32_t block, void** ptrs)
@@ -1120,5 +1182,9 @@ sd2_status sd2_drafter_free(sd2_drafter d)
     delete d;
     return st;
 }
+
+#ifdef SD2_TRACE
+void sd2_debug_set_trace(long long* device_buffer) { g_trace = device_buffer; }
+#endif
 
 }  // extern "C"

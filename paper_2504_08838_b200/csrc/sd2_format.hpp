@@ -12,43 +12,47 @@
 //                                             column 32w+b; bits at columns >= K are 0
 //            sec2  vals         u16[nnz]      kept bf16 patterns, row-major, ascending column
 //
-//   GAP4     sec0  rowdir       8 bytes per row: where its record starts, how many chunks
-//            sec1  row records  (see below), each a multiple of 16 bytes
+//   GAP4     sec0  tile_off     u32[T+1]      start of each tile record in sec1, in 16-byte units
+//            sec1  tiles        T tile records (see below), each a multiple of 16 bytes
 //            (sec2 is empty)
 //
-// GAP4 in detail.  The K columns are cut into 32 strips of B columns (B a multiple of 4,
-// 32 * B >= K), one per lane of a warp; a strip widened by V columns on both sides is that
-// lane's *window*.  A row is worked on by one warp: its kept entries, in ascending column order,
-// are dealt to the 32 lanes in consecutive runs, every lane the same number of whole 8-entry
-// chunks where the windows allow it (a lane must take what the next lane's window cannot reach
-// and cannot take what lies beyond its own); the last lane takes the rest.  A lane's run
-// becomes a list of (step, value) entries: a cursor starts at most 3 columns before the run's
-// first column (on a multiple of 4 counted from the window's start); an entry's 4-bit code is
-// how many columns the cursor moves to reach it, 0 .. 15, so an entry at column c after one at
-// column p is coded as c - p.  When the next kept column is more than 15 ahead, a filler entry
-// (value +0) is placed 15 columns ahead first.  The list is then filled up to a multiple of 8
-// with fillers of code 0 (value +0), which leave the cursor where it is.  Fillers sit on
-// masked-out columns or repeat a column and carry +0, so decoding still yields W.*mask bit for
-// bit; they are not counted in nnz, and their bytes are part of "compressed bytes" but never
-// called useful.  Eight consecutive entries form a chunk: 16 bytes of values + one 32-bit code
-// word whose nibble i (bits 4i..4i+3) is entry i's code.
+// GAP4 in detail.  The K columns are cut into S strips of B columns (S a power of two <= 32,
+// S * B >= K, B = 2 mod 4) and every strip, widened by V columns on both sides, is the *window* of
+// one lane.  A row's kept entries, in ascending column order, are dealt to the S lanes in
+// consecutive runs: every lane gets the same number of whole 8-entry chunks where the windows
+// allow it (a lane must take what the next lane's window cannot reach and cannot take what lies
+// beyond its own), the last lane takes the rest.  So the lanes of a row finish together and
+// only the last one pays padding.  A lane's run becomes a list of (gap, value) entries: a
+// cursor starts on the run's first column; an entry at column c is coded as g = c - cursor in
+// [0, 15] and moves the cursor to c + 1.  When the next kept column is more than 15 ahead, a
+// filler entry (value +0) is placed at cursor + 15 first.  The list is then filled up to a
+// multiple of 8 with gap-0 fillers (value +0), which may run up to 7 columns past the window's
+// end: kernels give every window 8 more rows and the decoder drops such columns.  Fillers sit
+// on masked-out columns (or outside the matrix) and carry +0, so decoding still yields
+// W.*mask bit for bit; they are not counted in nnz, and their bytes are part of "compressed
+// bytes" but never called useful.  Eight consecutive entries form a chunk: 16 bytes of values
+// + one 32-bit code word whose nibble i (bits 4i..4i+3) is entry i's gap.
 //
-// The lanes step through their chunks together.  cnt[l] = chunks of lane l; cmin = the smallest
-// cnt; steps 0 .. cmin-1 hold a chunk of every lane; step cmin + e (e < nx) holds a chunk of the
-// lanes in xmask[e] = { l : cnt[l] > cmin + e } only.  nx is at most 2: where the lanes of a row
-// would differ by more, the short ones get whole chunks of code-0 fillers.  A step is stored as
-// one contiguous run: its code words in lane order (padded to 16 bytes), then its values in the
-// same order, so a warp reads 128 B + 512 B per full step with every lane on its own 4 / 16
-// bytes, and any run of whole steps of a record is one contiguous piece of memory.
-// Rows keep their natural order.
+// Rows are ordered by chunk count (most first, ties by row index), so that rows of like
+// density share a tile.  A *paired* blob (header field `pairing` = 1; M even, S <= 16) orders
+// the row pairs (2i, 2i+1) instead, by the chunks of both rows together, and keeps each pair
+// in tile rows 2j and 2j+1: a kernel that holds gate row i as row 2i and up row i as row 2i+1
+// of one stacked matrix then finds both results of a pair in the same warp.  A tile is R = 32 / S consecutive rows of that order: 32 runs, one per
+// lane of a warp; lane l holds the run of window l % S of the tile's row l / S.  Lanes step
+// through their chunks together; step j of the tile stores chunk j of every lane that has
+// more than j chunks, in lane order, so each step is one contiguous, fully used run.
 //
-//   sec0  rowdir  {u32 off16, u16 C, u8 cmin, u8 nx, u32 xmask[2]}[M+1]
-//                                      off16: start of the row record in sec1 in 16-byte units;
-//                                      C = sum of cnt; unused xmask words are 0;
-//                                      entry M: off16 = end of sec1, rest 0
-//   sec1  row records, empty for a row without chunks, else
-//                 u8  start[32]        cursor start of each lane, in units of 4 columns from its window's start
-//                 per step: u32 code[lanes of the step] (pad to 16 bytes), u16 val[8 * lanes of the step]
+//   tile record   u16 cnt[32]          chunks of each lane's run
+//                 u32 n_chunks         sum of cnt
+//                 u32 cnt_range        smallest non-zero cnt | largest cnt << 16 (0 if all are zero)
+//                 u32 lane_mask        bit l set iff cnt[l] > 0
+//                 u32 reserved         0
+//                 u16 start[32]        first column of each lane's run, counted from its window's start
+//                 u32 row[R]           original row index of each tile row, 0xFFFFFFFF = none
+//                 (pad to 16 bytes)
+//                 u32 code[n_chunks]   step-major as described
+//                 (pad to 16 bytes)
+//                 u16 val[8*n_chunks]  same order, 16 bytes per chunk
 
 #pragma once
 
@@ -69,15 +73,14 @@ namespace sd2 {
 
 constexpr int kFormatBitmask = 1;
 constexpr int kFormatGap4 = 2;
-constexpr int kGap4Lanes = 32;         // strips per row = lanes of the warp that works on it
-constexpr int kGap4MaxStrip = 496;     // widest strip
-constexpr int kGap4MinOverlap = 32;    // V is picked per matrix between these two
-constexpr int kGap4MaxOverlap = 192;
-constexpr int kGap4MaxWindow = 792;    // B + 2 V at most: 792 window rows of 128 bytes are 99 KB of shared memory
-constexpr int kGap4MaxRagged = 2;      // ragged steps of a row at most
+constexpr int kGap4Slack = 8;          // zero columns kernels append to every lane's window
+constexpr int kGap4Overlap = 32;       // columns a lane's window reaches into the strips on either side
+constexpr int kGap4MaxStrip = 496;     // widest strip: at most 63 chunks per segment
+constexpr int kGap4MinStrip = 64;      // strips narrower than this pay too much padding
+constexpr int kGap4TileTarget = 2048;  // tiles a matrix should have, if its shape allows
 
 struct BlobHeader {
-    char magic[8];          // "SD2BLOB4"
+    char magic[8];          // "SD2BLOB2"
     uint32_t version;
     uint32_t format;
     uint32_t y_dtype;
@@ -87,101 +90,57 @@ struct BlobHeader {
     int64_t compressed_bytes;   // sum of section sizes: what a kernel reads for W
     uint64_t sec_off[4];
     uint64_t sec_bytes[4];
-    uint64_t n_chunks;          // GAP4: chunks in all rows; BITMASK: 0
+    uint64_t n_chunks;          // GAP4: chunks in all tiles; BITMASK: 0
     uint64_t checksum;          // FNV-1a over bytes [sizeof(BlobHeader), total_bytes)
+    uint32_t strips;            // GAP4: S
     uint32_t strip_cols;        // GAP4: B
+    uint32_t n_tiles;           // GAP4: T
+    uint32_t max_tile_bytes;    // GAP4: largest tile record
     uint32_t overlap;           // GAP4: V, columns a lane's window reaches into its neighbours' strips
-    uint32_t max_row_steps;     // GAP4: largest cmin + nx of any row
-    uint32_t reserved[5];
+    uint32_t pairing;           // GAP4: 1 = rows 2i and 2i+1 sit in tile rows 2j and 2j+1, else 0
+    uint32_t reserved[2];
     uint8_t pad[256 - 8 - 16 - 24 - 16 - 64 - 16 - 16 - 16];
 };
 static_assert(sizeof(BlobHeader) == 256, "header is 256 bytes");
 
-// One entry of a GAP4 row directory.
-struct Gap4Dir {
-    uint32_t off16;      // start of the row record, in 16-byte units from the start of sec1
-    uint16_t C;          // chunks of the row (all lanes)
-    uint8_t cmin;        // steps in which every lane has a chunk
-    uint8_t nx;          // further steps (at most kGap4MaxRagged), in which only the lanes of xmask[e] have one
-    uint32_t xmask[2];   // lanes of ragged step e; 0 beyond nx
-};
-static_assert(sizeof(Gap4Dir) == 16, "directory entries are 16 bytes");
-
 // Strip geometry of a GAP4 matrix.
 struct Gap4Geom {
-    int B;   // columns per strip (0: K is too large for the format)
+    int S;   // strips per row
+    int B;   // columns per strip
+    int R;   // rows per tile
     int V;   // overlap: a lane's window is its strip widened by V columns on both sides
 };
 
-// Columns per strip: the smallest multiple of 4 that is >= K / 32.
-inline int64_t gap4_strip_cols(int64_t K)
+// Header bytes of a tile record with R rows.
+SD2_HD int gap4_tile_header_bytes(int R) { return (144 + 4 * R + 15) & ~15; }
+
+// Picks S: enough tiles to spread over every SM's warps, strips neither too narrow (padding)
+// nor wider than the chunk counters allow.  B is twice an odd number: in a linear row of bf16
+// activations the strips then start on 32-bit words in distinct shared-memory banks, and so does
+// every fourth column of them, which is how a kernel spreads the row over the lanes' windows.
+// S == 0: K is too large.
+// Columns per strip: the smallest B >= K / S with B = 2 (mod 4).
+inline int64_t gap4_strip_cols(int64_t K, int S)
 {
-    const int64_t b = (K + kGap4Lanes - 1) / kGap4Lanes;
-    return (b + 3) & ~int64_t(3);
+    const int64_t b = (K + S - 1) / S;
+    return b + ((6 - (b & 3)) & 3);
 }
 
-// Integer square root, rounded down.
-inline int64_t isqrt64(int64_t x)
+// A paired stack counts as one of its two halves, so that it is cut like they are.
+inline Gap4Geom gap4_geometry(int64_t M, int64_t K, bool paired = false)
 {
-    int64_t r = 0;
-    while ((r + 1) * (r + 1) <= x) ++r;
-    return r;
-}
-
-// The overlap V is what lets the dealer give every lane the same number of chunks although the
-// kept columns are not spread evenly: the column of a row's n-th kept entry strays from its
-// mean by about sqrt(n (1 - d)) / d for density d, at most sqrt(K (1 - d) / (4 d)) =: sigma in
-// the middle of a row whose total is fixed.  V = 3 sigma + 16, in steps of 16, within
-// [kGap4MinOverlap, kGap4MaxOverlap] and the shared-memory limit on B + 2 V.  Integer arithmetic
-// only, so that every build picks the same V for the same (K, nnz / (M K)).
-inline Gap4Geom gap4_geometry(int64_t M, int64_t K, int64_t nnz)
-{
+    const int64_t Mt = paired ? M / 2 : M;
+    int S = 1;
+    while (S < 32 && Mt * S / 32 < kGap4TileTarget) S <<= 1;
+    while (S > 1 && (K + S - 1) / S < kGap4MinStrip) S >>= 1;
+    while (S < 32 && gap4_strip_cols(K, S) > kGap4MaxStrip) S <<= 1;
     Gap4Geom g;
-    g.B = (int)gap4_strip_cols(K);
-    g.V = kGap4MinOverlap;
-    if (g.B > kGap4MaxStrip) { g.B = 0; return g; }
-    const int64_t slots = M * K;
-    int64_t kept = nnz < 1 ? 1 : nnz;
-    if (kept * 64 < slots) kept = (slots + 63) / 64;                 // densities under 1/64 count as 1/64
-    const int64_t var = K * (slots - (nnz < slots ? nnz : slots)) / (4 * kept);   // K (1 - d) / (4 d)
-    int64_t v = 3 * isqrt64(var) + 16;
-    v = (v + 15) & ~int64_t(15);
-    if (v < kGap4MinOverlap) v = kGap4MinOverlap;
-    if (v > kGap4MaxOverlap) v = kGap4MaxOverlap;
-    const int64_t cap = ((kGap4MaxWindow - g.B) / 2) & ~int64_t(3);
-    if (v > cap) v = cap;
-    g.V = (int)v;
+    g.S = S;
+    g.B = (int)gap4_strip_cols(K, S);
+    g.R = 32 / S;
+    g.V = kGap4Overlap;
+    if (g.B > kGap4MaxStrip) g.S = 0;
     return g;
-}
-
-// Rows of a lane's window in shared memory.
-SD2_HD int gap4_window_rows(int B, int V) { return B + 2 * V; }
-
-// Bytes of a step in which p lanes have a chunk: code words (padded to 16 bytes), then values.
-SD2_HD uint32_t gap4_step_bytes(uint32_t p) { return ((p * 4u + 15u) & ~15u) + p * 16u; }
-constexpr uint32_t kGap4FullStepBytes = 32 * 4 + 32 * 16;   // 640
-constexpr uint32_t kGap4RecordHeader = 32;                  // the start bytes
-
-SD2_HD uint32_t popcount32(uint32_t x)
-{
-#if defined(__CUDA_ARCH__)
-    return (uint32_t)__popc(x);
-#else
-    return (uint32_t)__builtin_popcount(x);
-#endif
-}
-
-// Byte offset of step j of a record (j = cmin + nx: the record's size), from what its directory entry says.
-SD2_HD uint32_t gap4_step_offset(uint32_t j, uint32_t cmin, uint32_t xmask0, uint32_t xmask1)
-{
-    uint32_t o = kGap4RecordHeader + (j < cmin ? j : cmin) * kGap4FullStepBytes;
-    if (j > cmin) o += gap4_step_bytes(popcount32(xmask0));
-    if (j > cmin + 1) o += gap4_step_bytes(popcount32(xmask1));
-    return o;
-}
-SD2_HD uint32_t gap4_record_bytes(uint32_t C, uint32_t cmin, uint32_t nx, uint32_t xmask0, uint32_t xmask1)
-{
-    return C == 0 ? 0u : gap4_step_offset(cmin + nx, cmin, xmask0, xmask1);
 }
 
 inline uint64_t fnv1a(const uint8_t* p, size_t n)
@@ -216,8 +175,8 @@ inline void fill_header(BlobHeader& h, int format, int y_dtype, int64_t M, int64
                         const size_t sec_bytes[3], uint64_t n_chunks)
 {
     std::memset(&h, 0, sizeof h);
-    std::memcpy(h.magic, "SD2BLOB4", 8);
-    h.version = 4;
+    std::memcpy(h.magic, "SD2BLOB2", 8);
+    h.version = 2;
     h.format = (uint32_t)format;
     h.y_dtype = (uint32_t)y_dtype;
     h.n_sections = 3;
@@ -319,17 +278,16 @@ inline int unpack_bitmask(const BlobHeader& h, const uint8_t* blob, uint16_t* de
 
 // ---------------------------------------------------------------- GAP4
 
-// Deals the kept columns of one row (ascending, `E` of them) to the 32 lanes: lane l gets the
-// run cols[first[l] .. first[l+1]).  The aim is the same number of whole chunks in every lane
-// (the warp walks the lanes' chunks in lock step, so the longest lane sets the time, and only a
-// lane whose count is not a multiple of 8 pays padding), under the rule that a lane's columns
-// lie in its window [l*B - V, (l+1)*B + V): a lane must take what the next one cannot reach and
-// cannot take what lies beyond its own window.
-inline void gap4_deal_row(const int32_t* cols, int E, int B, int V, int* first)
+// Deals the kept columns of one row (ascending, `E` of them) to the S lanes: lane l gets the run
+// cols[first[l] .. first[l+1]).  The aim is the same number of whole chunks in every lane (the
+// warp walks the lanes' chunks in lock step, so the longest lane sets the time, and only a lane
+// whose count is not a multiple of 8 pays padding), under the rule that a lane's columns lie in
+// its window [l*B - V, (l+1)*B + V): a lane must take what the next one cannot reach and cannot
+// take what lies beyond its own window.
+inline void gap4_deal_row(const int32_t* cols, int E, int S, int B, int V, int* first)
 {
-    constexpr int S = kGap4Lanes;
-    const int chunks = (E + 7) / 8;   // the row's last chunk may be partly padding: it ends up in the last lane
-    const int base = chunks / S, extra = chunks % S;
+    const int full = E / 8;
+    const int base = full / S, extra = full % S;
     int e = 0;
     first[0] = 0;
     for (int l = 0; l < S; ++l) {
@@ -343,9 +301,7 @@ inline void gap4_deal_row(const int32_t* cols, int E, int B, int V, int* first)
             while (e + lo < E && cols[e + lo] < must_below) ++lo;
             hi = lo;
             while (e + hi < E && cols[e + hi] < can_below) ++hi;
-            // the `extra` chunks beyond `base` per lane go to lanes spread evenly over the row, so that
-            // the runs never stray from their strips by more than the columns of one chunk on that account
-            const int want = 8 * (base + ((l + 1) * extra / S - l * extra / S));
+            const int want = 8 * (base + (l < extra ? 1 : 0));
             n = want < lo ? lo : want > hi ? hi : want;
             if (n % 8) {   // whole chunks if the limits allow: up first, then down
                 const int up = (n + 7) / 8 * 8, down = n / 8 * 8;
@@ -358,12 +314,11 @@ inline void gap4_deal_row(const int32_t* cols, int E, int B, int V, int* first)
     }
 }
 
-// Entries (kept + far-step fillers) of a lane's run, before rounding up to 8: between two kept
-// columns g apart there are (g - 1) / 15 fillers.
+// Entries (kept + far-gap fillers) of a lane's run, before rounding up to 8.
 inline int gap4_run_entries(const int32_t* cols, int n)
 {
     int e = 0;
-    for (int i = 0; i < n; ++i) e += (i == 0 ? 0 : (cols[i] - cols[i - 1] - 1) / 15) + 1;
+    for (int i = 0; i < n; ++i) e += (i == 0 ? 0 : (cols[i] - cols[i - 1] - 1) / 16) + 1;
     return e;
 }
 
@@ -374,144 +329,153 @@ inline void gap4_row_cols(const uint16_t* W, const uint8_t* mask, int64_t m, int
         if (is_kept(W, mask, m * K + k)) cols.push_back((int32_t)k);
 }
 
-// Chunk counts of the 32 lanes of one row, from its kept columns.
-struct Gap4RowPlan {
-    int first[kGap4Lanes + 1];
-    int cnt[kGap4Lanes];     // chunks of each lane, whole chunks of fillers included
-    int C, cmin, cmax;
-};
-
-inline void gap4_plan_row(const std::vector<int32_t>& cols, int B, int V, Gap4RowPlan& p)
-{
-    gap4_deal_row(cols.data(), (int)cols.size(), B, V, p.first);
-    p.cmax = 0;
-    for (int l = 0; l < kGap4Lanes; ++l) {
-        const int n = p.first[l + 1] - p.first[l];
-        p.cnt[l] = n ? (gap4_run_entries(cols.data() + p.first[l], n) + 7) / 8 : 0;
-        if (p.cnt[l] > p.cmax) p.cmax = p.cnt[l];
-    }
-    // at most kGap4MaxRagged ragged steps: lanes that are further behind get whole chunks of fillers
-    p.C = 0;
-    p.cmin = 0x7FFFFFFF;
-    for (int l = 0; l < kGap4Lanes; ++l) {
-        if (p.cmax > 0 && p.cnt[l] < p.cmax - kGap4MaxRagged) p.cnt[l] = p.cmax - kGap4MaxRagged;
-        p.C += p.cnt[l];
-        if (p.cnt[l] < p.cmin) p.cmin = p.cnt[l];
-    }
-}
-
-inline void gap4_fill_dir(const Gap4RowPlan& p, Gap4Dir& d)
-{
-    d.C = (uint16_t)p.C;
-    d.cmin = (uint8_t)p.cmin;
-    d.nx = (uint8_t)(p.cmax - p.cmin);
-    d.xmask[0] = d.xmask[1] = 0u;
-    for (int e = 0; e < p.cmax - p.cmin && e < 2; ++e)
-        for (int l = 0; l < kGap4Lanes; ++l)
-            if (p.cnt[l] > p.cmin + e) d.xmask[e] |= 1u << l;
-}
-
-inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype)
+inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K, int y_dtype, bool pair_rows = false)
 {
     PackResult r;
-    int64_t nnz = 0;
-#pragma omp parallel for schedule(static) reduction(+ : nnz)
-    for (int64_t m = 0; m < M; ++m) {
-        int64_t c = 0;
-        for (int64_t k = 0; k < K; ++k) c += is_kept(W, mask, m * K + k);
-        nnz += c;
-    }
-    const Gap4Geom g = gap4_geometry(M, K, nnz);
-    if (g.B == 0) { r.status = -5; return r; }
-    const int B = g.B, V = g.V;
-    std::vector<Gap4Dir> dir((size_t)M + 1);
-    int bad = 0;
+    const Gap4Geom g = gap4_geometry(M, K, pair_rows);
+    if (g.S == 0) { r.status = -5; return r; }
+    if (pair_rows && ((M & 1) || g.R < 2)) { r.status = -5; return r; }
+    const int S = g.S, B = g.B, R = g.R, V = g.V;
+    // per row: where each lane's run starts, chunks of each lane
+    std::vector<int32_t> first((size_t)M * (S + 1));
+    std::vector<uint16_t> seg_chunks((size_t)M * S);
+    std::vector<int64_t> row_chunks((size_t)M, 0), row_kept((size_t)M, 0);
 #pragma omp parallel
     {
         std::vector<int32_t> cols;
-        Gap4RowPlan p;
-#pragma omp for schedule(static) reduction(| : bad)
+        std::vector<int> f((size_t)S + 1);
+#pragma omp for schedule(static)
         for (int64_t m = 0; m < M; ++m) {
             gap4_row_cols(W, mask, m, K, cols);
-            gap4_plan_row(cols, B, V, p);
-            if (p.C > 0xFFFF || p.cmax > 255) bad |= 1;
-            gap4_fill_dir(p, dir[(size_t)m]);
+            gap4_deal_row(cols.data(), (int)cols.size(), S, B, V, f.data());
+            int64_t tot = 0;
+            for (int l = 0; l < S; ++l) {
+                first[(size_t)m * (S + 1) + l] = f[(size_t)l];
+                const int c = (gap4_run_entries(cols.data() + f[(size_t)l], f[(size_t)l + 1] - f[(size_t)l]) + 7) / 8;
+                seg_chunks[(size_t)m * S + l] = (uint16_t)c;
+                tot += c;
+            }
+            first[(size_t)m * (S + 1) + S] = f[(size_t)S];
+            row_chunks[(size_t)m] = tot;
+            row_kept[(size_t)m] = (int64_t)cols.size();
         }
     }
-    if (bad) { r.status = -5; return r; }
-    int64_t units = 0, chunks = 0;
-    uint32_t max_steps = 0;
-    for (int64_t m = 0; m < M; ++m) {
-        Gap4Dir& d = dir[(size_t)m];
-        d.off16 = (uint32_t)units;
-        units += (int64_t)(gap4_record_bytes(d.C, d.cmin, d.nx, d.xmask[0], d.xmask[1]) / 16);
-        chunks += d.C;
-        if ((uint32_t)d.cmin + d.nx > max_steps) max_steps = (uint32_t)d.cmin + d.nx;
+    // rows by chunk count, most first, ties by index
+    std::vector<uint32_t> order((size_t)M);
+    std::iota(order.begin(), order.end(), 0u);
+    if (!pair_rows) {
+        std::stable_sort(order.begin(), order.end(),
+                         [&](uint32_t a, uint32_t b) { return row_chunks[a] > row_chunks[b]; });
+    } else {   // the same for pairs (2i, 2i+1), by the chunks of both rows
+        std::vector<uint32_t> pairs((size_t)(M / 2));
+        std::iota(pairs.begin(), pairs.end(), 0u);
+        std::stable_sort(pairs.begin(), pairs.end(), [&](uint32_t a, uint32_t b) {
+            return row_chunks[2 * (size_t)a] + row_chunks[2 * (size_t)a + 1] > row_chunks[2 * (size_t)b] + row_chunks[2 * (size_t)b + 1];
+        });
+        for (size_t i = 0; i < pairs.size(); ++i) {
+            order[2 * i] = 2 * pairs[i];
+            order[2 * i + 1] = 2 * pairs[i] + 1;
+        }
+    }
+    const int64_t T = (M + R - 1) / R;
+    const int hdr = gap4_tile_header_bytes(R);
+    std::vector<uint32_t> toff((size_t)T + 1, 0);
+    int64_t C = 0, nnz = 0, units = 0;
+    uint32_t max_tile = 0;
+    for (int64_t m = 0; m < M; ++m) nnz += row_kept[(size_t)m];
+    for (int64_t t = 0; t < T; ++t) {
+        int64_t ct = 0;
+        for (int rr = 0; rr < R; ++rr) {
+            const int64_t i = t * R + rr;
+            if (i < M) ct += row_chunks[order[(size_t)i]];
+        }
+        const size_t bytes = (size_t)hdr + align16((size_t)ct * 4) + (size_t)ct * 16;
+        toff[(size_t)t] = (uint32_t)units;
+        units += (int64_t)(bytes / 16);
+        C += ct;
+        if (bytes > max_tile) max_tile = (uint32_t)bytes;
         if (units > 0xFFFFFFF0ll) { r.status = -2; return r; }
     }
-    std::memset(&dir[(size_t)M], 0, sizeof(Gap4Dir));
-    dir[(size_t)M].off16 = (uint32_t)units;
-    size_t sec[3] = {(size_t)(M + 1) * sizeof(Gap4Dir), (size_t)units * 16, 0};
+    toff[(size_t)T] = (uint32_t)units;
+    size_t sec[3] = {(size_t)(T + 1) * 4, (size_t)units * 16, 0};
     BlobHeader h;
-    fill_header(h, kFormatGap4, y_dtype, M, K, nnz, sec, (uint64_t)chunks);
+    fill_header(h, kFormatGap4, y_dtype, M, K, nnz, sec, (uint64_t)C);
+    h.strips = (uint32_t)S;
     h.strip_cols = (uint32_t)B;
+    h.n_tiles = (uint32_t)T;
+    h.max_tile_bytes = max_tile;
     h.overlap = (uint32_t)V;
-    h.max_row_steps = max_steps;
+    h.pairing = pair_rows ? 1u : 0u;
     uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
     if (!blob) { r.status = -3; return r; }
-    std::memcpy(blob + h.sec_off[0], dir.data(), sec[0]);
-    uint8_t* recs = blob + h.sec_off[1];
+    std::memcpy(blob + h.sec_off[0], toff.data(), sec[0]);
+    uint8_t* tiles = blob + h.sec_off[1];
 #pragma omp parallel
     {
         std::vector<int32_t> cols;
-        std::vector<uint8_t> eg[kGap4Lanes];
-        std::vector<uint16_t> ev[kGap4Lanes];
-        Gap4RowPlan p;
-#pragma omp for schedule(dynamic, 16)
-        for (int64_t m = 0; m < M; ++m) {
-            const Gap4Dir& d = dir[(size_t)m];
-            if (d.C == 0) continue;
-            uint8_t* rec = recs + (size_t)d.off16 * 16;
-            gap4_row_cols(W, mask, m, K, cols);
-            gap4_plan_row(cols, B, V, p);
-            uint8_t* start = rec;
-            for (int l = 0; l < kGap4Lanes; ++l) {
-                const int c = p.cnt[l];
-                start[l] = 0;
-                eg[l].assign((size_t)c * 8, 0);
-                ev[l].assign((size_t)c * 8, 0);
-                const int e0 = p.first[l], e1 = p.first[l + 1];
-                if (e0 == e1) continue;   // only fillers (or nothing): the cursor rests on the window's first column
-                const int64_t wbase = (int64_t)l * B - V;
-                const int64_t q = (cols[(size_t)e0] - wbase) >> 2;   // cursor start, in units of 4 columns
-                start[l] = (uint8_t)q;
-                int64_t cursor = wbase + 4 * q;
-                size_t e = 0;
-                for (int x = e0; x < e1; ++x) {
-                    const int64_t k = cols[(size_t)x];
-                    while (k - cursor > 15) {  // filler 15 columns ahead
-                        eg[l][e] = 15;
-                        ev[l][e] = 0;
-                        ++e;
-                        cursor += 15;
-                    }
-                    eg[l][e] = (uint8_t)(k - cursor);
-                    ev[l][e] = W[m * K + k];
-                    ++e;
-                    cursor = k;
+        std::vector<uint8_t> eg[32];
+        std::vector<uint16_t> ev[32];
+#pragma omp for schedule(dynamic, 8)
+        for (int64_t t = 0; t < T; ++t) {
+            uint8_t* rec = tiles + (size_t)toff[(size_t)t] * 16;
+            uint16_t* cnt = (uint16_t*)rec;
+            uint32_t* nch = (uint32_t*)(rec + 64);
+            uint16_t* start = (uint16_t*)(rec + 80);
+            uint32_t* rows = (uint32_t*)(rec + 144);
+            uint32_t ct = 0, lane_mask = 0;
+            int maxc = 0, minc = 0xFFFF;
+            for (int rr = 0; rr < R; ++rr) {
+                const int64_t i = t * R + rr;
+                rows[rr] = i < M ? order[(size_t)i] : 0xFFFFFFFFu;
+                if (i >= M) {
+                    for (int s = 0; s < S; ++s) { cnt[rr * S + s] = 0; start[rr * S + s] = 0; }
+                    continue;
                 }
-                // entries e .. 8c-1 stay code 0 / value +0: the cursor rests on the last column
+                const int64_t m = order[(size_t)i];
+                gap4_row_cols(W, mask, m, K, cols);
+                for (int s = 0; s < S; ++s) {
+                    const int l = rr * S + s;
+                    const int e0 = first[(size_t)m * (S + 1) + s], e1 = first[(size_t)m * (S + 1) + s + 1];
+                    const int c = seg_chunks[(size_t)m * S + s];
+                    cnt[l] = (uint16_t)c;
+                    start[l] = 0;
+                    ct += (uint32_t)c;
+                    if (c > maxc) maxc = c;
+                    if (c == 0) continue;
+                    if (c < minc) minc = c;
+                    lane_mask |= 1u << l;
+                    eg[l].assign((size_t)c * 8, 0);
+                    ev[l].assign((size_t)c * 8, 0);
+                    // the cursor starts on the run's first column, given relative to the lane's window
+                    start[l] = (uint16_t)(cols[(size_t)e0] - ((int64_t)s * B - V));
+                    int64_t cursor = cols[(size_t)e0];
+                    size_t e = 0;
+                    for (int x = e0; x < e1; ++x) {
+                        const int64_t k = cols[(size_t)x];
+                        while (k - cursor > 15) {  // filler 15 columns ahead
+                            eg[l][e] = 15;
+                            ev[l][e] = 0;
+                            ++e;
+                            cursor += 16;
+                        }
+                        eg[l][e] = (uint8_t)(k - cursor);
+                        ev[l][e] = W[m * K + k];
+                        ++e;
+                        cursor = k + 1;
+                    }
+                    // entries e .. 8c-1 stay gap 0 / value +0
+                }
             }
-            uint8_t* at = rec + kGap4RecordHeader;
-            for (int j = 0; j < p.cmax; ++j) {
-                uint32_t lanes = 0;
-                for (int l = 0; l < kGap4Lanes; ++l)
-                    if (p.cnt[l] > j) ++lanes;
-                uint32_t* codes = (uint32_t*)at;
-                uint16_t* vals = (uint16_t*)(at + ((lanes * 4u + 15u) & ~15u));
-                size_t slot = 0;
-                for (int l = 0; l < kGap4Lanes; ++l) {
-                    if (p.cnt[l] <= j) continue;
+            nch[0] = ct;
+            nch[1] = lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u;
+            nch[2] = lane_mask;
+            nch[3] = 0;
+            uint32_t* codes = (uint32_t*)(rec + hdr);
+            uint16_t* vals = (uint16_t*)(rec + hdr + align16((size_t)ct * 4));
+            size_t slot = 0;
+            for (int j = 0; j < maxc; ++j) {
+                for (int l = 0; l < 32; ++l) {
+                    if (cnt[l] <= j) continue;
                     uint32_t code = 0;
                     for (int i = 0; i < 8; ++i) {
                         code |= (uint32_t)eg[l][(size_t)j * 8 + i] << (4 * i);
@@ -520,7 +484,6 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
                     codes[slot] = code;
                     ++slot;
                 }
-                at += gap4_step_bytes(lanes);
             }
         }
     }
@@ -531,77 +494,104 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     return r;
 }
 
-// Validates the directory and every row record (so that a kernel can trust them) and, if
-// `dense` is given, decodes.
+// Validates every tile record (so that a kernel can trust it) and, if `dense` is given, decodes.
 inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense)
 {
     const int64_t M = h.M, K = h.K;
-    const Gap4Geom g = gap4_geometry(M, K, h.nnz);
-    if (g.B == 0 || h.strip_cols != (uint32_t)g.B || h.overlap != (uint32_t)g.V) return -6;
-    const int B = g.B, V = g.V;
-    if (h.sec_bytes[0] != (uint64_t)(M + 1) * sizeof(Gap4Dir) || h.sec_bytes[2] != 0 || h.sec_bytes[1] % 16) return -6;
-    const Gap4Dir* dir = (const Gap4Dir*)(blob + h.sec_off[0]);
-    const uint8_t* recs = blob + h.sec_off[1];
+    if (h.pairing > 1) return -6;
+    const Gap4Geom g = gap4_geometry(M, K, h.pairing == 1);
+    if (g.S == 0 || h.strips != (uint32_t)g.S || h.strip_cols != (uint32_t)g.B || h.overlap != (uint32_t)g.V) return -6;
+    const int S = g.S, B = g.B, R = g.R, V = g.V;
+    const int64_t T = (M + R - 1) / R;
+    if (h.pairing > 1 || (h.pairing == 1 && ((M & 1) || R < 2))) return -6;
+    if (h.n_tiles != (uint64_t)T || h.sec_bytes[0] != (uint64_t)(T + 1) * 4 || h.sec_bytes[2] != 0) return -6;
+    if (h.sec_bytes[1] % 16) return -6;
+    const uint32_t* toff = (const uint32_t*)(blob + h.sec_off[0]);
+    const uint8_t* tiles = blob + h.sec_off[1];
     const uint64_t units = h.sec_bytes[1] / 16;
-    const int wrows = gap4_window_rows(B, V);   // window rows a kernel keeps per lane
-    if (dir[0].off16 != 0 || dir[M].off16 != units || dir[M].C != 0 || dir[M].cmin != 0 || dir[M].nx != 0 ||
-        dir[M].xmask[0] != 0 || dir[M].xmask[1] != 0)
-        return -6;
+    const int hdr = gap4_tile_header_bytes(R);
+    const int window = B + 2 * V;   // columns a lane may touch, before the slack
+    if (toff[0] != 0 || toff[T] != units) return -6;
+    for (int64_t t = 0; t < T; ++t)
+        if (toff[t + 1] <= toff[t]) return -6;
+    std::vector<uint8_t> seen((size_t)M, 0);
+    int bad = 0;
     int64_t chunks = 0;
-    uint32_t max_steps = 0;
-    for (int64_t m = 0; m < M; ++m) {
-        const Gap4Dir& d = dir[m];
-        if (dir[m + 1].off16 < d.off16) return -6;
-        if (d.nx > kGap4MaxRagged) return -6;
-        if (d.C == 0 && (d.cmin != 0 || d.nx != 0)) return -6;
-        if (d.C != 0 && d.cmin == 0 && d.nx == 0) return -6;
-        // ragged steps: each set of lanes non-empty, not all lanes, contained in the one before; none beyond nx
-        const uint32_t m0 = d.xmask[0], m1 = d.xmask[1];
-        if ((d.nx >= 1) != (m0 != 0) || (d.nx >= 2) != (m1 != 0)) return -6;
-        if (m0 == 0xFFFFFFFFu || (m1 & ~m0) != 0) return -6;
-        if ((int64_t)kGap4Lanes * d.cmin + __builtin_popcount(m0) + __builtin_popcount(m1) != (int64_t)d.C) return -6;
-        if ((uint64_t)(dir[m + 1].off16 - d.off16) * 16 != gap4_record_bytes(d.C, d.cmin, d.nx, m0, m1)) return -6;
-        chunks += d.C;
-        if ((uint32_t)d.cmin + d.nx > max_steps) max_steps = (uint32_t)d.cmin + d.nx;
+    for (int64_t t = 0; t < T; ++t) {  // row ids: a permutation of 0..M-1, checked serially
+        if ((uint64_t)(toff[t + 1] - toff[t]) * 16 < (uint64_t)hdr) return -6;
+        const uint32_t* rows = (const uint32_t*)(tiles + (size_t)toff[t] * 16 + 144);
+        for (int rr = 0; rr < R; ++rr) {
+            const int64_t i = t * R + rr;
+            if (i < M) {
+                if (rows[rr] >= (uint64_t)M || seen[rows[rr]]) return -6;
+                seen[rows[rr]] = 1;
+            } else if (rows[rr] != 0xFFFFFFFFu) {
+                return -6;
+            }
+        }
+        if (h.pairing == 1)
+            for (int rr = 0; rr + 1 < R; rr += 2) {
+                const bool none = rows[rr] == 0xFFFFFFFFu && rows[rr + 1] == 0xFFFFFFFFu;
+                if (!none && ((rows[rr] & 1u) || rows[rr + 1] != rows[rr] + 1u)) return -6;
+            }
     }
-    if (chunks != (int64_t)h.n_chunks || max_steps != h.max_row_steps) return -6;
     if (dense) {
 #pragma omp parallel for schedule(static)
         for (int64_t m = 0; m < M; ++m) std::memset(dense + m * K, 0, (size_t)K * 2);
     }
-    int bad = 0;
-#pragma omp parallel for schedule(dynamic, 16) reduction(| : bad)
-    for (int64_t m = 0; m < M; ++m) {
-        const Gap4Dir& d = dir[m];
-        if (d.C == 0) continue;
-        const uint8_t* rec = recs + (size_t)d.off16 * 16;
-        const uint8_t* start = rec;
-        int64_t cursor[kGap4Lanes], wbase[kGap4Lanes];
-        for (int l = 0; l < kGap4Lanes; ++l) {
-            wbase[l] = (int64_t)l * B - V;          // first column of the lane's window (may be negative)
-            if (4 * (int)start[l] >= wrows) bad |= 1;
-            cursor[l] = wbase[l] + 4 * (int64_t)start[l];
+#pragma omp parallel for schedule(dynamic, 8) reduction(| : bad) reduction(+ : chunks)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint8_t* rec = tiles + (size_t)toff[t] * 16;
+        const size_t rec_bytes = (size_t)(toff[t + 1] - toff[t]) * 16;
+        const uint16_t* cnt = (const uint16_t*)rec;
+        const uint32_t* meta = (const uint32_t*)(rec + 64);
+        const uint16_t* start = (const uint16_t*)(rec + 80);
+        const uint32_t ct = meta[0];
+        const uint32_t* rows = (const uint32_t*)(rec + 144);
+        uint32_t sum = 0, lane_mask = 0;
+        int maxc = 0, minc = 0xFFFF;
+        for (int l = 0; l < 32; ++l) {
+            if (cnt[l] > (window + kGap4Slack) / 8 + 1) bad |= 1;
+            if (rows[l / S] == 0xFFFFFFFFu && cnt[l] != 0) bad |= 1;
+            if (start[l] >= window + kGap4Slack) bad |= 1;
+            sum += cnt[l];
+            if (cnt[l] > maxc) maxc = cnt[l];
+            if (cnt[l] > 0) {
+                lane_mask |= 1u << l;
+                if (cnt[l] < minc) minc = cnt[l];
+            }
         }
-        const int steps = (int)d.cmin + (int)d.nx;
-        for (int j = 0; j < steps; ++j) {
-            const uint32_t mk = j < (int)d.cmin ? 0xFFFFFFFFu : d.xmask[j - d.cmin];
-            const uint8_t* at = rec + gap4_step_offset((uint32_t)j, d.cmin, d.xmask[0], d.xmask[1]);
-            const uint32_t lanes = (uint32_t)__builtin_popcount(mk);
-            const uint32_t* codes = (const uint32_t*)at;
-            const uint16_t* vals = (const uint16_t*)(at + ((lanes * 4u + 15u) & ~15u));
-            size_t slot = 0;
-            for (int l = 0; l < kGap4Lanes; ++l) {
-                if (!((mk >> l) & 1u)) continue;
+        if (meta[1] != (lane_mask ? (uint32_t)minc | ((uint32_t)maxc << 16) : 0u) || meta[2] != lane_mask || meta[3] != 0)
+            bad |= 1;
+        if (sum != ct || rec_bytes != (size_t)hdr + align16((size_t)ct * 4) + (size_t)ct * 16 ||
+            rec_bytes > h.max_tile_bytes) {
+            bad |= 1;
+            continue;
+        }
+        if (bad) continue;
+        chunks += ct;
+        const uint32_t* codes = (const uint32_t*)(rec + hdr);
+        const uint16_t* vals = (const uint16_t*)(rec + hdr + align16((size_t)ct * 4));
+        int64_t cursor[32], wbase[32];
+        for (int l = 0; l < 32; ++l) {
+            wbase[l] = (int64_t)(l % S) * B - V;          // first column of the lane's window (may be negative)
+            cursor[l] = wbase[l] + start[l];
+        }
+        size_t slot = 0;
+        for (int j = 0; j < maxc; ++j) {
+            for (int l = 0; l < 32; ++l) {
+                if (cnt[l] <= j) continue;
+                const int64_t m = rows[l / S];
                 const uint32_t code = codes[slot];
                 for (int i = 0; i < 8; ++i) {
                     const int64_t col = cursor[l] + ((code >> (4 * i)) & 15);
-                    cursor[l] = col;
+                    cursor[l] = col + 1;
                     const uint16_t v = vals[slot * 8 + i];
-                    // a kernel reads window row col - wbase: it must exist
-                    if (col - wbase[l] >= wrows) { bad |= 1; continue; }
+                    // a kernel reads window row col - wbase: it must exist (window + slack rows)
+                    if (col - wbase[l] >= window + kGap4Slack) { bad |= 1; continue; }
                     if (col >= 0 && col < K) {
                         if (dense && v != 0) {
-                            if (dense[m * K + col] != 0) bad |= 1;   // two entries claim one column
+                            if (dense[m * K + col] != 0) bad |= 1;   // two lanes claim one column
                             dense[m * K + col] = v;
                         }
                     } else if (v != 0) {
@@ -612,6 +602,7 @@ inline int unpack_gap4(const BlobHeader& h, const uint8_t* blob, uint16_t* dense
             }
         }
     }
+    if (chunks != (int64_t)h.n_chunks) bad |= 1;
     return bad ? -6 : 0;
 }
 
@@ -620,7 +611,7 @@ inline int check_header(const uint8_t* blob, int64_t bytes, BlobHeader& h, bool 
 {
     if (bytes < (int64_t)sizeof(BlobHeader)) return -6;
     std::memcpy(&h, blob, sizeof h);
-    if (std::memcmp(h.magic, "SD2BLOB4", 8) != 0 || h.version != 4) return -6;
+    if (std::memcmp(h.magic, "SD2BLOB2", 8) != 0 || h.version != 2) return -6;
     if (h.format != (uint32_t)kFormatBitmask && h.format != (uint32_t)kFormatGap4) return -6;
     if (h.y_dtype > 1 || h.n_sections != 3) return -6;
     if (h.M < 1 || h.K < 1 || h.nnz < 0 || h.nnz > h.M * h.K) return -6;

@@ -2,23 +2,20 @@
 // Y[n, m] = sum over kept k of W[m, k] X[n, k]  (bf16 in, fp32 accumulate, one rounding).
 //
 // The work is a streaming scan of a compressed matrix, bound by HBM bandwidth at N = 1
-// and by the load/store pipe and instruction issue as N grows; it is not a dense contraction,
-// so there are no tensor-core instructions here.  What matters instead:
-//   - every byte of the compressed weight is read from HBM exactly once, by asynchronous copies
-//     (cp.async, 16 bytes per lane, global -> shared without a register in between): every warp
-//     keeps a private ring of a few pieces of its coming rows in flight, across row and stage
-//     boundaries, so DRAM keeps streaming while the arithmetic waits for activations;
+// and by instruction issue as N grows; it is not a dense contraction, so there are no
+// tensor-core instructions here.  What matters instead:
+//   - every byte of the compressed weight is read from HBM exactly once, by bulk
+//     asynchronous copies (cp.async.bulk, global -> shared) that a producer warp issues tile
+//     by tile into a ring and that run ahead of the arithmetic, across stage boundaries;
 //   - the activations are staged once per stage in shared memory in a layout in which the
 //     32 lanes of a warp always read 32 different banks, whatever columns they gather;
-//   - position decoding is byte-parallel (prefix sums of eight 4-bit codes in two registers);
+//   - position decoding is byte-parallel (prefix sums of eight 4-bit gaps in two registers);
 //   - one row's sum order is fixed, so results are deterministic run to run.
 
 #pragma once
 
 #include <cuda_runtime.h>
 #include <stdint.h>
-
-#include <type_traits>
 
 #include "sd2_format.hpp"
 
@@ -67,97 +64,77 @@ __device__ __forceinline__ float warp_sum(float v)
 //
 // One persistent CTA per SM runs a *program* of stages.  A stage is one launch's worth of
 // work: up to four weights that read the same activations (q|k|v, gate|up, or one weight).
-// Consecutive stages depend on each other (the next one reads what this one wrote).
+// Consecutive stages depend on each other (the next one reads what this one wrote), so they
+// are separated by a grid-wide barrier; the weights, however, never depend on anything, and
+// the producer warp keeps copying the tiles of coming stages into the ring while the
+// consumer warps are still computing, waiting at the barrier or staging activations.
 //
-// Work is dealt in *units* of one row (two rows of a paired gate|up stack): unit v of a stage
-// goes to CTA v % gridDim.x, and the units of a CTA go round-robin to its 16 warps.  A warp owns
-// whole rows, so a row's sum is formed in one fixed order (deterministic, no atomics).
-// Everything about a warp's coming rows follows from the stage descriptors and the weights' row
-// directories, none of which depend on activations.  A warp cuts its rows into *pieces* of up to
-// kPieceSteps steps (a piece is one contiguous run of a row record), and keeps the next pieces,
-// those of the following stages included, in flight into its own ring of shared-memory slots:
-// the lanes copy a piece 16 bytes each per instruction (one commit group per piece) and the warp
-// later waits for that group.  No other warp ever touches the ring, so a slot is free again as
-// soon as the warp itself is done with it.  (One bulk copy per piece, cp.async.bulk, would be
-// fewer instructions, but an SM starts only a few of those per microsecond whatever their size:
-// at 2 to 3 KB a piece that is a tenth of the HBM rate.)
+// Tiles of a stage are dealt round-robin to the CTAs (tile v of the stage goes to CTA
+// v % gridDim.x) and, inside a CTA, round-robin to the consumer warps.  A warp owns whole
+// tiles, so a row's sum is formed in one fixed order (deterministic, no atomics).
 //
-// Per row, lane l owns the run of strip l (see sd2_format.hpp); per chunk: E = even nibbles,
-// O = odd nibbles as bytes; P = (E + O) * 0x01010100 is the exclusive prefix of the pair sums;
-// PE = P + E and PO = PE + O are the inclusive prefixes of the even and odd entries' codes; entry
-// i sits at window row cursor + prefix_i.  The activations live in shared memory as xs[window
-// row][lane][W words], 32 * W words per window row: a word holds one bf16 (NT = 1, in the high
-// half) or the bf16 values of two activation rows (row 2j in the low half, row 2j+1 in the high
-// half of word j), W = max(1, NT / 2).  Lane l reads only its own words, so one warp-wide gather
-// touches every bank W times.
+// Per tile, lane l owns one segment (strip l % S of tile row l / S) and walks its chunks;
+// per chunk: E = even nibbles, O = odd nibbles as bytes; P = (E + O) * 0x01010100 is the
+// exclusive prefix of the pair sums; PE = P + E and PO = PE + O are the inclusive gap
+// prefixes of the even and odd entries; entry i sits at local column cursor + prefix_i + i.
+// The activations live in shared memory as xs[column][groups][W words], 32 words per column: a
+// word holds one bf16 (NT = 1, in the high half) or the bf16 values of two activation rows
+// (row 2j in the low half, row 2j+1 in the high half of word j), W = max(1, NT / 2), groups =
+// 32 / W.  Lane l reads group l % groups, so one warp-wide gather touches every bank W times.
 //
-// Hand-off between stages is either a grid-wide barrier (programs over caller-owned
-// workspaces) or *tagged words* (drafters): every intermediate activation is also written as a
-// 32-bit word bf16 << 16 | tag, and the next stage polls exactly the words it needs until they
-// carry the tag it expects.  Value and tag share a word, so no fence is needed.  A tag is
-// (number of times that activation row has been produced & 0xFF) << 8 | (stage number + 1):
-// a word left by any earlier launch differs in the first field from the one this launch will
-// write, whatever rows the launches in between covered.
-//
-// Every wait on another SM (tag polls, grid barrier) is bounded by a cycle budget: when it runs
-// out the CTA raises the error word and winds down instead of hanging.
+// Every wait (ring barriers, grid barrier) is bounded by a cycle budget: when it runs out
+// the CTA raises the error word and winds down instead of hanging.
 
-constexpr int kConsumerWarps = 16;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kStreamThreads = kConsumerThreads;
-#ifndef SD2_PIECE_STEPS
-#define SD2_PIECE_STEPS 4
+#ifndef SD2_CONSUMER_WARPS
+#define SD2_CONSUMER_WARPS 16
 #endif
-constexpr int kPieceSteps = SD2_PIECE_STEPS;             // steps of a piece, at most
-constexpr int kSlotBytes = ((16 + (int)kGap4RecordHeader + kPieceSteps * (int)kGap4FullStepBytes) + 127) & ~127;
-constexpr int kMaxSlots = 4;                             // ring slots per warp, at most
-constexpr int kDirSlots = 8;                             // rows of a stage a warp looks up at a time
-constexpr int kMaxStagesInline = 4;
-constexpr int kStageSlots = 8;                           // stage descriptors kept in shared memory
-constexpr int kStageAhead = 6;                           // a CTA in stage s holds the descriptors of stages s - 1 .. s + kStageAhead:
-                                                         // a warp's piece iterator runs at most kMaxSlots stages ahead and looks
-                                                         // one stage further
-
+constexpr int kConsumerWarps = SD2_CONSUMER_WARPS;
 // words of staged activations a lane reads per gathered column, at a panel width of nt rows
 __host__ __device__ constexpr int xs_words(int nt) { return nt <= 2 ? 1 : nt / 2; }
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
+constexpr int kSlots = 64;                               // tiles in flight per CTA, at most
+constexpr int kMaxStagesInline = 8;
 
 struct SMat {
-    const uint4* rowdir;           // [M + 1] directory entries (Gap4Dir)
-    const unsigned char* stream;   // row records
-    void* y;                       // [N * M], may be NULL when yt is set (or in a paired stage)
-    uint32_t* yt;                  // [N * M] tagged words (bf16 << 16 | tag) for the next stage, or NULL
+    const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
+    const unsigned char* stream;   // tile records
+    void* y;                       // [N * M], may be NULL when yt is set
+    uint32_t* yt;                  // [N * M] tagged words (bf16 << 16 | stage tag) for the next stage, or NULL
     int M;
+    int T;
     int y_f32;                     // 1: fp32 output, 0: bf16
-    int unit0;                     // first unit of this weight in the stage's unit sequence
-    int voff;                      // the stage's overlap minus this weight's: window rows its cursors start later
+    int reserved;
 };
 
 struct SStage {
     SMat mat[kMaxFused];
-    const uint16_t* x;     // [N * K] bf16 (or tagged words, see tagged_in), or NULL in glue mode
-    const uint16_t* g;     // glue mode: t = bf16(silu(g) * u) is the activation; paired: g is an output
+    const uint16_t* x;     // [N * K] bf16, or NULL in glue mode
+    const uint16_t* g;     // glue mode: t = bf16(silu(g) * u) is the activation
     const uint16_t* u;
-    uint16_t* t_out;       // glue mode / paired: t is also written here as plain bf16 (may be NULL)
-    uint32_t* tt;          // paired: tagged copy of t for the next stage
+    uint16_t* t_out;       // glue mode: t is also written here as plain bf16 (may be NULL)
+    uint32_t* tt;          // tagged glue mode: tagged copy of t, computed once, a slice per CTA (or NULL)
     int count;             // weights in the stage
     int K;
+    int S;                 // strips; equal for all weights of a stage
     int B;                 // strip width
-    int V;                 // overlap of the staged windows: the largest of the weights' overlaps
-    int wrows;             // rows of a lane's window: B + 2 V
-    int units;             // units of all weights
-    int upr;               // rows per unit: 1, or 2 in a paired stage
-    int tagged_in;         // x points at tagged 32-bit words written by the previous stage
-    int paired;            // mat[0] stacks gate row i (row 2i) and up row i (row 2i+1): the stage stores
-                           // g, u, t_out (plain bf16, each may be NULL) and tt (tagged t)
-    int reserved[5];
+    int T_total;           // tiles of all weights
+    int hdr_bytes;         // tile header bytes (depends on S)
+    int log2S;
+    int tiles_div;         // T_total / grid size: CTA c runs tiles_div + (c < tiles_rem) tiles
+    int tiles_rem;         // T_total % grid size
+    int tagged_in;         // x / g / u point at tagged 32-bit words written by the previous stage
+    int V;                 // overlap: lane windows are strips widened by V columns on both sides
+    int paired;            // mat[0] stacks gate row i (row 2i) and up row i (row 2i+1), pairs share a tile:
+                           // the stage stores g, u, t_out (plain bf16, each may be NULL) and tt (tagged t)
+    int reserved[2];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
-constexpr int kStageWords = (int)(sizeof(SStage) / 4);
 
 struct SArgs {
     SStage inl[kMaxStagesInline];   // used when ext == NULL
-    const SStage* ext;              // device array of stages (longer programs)
-    const uint16_t* x_in;           // replaces stage 0's x when not NULL (plain bf16)
+    const SStage* ext;              // device array of stages (programs longer than four stages)
+    const uint16_t* x_in;           // replaces stage 0's x when not NULL
     void* y_out;                    // replaces the last stage's mat[0].y when not NULL
     unsigned int* gbar;             // grid barrier: [0] arrivals, [32] exits (two cache lines)
     int* err;                       // device error word
@@ -165,15 +142,24 @@ struct SArgs {
     int n_stages;
     int N;                          // activation rows of this launch, 1..NT
     int n0;                         // first activation row: every X / Y pointer is advanced by n0 rows
-    int xs_odd;                     // staged activations: even stages at offset 0, odd stages at this offset of
-    int xs_total;                   // the activation area of xs_total bytes (0 and xs_total / 1: one buffer)
-    int xs_single;                  // 1: both offsets are 0 (one buffer): one more CTA barrier per stage
-    int nslot;                      // ring slots per warp, 2 .. kMaxSlots
+    int xs_bytes;                   // shared memory for the transposed activations
+    int xlin_bytes;                 // shared memory for one linear activation row
+    int ring_bytes;
     int tagged;                     // 1: stages hand activations over as tagged words, no grid barrier
-    unsigned int* rowseq;           // tagged programs: per activation row, how often it has been produced
-    int hinted;                     // 1: weight copies carry an L2 evict-first policy
-    int reserved;
+    unsigned int* seq;              // tagged programs: launch counter (device word), bumped by the last CTA out
+    int free_tiles;                 // 1: a consumer warp that is done draws the next tile from a shared counter;
+                                    // 0: tile k of a stage goes to warp k % 16 (see the consumer loop)
+    long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
 };
+
+#ifdef SD2_TRACE
+// per-tile stamps of CTA 0 (issue, wait begin, start, end, producer waits for its release: begin, end)
+#define SD2_TILE_STAMP(q, slot) do { if (a.trace && cta == 0 && (q) < 4096u) a.trace[(size_t)gridDim.x * a.n_stages * 8 + (size_t)(q) * 8 + (slot)] = clock64(); } while (0)
+#define SD2_STAMP(slot) do { if (a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define SD2_STAMP(slot) do { } while (0)
+#define SD2_TILE_STAMP(q, slot) do { } while (0)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -182,8 +168,18 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 // A waiting thread is parked by the hardware until the phase completes or this many
-// nanoseconds pass, instead of spinning.
+// nanoseconds pass, instead of spinning through the shared-memory pipe that working warps need.
 constexpr uint32_t kSuspendHintNs = 20000;
 
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
@@ -199,39 +195,44 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
-// 16 bytes global -> shared, asynchronously (no register in between, no L1 allocation); completion is
-// tracked per thread in groups (cp_async_commit / cp_async_wait)
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src)
+// non-blocking: has the phase of this parity completed?
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint64_t policy)
+
+// global -> this CTA's shared memory, completion counted in bytes on `bar`
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
 {
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-// waits until at most `pending` of this thread's most recent groups are still under way (0 .. 3)
-__device__ __forceinline__ void cp_async_wait(uint32_t pending)
+// the same with an L2 cache policy (see l2_evict_first)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy)
 {
-    if (pending == 0u) asm volatile("cp.async.wait_group 0;" ::: "memory");
-    else if (pending == 1u) asm volatile("cp.async.wait_group 1;" ::: "memory");
-    else if (pending == 2u) asm volatile("cp.async.wait_group 2;" ::: "memory");
-    else asm volatile("cp.async.wait_group 3;" ::: "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+                 : "memory");
 }
 
 // Weights are read once per launch: their lines are the first to go when L2 needs room, so that the
 // stream does not push the (small, shared, re-read) activation words of the hand-off out to DRAM.
+// Only programs of several stages have such words; a single-stage launch measured 13 % slower with
+// the hint than without, and goes without.
 __device__ __forceinline__ uint64_t l2_evict_first()
 {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
-}
-
-// ask L2 to fetch [p, p + bytes) (16-byte aligned, a multiple of 16 bytes); nothing is returned
-__device__ __forceinline__ void l2_prefetch_bulk(const void* p, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ uint32_t lds_u32(uint32_t a)
@@ -240,10 +241,10 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t a)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
-__device__ __forceinline__ uint32_t lds_u8(uint32_t a)
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a)
 {
-    uint32_t v;
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
     return v;
 }
 __device__ __forceinline__ uint4 lds_v4(uint32_t a)
@@ -251,10 +252,6 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t a)
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
-}
-__device__ __forceinline__ void sts_v4(uint32_t a, uint4 v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 template <int OFF>
 __device__ __forceinline__ uint32_t lds_u32_off(uint32_t a)
@@ -270,13 +267,12 @@ __device__ __forceinline__ uint2 lds_u32x2_off(uint32_t a)
     asm volatile("ld.shared.v2.u32 {%0,%1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(a), "n"(OFF));
     return v;
 }
-__device__ __forceinline__ void sts_u32(uint32_t a, uint32_t v)
+template <int OFF>
+__device__ __forceinline__ uint4 lds_u32x4_off(uint32_t a)
 {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-__device__ __forceinline__ void sts_u32x2(uint32_t a, uint32_t v0, uint32_t v1)
-{
-    asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(a), "r"(v0), "r"(v1) : "memory");
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a), "n"(OFF));
+    return v;
 }
 
 // c + 128 * byte K8 of p (one integer dot-product instruction with a one-hot operand)
@@ -299,39 +295,18 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p)
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ uint4 ld_relaxed_v4(const uint32_t* p)
-{
-    uint4 v;
-    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p)
-{
-    uint32_t v;
-    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_relaxed_u32(uint32_t* p, uint32_t v)
-{
-    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 
-// Shared-memory bookkeeping of one CTA (placed before the rings and the staged activations).
-struct DirSlot {             // what a warp knows of one of its rows
-    uint32_t rec_lo, rec_hi; // address of the row record
-    uint32_t meta;           // C | cmin << 16 | nx << 24
-    uint32_t row;            // row | weight index << 28
-    uint32_t xmask[2];
-    uint32_t pad[2];
-};
+// Shared-memory bookkeeping of one CTA (placed after xs and xlin).
 struct StreamShared {
-    SStage stage[kStageSlots];                        // descriptor of stage s sits in slot s % kStageSlots while it is needed
-    DirSlot wdir[kConsumerWarps][kDirSlots];          // per warp: its next rows of the stage its piece iterator is in
-    uint32_t tag_base[4];                             // tagged programs: (rowseq[n0 + n] & 0xFF) << 8 for the panel's rows
-    int abort_flag;                                   // any thread: a bounded wait ran out
-    int pad[3];
+    SStage stage[2];                   // descriptors of the current and the next stage
+    int4 desc[kSlots];                 // x: ring offset, y: weight index, z: tile index, w: bytes
+    unsigned long long full[kSlots];   // mbarriers: tile landed
+    unsigned long long empty[kSlots];  // mbarriers: tile consumed
+    int abort_flag;                    // any warp: a bounded wait ran out
+    int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
+    unsigned int tag_base;             // tagged programs: (launch counter & 0xFF) << 8
+    unsigned int next_q;               // next tile (sequence number) no consumer warp has taken yet
 };
-constexpr int kCtrlBytes = (int)((sizeof(StreamShared) + 127) & ~127);
 
 struct WaitCtx {
     volatile int* abort_flag;
@@ -356,6 +331,8 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, const 
     return true;
 }
 
+// acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`;
+// w is the low (HI = 0) or high (HI = 1) bf16 of `wpair`.
 // c + w * x for bf16 w and x with an fp32 sum (the product of two bf16 values is exact in fp32,
 // so this equals an fp32 fused multiply-add of the widened values): w = half WH of wpair,
 // x = half XH of xword (0: low, 1: high)
@@ -383,10 +360,16 @@ __device__ __forceinline__ void fma_at(float (&acc)[NT], uint32_t wpair, uint32_
     uint32_t x[W];
     if (W == 1) {
         x[0] = lds_u32_off<OFF>(addr);
-    } else {
+    } else if (W == 2) {
         const uint2 t = lds_u32x2_off<OFF>(addr);
         x[0] = t.x;
         x[W - 1] = t.y;
+    } else {
+        const uint4 t = lds_u32x4_off<OFF>(addr);
+        x[0] = t.x;
+        x[1 % W] = t.y;
+        x[2 % W] = t.z;
+        x[3 % W] = t.w;
     }
     if (NT == 1) {
         acc[0] = fma_bf16_sel<HI, 1>(wpair, x[0], acc[0]);
@@ -399,645 +382,686 @@ __device__ __forceinline__ void fma_at(float (&acc)[NT], uint32_t wpair, uint32_
     }
 }
 
-// One chunk: eight (code, value) entries against the activations at `xb` (the lane's cursor, a
-// shared-memory address; a window row is 128 * W bytes).  Returns the cursor after the chunk.
-// Two accumulator sets keep two FMA chains in flight.
+// One chunk: eight (gap, value) entries against the activations at `xb` (the lane's cursor).
+// Returns the cursor after the chunk.  Two accumulator sets keep two FMA chains in flight.
 template <int NT>
 __device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uint32_t xb, float (&a0)[NT], float (&a1)[NT])
 {
-    constexpr int W = xs_words(NT);
-    static_assert(W == 1 || W == 2, "a code prefix (at most 120) times W must fit a byte");
     const uint32_t E = code & 0x0F0F0F0Fu;
     const uint32_t O = (code >> 4) & 0x0F0F0F0Fu;
-    uint32_t PE = (E + O) * 0x01010100u + E;
-    uint32_t PO = PE + O;
-    if (W == 2) { PE <<= 1; PO <<= 1; }   // bytes stay below 256: the dot product then scales by 128 * 2
+    const uint32_t PE = (E + O) * 0x01010100u + E;
+    const uint32_t PO = PE + O;
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #define SD2_PAIR(k)                                                              \
     {                                                                            \
         const uint32_t ae = byte_times_128_plus<k>(PE, xb);                      \
         const uint32_t ao = byte_times_128_plus<k>(PO, xb);                      \
-        fma_at<NT, 0, 0>(a0, w[k], ae);                                          \
-        fma_at<NT, 0, 1>(a1, w[k], ao);                                          \
+        fma_at<NT, (2 * (k)) * 128, 0>(a0, w[k], ae);                            \
+        fma_at<NT, (2 * (k) + 1) * 128, 1>(a1, w[k], ao);                        \
     }
     SD2_PAIR(0)
     SD2_PAIR(1)
     SD2_PAIR(2)
     SD2_PAIR(3)
 #undef SD2_PAIR
-    return byte_times_128_plus<3>(PO, xb);
+    return byte_times_128_plus<3>(PO, xb + 1024u);
 }
 
-// ---- staging the activations of one stage ---------------------------------------------------
-//
-// xs[c][l][W words]: window row c of lane l holds the activation of column l * B - V + c (zero
-// outside the matrix), for every panel row.  Thread (warp w, lane l) fetches groups w, w + 16,
-// ... of CG columns of strip l and writes each column into the window of every lane that can see
-// it (lanes l - Dn .. l + Dn): the 32 threads of a warp then write 32 different banks.  Global
-// memory is read in pieces of 16 bytes (tagged words) or 8 bytes (bf16), strip by strip.
-//
-// kind 0: x is plain bf16; kind 1: x is tagged words, polled until they carry tags[n]; kind 2:
-// the activation is bf16(silu(g) * u) of plain bf16 g and u (CTA 0 also publishes it to t_out).
-// Pointers already point at the launch's first activation row.  CG = 4 needs K, B and V to be
-// multiples of 4 (B and V always are) and aligned pointers; CG = 1 serves everything else.
-template <int NT, int CG>
-__device__ __forceinline__ void stage_x(const SStage& st, int N, int kind, const void* xp, const uint16_t* gp, const uint16_t* up,
-                                        uint16_t* t_out, uint32_t xs, int warp, int lane, const uint32_t* tags, const WaitCtx& wc)
+// Stage the activations of one stage: xs[plane][window row c][group][NT] (fp32) with
+// value = X[n][strip * B - V + c] where strip = plane * groups + group % S (for S <= groups the
+// strips repeat across the groups), zero outside the matrix, in the slack rows and for n >= N.
+// Row by row through `xlin` (bf16, linear) so that global memory is read with 128-bit loads.
+// x_src, g, u, t_out already point at the launch's first activation row.
+// One 128-bit load of four tagged words, repeated until all four carry `tag` (their producers,
+// on other SMs, have stored them) or the wait budget runs out.  Value and tag share a 32-bit
+// word, so a word that shows the tag also shows its value: no fence is needed.
+__device__ __forceinline__ uint4 poll_tagged(const uint32_t* p, uint32_t tag, const WaitCtx& w)
+{
+    uint4 v;
+    long long t0 = 0;
+    uint32_t it = 0;
+    while (true) {
+        asm volatile("ld.relaxed.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+        if (((v.x ^ tag) & 0xFFFFu) == 0 && ((v.y ^ tag) & 0xFFFFu) == 0 && ((v.z ^ tag) & 0xFFFFu) == 0 && ((v.w ^ tag) & 0xFFFFu) == 0) break;
+        if (it == 0) t0 = clock64();
+        if ((++it & 7u) == 0u) {
+            if (*w.abort_flag) break;
+            if (clock64() - t0 > w.budget) { *w.abort_flag = 1; break; }
+        }
+    }
+    return v;
+}
+__device__ __forceinline__ uint32_t poll_tagged1(const uint32_t* p, uint32_t tag, const WaitCtx& w)
+{
+    uint32_t v;
+    long long t0 = 0;
+    uint32_t it = 0;
+    while (true) {
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (((v ^ tag) & 0xFFFFu) == 0) break;
+        if (it == 0) t0 = clock64();
+        if ((++it & 7u) == 0u) {
+            if (*w.abort_flag) break;
+            if (clock64() - t0 > w.budget) { *w.abort_flag = 1; break; }
+        }
+    }
+    return v;
+}
+
+// Linear phase of the staging for tagged inputs: xlin[k] = bf16 of word k of row n (or of
+// silu(g) * u in glue mode), waiting for each word's tag.
+__device__ __forceinline__ void stage_linear_tagged(int K, const uint32_t* x, const uint32_t* g, const uint32_t* u,
+                                                    uint16_t* t_out, bool pub, uint16_t* xlin, uint32_t tag, const WaitCtx& w, int ctid)
+{
+    const bool glue = x == nullptr;
+    const bool vec = (K % 4 == 0) && ((((uintptr_t)x | (uintptr_t)g | (uintptr_t)u) & 15) == 0) && ((((uintptr_t)t_out) & 7) == 0);
+    if (vec) {
+        for (int i = ctid; i < (K >> 2); i += kConsumerThreads) {
+            uint32_t lo, hi;
+            if (!glue) {
+                const uint4 v = poll_tagged(x + 4 * i, tag, w);
+                lo = __byte_perm(v.x, v.y, 0x7632);
+                hi = __byte_perm(v.z, v.w, 0x7632);
+            } else {
+                const uint4 gv = poll_tagged(g + 4 * i, tag, w);
+                const uint4 uv = poll_tagged(u + 4 * i, tag, w);
+                lo = silu_mul_pair(__byte_perm(gv.x, gv.y, 0x7632), __byte_perm(uv.x, uv.y, 0x7632));
+                hi = silu_mul_pair(__byte_perm(gv.z, gv.w, 0x7632), __byte_perm(uv.z, uv.w, 0x7632));
+                if (pub) ((uint2*)t_out)[i] = make_uint2(lo, hi);
+            }
+            ((uint2*)xlin)[i] = make_uint2(lo, hi);
+        }
+    } else {
+        for (int i = ctid; i < K; i += kConsumerThreads) {
+            uint16_t v;
+            if (!glue) {
+                v = (uint16_t)(poll_tagged1(x + i, tag, w) >> 16);
+            } else {
+                v = silu_mul_bits((uint16_t)(poll_tagged1(g + i, tag, w) >> 16), (uint16_t)(poll_tagged1(u + i, tag, w) >> 16));
+                if (pub) t_out[i] = v;
+            }
+            xlin[i] = v;
+        }
+    }
+}
+
+// Tagged glue, first half: t = bf16(silu(g) * u) is computed once per launch instead of once
+// per CTA.  CTA c takes the c-th slice of every row, waits for exactly the g and u words it
+// needs, and publishes its slice of t as tagged words (and as plain bf16 if asked); every CTA
+// then stages the whole of t like any tagged activation.
+__device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g, const uint32_t* u, uint32_t* tt,
+                                                uint16_t* t_out, uint32_t tag, const WaitCtx& w, int ctid)
+{
+    const int G = gridDim.x;
+    const int slice = ((K + G - 1) / G + 3) & ~3;
+    const int k0 = (int)blockIdx.x * slice;
+    const bool vec = (K % 4 == 0) && ((((uintptr_t)g | (uintptr_t)u | (uintptr_t)tt) & 15) == 0);
+    for (int i = ctid; i < N * slice; i += kConsumerThreads) {
+        const int n = i / slice, k = k0 + (i - n * slice);
+        if (k >= K) continue;
+        const size_t at = (size_t)n * K + k;
+        if (vec) {
+            if (k & 3) continue;   // one thread per group of four
+            const uint4 gv = poll_tagged(g + at, tag, w);
+            const uint4 uv = poll_tagged(u + at, tag, w);
+            const uint32_t lo = silu_mul_pair(__byte_perm(gv.x, gv.y, 0x7632), __byte_perm(uv.x, uv.y, 0x7632));
+            const uint32_t hi = silu_mul_pair(__byte_perm(gv.z, gv.w, 0x7632), __byte_perm(uv.z, uv.w, 0x7632));
+            *(uint4*)(tt + at) = make_uint4((lo << 16) | tag, (lo & 0xFFFF0000u) | tag, (hi << 16) | tag, (hi & 0xFFFF0000u) | tag);
+            if (t_out) {
+                t_out[at] = (uint16_t)lo; t_out[at + 1] = (uint16_t)(lo >> 16);
+                t_out[at + 2] = (uint16_t)hi; t_out[at + 3] = (uint16_t)(hi >> 16);
+            }
+        } else {
+            const uint16_t v = silu_mul_bits((uint16_t)(poll_tagged1(g + at, tag, w) >> 16), (uint16_t)(poll_tagged1(u + at, tag, w) >> 16));
+            tt[at] = ((uint32_t)v << 16) | tag;
+            if (t_out) t_out[at] = v;
+        }
+    }
+}
+
+// `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged).
+// Panels of four and eight rows go two rows at a time: both rows are fetched into their own linear
+// buffer (xlin holds two, `xlin_row` elements apart), then one scatter writes the packed words.
+// (Panels of two keep one buffer and take a pass per row: the second buffer would come out of the
+// weight ring, which costs them more than the extra pass.)
+template <int NT>
+__device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
+                                        const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int xlin_row, int ctid,
+                                        uint32_t tag, const WaitCtx& wc)
 {
     constexpr int W = xs_words(NT);
-    constexpr uint32_t RS = 128u * W;             // bytes per window row
-    constexpr int ITC = CG == 4 ? (4 / NT) : 1;   // groups a thread keeps in flight, times NT rows
-    const int K = st.K, B = st.B, V = st.V, wrows = st.wrows;
-    // window rows whose column lies outside [0, 32 B): nothing below writes them.  Four rows at a
-    // time: B and V are multiples of 4, so a group of four rows is inside or outside as a whole.
-    for (int i = warp * 32 + lane; i < 8 * V; i += kConsumerThreads) {   // 32 lanes x V / 4 groups
-        const int l = i & 31, c = (i >> 5) << 2;
-        if (l * B - V + c < 0) {
-            const uint32_t at = xs + (uint32_t)(c * 32 + l) * (4u * W);
+    constexpr int kGroups = 32 / W;
+    constexpr int kRowsPerPass = NT <= 2 ? 1 : 2;
+    const int K = st.K, S = st.S, B = st.B;
+    const bool glue = x_src == nullptr;
+    const int planes = S > kGroups ? S / kGroups : 1;
+    const int rows = B + 2 * st.V + kGap4Slack;     // a lane's window and the slack
+    const int rows4 = (rows + 3) & ~3;              // the scatter works on four rows at a time
+    const int tail_pad = S * B - K + st.V + 48;
+    const bool vec = (K % 8 == 0) && ((((uintptr_t)x_src | (uintptr_t)g | (uintptr_t)u | (uintptr_t)t_out) & 15) == 0);
+    const bool pub = glue && t_out && blockIdx.x == 0;
+    for (int n0 = 0; n0 < NT; n0 += kRowsPerPass) {
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int w = 0; w < W; ++w) sts_u32(at + r * RS + 4u * w, 0u);
-        }
-        const int ch = wrows - 4 - c;
-        if (l * B - V + ch >= 32 * B) {
-            const uint32_t at = xs + (uint32_t)(ch * 32 + l) * (4u * W);
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-#pragma unroll
-                for (int w = 0; w < W; ++w) sts_u32(at + r * RS + 4u * w, 0u);
-        }
-    }
-    const int ngrp = B / CG;
-    const int Dn = (V + B - 1) / B;   // strips to either side whose windows see a column
-    const uint32_t* xt = (const uint32_t*)xp;
-    const uint16_t* xb = (const uint16_t*)xp;
-    const bool pub = kind == 2 && t_out != nullptr && blockIdx.x == 0;
-    for (int g0 = warp; g0 < ngrp; g0 += kConsumerWarps * ITC) {
-        uint32_t wv[ITC][NT][CG];   // the group's activations, bf16 in the high half of each word
-        bool pend[ITC][NT];
-#pragma unroll
-        for (int ii = 0; ii < ITC; ++ii) {
-            const int gi = g0 + kConsumerWarps * ii;
-            const int k0 = lane * B + CG * gi;
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                const bool valid = gi < ngrp && k0 < K && n < N;
-                pend[ii][n] = false;
-#pragma unroll
-                for (int j = 0; j < CG; ++j) wv[ii][n][j] = 0u;
-                if (!valid) continue;
-                const size_t at = (size_t)n * K + k0;
-                if (kind == 1) {
-                    if (CG == 4) {
-                        const uint4 v = ld_relaxed_v4(xt + at);
-                        wv[ii][n][0] = v.x; wv[ii][n][1 % CG] = v.y; wv[ii][n][2 % CG] = v.z; wv[ii][n][3 % CG] = v.w;
+        for (int r = 0; r < kRowsPerPass; ++r) {
+            const int n = n0 + r;
+            if (n >= N) continue;   // the scatter writes zeros for this row
+            // the linear row sits V elements into its buffer, with zeros before it and behind it, so
+            // that the scatter can read any window without bounds checks
+            uint16_t* xb = xlin + (size_t)r * xlin_row;
+            uint16_t* xl = xb + st.V;
+            for (int i = ctid; i < st.V; i += kConsumerThreads) xb[i] = 0;
+            for (int i = ctid; i < tail_pad; i += kConsumerThreads) xl[K + i] = 0;
+            if (tag != 0u) {
+                stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
+                                    g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
+                                    t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag, wc, ctid);
+            } else if (vec) {
+                for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
+                    uint4 v;
+                    if (!glue) {
+                        v = __ldcg((const uint4*)(x_src + (size_t)n * K) + i);
                     } else {
-                        wv[ii][n][0] = ld_relaxed_u32(xt + at);
+                        const uint4 gv = __ldcg((const uint4*)(g + (size_t)n * K) + i);
+                        const uint4 uv = __ldcg((const uint4*)(u + (size_t)n * K) + i);
+                        const uint32_t gg[4] = {gv.x, gv.y, gv.z, gv.w}, uu[4] = {uv.x, uv.y, uv.z, uv.w};
+                        uint32_t w[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) w[q] = silu_mul_pair(gg[q], uu[q]);
+                        v = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (pub) ((uint4*)(t_out + (size_t)n * K))[i] = v;
                     }
-                    pend[ii][n] = true;
-                } else if (kind == 0) {
-                    if (CG == 4) {
-                        const uint2 v = __ldcg((const uint2*)(xb + at));
-                        wv[ii][n][0] = v.x << 16; wv[ii][n][1 % CG] = v.x & 0xFFFF0000u;
-                        wv[ii][n][2 % CG] = v.y << 16; wv[ii][n][3 % CG] = v.y & 0xFFFF0000u;
+                    ((uint4*)xl)[i] = v;
+                }
+            } else {
+                for (int i = ctid; i < K; i += kConsumerThreads) {
+                    uint16_t v;
+                    if (!glue) {
+                        v = __ldcg(x_src + (size_t)n * K + i);
                     } else {
-                        wv[ii][n][0] = (uint32_t)__ldcg(xb + at) << 16;
+                        v = silu_mul_bits(__ldcg(g + (size_t)n * K + i), __ldcg(u + (size_t)n * K + i));
+                        if (pub) t_out[(size_t)n * K + i] = v;
                     }
-                } else {
-                    if (CG == 4) {
-                        const uint2 gv = __ldcg((const uint2*)(gp + at));
-                        const uint2 uv = __ldcg((const uint2*)(up + at));
-                        const uint32_t lo = silu_mul_pair(gv.x, uv.x), hi = silu_mul_pair(gv.y, uv.y);
-                        if (pub) *(uint2*)(t_out + at) = make_uint2(lo, hi);
-                        wv[ii][n][0] = lo << 16; wv[ii][n][1 % CG] = lo & 0xFFFF0000u;
-                        wv[ii][n][2 % CG] = hi << 16; wv[ii][n][3 % CG] = hi & 0xFFFF0000u;
-                    } else {
-                        const uint16_t t = silu_mul_bits(__ldcg(gp + at), __ldcg(up + at));
-                        if (pub) t_out[at] = t;
-                        wv[ii][n][0] = (uint32_t)t << 16;
-                    }
+                    xl[i] = v;
                 }
             }
-        }
-        if (kind == 1) {
-            // poll: a word that shows its row's tag also shows its value
-            long long t0 = 0;
-            uint32_t spins = 0;
-            while (true) {
-                bool all = true;
-#pragma unroll
-                for (int ii = 0; ii < ITC; ++ii) {
-#pragma unroll
-                    for (int n = 0; n < NT; ++n) {
-                        if (!pend[ii][n]) continue;
-                        uint32_t diff = 0;
-#pragma unroll
-                        for (int j = 0; j < CG; ++j) diff |= (wv[ii][n][j] ^ tags[n]) & 0xFFFFu;
-                        if (diff == 0) pend[ii][n] = false;
-                        else all = false;
-                    }
-                }
-                if (all) break;
-                if (spins == 0) t0 = clock64();
-                if ((++spins & 7u) == 0u) {
-                    if (*wc.abort_flag) break;
-                    if (clock64() - t0 > wc.budget) { *wc.abort_flag = 1; break; }
-                }
-                __nanosleep(40);
-#pragma unroll
-                for (int ii = 0; ii < ITC; ++ii) {
-                    const int gi = g0 + kConsumerWarps * ii;
-                    const int k0 = lane * B + CG * gi;
-#pragma unroll
-                    for (int n = 0; n < NT; ++n) {
-                        if (!pend[ii][n]) continue;
-                        const size_t at = (size_t)n * K + k0;
-                        if (CG == 4) {
-                            const uint4 v = ld_relaxed_v4(xt + at);
-                            wv[ii][n][0] = v.x; wv[ii][n][1 % CG] = v.y; wv[ii][n][2 % CG] = v.z; wv[ii][n][3 % CG] = v.w;
-                        } else {
-                            wv[ii][n][0] = ld_relaxed_u32(xt + at);
-                        }
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int ii = 0; ii < ITC; ++ii) {
-            const int gi = g0 + kConsumerWarps * ii;
-            if (gi >= ngrp) continue;
-            uint32_t word[CG][W];
-#pragma unroll
-            for (int j = 0; j < CG; ++j) {
-                if (NT == 1) {
-                    word[j][0] = wv[ii][0][j] & 0xFFFF0000u;
-                } else {
-#pragma unroll
-                    for (int w = 0; w < W; ++w) word[j][w] = __byte_perm(wv[ii][2 * w][j], wv[ii][2 * w + 1 < NT ? 2 * w + 1 : 2 * w][j], 0x7632);
-                }
-            }
-            const int cs = CG * gi;   // first column of the group inside the strip
-            for (int dl = -Dn; dl <= Dn; ++dl) {
-                const int l2 = lane + dl;
-                const int c = cs + V - dl * B;
-                if (l2 < 0 || l2 >= 32 || c < 0 || c >= wrows) continue;   // CG = 4: the four rows are in or out together
-                const uint32_t at = xs + (uint32_t)((c * 32 + l2) * W) * 4u;
-#pragma unroll
-                for (int j = 0; j < CG; ++j) {
-                    if (W == 1) sts_u32(at + j * RS, word[j][0]);
-                    else sts_u32x2(at + j * RS, word[j][0], word[j][W - 1]);
-                }
-            }
-        }
-    }
-}
-
-// shared-memory address of the staged activations of stage s
-__device__ __forceinline__ uint32_t xs_of_stage(const SArgs& a, uint32_t xs_base, int s)
-{
-    return xs_base + ((s & 1) ? (uint32_t)a.xs_odd : 0u);
-}
-
-// Enters stage s: waits for its inputs and stages them.  false: a wait ran out somewhere in the CTA.
-// Called by all threads (not inlined: it is called from one place, but is large and rarely run).
-template <int NT>
-__device__ __noinline__ bool enter_stage(const SArgs& a, StreamShared* sh, const SStage* gstages, const int s, const uint32_t xs_base)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int G = gridDim.x, N = a.N, n_stages = a.n_stages;
-    WaitCtx wc;
-    wc.abort_flag = &sh->abort_flag;
-    wc.budget = a.wait_cycles;
-    const SStage& st = sh->stage[s & (kStageSlots - 1)];
-    if (s + kStageAhead < n_stages)
-        for (int i = tid; i < kStageWords; i += kConsumerThreads)
-            ((uint32_t*)&sh->stage[(s + kStageAhead) & (kStageSlots - 1)])[i] = ((const uint32_t*)(gstages + s + kStageAhead))[i];
-    if (s > 0 && !a.tagged) {
-        // grid barrier: every CTA has written the previous stage's outputs
-        named_bar_sync(1, kConsumerThreads);
-        if (tid == 0) {
-            __threadfence();
-            atomicAdd(a.gbar, 1u);
-            const unsigned int target = (unsigned int)s * (unsigned int)G;
-            const long long t0 = clock64();
-            uint32_t it = 0;
-            while ((int)(ld_acquire_gpu(a.gbar) - target) < 0) {
-                if ((++it & 15u) == 0u) {
-                    if (sh->abort_flag) break;
-                    if (clock64() - t0 > wc.budget) { sh->abort_flag = 1; break; }
-                }
-            }
-            __threadfence();
         }
         named_bar_sync(1, kConsumerThreads);
-    } else if (s > 0 && a.xs_single) {
-        named_bar_sync(1, kConsumerThreads);   // every warp is done reading the one buffer
+        // scatter: consecutive threads take consecutive groups; each takes four window rows of its
+        // group from two aligned 32-bit reads per activation row (window row c of strip s is element
+        // s * B + c of the linear buffer; B is even and c a multiple of 4, and B / 2 is odd, so the
+        // threads of a warp read 32 different banks)
+        const int per_plane = (rows4 >> 2) * kGroups;
+        const uint32_t* xa32 = (const uint32_t*)xlin;
+        const uint32_t* xb32 = (const uint32_t*)(xlin + xlin_row);
+        const bool have_a = n0 < N, have_b = n0 + 1 < N;
+        for (int p = 0; p < planes; ++p) {
+            float* xp = xs + (size_t)p * rows4 * 32;
+            const int grp = ctid % kGroups;
+            const int strip = S > kGroups ? p * kGroups + grp : grp & (S - 1);   // fixed per thread
+#pragma unroll 2
+            for (int i = ctid; i < per_plane; i += kConsumerThreads) {
+                const int c = (i / kGroups) << 2;
+                const int e = (strip * B + c) >> 1;
+                uint32_t t0 = 0u, t1 = 0u;
+                if (have_a) { t0 = xa32[e]; t1 = xa32[e + 1]; }
+                if (NT == 1) {   // one word per column, the value in its high half
+                    float* dst = xp + (size_t)c * 32 + grp;
+                    dst[0] = bf16_lo(t0);
+                    dst[32] = bf16_hi(t0);
+                    dst[64] = bf16_lo(t1);
+                    dst[96] = bf16_hi(t1);
+                } else if (kRowsPerPass == 1) {   // row n0 is half n0 % 2 of word n0 / 2
+                    uint16_t* dst = (uint16_t*)xp + ((size_t)c * 32 + grp * W) * 2 + n0;
+                    dst[0] = (uint16_t)t0;
+                    dst[64] = (uint16_t)(t0 >> 16);
+                    dst[128] = (uint16_t)t1;
+                    dst[192] = (uint16_t)(t1 >> 16);
+                } else {         // rows n0 and n0 + 1 are the two halves of word n0 / 2
+                    uint32_t u0 = 0u, u1 = 0u;
+                    if (have_b) { u0 = xb32[e]; u1 = xb32[e + 1]; }
+                    uint32_t* dst = (uint32_t*)xp + (size_t)c * 32 + grp * W + (n0 >> 1);
+                    dst[0] = __byte_perm(t0, u0, 0x5410);
+                    dst[32] = __byte_perm(t0, u0, 0x7632);
+                    dst[64] = __byte_perm(t1, u1, 0x5410);
+                    dst[96] = __byte_perm(t1, u1, 0x7632);
+                }
+            }
+        }
+        named_bar_sync(1, kConsumerThreads);
     }
-    const uint32_t xs = xs_of_stage(a, xs_base, s);
-    const int K = st.K;
-    const bool first_in = s == 0 && a.x_in != nullptr;
-    const uint16_t* x_src = first_in ? a.x_in : st.x;
-    const size_t xoff = (size_t)a.n0 * K;
-    const bool tin = a.tagged && st.tagged_in && !first_in;
-    uint32_t tags[NT];
-#pragma unroll
-    for (int n = 0; n < NT; ++n) tags[n] = sh->tag_base[n] | (uint32_t)s;
-    const int kind = tin ? 1 : (x_src ? 0 : 2);
-    const void* xp = tin ? (const void*)((const uint32_t*)x_src + xoff) : (const void*)(x_src ? x_src + xoff : nullptr);
-    const uint16_t* gp = kind == 2 ? st.g + xoff : nullptr;
-    const uint16_t* up = kind == 2 ? st.u + xoff : nullptr;
-    uint16_t* tp = (kind == 2 && st.t_out) ? st.t_out + xoff : nullptr;
-    const uintptr_t al = (uintptr_t)xp | (uintptr_t)gp | (uintptr_t)up | (uintptr_t)tp;
-    const bool vec = (K % 4 == 0) && ((al & (kind == 1 ? 15u : 7u)) == 0);
-    if (vec) stage_x<NT, 4>(st, N, kind, xp, gp, up, tp, xs, warp, lane, tags, wc);
-    else stage_x<NT, 1>(st, N, kind, xp, gp, up, tp, xs, warp, lane, tags, wc);
-    named_bar_sync(1, kConsumerThreads);
-    return sh->abort_flag == 0;
 }
-
-// One warp's walk through its rows of all stages.
-//
-// The *piece iterator* (it_*, r_*) runs ahead: it names the warp's pieces in order and the lanes
-// start the copy of each into the next free ring slot, with a 16-byte descriptor in front of
-// the data.  The warp then takes the slots in the same order: wait for the copy, read the
-// descriptor, enter the stage if the piece is the first of one, walk the piece's steps, finish
-// the row if it is the row's last.  Pieces without data (a row without chunks; the marker of a
-// stage in which the warp has no row) go through the ring like the others, so that everything
-// happens in one order.
-template <int NT>
-struct WarpWalk {
-    static constexpr int W = xs_words(NT);
-    static constexpr uint32_t RS = 128u * W;
-
-    const SArgs& a;
-    StreamShared* sh;
-    const SStage* gstages;
-    uint32_t xs_base, ring;   // shared-memory addresses: activations, this warp's ring
-    int lane, warp, cta, G, N, n_stages, nslot;
-    uint32_t lt;
-    uint64_t policy;
-    WaitCtx wc;
-
-    // ---- piece iterator
-    int it_stage, it_t, it_nt, it_more;
-    bool it_new;        // the next piece is the first one of it_stage
-    bool it_done;
-    uint32_t r_lo, r_hi, r_meta, r_row, r_xm0, r_xm1;   // the row whose pieces are being named
-    uint32_t r_j, r_n;                                  // next step of it, its steps
-    // directory entry of this lane's slot of stage it_stage + 1, asked for when it_stage was entered
-    uint4 pd;
-    uint32_t pd_row;
-    int pd_stage;       // -1: none
-
-    // ---- ring
-    uint32_t issued, taken;   // pieces named / worked through
-    int islot, tslot;         // their ring slots
-
-    // ---- arithmetic
-    float a0[NT], a1[NT], rg[NT];
-    uint32_t xb;    // the lane's cursor: a shared-memory address
-    bool dead;      // a bounded wait ran out somewhere in the CTA: all its threads stop after the same barrier
-
-    __device__ __forceinline__ WarpWalk(const SArgs& a_, StreamShared* sh_, const SStage* gs, uint32_t xs_base_, uint32_t ring_base)
-        : a(a_), sh(sh_), gstages(gs), xs_base(xs_base_)
-    {
-        lane = threadIdx.x & 31;
-        warp = threadIdx.x >> 5;
-        cta = blockIdx.x;
-        G = gridDim.x;
-        N = a.N;
-        n_stages = a.n_stages;
-        nslot = a.nslot;
-        ring = ring_base + (uint32_t)(warp * nslot) * (uint32_t)kSlotBytes;
-        lt = (1u << lane) - 1u;
-        policy = l2_evict_first();
-        wc.abort_flag = &sh->abort_flag;
-        wc.budget = a.wait_cycles;
-        it_stage = it_t = it_nt = 0;
-        it_more = -1;
-        it_new = true;
-        it_done = false;
-        r_lo = r_hi = r_meta = r_row = r_xm0 = r_xm1 = r_j = r_n = 0u;
-        pd = make_uint4(0u, 0u, 0u, 0u);
-        pd_row = 0u;
-        pd_stage = -1;
-        issued = taken = 0u;
-        islot = tslot = 0;
-#pragma unroll
-        for (int n = 0; n < NT; ++n) a0[n] = a1[n] = rg[n] = 0.f;
-        xb = 0u;
-        dead = false;
-    }
-
-    // Row slots of this warp in stage s from slot index ibase on: how many of the next kDirSlots
-    // exist (nt) and, if there are more after them, where they start (more, else -1).
-    __device__ __forceinline__ void slot_count(int s, int ibase, int& nt, int& more) const
-    {
-        const SStage& st = sh->stage[s & (kStageSlots - 1)];
-        const int sh_u = st.upr - 1;   // 0 or 1
-        const int units = st.units;
-        const int n_c = units > cta ? (units - cta + G - 1) / G : 0;
-        const int n_w = n_c > warp ? (n_c - warp + kConsumerWarps - 1) / kConsumerWarps : 0;
-        const int left = (n_w - ibase) << sh_u;   // row slots left
-        nt = left < 0 ? 0 : left > kDirSlots ? kDirSlots : left;
-        more = left > kDirSlots ? ibase + (kDirSlots >> sh_u) : -1;
-    }
-
-    // Asks for the directory entries of this warp's row slots ibase .. of stage s (lane t: slot t).
-    __device__ __forceinline__ void dir_ask(int s, int ibase)
-    {
-        const SStage& st = sh->stage[s & (kStageSlots - 1)];
-        const int sh_u = st.upr - 1;
-        int nt, more;
-        slot_count(s, ibase, nt, more);
-        pd = make_uint4(0u, 0u, 0u, 0u);
-        pd_row = 0u;
-        pd_stage = s;
-        if (lane < nt) {
-            const int i = ibase + (lane >> sh_u);
-            const int v = cta + G * (warp + kConsumerWarps * i);
-            int mi = 0;
-#pragma unroll
-            for (int m = 1; m < kMaxFused; ++m)
-                if (m < st.count && v >= st.mat[m].unit0) mi = m;
-            const SMat& md = st.mat[mi];
-            const uint32_t r = ((uint32_t)(v - md.unit0) << sh_u) + (uint32_t)(lane & sh_u);
-            pd = __ldg(md.rowdir + r);
-            pd_row = r | ((uint32_t)mi << 28);
-        }
-    }
-    // ... and puts them where the iterator reads them (waits for them if they are still on their way).
-    __device__ __forceinline__ void dir_put()
-    {
-        const SStage& st = sh->stage[pd_stage & (kStageSlots - 1)];
-        __syncwarp();   // every lane is done with what the slots held before
-        if (lane < kDirSlots) {
-            const unsigned long long rec = (unsigned long long)st.mat[pd_row >> 28].stream + (unsigned long long)pd.x * 16ull;
-            DirSlot d;
-            d.rec_lo = (uint32_t)rec;
-            d.rec_hi = (uint32_t)(rec >> 32);
-            d.meta = pd.y;
-            d.row = pd_row;
-            d.xmask[0] = pd.z;
-            d.xmask[1] = pd.w;
-            d.pad[0] = d.pad[1] = 0u;
-            const uint32_t at = smem_u32(&sh->wdir[warp][lane]);
-            sts_v4(at, make_uint4(d.rec_lo, d.rec_hi, d.meta, d.row));
-            sts_v4(at + 16u, make_uint4(d.xmask[0], d.xmask[1], 0u, 0u));
-        }
-        pd_stage = -1;
-        __syncwarp();
-    }
-
-    __device__ __forceinline__ void begin()
-    {
-        dir_ask(0, 0);
-        dir_put();
-        slot_count(0, 0, it_nt, it_more);
-        if (n_stages > 1) dir_ask(1, 0);
-    }
-
-    // Names the next piece and starts its copy into ring slot `islot`.  false: no piece is left.
-    __device__ __forceinline__ bool issue_piece()
-    {
-        uint32_t ctx, rowinfo = 0u, xm0 = 0u, xm1 = 0u, bytes = 0u;
-        const unsigned char* src = nullptr;
-        while (true) {
-            if (r_j < r_n) {
-                const uint32_t cmin = (r_meta >> 16) & 0xFFu;
-                const uint32_t left = r_n - r_j;
-                const uint32_t ns = left < (uint32_t)kPieceSteps ? left : (uint32_t)kPieceSteps;
-                const uint32_t first = r_j == 0u ? 1u : 0u;
-                const uint32_t o0 = first ? 0u : gap4_step_offset(r_j, cmin, r_xm0, r_xm1);
-                const uint32_t o1 = gap4_step_offset(r_j + ns, cmin, r_xm0, r_xm1);
-                const uint32_t nfull = r_j >= cmin ? 0u : (cmin - r_j < ns ? cmin - r_j : ns);
-                const uint32_t e0 = r_j > cmin ? r_j - cmin : 0u;   // index of the piece's first ragged step
-                r_j += ns;
-                const uint32_t last = r_j == r_n ? 1u : 0u;
-                ctx = ns | (first << 4) | (last << 5) | (1u << 6) | ((it_new ? 1u : 0u) << 7) | ((uint32_t)it_stage << 8) | (nfull << 24) | (e0 << 28);
-                rowinfo = r_row;
-                xm0 = r_xm0;
-                xm1 = r_xm1;
-                src = (const unsigned char*)(((unsigned long long)r_hi << 32) | r_lo) + o0;
-                bytes = o1 - o0;
-                break;
-            }
-            if (it_t < it_nt) {
-                const uint32_t at = smem_u32(&sh->wdir[warp][it_t]);
-                const uint4 d0 = lds_v4(at), d1 = lds_v4(at + 16u);
-                ++it_t;
-                r_lo = d0.x; r_hi = d0.y; r_meta = d0.z; r_row = d0.w; r_xm0 = d1.x; r_xm1 = d1.y;
-                if ((r_meta & 0xFFFFu) == 0u) {   // a row without chunks: its output is +0
-                    ctx = (1u << 4) | (1u << 5) | (1u << 6) | ((it_new ? 1u : 0u) << 7) | ((uint32_t)it_stage << 8);
-                    rowinfo = r_row;
-                    break;
-                }
-                r_n = ((r_meta >> 16) & 0xFFu) + (r_meta >> 24);
-                r_j = 0u;
-                continue;
-            }
-            if (it_more >= 0) {   // more row slots in this stage than are looked up at a time: the next ones
-                const int ibase = it_more;
-                // (the entries asked for on behalf of the next stage are dropped and asked for again below)
-                dir_ask(it_stage, ibase);
-                dir_put();
-                slot_count(it_stage, ibase, it_nt, it_more);
-                it_t = 0;
-                if (it_more < 0 && it_stage + 1 < n_stages) dir_ask(it_stage + 1, 0);
-                continue;
-            }
-            if (it_new) {   // no row of this stage is this warp's: the stage still has to be entered
-                ctx = (1u << 7) | ((uint32_t)it_stage << 8);
-                break;
-            }
-            if (it_stage + 1 >= n_stages) { it_done = true; return false; }
-            ++it_stage;
-            dir_put();   // the entries of this stage were asked for when the one before it was entered
-            slot_count(it_stage, 0, it_nt, it_more);
-            it_t = 0;
-            it_new = true;
-            if (it_more < 0 && it_stage + 1 < n_stages) dir_ask(it_stage + 1, 0);
-        }
-        it_new = false;
-        // descriptor, then the copy: one commit group per piece (an empty one for a piece without data)
-        const uint32_t slot = ring + (uint32_t)islot * (uint32_t)kSlotBytes;
-        if (lane == 0) sts_v4(slot, make_uint4(ctx, rowinfo, xm0, xm1));
-        if (a.hinted) {
-            for (uint32_t o = 16u * (uint32_t)lane; o < bytes; o += 512u) cp_async16(slot + 16u + o, src + o, policy);
-        } else {
-            for (uint32_t o = 16u * (uint32_t)lane; o < bytes; o += 512u) cp_async16(slot + 16u + o, src + o);
-        }
-        cp_async_commit();
-        ++issued;
-        islot = islot + 1 == nslot ? 0 : islot + 1;
-        return true;
-    }
-
-    // the current row is complete: reduce over the lanes and store
-    __device__ __forceinline__ void finish_row(const int s, const uint32_t rowinfo)
-    {
-        const SStage& st = sh->stage[s & (kStageSlots - 1)];
-        float r[NT];
-#pragma unroll
-        for (int n = 0; n < NT; ++n) r[n] = warp_sum(a0[n] + a1[n]);
-        const uint32_t mi = rowinfo >> 28, row = rowinfo & 0x0FFFFFFFu;
-        if (st.paired) {
-            // rows 2i and 2i+1 are gate row i and up row i: the gate result waits in rg for the up
-            // result, and t = bf16(silu(bf16 g) * bf16 u) is formed right here
-            if (!(row & 1u)) {
-#pragma unroll
-                for (int n = 0; n < NT; ++n) rg[n] = r[n];
-            } else if (lane == 0) {
-                const size_t I = (size_t)st.mat[0].M >> 1;
-                uint16_t* gp = (uint16_t*)st.g;
-                uint16_t* up = (uint16_t*)st.u;
-#pragma unroll
-                for (int n = 0; n < NT; ++n) {
-                    if (n < N) {
-                        const size_t at = (size_t)(a.n0 + n) * I + (row >> 1);
-                        const uint16_t gb = f32_to_bf16_rne(rg[n]), ub = f32_to_bf16_rne(r[n]);
-                        const uint16_t tv = silu_mul_bits(gb, ub);
-                        if (st.tt) st_relaxed_u32(st.tt + at, ((uint32_t)tv << 16) | sh->tag_base[n] | (uint32_t)(s + 1));
-                        if (gp) gp[at] = gb;
-                        if (up) up[at] = ub;
-                        if (st.t_out) st.t_out[at] = tv;
-                    }
-                }
-            }
-        } else if (lane == 0) {
-            const SMat& md = st.mat[mi];
-            void* yp = (s == n_stages - 1 && a.y_out && mi == 0u) ? a.y_out : md.y;
-            const size_t M = (size_t)md.M;
-            uint32_t* yt = a.tagged ? md.yt : nullptr;
-#pragma unroll
-            for (int n = 0; n < NT; ++n) {
-                if (n < N) {
-                    const size_t at = (size_t)(a.n0 + n) * M + row;
-                    if (md.y_f32 && yp) {
-                        ((float*)yp)[at] = r[n];
-                        if (yt) st_relaxed_u32(yt + at, ((uint32_t)f32_to_bf16_rne(r[n]) << 16) | sh->tag_base[n] | (uint32_t)(s + 1));
-                    } else {
-                        const uint32_t bits = f32_to_bf16_rne(r[n]);
-                        if (yt) st_relaxed_u32(yt + at, (bits << 16) | sh->tag_base[n] | (uint32_t)(s + 1));
-                        if (yp) ((uint16_t*)yp)[at] = (uint16_t)bits;
-                    }
-                }
-            }
-        }
-    }
-
-    // Works through the piece in ring slot `tslot`.  false: a wait ran out somewhere in the CTA.
-    __device__ __forceinline__ bool take_piece()
-    {
-        const uint32_t slot = ring + (uint32_t)tslot * (uint32_t)kSlotBytes;
-        cp_async_wait(issued - taken - 1u);   // this piece's group and all older ones are done
-        __syncwarp();                         // ... in every lane: the piece is complete
-        const uint4 d = lds_v4(slot);
-        const uint32_t ctx = d.x;
-        const int s = (int)((ctx >> 8) & 0xFFFFu);
-        if (ctx & (1u << 7)) {
-            if (!enter_stage<NT>(a, sh, gstages, s, xs_base)) return false;
-        }
-        if (ctx & (1u << 6)) {
-            uint32_t at = slot + 16u;
-            if (ctx & (1u << 4)) {
-                const SStage& st = sh->stage[s & (kStageSlots - 1)];
-                const uint32_t start = (ctx & 15u) ? lds_u8(at + (uint32_t)lane) : 0u;
-                xb = xs_of_stage(a, xs_base, s) + (uint32_t)lane * (4u * W) + RS * (4u * start + (uint32_t)st.mat[d.y >> 28].voff);
-#pragma unroll
-                for (int n = 0; n < NT; ++n) a0[n] = a1[n] = 0.f;
-                at += kGap4RecordHeader;
-            }
-            const uint32_t ns = ctx & 15u, nfull = (ctx >> 24) & 15u;
-#pragma unroll
-            for (int i = 0; i < kPieceSteps; ++i) {
-                if ((uint32_t)i < nfull) {
-                    const uint32_t code = lds_u32(at + 4u * (uint32_t)lane);
-                    const uint4 v = lds_v4(at + 128u + 16u * (uint32_t)lane);
-                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
-                    at += kGap4FullStepBytes;
-                }
-            }
-            if (nfull < ns) {   // ragged steps: only the lanes of the step's mask have a chunk
-                uint32_t e = ctx >> 28;
-                for (uint32_t i = nfull; i < ns; ++i, ++e) {
-                    const uint32_t m = e == 0u ? d.z : d.w;
-                    const uint32_t p = (uint32_t)__popc(m), idx = (uint32_t)__popc(m & lt);
-                    if ((m >> lane) & 1u) {
-                        const uint32_t code = lds_u32(at + 4u * idx);
-                        const uint4 v = lds_v4(at + ((p * 4u + 15u) & ~15u) + 16u * idx);
-                        xb = chunk_fma<NT>(code, v, xb, a0, a1);
-                    }
-                    at += gap4_step_bytes(p);
-                }
-            }
-            if (ctx & (1u << 5)) finish_row(s, d.y);
-        }
-        __syncwarp();   // every lane is done reading the slot before lane 0 starts a copy into it
-        ++taken;
-        tslot = tslot + 1 == nslot ? 0 : tslot + 1;
-        return true;
-    }
-
-    __device__ __forceinline__ void run()
-    {
-        begin();
-        while (true) {
-            while (!it_done && issued - taken < (uint32_t)nslot) {
-                if (!issue_piece()) break;
-            }
-            if (taken == issued) break;
-            if (!take_piece()) { dead = true; break; }
-        }
-        cp_async_wait(0u);   // (after a wait that ran out: copies under way land before the shared memory is given up)
-    }
-};
 
 template <int NT>
 __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_constant__ SArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    StreamShared* sh = (StreamShared*)smem;
-    const uint32_t ring_base = smem_u32(smem + kCtrlBytes);
-    const uint32_t xs_base = ring_base + (uint32_t)(kConsumerWarps * a.nslot * kSlotBytes);
+    float* xs = (float*)smem;
+    uint16_t* xlin = (uint16_t*)(smem + a.xs_bytes);
+    StreamShared* sh = (StreamShared*)(smem + a.xs_bytes + a.xlin_bytes);
+    unsigned char* ring = smem + a.xs_bytes + a.xlin_bytes + ((sizeof(StreamShared) + 127) & ~127);
     const int tid = threadIdx.x;
-    const SStage* gstages = a.ext ? a.ext : a.inl;
-    const int n_stages = a.n_stages;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int cta = blockIdx.x;
+    const int G = gridDim.x;
+    const uint32_t full0 = smem_u32(&sh->full[0]);
+    const uint32_t empty0 = smem_u32(&sh->empty[0]);
+    const uint32_t ring0 = smem_u32(ring);
 
-    for (int s = 0; s < kStageAhead && s < n_stages; ++s)
-        for (int i = tid; i < kStageWords; i += kStreamThreads) ((uint32_t*)&sh->stage[s])[i] = ((const uint32_t*)(gstages + s))[i];
-    if (tid == 0) sh->abort_flag = 0;
-    if (tid < 4) sh->tag_base[tid] = (a.tagged && tid < a.N) ? ((*(volatile unsigned int*)(a.rowseq + a.n0 + tid)) & 0xFFu) << 8 : 0u;
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, 1);
+        }
+        sh->abort_flag = 0;
+        sh->stage_dead = 0;
+        sh->next_q = (unsigned int)kConsumerWarps;   // warp w starts on tile w
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     __syncthreads();
 
-    // All threads meet at named barrier 1, once per stage, after staging, and once more here.  The
-    // decision to stop after a wait that ran out is taken by all of them together, right after one
-    // of these barriers.
-    WarpWalk<NT> w(a, sh, gstages, xs_base, ring_base);
-    w.run();
-    named_bar_sync(1, kConsumerThreads);
-    if (sh->abort_flag) {   // a bounded wait ran out somewhere in this CTA
-        if (tid == 0 && a.err) atomicExch(a.err, 1);
+    WaitCtx wc;
+    wc.abort_flag = &sh->abort_flag;
+    wc.budget = a.wait_cycles;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------------------ producer warp
+        // Walks this CTA's tiles of all stages in order, one batch of up to 32 tiles (one per
+        // lane) at a time.  Everything it needs is fetched ahead: the descriptor fields of
+        // stage s + 2 and the tile offsets of stage s + 1 are loaded while the copies of stage
+        // s are issued, so its own global-memory latencies stay off the ring's critical path.
+        // Room in the ring is found for a whole run of tiles at once (a warp prefix sum of
+        // their sizes against the free stretch), and every lane that got a place issues its
+        // own copy in the same instruction: one thread can start only about three bulk copies
+        // per microsecond, whatever their size.
+        struct PStage {          // what the producer needs of a stage (the same in every lane)
+            int count, n_cta;
+            int T[kMaxFused];
+            const uint32_t* toff[kMaxFused];
+            const unsigned char* strm[kMaxFused];
+        };
+        struct PBatch {          // one tile per lane
+            uint32_t bytes;
+            unsigned long long src;
+            int mi, ti;
+        };
+        auto load_stage = [&](int s) {
+            PStage p;
+            const SStage* st = a.ext ? a.ext + s : &a.inl[s];
+            p.count = st->count;
+            p.n_cta = st->tiles_div + (cta < st->tiles_rem ? 1 : 0);
+#pragma unroll
+            for (int m = 0; m < kMaxFused; ++m) {
+                p.T[m] = st->mat[m].T;
+                p.toff[m] = st->mat[m].tile_off;
+                p.strm[m] = st->mat[m].stream;
+            }
+            return p;
+        };
+        auto load_batch = [&](const PStage& p, int k0) {
+            PBatch b;
+            b.bytes = 0; b.src = 0; b.mi = 0; b.ti = 0;
+            const int k = k0 + lane;
+            if (k < p.n_cta) {
+                int v = cta + k * G;
+                int mi = 0;
+#pragma unroll
+                for (int m = 0; m + 1 < kMaxFused; ++m)
+                    if (mi == m && m + 1 < p.count && v >= p.T[m]) { v -= p.T[m]; mi = m + 1; }
+                const uint32_t* toff = p.toff[0];
+                const unsigned char* strm = p.strm[0];
+#pragma unroll
+                for (int m = 1; m < kMaxFused; ++m)
+                    if (mi == m) { toff = p.toff[m]; strm = p.strm[m]; }
+                const uint32_t o0 = __ldg(toff + v);
+                const uint32_t o1 = __ldg(toff + v + 1);
+                b.bytes = (o1 - o0) * 16u;
+                b.src = (unsigned long long)(strm + (size_t)o0 * 16);
+                b.mi = mi;
+                b.ti = v;
+            }
+            return b;
+        };
+
+        const uint64_t weight_policy = l2_evict_first();
+        const bool hinted = a.n_stages > 1;
+        uint32_t q = 0, oldest = 0;         // tile sequence numbers of this CTA
+        uint32_t head = 0, tail = 0;        // ring bytes: [tail, head) is in use (mod wrap)
+        const uint32_t ring_bytes = (uint32_t)a.ring_bytes;
+        bool ok = true;
+        PStage ps_cur = load_stage(0);
+        PStage ps_next = a.n_stages > 1 ? load_stage(1) : ps_cur;
+        PBatch pb_cur = load_batch(ps_cur, 0);
+        for (int s = 0; s < a.n_stages && ok; ++s) {
+            // fetch ahead: first batch of stage s + 1, fields of stage s + 2
+            PBatch pb_next = pb_cur;
+            PStage ps_next2 = ps_next;
+            if (s + 1 < a.n_stages) pb_next = load_batch(ps_next, 0);
+            if (s + 2 < a.n_stages) ps_next2 = load_stage(s + 2);
+            const int n_cta = ps_cur.n_cta;
+            for (int k0 = 0; k0 < n_cta && ok; k0 += 32) {
+                if (k0 > 0) pb_cur = load_batch(ps_cur, k0);   // stages of more than 32 tiles per CTA: not fetched ahead
+                const uint32_t bytes = pb_cur.bytes;
+                const int cnt = min(32, n_cta - k0);
+                int i0 = 0;
+                while (i0 < cnt && ok) {
+                    const uint32_t outstanding = q - oldest;
+                    if (outstanding == 0) head = tail = 0;
+                    // free stretch that starts at head: up to the ring's end, or up to just before tail
+                    const uint32_t limit = head >= tail ? ring_bytes : tail - 1u;
+                    const bool cand = lane >= i0 && lane < cnt;
+                    uint32_t incl = cand ? bytes : 0u;
+#pragma unroll
+                    for (int dd = 1; dd < 32; dd <<= 1) {
+                        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, dd);
+                        if (lane >= dd) incl += up;
+                    }
+                    const uint32_t fit_mask = __ballot_sync(0xFFFFFFFFu, cand && head + incl <= limit);
+                    int nfit = __popc(fit_mask);                       // a run of lanes starting at i0
+                    const int slots_free = kSlots - (int)outstanding;
+                    if (nfit > slots_free) nfit = slots_free;
+                    if (nfit > 0) {
+                        if (cand && lane < i0 + nfit) {
+                            const uint32_t my_head = head + incl - bytes;
+                            const uint32_t my_q = q + (uint32_t)(lane - i0);
+                            const uint32_t my_slot = my_q % kSlots;
+                            SD2_TILE_STAMP(my_q, 0);
+                            sh->desc[my_slot] = make_int4((int)my_head, pb_cur.mi, pb_cur.ti, (int)bytes);
+                            mbar_expect_tx(full0 + 8 * my_slot, bytes);
+                            if (hinted) bulk_g2s(ring0 + my_head, (const void*)pb_cur.src, bytes, full0 + 8 * my_slot, weight_policy);
+                            else bulk_g2s(ring0 + my_head, (const void*)pb_cur.src, bytes, full0 + 8 * my_slot);
+                        }
+                        __syncwarp();
+                        head += __shfl_sync(0xFFFFFFFFu, incl, i0 + nfit - 1);
+                        q += (uint32_t)nfit;
+                        i0 += nfit;
+                        continue;
+                    }
+                    const uint32_t b_next = __shfl_sync(0xFFFFFFFFu, bytes, i0);
+                    if (slots_free > 0 && head >= tail && b_next < tail) {   // nothing fits at the end: start over at the front
+                        head = 0;
+                        continue;
+                    }
+                    // no room: wait until the oldest tile in the ring has been consumed, and take
+                    // along every further tile that is already done
+                    if (lane == 0) SD2_TILE_STAMP(oldest, 4);
+                    if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
+                    if (lane == 0) SD2_TILE_STAMP(oldest, 5);
+                    ++oldest;
+                    while (oldest != q) {   // each lane looks at one of the next 32 tiles; the leading run of done ones goes
+                        const uint32_t t = oldest + (uint32_t)lane;
+                        const bool done = (int)(q - t) > 0 && mbar_test_wait(empty0 + 8 * (t % kSlots), (t / kSlots) & 1u);
+                        const uint32_t run = __ffs(~__ballot_sync(0xFFFFFFFFu, done)) - 1;   // 32 if all are done
+                        oldest += run > 32u ? 32u : run;
+                        if (run < 32u) break;
+                    }
+                    tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
+                }
+            }
+            if (lane == 0) SD2_STAMP(6);
+            ps_cur = ps_next;
+            ps_next = ps_next2;
+            pb_cur = pb_next;
+        }
+        if (!ok) {
+            // give the copies already issued time to land before this CTA's memory is released
+            for (uint32_t t = oldest; t != q; ++t) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(full0 + 8 * (t % kSlots), (t / kSlots) & 1u))
+                    if (clock64() - t0 > wc.budget) break;
+            }
+            if (lane == 0 && a.err) atomicExch(a.err, 1);
+        }
         return;
     }
-    // leave the barrier words as they were found: the last CTA out clears them and counts the
-    // launch's activation rows as produced once more
-    if (tid == 0 && (n_stages > 1 || a.tagged)) {
-        __threadfence();
+
+    // ---------------------------------------------------------------------- consumer warps
+    // Consumer threads meet at named barrier 1.  A warp that gave up on a wait keeps meeting
+    // the others there; the decision to stop is taken by all of them together, right after
+    // a barrier, from a word that only thread 0 writes.
+    // The descriptor of stage s sits in sh->stage[s & 1]: warp 1 fetches the next stage's while
+    // the current one is computed; the barrier at the end of the stage makes it visible.
+    constexpr int kGroups = 32 / xs_words(NT);
+    constexpr int kStageWords = (int)(sizeof(SStage) / 4);
+    const int ctid = tid;   // consumer threads are 0 .. kConsumerThreads - 1
+    const int N = a.N;
+    const int xlin_row = NT <= 2 ? 0 : a.xlin_bytes >> 2;   // elements between the two linear buffers of a pass
+    // With free_tiles, tiles go to whichever consumer warp is free next: a warp holds one sequence
+    // number and draws the next from a shared counter when it is done.  Numbers run on across
+    // stages, so a number drawn past the end of a stage is simply the warp's first tile of the next
+    // one.  That evens out the warps' loads where stages have more tiles than warps; where they have
+    // fewer, the fixed deal (tile k to warp k % 16) keeps the busy warps spread over the SM's four
+    // schedulers, and measures faster.
+    uint32_t qbase = 0;
+    uint32_t q_mine = (uint32_t)warp;
+    bool failed = false;
+    if (warp == 1) {
+        const uint32_t* src = (const uint32_t*)(a.ext ? a.ext : &a.inl[0]);
+        for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[0])[i] = src[i];
+    }
+    if (ctid == 0) sh->tag_base = a.tagged ? ((*(volatile unsigned int*)a.seq) & 0xFFu) << 8 : 0u;
+    int s = 0;
+    for (; s < a.n_stages; ++s) {
+        if (ctid == 0) {
+            SD2_STAMP(0);
+            if (s > 0 && !a.tagged) {
+                // grid barrier: every CTA has written the previous stage's outputs
+                const unsigned int target = (unsigned int)s * (unsigned int)G;
+                const long long t0 = clock64();
+                uint32_t it = 0;
+                while ((int)(ld_acquire_gpu(a.gbar) - target) < 0) {
+                    if ((++it & 15u) == 0u) {
+                        if (sh->abort_flag) break;
+                        if (clock64() - t0 > wc.budget) { sh->abort_flag = 1; break; }
+                    }
+                }
+                __threadfence();
+            }
+            sh->stage_dead = sh->abort_flag;
+            SD2_STAMP(1);
+        }
+        named_bar_sync(1, kConsumerThreads);
+        if (sh->stage_dead) break;
+        const SStage& st = sh->stage[s & 1];
+
+        const int K = st.K;
+        const uint16_t* x_src = (s == 0 && a.x_in) ? a.x_in : st.x;
+        const size_t xoff = (size_t)a.n0 * K;
+        // tagged inputs are 32-bit words: twice the stride of bf16; stage s reads what stage s - 1 tagged
+        const bool tin = a.tagged && st.tagged_in && !(s == 0 && a.x_in);
+        const size_t xw = tin ? 2 * xoff : xoff;
+        const uint32_t tag_in = tin ? (sh->tag_base | (uint32_t)s) : 0u;
+        const uint32_t tag_out = sh->tag_base | (uint32_t)(s + 1);
+        if (tin && !x_src && st.tt) {
+            // glue: this CTA's share of t first, then all of t like any tagged activation
+            publish_t_slice(K, N, (const uint32_t*)st.g + xoff, (const uint32_t*)st.u + xoff, st.tt + xoff,
+                            st.t_out ? st.t_out + xoff : nullptr, tag_in, wc, ctid);
+            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+        } else if (st.paired) {   // g, u, t_out are this stage's outputs
+            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+        } else {
+            stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
+                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+        }
+        if (ctid == 0) SD2_STAMP(2);
+        if (warp == 1 && s + 1 < a.n_stages) {
+            const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);
+            for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[(s + 1) & 1])[i] = src[i];
+        }
+
+        const int S = st.S;
+        const int n_cta = st.tiles_div + (cta < st.tiles_rem ? 1 : 0);
+        const uint32_t hdr_bytes = (uint32_t)st.hdr_bytes;
+        const int strip = lane & (S - 1);
+        const int plane = S > kGroups ? strip / kGroups : 0;
+        const uint32_t xs_lane = smem_u32(xs) + (uint32_t)plane * (uint32_t)(((st.B + 2 * st.V + kGap4Slack + 3) & ~3) * 128) +
+                                 (uint32_t)(lane % kGroups) * (4u * xs_words(NT));
+        const uint32_t lt = (1u << lane) - 1u;
+        const bool last_stage = s == a.n_stages - 1;
+
+#ifdef SD2_TRACE
+        long long trace_wait = 0;   // cycles this warp waited for tiles to land, stored once per stage
+#endif
+        if (!a.free_tiles) q_mine = qbase + (uint32_t)warp;
+        while ((int)(q_mine - (qbase + (uint32_t)n_cta)) < 0 && !failed) {
+            const uint32_t q = q_mine;
+            const uint32_t slot = q % kSlots;
+#ifdef SD2_TRACE
+            const long long tw0 = clock64();
+            if (lane == 0) SD2_TILE_STAMP(q, 1);
+#endif
+            if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
+#ifdef SD2_TRACE
+            trace_wait += clock64() - tw0;
+#endif
+            if (ctid == 0 && q == qbase) SD2_STAMP(3);
+            if (lane == 0) SD2_TILE_STAMP(q, 2);
+            const int4 d = sh->desc[slot];
+            const uint32_t tb = ring0 + (uint32_t)d.x;
+            const uint32_t cnt = lds_u16(tb + 2u * lane);
+            const uint4 meta = lds_v4(tb + 64u);                           // n_chunks, min | max << 16, lane mask
+            const uint32_t cb = tb + hdr_bytes;                           // code words
+            const uint32_t vb = cb + ((meta.x * 4u + 15u) & ~15u);        // values
+            const uint32_t jmin = meta.y & 0xFFFFu, jmax = meta.y >> 16;
+            const uint32_t bal0 = meta.z;
+            const uint32_t n0 = __popc(bal0);
+
+            float a0[NT], a1[NT];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) a0[n] = a1[n] = 0.f;
+            uint32_t xb = xs_lane + 128u * lds_u16(tb + 80u + 2u * lane);   // the cursor starts inside the window
+
+            // steps every populated lane takes: addresses advance by a constant
+            if (cnt > 0) {
+                const uint32_t rank0 = __popc(bal0 & lt);
+                uint32_t ca = cb + rank0 * 4u, va = vb + rank0 * 16u;
+                uint32_t code = lds_u32(ca);
+                uint4 v = lds_v4(va);
+                for (uint32_t jj = 1; jj < jmin; ++jj) {
+                    ca += n0 * 4u;
+                    va += n0 * 16u;
+                    const uint32_t code_n = lds_u32(ca);
+                    const uint4 v_n = lds_v4(va);
+                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                    code = code_n;
+                    v = v_n;
+                }
+                xb = chunk_fma<NT>(code, v, xb, a0, a1);
+            }
+            __syncwarp();
+            // ragged tail: the set of lanes that still have a chunk shrinks step by step
+            uint32_t off = n0 * jmin;
+            for (uint32_t j = jmin; j < jmax; ++j) {
+                const bool act = j < cnt;
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, act);
+                if (act) {
+                    const uint32_t idx = off + __popc(bal & lt);
+                    const uint32_t code = lds_u32(cb + idx * 4u);
+                    const uint4 v = lds_v4(vb + idx * 16u);
+                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                }
+                off += __popc(bal);
+            }
+
+            // the S lanes of a row add up; the lane of strip 0 stores
+            float r[NT];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                r[n] = a0[n] + a1[n];
+                for (int dd = 1; dd < S; dd <<= 1) r[n] += __shfl_xor_sync(0xFFFFFFFFu, r[n], dd);
+            }
+            if (st.paired) {
+                // tile rows 2j and 2j+1 are gate row i and up row i: the up result comes over from
+                // S lanes further on, and t = bf16(silu(bf16 g) * bf16 u) is formed right here
+                float ru[NT];
+#pragma unroll
+                for (int n = 0; n < NT; ++n) ru[n] = __shfl_down_sync(0xFFFFFFFFu, r[n], (unsigned)S);
+                const uint32_t trow = (uint32_t)(lane >> st.log2S);
+                if (strip == 0 && !(trow & 1u)) {
+                    const uint32_t row = lds_u32(tb + 144u + 4u * trow);
+                    if (row != 0xFFFFFFFFu) {
+                        const size_t I = (size_t)st.mat[0].M >> 1;
+                        uint16_t* gp = (uint16_t*)st.g;
+                        uint16_t* up = (uint16_t*)st.u;
+#pragma unroll
+                        for (int n = 0; n < NT; ++n) {
+                            if (n < N) {
+                                const size_t at = (size_t)(a.n0 + n) * I + (row >> 1);
+                                const uint16_t gb = f32_to_bf16_rne(r[n]), ub = f32_to_bf16_rne(ru[n]);
+                                const uint16_t tv = silu_mul_bits(gb, ub);
+                                st.tt[at] = ((uint32_t)tv << 16) | tag_out;
+                                if (gp) gp[at] = gb;
+                                if (up) up[at] = ub;
+                                if (st.t_out) st.t_out[at] = tv;
+                            }
+                        }
+                    }
+                }
+            } else if (strip == 0) {
+                const uint32_t row = lds_u32(tb + 144u + 4u * (uint32_t)(lane >> st.log2S));
+                if (row != 0xFFFFFFFFu) {
+                    const SMat& md = st.mat[d.y];
+                    void* yp = (last_stage && a.y_out && d.y == 0) ? a.y_out : md.y;
+                    const size_t M = (size_t)md.M;
+                    const bool f32 = md.y_f32 != 0;
+                    uint32_t* yt = a.tagged ? md.yt : nullptr;
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        if (n < N) {
+                            const size_t at = (size_t)(a.n0 + n) * M + row;
+                            if (yt) {   // value and tag in one word: the next stage polls it
+                                const uint32_t bits = f32_to_bf16_rne(r[n]);
+                                yt[at] = (bits << 16) | tag_out;
+                                if (yp) ((uint16_t*)yp)[at] = (uint16_t)bits;
+                            } else if (f32) {
+                                ((float*)yp)[at] = r[n];
+                            } else {
+                                ((uint16_t*)yp)[at] = f32_to_bf16_rne(r[n]);
+                            }
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) SD2_TILE_STAMP(q, 3);
+            uint32_t q_next = q + (uint32_t)kConsumerWarps;
+            if (lane == 0) {
+                mbar_arrive(empty0 + 8 * slot);
+                if (a.free_tiles) q_next = atomicAdd(&sh->next_q, 1u);
+            }
+            q_mine = __shfl_sync(0xFFFFFFFFu, q_next, 0);
+        }
+        qbase += (uint32_t)n_cta;
+        if (ctid == 0) SD2_STAMP(4);
+#ifdef SD2_TRACE
+        if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] = trace_wait;
+#endif
+        // everything this CTA wrote in the stage is visible before it arrives at the barrier
+        named_bar_sync(1, kConsumerThreads);
+        if (ctid == 0) SD2_STAMP(5);
+        if (s + 1 < a.n_stages && ctid == 0 && !a.tagged) {
+            __threadfence();
+            atomicAdd(a.gbar, 1u);
+        }
+    }
+    if (s < a.n_stages || sh->abort_flag) {   // a bounded wait ran out somewhere in this CTA
+        if (ctid == 0 && a.err) atomicExch(a.err, 1);
+        return;
+    }
+    // leave the barrier words as they were found: the last CTA out clears them
+    if (a.n_stages > 1 && ctid == 0) {
         const unsigned int prev = atomicAdd(a.gbar + 32, 1u);
-        if (prev == (unsigned int)gridDim.x - 1u) {
+        if (prev == (unsigned int)G - 1u) {
             atomicExch(a.gbar, 0u);
             atomicExch(a.gbar + 32, 0u);
-            if (a.tagged)
-                for (int n = 0; n < a.N; ++n) atomicAdd(a.rowseq + a.n0 + n, 1u);
+            if (a.tagged) atomicAdd(a.seq, 1u);   // the next launch tags its words differently
         }
     }
 }
 
-// Diagnostic: one warp waits, with the same kind of bounded wait the stream kernel uses, on an
-// mbarrier that nothing ever arrives at.  The wait must run out, raise the error word and let the
-// kernel end normally (no trap, no hang).
+// Diagnostic: one warp waits, with the same bounded wait the stream kernel uses, on an mbarrier
+// that nothing ever arrives at.  The wait must run out, raise the error word and let the kernel
+// end normally (no trap, no hang).
 __global__ void __launch_bounds__(32, 1) wait_selftest_kernel(int* err, long long budget)
 {
     __shared__ unsigned long long bar;

@@ -62,7 +62,7 @@ def test_zero_and_full_masks(fmt):
     if fmt == sd2.SD2_FORMAT_BITMASK:
         assert info["compressed_bytes"] == 4 * 11 + 4 * 10 * 7      # offsets + mask words, no values
     else:
-        assert info["compressed_bytes"] == 16 * 11                 # the row directory, no records
+        assert info["compressed_bytes"] == _gap4_bytes(zero)       # tile offsets and tile headers, no chunks
     full = np.ones((10, 200), np.uint8)
     dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, full, fmt))
     assert np.array_equal(dense, W) and info["nnz"] == 2000
@@ -85,68 +85,98 @@ def test_bitmask_byte_count_closed_form():
     assert info["compressed_bytes"] == 4 * (M + 1) + 4 * M * ((K + 31) // 32) + 2 * int(mask.sum())
 
 
-def _gap4_directory(blob):
-    """(M, K, B, V, directory rows [off16, C, cmin, nx, xmask0, xmask1], record section bytes), read from
-    the blob by the layout documented with the format."""
-    M, K = struct.unpack_from("<qq", blob, 24)
-    sec_off = struct.unpack_from("<4Q", blob, 64)
-    sec_bytes = struct.unpack_from("<4Q", blob, 96)
-    B, V = struct.unpack_from("<2I", blob, 144)
-    raw = np.frombuffer(blob, np.uint32, 4 * (M + 1), sec_off[0]).reshape(M + 1, 4)
-    rows = np.stack([raw[:, 0], raw[:, 1] & 0xFFFF, (raw[:, 1] >> 16) & 0xFF, raw[:, 1] >> 24, raw[:, 2], raw[:, 3]],
-                    axis=1).astype(np.int64)
-    return M, K, B, V, rows, sec_bytes[1]
+GAP4_OVERLAP = 32
 
 
-def _a16(x):
-    return (x + 15) // 16 * 16
+def _gap4_geometry(M, K, paired=False):
+    """Strip geometry (S strips of B columns, R rows per tile) from the format's definition."""
+    Mt = M // 2 if paired else M            # a paired stack is cut like one of its halves
+    S = 1
+    while S < 32 and Mt * S // 32 < 2048:
+        S *= 2
+    while S > 1 and (K + S - 1) // S < 64:
+        S //= 2
+    def strip_cols(S):                      # the smallest B >= K / S that is twice an odd number
+        b = (K + S - 1) // S
+        while b % 4 != 2:
+            b += 1
+        return b
+    while S < 32 and strip_cols(S) > 496:
+        S *= 2
+    return S, strip_cols(S), 32 // S
 
 
-def _step_bytes(p):
-    return _a16(4 * p) + 16 * p
+def _gap4_deal_row(cols, S, B, V):
+    """Runs of a row's kept columns per lane: equal whole chunks where the lane windows allow."""
+    E = len(cols)
+    full = E // 8
+    base, extra = full // S, full % S
+    e, first = 0, [0]
+    for l in range(S):
+        if l == S - 1:
+            n = E - e
+        else:
+            lo = 0
+            while e + lo < E and cols[e + lo] < (l + 1) * B - V:
+                lo += 1
+            hi = lo
+            while e + hi < E and cols[e + hi] < (l + 1) * B + V:
+                hi += 1
+            want = 8 * (base + (1 if l < extra else 0))
+            n = min(max(want, lo), hi)
+            if n % 8:
+                up, down = (n + 7) // 8 * 8, n // 8 * 8
+                if up <= hi:
+                    n = up
+                elif down >= lo:
+                    n = down
+        e += n
+        first.append(e)
+    return first
 
 
-def test_gap4_byte_count_follows_from_the_chunk_counts():
-    # a row's record: 32 start bytes, then per step the code words of its lanes (padded to 16 bytes) and
-    # their values: 640 bytes for each of the cmin steps that all 32 lanes take, less for the (at most two)
-    # ragged ones; the directory takes 16 bytes per row and one terminator.  A row needs at least
-    # ceil(kept / 8) chunks and, with a whole chunk of padding in every lane and a filler per 15 skipped
-    # columns, not more than the bound below
+def _gap4_run_chunks(cols):
+    """Chunks of one lane's run: kept entries plus one filler per 16 skipped columns, rounded up to 8."""
+    e = 0
+    for i, c in enumerate(cols):
+        e += (0 if i == 0 else (c - cols[i - 1] - 1) // 16) + 1
+    return (e + 7) // 8
+
+
+def _gap4_bytes(mask, paired=False):
+    """Compressed bytes of a mask: tile offsets + per tile (header, code words, values)."""
+    M, K = mask.shape
+    S, B, R = _gap4_geometry(M, K, paired)
+    row_chunks = []
+    for m in range(M):
+        cols = np.nonzero(mask[m])[0].tolist()
+        first = _gap4_deal_row(cols, S, B, GAP4_OVERLAP)
+        row_chunks.append(sum(_gap4_run_chunks(cols[first[l]:first[l + 1]]) for l in range(S)))
+    row_chunks = np.array(row_chunks)
+    if paired:      # pairs (2i, 2i+1) ordered by the chunks of both rows, each pair kept together
+        pair_order = np.argsort(-(row_chunks[0::2] + row_chunks[1::2]), kind="stable")
+        order = np.stack([2 * pair_order, 2 * pair_order + 1], axis=1).reshape(-1)
+    else:
+        order = np.argsort(-row_chunks, kind="stable")
+    T = (M + R - 1) // R
+    hdr = (144 + 4 * R + 15) // 16 * 16
+    total = 4 * (T + 1)
+    for t in range(T):
+        ct = int(row_chunks[order[t * R:(t + 1) * R]].sum())
+        total += hdr + (4 * ct + 15) // 16 * 16 + 16 * ct
+    return total
+
+
+def test_gap4_byte_count_closed_form():
     for M, K in ((29, 700), (70, 2048), (5, 11008), (300, 257)):
         for d in (0.5, 0.1, 0.03, 0.97):
             W, mask = _case(31, M, K, d)
-            blob = sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4)
-            _, info = sd2.sd2_unpack_host(blob, want_dense=False)
-            M_, K_, B, V, rows, rec_bytes = _gap4_directory(blob)
-            assert (M_, K_) == (M, K) and 32 * B >= K and B % 4 == 0 and V >= 32 and V % 4 == 0
-            total = 0
-            for m in range(M):
-                off16, C, cmin, nx, xm0, xm1 = (int(v) for v in rows[m])
-                assert off16 * 16 == total
-                kept = int(mask[m].sum())
-                assert (C == 0) == (kept == 0)
-                assert nx <= 2 and (nx >= 1) == (xm0 != 0) and (nx >= 2) == (xm1 != 0) and (xm1 & ~xm0) == 0
-                p0, p1 = bin(xm0).count("1"), bin(xm1).count("1")
-                assert C == 32 * cmin + p0 + p1
-                if nx < 2:       # (with two ragged steps the short lanes may have been given filler chunks)
-                    assert (kept + 7) // 8 <= C <= (kept + 7) // 8 + 32 + K // 15
-                total += 0 if C == 0 else 32 + 640 * cmin + (_step_bytes(p0) if nx >= 1 else 0) + (_step_bytes(p1) if nx >= 2 else 0)
-            assert rows[M, 0] * 16 == total == rec_bytes
-            assert info["compressed_bytes"] == 16 * (M + 1) + total
+            _, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
+            assert info["compressed_bytes"] == _gap4_bytes(mask)
 
 
-def test_gap4_lanes_of_a_row_get_the_same_number_of_chunks():
-    # what the format is for: at even density the 32 lanes of a row walk in lock step, at most one
-    # ragged step (two where a far gap needs a filler) on top of the steps every lane takes
-    W, mask = _case(33, 256, 2048, 0.5)
-    _, _, _, _, rows, _ = _gap4_directory(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
-    assert (rows[:-1, 3] <= 1).mean() > 0.95
-    kept = mask.sum(axis=1)
-    assert (rows[:-1, 2] >= kept // 256 - 1).all()               # cmin: whole steps of 256 entries
-
-
-def test_gap4_ragged_rows():
-    # rows of very different lengths, empty and full rows, tiny and wide matrices
+def test_gap4_geometries_and_ragged_tiles():
+    # every strip count, tiles with missing rows, rows of very different lengths
     for M, K in ((3, 11008), (100, 64), (2500, 100), (5000, 70), (33, 2048), (9000, 130), (20000, 3)):
         W, mask = _case(41 + M, M, K, 0.5)
         if M >= 33:
@@ -154,7 +184,9 @@ def test_gap4_ragged_rows():
             mask[1::11, :] = 1                   # full rows
         dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
         assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
-    # every run length from 0 to a full row, all entries at the front of the row
+        if M * K < 400000:
+            assert info["compressed_bytes"] == _gap4_bytes(mask)
+    # every segment length from 0 to a full strip
     K = 257
     mask = np.zeros((K + 1, K), np.uint8)
     for m in range(K + 1):
@@ -162,20 +194,58 @@ def test_gap4_ragged_rows():
     W = synth.normal_bf16(43, (K + 1, K), 0.02)
     dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
     assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
-    # columns kept in clusters: lanes cannot share the entries evenly, rows turn ragged, still lossless
-    mask = np.zeros((40, 4096), np.uint8)
-    mask[:, 100:700] = 1
-    mask[::2, 3000:3100] = 1
-    W = synth.normal_bf16(44, (40, 4096), 0.02)
-    dense, info = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
-    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
 
 
-def test_a_blob_with_a_tampered_directory_is_rejected():
-    W, mask = _case(97, 64, 300, 0.5)
-    blob = bytearray(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+def _tile_rows(blob):
+    """Row ids of every tile, read from the records (header layout as documented with the format)."""
+    M, K = struct.unpack_from("<qq", blob, 24)
     sec_off = struct.unpack_from("<4Q", blob, 64)
-    struct.pack_into("<H", blob, sec_off[0] + 16 * 3 + 4, 1)      # row 3 claims a single chunk
+    S, B, T = struct.unpack_from("<3I", blob, 144)
+    R = 32 // S
+    toff = np.frombuffer(blob, np.uint32, T + 1, sec_off[0])
+    return [np.frombuffer(blob, np.uint32, R, sec_off[1] + 16 * int(toff[t]) + 144) for t in range(T)], M
+
+
+def test_paired_blobs_keep_row_pairs_in_one_tile():
+    for M, K, d in ((64, 300, 0.5), (1000, 1024, 0.5), (4098, 130, 0.3), (2, 300, 0.5)):
+        W, mask = _case(91 + M, M, K, d)
+        mask[4::10, :] = 0                                        # some pairs of very different rows
+        blob = sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)
+        dense, info = sd2.sd2_unpack_host(blob)
+        assert info["format"] == sd2.SD2_FORMAT_GAP4              # an ordering of GAP4, not another format
+        assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))
+        assert info["compressed_bytes"] == _gap4_bytes(mask, paired=True)
+        tiles, M_hdr = _tile_rows(blob)
+        assert M_hdr == M
+        seen = []
+        for rows in tiles:
+            for j in range(0, len(rows), 2):
+                a, b = int(rows[j]), int(rows[j + 1])
+                if a == 0xFFFFFFFF:
+                    assert b == 0xFFFFFFFF
+                else:
+                    assert a % 2 == 0 and b == a + 1
+                    seen.append(a)
+        assert sorted(seen) == list(range(0, M, 2))
+
+
+def test_paired_needs_even_rows_and_two_rows_per_tile():
+    W, mask = _case(95, 7, 300, 0.5)
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)    # odd M
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+    W, mask = _case(96, 2048, 4096, 0.05)                         # 32 strips: one row per tile
+    assert _gap4_geometry(2048, 4096, paired=True)[2] == 1
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED)
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+
+
+def test_a_blob_that_claims_pairing_without_it_is_rejected():
+    W, mask = _case(97, 64, 300, 0.5)
+    mask[::3, :] = 0                                              # the plain order splits pairs
+    blob = bytearray(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4))
+    struct.pack_into("<I", blob, 164, 1)                          # header field `pairing`
     with pytest.raises(sd2.Sd2Error) as e:
         sd2.sd2_unpack_host(bytes(blob))
     assert e.value.status == sd2.SD2_ERR_CORRUPT
@@ -191,13 +261,13 @@ def test_gap4_is_unsupported_for_very_wide_matrices():
 
 
 def test_sizes_at_half_density_match_the_format_arithmetic():
-    M, K = 8192, 2048                                            # a gate / up projection: 32 strips of 64 columns
+    M, K = 8192, 2048                                            # a gate / up projection: strips of 257 columns
     W, mask = _case(51, M, K, 0.5)
     nnz = int(mask.sum())
     _, bm = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_BITMASK), want_dense=False)
     _, g4 = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_GAP4), want_dense=False)
     assert abs(bm["compressed_bytes"] / nnz - 2.25) < 0.01       # 2 B value + 2 bits of mask per kept weight
-    assert 2.5 <= g4["compressed_bytes"] / nnz < 2.58            # 2 B value + 4-bit gap + a little padding + row headers
+    assert 2.5 <= g4["compressed_bytes"] / nnz < 2.56            # 2 B value + 4-bit gap + a little padding + headers
     assert g4["compressed_bytes"] < 0.66 * 2 * M * K             # well under the dense bf16 bytes
 
 

@@ -275,7 +275,23 @@ def _read_u16(ptr, count):
     return buf
 
 
-# (hidden, kv, inter): a narrow and a wide hidden size (one and four groups of activations per thread)
+def test_paired_stack_is_the_same_linear():
+    # a stack ordered in row pairs is still W.*mask: same product, rows where they belong
+    M, K, N = 600, 1024, 3
+    W, mask, X = case(77, M, K, 0.5, N)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_PAIRED, sd2.SD2_DTYPE_F32)
+    assert h.format == sd2.SD2_FORMAT_GAP4
+    Y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_spmm(h, dev_bf16(X), Y)
+    sd2.sd2_stream_check()
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(Y.cpu().numpy().astype(np.float64), Yr, S, True)
+    assert np.array_equal(sd2.sd2_decompress(h), oracle.roundtrip_ref(W, mask))
+    sd2.sd2_free(h)
+
+
+# (hidden, kv, inter): the first lets the drafter pair gate and up rows in one stack; the second
+# gives that stack one row per tile, so gate and up stay apart and t is formed by the down stage
 @pytest.mark.parametrize("dims3", [(256, 64, 1024), (2048, 128, 1024)])
 @pytest.mark.parametrize("N", [1, 3, 6])
 def test_drafter_step_teacher_forced(N, dims3):
