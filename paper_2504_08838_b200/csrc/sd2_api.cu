@@ -44,7 +44,6 @@ struct sd2_drafter_s {
     unsigned int* d_gbar;
     uint32_t* d_tags;          // tagged copies of q, hdn, g, u and the block output of every block (or NULL)
     int64_t tags_bytes;
-    int64_t last_n;            // rows of the previous step: a change clears d_tags (stale tags of other rows)
     int K_max, max_tile;       // what decides the shared-memory split
     int free_tiles;            // every stage has enough tiles per CTA for free tile assignment
     int xs_need[4];            // bytes of staged activations at panel widths 1, 2, 4, 8
@@ -60,6 +59,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kBarrierPool = 64;             // grid-barrier word pairs handed out round-robin
 constexpr int kBarrierStrideWords = 64;      // 256 bytes apart
 constexpr int kSmemMax = 227 * 1024;         // dynamic shared memory a CTA may opt in to
+constexpr int kDrafterWordsBytes = 512;      // a drafter's device words: barrier (two lines), then 64 production counts
 
 struct DeviceState {
     bool ready;
@@ -826,7 +826,10 @@ sd2_status sd2_stream_check(void* cuda_stream)
         {
             std::lock_guard<std::mutex> lk(g_mu);
             for (sd2_drafter d : g_live_drafters)
-                if (d->device == dev) { cudaMemset(d->d_gbar, 0, 256); d->last_n = -1; }
+                if (d->device == dev) {   // barrier words, production counts and every tagged word start over
+                    cudaMemset(d->d_gbar, 0, kDrafterWordsBytes);
+                    if (d->d_tags) cudaMemset(d->d_tags, 0, (size_t)d->tags_bytes);
+                }
         }
         cudaGetLastError();
         return SD2_ERR_TIMEOUT;
@@ -1039,7 +1042,6 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
     std::vector<int64_t> tag_off((size_t)L * 6 + 1, 0);
     d->d_tags = nullptr;
     d->tags_bytes = 0;
-    d->last_n = -1;
     if (tagged) {
         int64_t to = 0;
         for (int b = 0; b < L; ++b) {
@@ -1094,7 +1096,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         d->n_stages = n;
         ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
              cudaMemcpy(d->d_stages, stages.data(), sizeof(SStage) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMalloc((void**)&d->d_gbar, 256) == cudaSuccess && cudaMemset(d->d_gbar, 0, 256) == cudaSuccess;
+             cudaMalloc((void**)&d->d_gbar, kDrafterWordsBytes) == cudaSuccess && cudaMemset(d->d_gbar, 0, kDrafterWordsBytes) == cudaSuccess;
     }
     if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
         for (sd2_handle p : d->owned) sd2_free(p);
@@ -1143,13 +1145,11 @@ sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, vo
     a.wait_cycles = wait_budget(dev);
     if (d->d_tags) {
         a.tagged = 1;
-        a.seq = d->d_gbar + 48;   // third cache-line-sized slot of the 256-byte block
-        // Only rows [0, N) are written and polled in a step.  When N changes, rows written long ago
-        // could carry a tag that comes round again (tags are 16 bits): start from clean words.
-        if (d->last_n != N) {
-            if (cudaMemsetAsync(d->d_tags, 0, (size_t)d->tags_bytes, (cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
-            d->last_n = N;
-        }
+        // How often each activation row has been produced is the first half of every tag.  A word left by
+        // an earlier launch (or by launches that covered other rows) can never show the tag this launch
+        // waits for: a row's count moves only when the row is produced, so its previous tag is always one
+        // behind.  Steps of any N, eager or replayed from a CUDA graph, can therefore follow each other.
+        a.rowseq = d->d_gbar + 64;
     }
     // Rows of X are independent through the whole drafter: panels run one after another.  Row n
     // of every buffer starts at n * width, whatever N is.

@@ -95,6 +95,10 @@ constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kStreamThreads = kConsumerThreads + 32;   // + the producer warp
 constexpr int kSlots = 64;                               // tiles in flight per CTA, at most
 constexpr int kMaxStagesInline = 8;
+#ifndef SD2_UNROLL
+#define SD2_UNROLL 4
+#endif
+constexpr int kUnroll = SD2_UNROLL;                      // uniform steps of a tile taken as one run of code
 
 struct SMat {
     const uint32_t* tile_off;      // [T + 1], 16-byte units into `stream`
@@ -146,7 +150,8 @@ struct SArgs {
     int xlin_bytes;                 // shared memory for one linear activation row
     int ring_bytes;
     int tagged;                     // 1: stages hand activations over as tagged words, no grid barrier
-    unsigned int* seq;              // tagged programs: launch counter (device word), bumped by the last CTA out
+    unsigned int* rowseq;           // tagged programs: per activation row, how often it has been produced (device
+                                    // words, bumped by the last CTA out)
     int free_tiles;                 // 1: a consumer warp that is done draws the next tile from a shared counter;
                                     // 0: tile k of a stage goes to warp k % 16 (see the consumer loop)
     long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
@@ -289,6 +294,15 @@ __device__ __forceinline__ void named_bar_sync(int id, int threads)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+__device__ __forceinline__ void st_relaxed_u32(uint32_t* p, uint32_t v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_v4(uint32_t* p, uint4 v)
+{
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
 __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p)
 {
     unsigned int v;
@@ -304,7 +318,7 @@ struct StreamShared {
     unsigned long long empty[kSlots];  // mbarriers: tile consumed
     int abort_flag;                    // any warp: a bounded wait ran out
     int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
-    unsigned int tag_base;             // tagged programs: (launch counter & 0xFF) << 8
+    unsigned int tag_base[8];          // tagged programs: (production count of activation row n0 + n & 0xFF) << 8
     unsigned int next_q;               // next tile (sequence number) no consumer warp has taken yet
 };
 
@@ -490,7 +504,7 @@ __device__ __forceinline__ void stage_linear_tagged(int K, const uint32_t* x, co
 // needs, and publishes its slice of t as tagged words (and as plain bf16 if asked); every CTA
 // then stages the whole of t like any tagged activation.
 __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g, const uint32_t* u, uint32_t* tt,
-                                                uint16_t* t_out, uint32_t tag, const WaitCtx& w, int ctid)
+                                                uint16_t* t_out, uint32_t stage_tag, const unsigned int* tagb, const WaitCtx& w, int ctid)
 {
     const int G = gridDim.x;
     const int slice = ((K + G - 1) / G + 3) & ~3;
@@ -499,6 +513,7 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
     for (int i = ctid; i < N * slice; i += kConsumerThreads) {
         const int n = i / slice, k = k0 + (i - n * slice);
         if (k >= K) continue;
+        const uint32_t tag = stage_tag | tagb[n];
         const size_t at = (size_t)n * K + k;
         if (vec) {
             if (k & 3) continue;   // one thread per group of four
@@ -506,20 +521,21 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
             const uint4 uv = poll_tagged(u + at, tag, w);
             const uint32_t lo = silu_mul_pair(__byte_perm(gv.x, gv.y, 0x7632), __byte_perm(uv.x, uv.y, 0x7632));
             const uint32_t hi = silu_mul_pair(__byte_perm(gv.z, gv.w, 0x7632), __byte_perm(uv.z, uv.w, 0x7632));
-            *(uint4*)(tt + at) = make_uint4((lo << 16) | tag, (lo & 0xFFFF0000u) | tag, (hi << 16) | tag, (hi & 0xFFFF0000u) | tag);
+            st_relaxed_v4(tt + at, make_uint4((lo << 16) | tag, (lo & 0xFFFF0000u) | tag, (hi << 16) | tag, (hi & 0xFFFF0000u) | tag));
             if (t_out) {
                 t_out[at] = (uint16_t)lo; t_out[at + 1] = (uint16_t)(lo >> 16);
                 t_out[at + 2] = (uint16_t)hi; t_out[at + 3] = (uint16_t)(hi >> 16);
             }
         } else {
             const uint16_t v = silu_mul_bits((uint16_t)(poll_tagged1(g + at, tag, w) >> 16), (uint16_t)(poll_tagged1(u + at, tag, w) >> 16));
-            tt[at] = ((uint32_t)v << 16) | tag;
+            st_relaxed_u32(tt + at, ((uint32_t)v << 16) | tag);
             if (t_out) t_out[at] = v;
         }
     }
 }
 
-// `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged).
+// `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged); row n's words carry
+// tag | tagb[n].
 // Panels of four and eight rows go two rows at a time: both rows are fetched into their own linear
 // buffer (xlin holds two, `xlin_row` elements apart), then one scatter writes the packed words.
 // (Panels of two keep one buffer and take a pass per row: the second buffer would come out of the
@@ -527,7 +543,7 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
 template <int NT>
 __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
                                         const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int xlin_row, int ctid,
-                                        uint32_t tag, const WaitCtx& wc)
+                                        uint32_t tag, const unsigned int* tagb, const WaitCtx& wc)
 {
     constexpr int W = xs_words(NT);
     constexpr int kGroups = 32 / W;
@@ -554,7 +570,7 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
             if (tag != 0u) {
                 stage_linear_tagged(K, x_src ? (const uint32_t*)x_src + (size_t)n * K : nullptr,
                                     g ? (const uint32_t*)g + (size_t)n * K : nullptr, u ? (const uint32_t*)u + (size_t)n * K : nullptr,
-                                    t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag, wc, ctid);
+                                    t_out ? t_out + (size_t)n * K : nullptr, pub, xl, tag | tagb[n], wc, ctid);
             } else if (vec) {
                 for (int i = ctid; i < (K >> 3); i += kConsumerThreads) {
                     uint4 v;
@@ -839,7 +855,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const uint32_t* src = (const uint32_t*)(a.ext ? a.ext : &a.inl[0]);
         for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[0])[i] = src[i];
     }
-    if (ctid == 0) sh->tag_base = a.tagged ? ((*(volatile unsigned int*)a.seq) & 0xFFu) << 8 : 0u;
+    if (ctid < 8) sh->tag_base[ctid] = (a.tagged && ctid < a.N) ? ((*(volatile unsigned int*)(a.rowseq + a.n0 + ctid)) & 0xFFu) << 8 : 0u;
     int s = 0;
     for (; s < a.n_stages; ++s) {
         if (ctid == 0) {
@@ -870,18 +886,19 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         // tagged inputs are 32-bit words: twice the stride of bf16; stage s reads what stage s - 1 tagged
         const bool tin = a.tagged && st.tagged_in && !(s == 0 && a.x_in);
         const size_t xw = tin ? 2 * xoff : xoff;
-        const uint32_t tag_in = tin ? (sh->tag_base | (uint32_t)s) : 0u;
-        const uint32_t tag_out = sh->tag_base | (uint32_t)(s + 1);
+        const uint32_t tag_in = tin ? (uint32_t)s : 0u;      // the stage part of a tag; the row part is tag_base[n]
+        const uint32_t tag_out = (uint32_t)(s + 1);
+        const unsigned int* tagb = sh->tag_base;
         if (tin && !x_src && st.tt) {
             // glue: this CTA's share of t first, then all of t like any tagged activation
             publish_t_slice(K, N, (const uint32_t*)st.g + xoff, (const uint32_t*)st.u + xoff, st.tt + xoff,
-                            st.t_out ? st.t_out + xoff : nullptr, tag_in, wc, ctid);
-            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+                            st.t_out ? st.t_out + xoff : nullptr, tag_in, tagb, wc, ctid);
+            stage_x<NT>(st, N, (const uint16_t*)(st.tt + xoff), nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         } else if (st.paired) {   // g, u, t_out are this stage's outputs
-            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+            stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         } else {
             stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
-                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, wc);
+                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         }
         if (ctid == 0) SD2_STAMP(2);
         if (warp == 1 && s + 1 < a.n_stages) {
@@ -935,18 +952,30 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             if (cnt > 0) {
                 const uint32_t rank0 = __popc(bal0 & lt);
                 uint32_t ca = cb + rank0 * 4u, va = vb + rank0 * 16u;
-                uint32_t code = lds_u32(ca);
-                uint4 v = lds_v4(va);
-                for (uint32_t jj = 1; jj < jmin; ++jj) {
-                    ca += n0 * 4u;
-                    va += n0 * 16u;
-                    const uint32_t code_n = lds_u32(ca);
-                    const uint4 v_n = lds_v4(va);
-                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
-                    code = code_n;
-                    v = v_n;
+                const uint32_t dc = n0 * 4u, dv = n0 * 16u;
+                uint32_t jj = 0;
+                // four steps at a time as one straight run of code: their loads go ahead of the
+                // arithmetic, and the decoding of one step overlaps the multiply-adds of another
+                for (; jj + kUnroll <= jmin; jj += kUnroll) {
+                    uint32_t code[kUnroll];
+                    uint4 v[kUnroll];
+#pragma unroll
+                    for (int i = 0; i < kUnroll; ++i) {
+                        code[i] = lds_u32(ca + (uint32_t)i * dc);
+                        v[i] = lds_v4(va + (uint32_t)i * dv);
+                    }
+#pragma unroll
+                    for (int i = 0; i < kUnroll; ++i) xb = chunk_fma<NT>(code[i], v[i], xb, a0, a1);
+                    ca += kUnroll * dc;
+                    va += kUnroll * dv;
                 }
-                xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                for (; jj < jmin; ++jj) {
+                    const uint32_t code = lds_u32(ca);
+                    const uint4 v = lds_v4(va);
+                    xb = chunk_fma<NT>(code, v, xb, a0, a1);
+                    ca += dc;
+                    va += dv;
+                }
             }
             __syncwarp();
             // ragged tail: the set of lanes that still have a chunk shrinks step by step
@@ -989,7 +1018,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                                 const size_t at = (size_t)(a.n0 + n) * I + (row >> 1);
                                 const uint16_t gb = f32_to_bf16_rne(r[n]), ub = f32_to_bf16_rne(ru[n]);
                                 const uint16_t tv = silu_mul_bits(gb, ub);
-                                st.tt[at] = ((uint32_t)tv << 16) | tag_out;
+                                st_relaxed_u32(st.tt + at, ((uint32_t)tv << 16) | tag_out | tagb[n]);
                                 if (gp) gp[at] = gb;
                                 if (up) up[at] = ub;
                                 if (st.t_out) st.t_out[at] = tv;
@@ -1011,7 +1040,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                             const size_t at = (size_t)(a.n0 + n) * M + row;
                             if (yt) {   // value and tag in one word: the next stage polls it
                                 const uint32_t bits = f32_to_bf16_rne(r[n]);
-                                yt[at] = (bits << 16) | tag_out;
+                                st_relaxed_u32(yt + at, (bits << 16) | tag_out | tagb[n]);
                                 if (yp) ((uint16_t*)yp)[at] = (uint16_t)bits;
                             } else if (f32) {
                                 ((float*)yp)[at] = r[n];
@@ -1054,7 +1083,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         if (prev == (unsigned int)G - 1u) {
             atomicExch(a.gbar, 0u);
             atomicExch(a.gbar + 32, 0u);
-            if (a.tagged) atomicAdd(a.seq, 1u);   // the next launch tags its words differently
+            if (a.tagged)   // the launch's activation rows have been produced once more: their next tags differ
+                for (int n = 0; n < a.N; ++n) atomicAdd(a.rowseq + a.n0 + n, 1u);
         }
     }
 }

@@ -345,38 +345,92 @@ def test_drafter_step_teacher_forced(N, dims3):
             sd2.sd2_free(h)
 
 
-def test_drafter_steps_repeat_bit_for_bit_across_tag_wraparound():
-    # the launch counter that tags the hand-off words is 8 bits wide: 600 steps wrap it twice; every
-    # step must give the first step's result, bit for bit (one row's sum order is fixed)
-    shape = synth.DrafterShape("tiny", 256, 64, 1024, 2)
+def _tiny_drafter(L, n_max, dims=(256, 64, 1024)):
+    shape = synth.DrafterShape("tiny", dims[0], dims[1], dims[2], L)
     blocks = []
-    for b in range(2):
+    for b in range(L):
         lin = synth.make_block(2, b, shape, 0.5)
-        blocks.append([sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32 if (b == 1 and i == 6) else sd2.SD2_DTYPE_BF16)
+        blocks.append([sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32 if (b == L - 1 and i == 6) else sd2.SD2_DTYPE_BF16)
                        for i, (W, m) in enumerate(lin)])
-    d = sd2.sd2_drafter_create(blocks, n_max=4)
-    N = 3
-    xd = dev_bf16(synth.make_activations(2, 0, 0, N, shape.hidden))
-    y0 = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
-    sd2.sd2_drafter_step(d, xd, y0)
+    return shape, blocks, sd2.sd2_drafter_create(blocks, n_max=n_max)
+
+
+def _block_chain(blocks, shape, xd):
+    """The same token through one sd2_block_step per block (grid barriers, caller's workspace): an
+    independent hand-off mechanism over the same kernels, so results must agree bit for bit."""
+    N = xd.shape[0]
+    ws = torch.zeros(sd2.sd2_block_workspace_bytes(blocks[0], N) // 2, dtype=torch.bfloat16, device="cuda")
+    cur = xd
+    for b, hs in enumerate(blocks):
+        last = b == len(blocks) - 1
+        out = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32 if last else torch.bfloat16, device="cuda")
+        sd2.sd2_block_step(hs, cur, out, ws)
+        cur = out
     sd2.sd2_stream_check()
-    assert not torch.isnan(y0).any()
-    y = torch.empty_like(y0)
+    return cur
+
+
+def test_drafter_steps_with_changing_inputs_across_tag_wraparound():
+    # the production counts that tag the hand-off words are 8 bits wide: 600 steps wrap them twice.  The
+    # input changes every step, so a word consumed before its producer has rewritten it (a stale tag
+    # taken for a fresh one) would show as a wrong result
+    shape, blocks, d = _tiny_drafter(2, 4)
+    N = 3
+    xs = [dev_bf16(synth.make_activations(2, 0, j, N, shape.hidden)) for j in range(7)]
+    refs = [_block_chain(blocks, shape, x) for x in xs]
+    y = torch.empty((N, shape.hidden), dtype=torch.float32, device="cuda")
     for k in range(600):
-        if k % 97 == 0:
+        if k % 97 == 0 or k == 599:
             y.fill_(float("nan"))
-        sd2.sd2_drafter_step(d, xd, y)
+        sd2.sd2_drafter_step(d, xs[k % 7], y)
         if k % 97 == 0 or k == 599:
             sd2.sd2_stream_check()
-            assert torch.equal(y, y0), "step %d differs" % k
+            assert torch.equal(y, refs[k % 7]), "step %d differs" % k
     # a different number of rows in between, then back
     y1 = torch.full((1, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
-    sd2.sd2_drafter_step(d, xd[:1], y1)
+    sd2.sd2_drafter_step(d, xs[3][:1], y1)
     sd2.sd2_stream_check()
-    assert torch.equal(y1[0], y0[0])
-    sd2.sd2_drafter_step(d, xd, y)
+    assert torch.equal(y1[0], refs[3][0])
+    sd2.sd2_drafter_step(d, xs[4], y)
     sd2.sd2_stream_check()
-    assert torch.equal(y, y0)
+    assert torch.equal(y, refs[4])
+    sd2.sd2_drafter_free(d)
+    for hs in blocks:
+        for h in hs:
+            sd2.sd2_free(h)
+
+
+def test_graph_replays_mixed_with_eager_steps_of_another_row_count():
+    # rows 1 and 2 are produced by an eager step, then a captured one-row step is replayed 256 times
+    # (row 0's production count comes round, rows 1 and 2 keep theirs and their old words), then rows
+    # 0..2 are produced again from other inputs: every stage must wait for the new words of rows 1, 2
+    shape, blocks, d = _tiny_drafter(2, 4)
+    xa = dev_bf16(synth.make_activations(2, 0, 1, 3, shape.hidden))
+    xb = dev_bf16(synth.make_activations(2, 0, 2, 3, shape.hidden))
+    x1 = dev_bf16(synth.make_activations(2, 0, 3, 1, shape.hidden))
+    ref_a, ref_b, ref_1 = (_block_chain(blocks, shape, x) for x in (xa, xb, x1))
+    y3 = torch.full((3, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    y1 = torch.full((1, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            sd2.sd2_drafter_step(d, x1, y1)                  # warm up on the capture stream
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            sd2.sd2_drafter_step(d, x1, y1)
+        sd2.sd2_drafter_step(d, xa, y3)                      # eager, three rows
+        stream.synchronize()
+        assert torch.equal(y3, ref_a)
+        for _ in range(256):
+            graph.replay()
+        stream.synchronize()
+        assert torch.equal(y1, ref_1)
+        y3.fill_(float("nan"))
+        sd2.sd2_drafter_step(d, xb, y3)                      # eager again, other inputs
+        stream.synchronize()
+    sd2.sd2_stream_check()
+    assert torch.equal(y3, ref_b)
     sd2.sd2_drafter_free(d)
     for hs in blocks:
         for h in hs:
