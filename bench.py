@@ -3,13 +3,15 @@
 
 A "step" is one token through every decoder-block linear of the drafter: one call of
 ``sd2_drafter_step``, a single persistent launch that runs the 4 x ``blocks`` dependent stages
-(q|k|v, o, gate|up, down of every block; seven sparse linears per block) separated by grid-wide
-barriers, replayed as a CUDA graph.  Default workload: Llama-3.2-1B-shaped drafter, 16
+(q|k|v, o, gate|up, down of every block; seven sparse linears per block), each stage handing its
+outputs to the next as tagged words, replayed as a CUDA graph.  Default workload: Llama-3.2-1B-shaped drafter, 16
 blocks, 50 % unstructured sparsity, one activation row (the configuration the metric is quoted
 on).  Every block has its own seeded weights, so one step streams about 1.2 GB of compressed
 weights, far more than the 126 MB L2: each launch reads its weights from HBM.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --workload config1      # one 2048 x 2048 linear, 128 rotating copies (cold) and L2-warm
+    python bench.py --workload sweep        # sparsity sweep on single matrices against cuBLAS dense
 
 With ``--gpus N`` > 1 (under torchrun) every rank runs an independent replica of the drafter
 (the path does not shard: replicas only); the value is the job's aggregate time per token.
@@ -49,7 +51,13 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama-3.2-1b", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="llama-3.2-1b", choices=sorted(WORKLOADS) + ["config1", "sweep"])
+    ap.add_argument("--sparsities", default="0.3,0.4,0.5,0.6,0.66,0.7,0.75,0.8,0.9", help="sweep: sparsity grid")
+    ap.add_argument("--sweep-n", default="1,16,64", help="sweep: activation rows")
+    ap.add_argument("--dense-glue", choices=["auto", "eager", "vllm", "compiled"], default="auto",
+                    help="silu(g)*u of the fused dense cuBLAS arm: vllm's silu_and_mul kernel (one launch), one torch.compile'd "
+                         "kernel, or two eager elementwise launches; auto = vllm's if it loads, else eager")
+    ap.add_argument("--quick", action="store_true", help="sweep: first shape only")
     ap.add_argument("--sparsity", type=float, default=0.5)
     ap.add_argument("--mask", default="bernoulli", choices=["bernoulli", "magnitude", "2:4"],
                     help="mask recipe; 2:4 keeps two of every four columns (sparsity is then 0.5)")
@@ -153,8 +161,30 @@ class ClockSampler:
 # the CPU oracle as a timed baseline (the only place bench.py executes oracle/)
 # ------------------------------------------------------------------------------------------
 
-def time_oracle(shape, cfg_id, density, n_rows, blocks_sample, mask_kind="bernoulli"):
-    """Seconds the oracle needs for `blocks_sample` blocks' seven linears (single thread)."""
+def host_cores():
+    """Cores this process may run on (the count the all-cores oracle timing uses)."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def oracle_linear_threads(oracle, W, m, X, threads):
+    """The oracle, as it stands, on `threads` host threads: its rows are independent, so every thread
+    calls it on its own slice of the rows (the C call releases the interpreter lock)."""
+    if threads <= 1:
+        return oracle.masked_linear(W, m, X)
+    from concurrent.futures import ThreadPoolExecutor
+    M = W.shape[0]
+    cuts = [M * i // threads for i in range(threads + 1)]
+    parts = [(cuts[i], cuts[i + 1]) for i in range(threads) if cuts[i + 1] > cuts[i]]
+    with ThreadPoolExecutor(len(parts)) as ex:
+        res = list(ex.map(lambda ab: oracle.masked_linear(W[ab[0]:ab[1]], None if m is None else m[ab[0]:ab[1]], X), parts))
+    return np.concatenate([r[0] for r in res], axis=1), np.concatenate([r[1] for r in res], axis=1)
+
+
+def time_oracle(shape, cfg_id, density, n_rows, blocks_sample, mask_kind="bernoulli", threads=1):
+    """Seconds the oracle needs for `blocks_sample` blocks' seven linears on `threads` host threads."""
     from oracle import oracle
     total = 0.0
     for b in range(blocks_sample):
@@ -162,7 +192,7 @@ def time_oracle(shape, cfg_id, density, n_rows, blocks_sample, mask_kind="bernou
         for i, (W, m) in enumerate(lin):
             X = synth.make_activations(cfg_id, b, i, n_rows, W.shape[1])
             t0 = time.perf_counter()
-            oracle.masked_linear(W, m, X)
+            oracle_linear_threads(oracle, W, m, X, threads)
             total += time.perf_counter() - t0
     return total
 
@@ -183,12 +213,14 @@ def run_reference(args):
     xs = [[synth.make_activations(cfg_id, b, i, args.n, W.shape[1]) for i, (W, _) in enumerate(lin)]
           for b, lin in enumerate(pool)]
 
+    cores = host_cores()
+
     def one_block(b, frac):
         total = 0.0
         for i, (W, m) in enumerate(pool[b]):
             rows = max(1, int(round(frac * W.shape[0])))
             t0 = time.perf_counter()
-            oracle.masked_linear(W[:rows], m[:rows], xs[b][i])
+            oracle_linear_threads(oracle, W[:rows], m[:rows], xs[b][i], cores)
             total += (time.perf_counter() - t0) * W.shape[0] / rows
         return total
 
@@ -199,14 +231,14 @@ def run_reference(args):
         one_block(k % len(pool), frac)
     per_step = [one_block(k % len(pool), frac) * blocks for k in range(args.steps)]
     us = float(np.mean(per_step)) * 1e6 if per_step else float("nan")
-    sample_txt = ("per step: the first %.1f %% of the rows of all 7 linears of one block (N=%d), scaled to all rows "
-                  "and by %d blocks" % (100 * frac, args.n, blocks))
+    sample_txt = ("per step: the first %.1f %% of the rows of all 7 linears of one block (N=%d), rows split over %d threads, "
+                  "scaled to all rows and by %d blocks" % (100 * frac, args.n, cores, blocks))
     line = {
         "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config_dict(args, shape, blocks),
-        "cpu_baseline": {"value": us, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample_txt},
         "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -225,7 +257,8 @@ def measured_peak():
 
 
 def ncu_traffic_ratio():
-    """DRAM bytes per algorithmic byte of the dominant kernel, from the committed ncu summary."""
+    """DRAM bytes per streamed byte of the dominant kernel, as stored in the committed ncu summary (not
+    measured in this run: the JSON line labels it so)."""
     import re
     name = "stream_kernel_nt1_llama1b_2blocks.md"
     try:
@@ -247,6 +280,46 @@ def aggregate_replicas(t_step, world, dist, device):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         t_step = float(t.item())
     return t_step, t_step * 1e3 / world
+
+
+def read_device_u16(ptr, count):
+    """`count` bf16 patterns from a raw device address (the CUDA runtime torch already loaded)."""
+    import ctypes
+    rt = ctypes.CDLL("libcudart.so.12")
+    rt.cudaMemcpy.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int]
+    rt.cudaMemcpy.restype = ctypes.c_int
+    buf = np.empty(count, np.uint16)
+    if rt.cudaMemcpy(buf.ctypes.data, ptr, count * 2, 2) != 0:          # 2 = device to host
+        raise RuntimeError("cudaMemcpy from a drafter buffer failed")
+    return buf
+
+
+def check_block0(sd2, drafter, shape, cfg_id, density, mask_kind, N, x_bits, threads):
+    """Block 0 of the step just run against the oracle: each of its seven linears on the input the
+    device gave it (teacher forcing), t against silu(g) * u.  Returns the largest |y - y_ref| / S over
+    the linears (S = sum |w x| of the row, the oracle's error scale; bf16 outputs carry their own
+    rounding, at most 2^-9 |y| <= 2^-9 S) and the largest bf16 ulp distance of t."""
+    from oracle import oracle
+    oracle.build()
+    lin = synth.make_block(cfg_id, 0, shape, density, mask_kind)
+    dims = [shape.hidden, shape.kv, shape.kv, shape.hidden, shape.inter, shape.inter, shape.inter, shape.hidden]
+    ptrs = sd2.sd2_drafter_buffers(drafter, 0)
+    q, k, v, hdn, g, u, t, out = [read_device_u16(p, N * dm).reshape(N, dm) for p, dm in zip(ptrs, dims)]
+    worst = 0.0
+    for idx, inp, got in ((0, x_bits, q), (1, x_bits, k), (2, x_bits, v), (3, q, hdn), (4, hdn, g), (5, hdn, u), (6, t, out)):
+        Yr, S = oracle_linear_threads(oracle, lin[idx][0], lin[idx][1], inp, threads)
+        y = synth.bf16_bits_to_f32(got).astype(np.float64)
+        err = np.abs(y - Yr) / np.maximum(S, 1e-300)
+        err[S == 0] = np.abs(y[S == 0])
+        worst = max(worst, float(err.max()))
+    t_ref = oracle.silu_mul(g, u)
+    t_bits = np.array([oracle.f64_to_bf16_rne(float(z)) for z in np.asarray(t_ref).ravel()], np.uint16).reshape(t.shape)
+
+    def key(b):
+        b = b.astype(np.int32)
+        return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    return {"block": 0, "linears": 7, "max_abs_err_over_S": worst, "bound_over_S": 2.0 ** -8 + 2e-3,
+            "silu_mul_max_bf16_ulps": int(np.abs(key(t) - key(t_bits)).max()), "against": "oracle, teacher-forced"}
 
 
 def run_ours(args):
@@ -295,8 +368,9 @@ def run_ours(args):
     acts = [x_dev] + [torch.zeros((N, shape.hidden), dtype=torch.bfloat16, device="cuda") for _ in range(blocks)]
     y_host = torch.zeros((N, shape.hidden), dtype=torch.bfloat16).pin_memory()
     harr = [sd2._handle_array(hs) for hs in handles]
-    launches_per_step = (N + 3) // 4          # one persistent launch per panel of at most 4 rows
     drafter = sd2.sd2_drafter_create(handles, n_max=N)
+    facts = sd2.sd2_drafter_query(drafter, N)          # launches per step, panel width, bytes: the library's own figures
+    launches_per_step = facts["launches"]
     y_dev = acts[blocks]
 
     def token():
@@ -335,6 +409,23 @@ def run_ours(args):
         torch.cuda.synchronize()
         clocks = sampler.stop()
 
+        # ---- spread: some replays timed one by one (an event pair each; the value above is the aggregate)
+        n_single = min(args.steps, 200)
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_single)]
+        for a0, a1 in pairs:
+            a0.record(stream)
+            graph.replay()
+            a1.record(stream)
+        stream.synchronize()
+        singles = sorted(a0.elapsed_time(a1) * 1e3 for a0, a1 in pairs)
+        spread = {"replays": n_single, "median_us": singles[n_single // 2], "min_us": singles[0], "max_us": singles[-1]}
+
+        # ---- the timed step against the oracle: block 0, every linear on the input the device gave it
+        parity = None
+        if not args.no_cpu and rank == 0 and N <= 8:
+            x_bits = synth.make_activations(cfg_id, 0, 0, N, shape.hidden)
+            parity = check_block0(sd2, drafter, shape, cfg_id, density, args.mask, N, x_bits, host_cores())
+
         # ---- end to end: pinned host x -> device, the token, device y -> pinned host, every step
         def e2e_step():
             acts[0].copy_(x_host, non_blocking=True)
@@ -361,20 +452,25 @@ def run_ours(args):
         stream.synchronize()
         ms_stream = e0.elapsed_time(e1) / 50
 
-        # ---- cuBLAS dense bf16 on the same masked weights, same chaining, same graph treatment
-        dense_us = None
+        # ---- cuBLAS dense bf16 on the same masked weights, same chaining, same graph treatment.
+        # Two arms: "fused" is what a tuned dense decoder does (q|k|v as one GEMM, gate|up as one GEMM,
+        # silu(g) * u as one elementwise kernel into a preallocated buffer: 5 launches per block);
+        # "unfused" issues the seven GEMMs one by one.  Per-shape single-launch times come with them.
+        dense_res = None
         if not args.no_dense:
             hid, kv, inter = shape.hidden, shape.kv, shape.inter
-            bufs = {"q": torch.zeros((N, hid), dtype=torch.bfloat16, device="cuda"),
-                    "k": torch.zeros((N, kv), dtype=torch.bfloat16, device="cuda"),
-                    "v": torch.zeros((N, kv), dtype=torch.bfloat16, device="cuda"),
-                    "h": torch.zeros((N, hid), dtype=torch.bfloat16, device="cuda"),
-                    "g": torch.zeros((N, inter), dtype=torch.bfloat16, device="cuda"),
-                    "u": torch.zeros((N, inter), dtype=torch.bfloat16, device="cuda"),
-                    "t": torch.zeros((N, inter), dtype=torch.bfloat16, device="cuda")}
-            dacts = [x_dev.clone()] + [torch.zeros((N, hid), dtype=torch.bfloat16, device="cuda") for _ in range(blocks)]
+            bf = dict(dtype=torch.bfloat16, device="cuda")
+            bufs = {"q": torch.zeros((N, hid), **bf), "k": torch.zeros((N, kv), **bf), "v": torch.zeros((N, kv), **bf),
+                    "h": torch.zeros((N, hid), **bf), "g": torch.zeros((N, inter), **bf), "u": torch.zeros((N, inter), **bf),
+                    "t": torch.zeros((N, inter), **bf), "qkv": torch.zeros((N, hid + 2 * kv), **bf),
+                    "gu": torch.zeros((N, 2 * inter), **bf)}
+            dacts = [x_dev.clone()] + [torch.zeros((N, hid), **bf) for _ in range(blocks)]
+            fused_w = []
+            for b in range(blocks):
+                Wq, Wk, Wv, Wo, Wg, Wu, Wd = dense[7 * b:7 * b + 7]
+                fused_w.append((torch.cat([Wq, Wk, Wv], 0).contiguous(), Wo, torch.cat([Wg, Wu], 0).contiguous(), Wd))
 
-            def dense_token():
+            def dense_token_unfused():
                 for b in range(blocks):
                     Wq, Wk, Wv, Wo, Wg, Wu, Wd = dense[7 * b:7 * b + 7]
                     torch.matmul(dacts[b], Wq.t(), out=bufs["q"])
@@ -385,22 +481,94 @@ def run_ours(args):
                     torch.matmul(bufs["h"], Wu.t(), out=bufs["u"])
                     torch.mul(torch.nn.functional.silu(bufs["g"]), bufs["u"], out=bufs["t"])
                     torch.matmul(bufs["t"], Wd.t(), out=dacts[b + 1])
-            for _ in range(3):
-                dense_token()
-            stream.synchronize()
-            dgraph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(dgraph, stream=stream):
-                dense_token()
-            for _ in range(10):
-                dgraph.replay()
-            stream.synchronize()
+
+            glue, glue_txt = None, "as two eager elementwise launches"
+            if args.dense_glue in ("auto", "vllm"):
+                try:
+                    import vllm._custom_ops  # noqa: F401  (registers torch.ops._C)
+                    op = torch.ops._C.silu_and_mul
+                    op(bufs["t"], bufs["gu"])
+                    glue, glue_txt = (lambda gu, t: op(t, gu)), "as one launch of vllm's silu_and_mul"
+                except Exception as exc:
+                    if args.dense_glue == "vllm":
+                        raise
+                    sys.stderr.write("dense arm: vllm's silu_and_mul unavailable (%s); two eager launches instead\n" % type(exc).__name__)
+            elif args.dense_glue == "compiled":
+                fn = torch.compile(lambda gu: torch.nn.functional.silu(gu[:, :inter]) * gu[:, inter:])
+                glue, glue_txt = (lambda gu, t: t.copy_(fn(gu))), "as one torch.compile'd kernel plus a copy"
+
+            def dense_token_fused():
+                for b in range(blocks):
+                    Wqkv, Wo, Wgu, Wd = fused_w[b]
+                    torch.matmul(dacts[b], Wqkv.t(), out=bufs["qkv"])
+                    torch.matmul(bufs["qkv"][:, :hid], Wo.t(), out=bufs["h"])
+                    torch.matmul(bufs["h"], Wgu.t(), out=bufs["gu"])
+                    if glue is not None:
+                        glue(bufs["gu"], bufs["t"])
+                    else:                                  # silu in place on the gate half, then one multiply
+                        torch.nn.functional.silu(bufs["gu"][:, :inter], inplace=True)
+                        torch.mul(bufs["gu"][:, :inter], bufs["gu"][:, inter:], out=bufs["t"])
+                    torch.matmul(bufs["t"], Wd.t(), out=dacts[b + 1])
+
+            def time_graph(fn, steps):
+                for _ in range(3):
+                    fn()
+                stream.synchronize()
+                gr = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gr, stream=stream):
+                    fn()
+                for _ in range(10):
+                    gr.replay()
+                stream.synchronize()
+                e0.record(stream)
+                for _ in range(steps):
+                    gr.replay()
+                e1.record(stream)
+                stream.synchronize()
+                return e0.elapsed_time(e1) / steps * 1e3
+
             dsteps = max(20, args.steps // 4)
-            e0.record(stream)
-            for _ in range(dsteps):
-                dgraph.replay()
-            e1.record(stream)
-            stream.synchronize()
-            dense_us = e0.elapsed_time(e1) / dsteps * 1e3
+            dense_res = {"unfused_us_per_token": time_graph(dense_token_unfused, dsteps),
+                         "fused_us_per_token": time_graph(dense_token_fused, dsteps),
+                         "fused_launches_per_block": 5 if glue is not None else 6, "unfused_launches_per_block": 9,
+                         "note": "cuBLAS bf16 via torch.matmul on W.*mask stored dense, CUDA-graph replays; fused = q|k|v and "
+                                 "gate|up concatenated, silu*mul " + glue_txt}
+
+            # ---- per shape: one launch of ours against one cuBLAS GEMM, each over a ring of copies larger than L2
+            per_shape = []
+            seen = set()
+            for i in range(7):
+                W = dense[i]
+                if tuple(W.shape) in seen:
+                    continue
+                seen.add(tuple(W.shape))
+                M_, K_ = W.shape
+                same = [j for j in range(len(dense)) if tuple(dense[j].shape) == (M_, K_)]
+                xin = torch.zeros((N, K_), **bf).normal_()
+                yo = torch.zeros((N, M_), **bf)
+                hs_same = [handles[j // 7][j % 7] for j in same]
+                reps = max(1, 200 // len(same))
+
+                def ours():
+                    for h in hs_same:
+                        sd2.sd2_spmm(h, xin, yo)
+
+                def theirs():
+                    for j in same:
+                        torch.matmul(xin, dense[j].t(), out=yo)
+                out_t = []
+                for fn in (ours, theirs):
+                    fn()
+                    stream.synchronize()
+                    e0.record(stream)
+                    for _ in range(reps):
+                        fn()
+                    e1.record(stream)
+                    stream.synchronize()
+                    out_t.append(e0.elapsed_time(e1) / (reps * len(same)) * 1e3)
+                per_shape.append({"M": int(M_), "K": int(K_), "copies_cycled": len(same), "sd2_spmm_us": out_t[0],
+                                  "cublas_dense_us": out_t[1], "ratio": out_t[1] / out_t[0]})
+            dense_res["per_shape_single_launch"] = per_shape
 
     ms_step = ms_total / args.steps
     ms_step, us_token = aggregate_replicas(ms_step, world, dist, "cuda")
@@ -409,53 +577,237 @@ def run_ours(args):
 
     if rank == 0:
         peak, peak_src = measured_peak()
-        achieved = comp_bytes / (ms_step * 1e-3) / 1e9           # per replica: bytes of one token / its time
+        t_launch = ms_step * 1e-3 / launches_per_step              # seconds per launch (one panel of the step)
+        kept = facts["kept_weights"]
+        streamed = facts["streamed_bytes"]                         # what one launch reads of the compressed drafter
+        useful = 2.5 * kept                                        # a bf16 value and a 4-bit column code per kept weight
+        bitmask_eq = 2.0 * kept + dense_elems / 8.0                # values + one mask bit per position
         traffic = ncu_traffic_ratio()
         roofline = {
-            "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "peak_source": peak_src, "frac_of_8TBps_nominal": achieved / 8000.0,
-            "kernel": "stream_kernel<%d>" % min(4, 1 << max(0, (min(N, 4) - 1).bit_length())),
-            "algorithmic_bytes_per_launch": comp_bytes / launches_per_step,
-            "avg_launch_us": ms_step * 1e3 / launches_per_step,
-            "traffic": (traffic["dram_bytes_per_algorithmic_byte"] * comp_bytes / launches_per_step) if traffic else None,
-            "traffic_source": traffic.get("source") if traffic else None,
+            "bound": "hbm", "achieved": useful / t_launch / 1e9, "peak": peak, "unit": "GB/s",
+            "frac": useful / t_launch / 1e9 / peak, "peak_source": peak_src,
+            "useful_bytes": useful, "padding_bytes": streamed - useful,
+            "useful_is": "2.5 B per kept weight (bf16 value + 4-bit column code); padding = tile headers, filler entries, alignment",
+            "achieved_streamed": streamed / t_launch / 1e9, "frac_streamed": streamed / t_launch / 1e9 / peak,
+            "achieved_bitmask_equivalent": bitmask_eq / t_launch / 1e9, "frac_bitmask_equivalent": bitmask_eq / t_launch / 1e9 / peak,
+            "kernel": "stream_kernel<%d>" % (1 << max(0, (min(N, facts["panel_rows"]) - 1).bit_length())),
+            "launches_per_step": launches_per_step, "panel_rows": facts["panel_rows"],
+            "avg_launch_us": t_launch * 1e6,
+            "traffic": (traffic["dram_bytes_per_algorithmic_byte"] * streamed) if traffic else None,
+            "traffic_source": ("stored: %s (DRAM bytes per streamed byte of an earlier capture x this launch's streamed bytes; "
+                               "not measured in this run)" % traffic.get("source")) if traffic else None,
         }
         cpu = None
         if not args.no_cpu and N == 1:
             from oracle import oracle
             oracle.build()
+            cores = host_cores()
             sample = min(blocks, 8)
-            sec = time_oracle(shape, cfg_id, density, N, sample, args.mask)
-            cpu = {"value": sec * blocks / sample * 1e6, "unit": UNIT, "cores": 1, "kind": "oracle",
-                   "sample": "%d of %d blocks (all 7 linears, N=1), one pass, scaled by %d/%d" % (sample, blocks, blocks, sample)}
+            sec_all = time_oracle(shape, cfg_id, density, N, sample, args.mask, threads=cores)
+            sample1 = min(blocks, 2)
+            sec_one = time_oracle(shape, cfg_id, density, N, sample1, args.mask, threads=1)
+            cpu = {"value": sec_all * blocks / sample * 1e6, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": "%d of %d blocks (all 7 linears, N=1), one pass, rows split over %d threads, scaled by %d/%d"
+                             % (sample, blocks, cores, blocks, sample),
+                   "one_core": {"value": sec_one * blocks / sample1 * 1e6, "unit": UNIT, "cores": 1,
+                                "sample": "%d of %d blocks, one thread" % (sample1, blocks)}}
         line = {
             "metric": METRIC, "value": us_token, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": config_dict(args, shape, blocks, {
                 "parallelism": "replicas x%d" % world, "compressed_bytes_per_token": comp_bytes,
-                "bytes_per_kept_weight": comp_bytes / max(nnz, 1), "dense_bf16_bytes_per_token": 2 * dense_elems,
-                "timing": "CUDA events around %d CUDA-graph replays of sd2_drafter_step (one persistent launch per token)" % args.steps,
+                "arithmetic": "bf16 weights and activations, exact products, fp32 accumulation, bf16 outputs",
+                "bytes_per_kept_weight": streamed / max(kept, 1), "dense_bf16_bytes_per_token": 2 * dense_elems,
+                "drafter_device_bytes": facts["owned_bytes"],
+                "timing": "CUDA events around %d CUDA-graph replays of sd2_drafter_step (%d persistent launch%s per step)"
+                          % (args.steps, launches_per_step, "" if launches_per_step == 1 else "es"),
+                "l2": "the step streams %.0f MB, more than the 126 MB L2; no flush between steps" % (streamed / 1e6),
                 "setup_seconds": round(setup_s, 1)}),
             "clocks": clocks,
+            "spread": spread,
             "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 2),
                     "d2h_bytes_per_step": int(y_host.numel() * 2), "steps": e2e_steps,
-                    "how": "wall clock per token: pinned-host x -> device, graph replay, device y -> pinned host, sync"},
+                    "how": "wall clock per step: pinned-host x -> device, graph replay, device y -> pinned host, sync"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline,
             "cpu_baseline": cpu,
+            "parity": parity,
             "block_step_launches_us_per_token": ms_stream * 1e3,
-            "cublas_dense_bf16_us_per_token": dense_us,
-            "speedup_vs_cublas_dense": (dense_us / (ms_step * 1e3)) if dense_us else None,
+            "cublas_dense": dense_res,
+            "cublas_dense_bf16_us_per_token": dense_res["fused_us_per_token"] if dense_res else None,
+            "speedup_vs_cublas_dense": (dense_res["fused_us_per_token"] / (ms_step * 1e3)) if dense_res else None,
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
 
+def time_graph_us(torch, fn, reps, stream=None):
+    """Microseconds per replay of a CUDA graph of `fn`, timed with events on the launch stream."""
+    stream = stream or torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        fn()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) / reps * 1e3
+
+
+def run_sweep(args):
+    """Sparsity sweep on single matrices (the paper's kernel-level speed-up figure): sd2_spmm against
+    cuBLAS dense bf16 with every launch reading its matrix from HBM.  For each shape, sparsity and N the
+    matrix is compressed once and loaded R times, R copies being at least four times the L2; a CUDA
+    graph holds one launch per copy.  The dense arm is torch.matmul on the masked weight stored
+    densely, rotated and captured the same way.  Prints a markdown table and, per shape and N, the
+    lowest sparsity from which the sparse launch is the faster one (linear interpolation)."""
+    import torch
+    from paper_2504_08838_b200 import binding as sd2
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    sd2.lib()
+    sparsities = [float(v) for v in args.sparsities.split(",")]
+    ns = [int(v) for v in args.sweep_n.split(",")]
+    shapes = synth.SWEEP_SHAPES[:1] if args.quick else synth.SWEEP_SHAPES
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    print("| M x K | N | sparsity | B / kept weight | sparse us | sparse GB/s | dense us | dense / sparse |")
+    print("|---|---|---|---|---|---|---|---|")
+    summary = []
+    for (M, K) in shapes:
+        W = synth.normal_bf16(synth.stream_seed(5, 0, 0, synth.WHAT_W) + M, (M, K), 0.02)
+        cross = {n: [] for n in ns}
+        for sp in sparsities:
+            mask = synth.bernoulli_mask(synth.stream_seed(5, 0, 0, synth.WHAT_MASK) + M + int(1000 * sp), (M, K), 1.0 - sp)
+            blob = sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_AUTO, sd2.SD2_DTYPE_BF16)
+            h0 = sd2.sd2_load_blob(blob)
+            R = max(2, int(np.ceil(4.0 * l2 / h0.compressed_bytes)))
+            hs = [h0] + [sd2.sd2_load_blob(blob) for _ in range(R - 1)]
+            Wd0 = torch.from_numpy(np.where(mask != 0, W, np.uint16(0)).view(np.int16)).cuda().view(torch.bfloat16)
+            Rd = max(2, int(np.ceil(4.0 * l2 / (2 * M * K))))
+            Wd = [Wd0] + [Wd0.clone() for _ in range(Rd - 1)]
+            for N in ns:
+                X = torch.from_numpy(synth.make_activations(5, 0, 0, N, K).view(np.int16).copy()).cuda().view(torch.bfloat16)
+                Y = torch.zeros((N, M), dtype=torch.bfloat16, device="cuda")
+
+                def sparse_all():
+                    for h in hs:
+                        sd2.sd2_spmm(h, X, Y)
+
+                def dense_all():
+                    for w in Wd:
+                        torch.matmul(X, w.t(), out=Y)
+
+                us_s = time_graph_us(torch, sparse_all, 20) / R
+                us_d = time_graph_us(torch, dense_all, 20) / Rd
+                cross[N].append((sp, us_s, us_d))
+                print("| %dx%d | %d | %.2f | %.3f | %.2f | %.0f | %.2f | %.2f |" % (
+                    M, K, N, sp, h0.compressed_bytes / max(h0.nnz, 1), us_s, h0.compressed_bytes / us_s / 1e3, us_d, us_d / us_s), flush=True)
+            for h in hs:
+                sd2.sd2_free(h)
+            del Wd, Wd0
+            torch.cuda.empty_cache()
+        for N in ns:
+            pts = cross[N]
+            where = "never on this grid"
+            if pts[0][1] < pts[0][2]:
+                where = "<= %.2f (already faster at the lowest grid point)" % pts[0][0]
+            else:
+                for (s0, a0, d0), (s1, a1, d1) in zip(pts, pts[1:]):
+                    if a0 >= d0 and a1 < d1:
+                        f0, f1 = a0 - d0, a1 - d1
+                        where = "%.3f" % (s0 + (s1 - s0) * f0 / (f0 - f1))
+                        break
+            summary.append({"M": M, "K": K, "N": N, "crossover_sparsity": where})
+            print("crossover %dx%d N=%d: sparse faster than cuBLAS dense from sparsity %s" % (M, K, N, where), flush=True)
+    print(json.dumps({"workload": "sweep", "crossovers": summary}))
+
+
+def run_config1(args):
+    """The single sparse linear (2048 x 2048, 50 % Bernoulli, N = 1): R = 128 independently seeded copies
+    (about 600 MB compressed, far more than the L2) launched round-robin give the HBM-cold time per
+    launch; the same launch repeated on one copy gives the L2-warm time, labelled as such."""
+    import torch
+    from paper_2504_08838_b200 import binding as sd2
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    sd2.lib()
+    M = K = 2048
+    R = 128
+    N = args.n
+    density = 1.0 - args.sparsity
+    fmt = {"auto": sd2.SD2_FORMAT_AUTO, "bitmask": sd2.SD2_FORMAT_BITMASK, "gap4": sd2.SD2_FORMAT_GAP4}[args.format]
+    hs, dense = [], []
+    for r in range(R):
+        W, m = synth.make_linear(1, r, 0, M, K, density, args.mask)
+        hs.append(sd2.sd2_compress(W, m, fmt, sd2.SD2_DTYPE_BF16))
+        if not args.no_dense:
+            dense.append(torch.from_numpy(np.where(m != 0, W, np.uint16(0)).view(np.int16)).cuda().view(torch.bfloat16))
+    x_bits = synth.make_activations(1, 0, 0, N, K)
+    X = torch.from_numpy(x_bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    Y = torch.zeros((N, M), dtype=torch.bfloat16, device="cuda")
+    sampler = ClockSampler(0)
+    sampler.start()
+    cold = time_graph_us(torch, lambda: [sd2.sd2_spmm(h, X, Y) for h in hs], max(3, args.steps // R)) / R
+    clocks = sampler.stop()
+    warm = time_graph_us(torch, lambda: [sd2.sd2_spmm(hs[0], X, Y) for _ in range(R)], max(3, args.steps // R)) / R
+    dcold = dwarm = None
+    if dense:
+        dcold = time_graph_us(torch, lambda: [torch.matmul(X, w.t(), out=Y) for w in dense], max(3, args.steps // R)) / R
+        dwarm = time_graph_us(torch, lambda: [torch.matmul(X, dense[0].t(), out=Y) for _ in range(R)], max(3, args.steps // R)) / R
+    parity = None
+    if not args.no_cpu:
+        from oracle import oracle
+        oracle.build()
+        W, m = synth.make_linear(1, 0, 0, M, K, density, args.mask)
+        sd2.sd2_spmm(hs[0], X, Y)
+        torch.cuda.synchronize()
+        Yr, S = oracle.masked_linear(W, m, x_bits)
+        y = Y.float().cpu().numpy().astype(np.float64)
+        parity = {"max_abs_err_over_S": float((np.abs(y - Yr) / np.maximum(S, 1e-300)).max()), "bound_over_S": 2.0 ** -8 + 2e-3,
+                  "against": "oracle, copy 0"}
+    peak, peak_src = measured_peak()
+    comp = sum(h.compressed_bytes for h in hs) / R
+    kept = sum(h.nnz for h in hs) / R
+    line = {
+        "metric": "single sparse linear us per launch at N=%d" % N, "value": cold, "unit": "us/launch", "n_gpus": 1,
+        "steps": max(3, args.steps // R) * R, "warmup": 3 * R, "ms_per_step": cold / 1e3, "higher_is_better": False,
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "config1: one %dx%d linear, %d%% Bernoulli sparsity, bf16 N(0,0.02), X %dx%d N(0,1); "
+                               "%d independently seeded copies launched round-robin (%.0f MB compressed > L2)"
+                               % (M, K, round(100 * args.sparsity), N, K, R, comp * R / 1e6),
+                   "timing": "CUDA events around replays of a CUDA graph holding one sd2_spmm per copy"},
+        "clocks": clocks, "gpu_launches": max(3, args.steps // R) * R,
+        "l2_warm_us_per_launch": warm, "l2_warm_note": "same copy every launch: the 4.7 MB matrix stays in L2; not an HBM figure",
+        "roofline": {"bound": "hbm", "achieved": 2.5 * kept / cold / 1e3, "peak": peak, "unit": "GB/s",
+                     "frac": 2.5 * kept / cold / 1e3 / peak, "peak_source": peak_src, "useful_bytes": 2.5 * kept,
+                     "padding_bytes": comp - 2.5 * kept, "achieved_streamed": comp / cold / 1e3,
+                     "frac_streamed": comp / cold / 1e3 / peak, "kernel": "stream_kernel<%d>" % max(1, min(8, 1 << max(0, (N - 1).bit_length()))),
+                     "avg_launch_us": cold, "traffic": None,
+                     "note": "a 4.7 MB launch lasts a few microseconds: launch and pipeline-fill latency, not bandwidth, bound it"},
+        "cublas_dense": {"cold_us_per_launch": dcold, "l2_warm_us_per_launch": dwarm} if dense else None,
+        "parity": parity,
+    }
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.workload in ("config1", "sweep"):
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the oracle arm times the drafter workloads only"}))
+        elif int(os.environ.get("RANK", "0")) == 0:
+            (run_config1 if args.workload == "config1" else run_sweep)(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

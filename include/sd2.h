@@ -51,7 +51,7 @@ typedef enum {
     SD2_ERR_CUDA = -4,        /* CUDA runtime error (no device, launch failure, ...)     */
     SD2_ERR_UNSUPPORTED = -5, /* valid request this build cannot serve (e.g. huge K)     */
     SD2_ERR_CORRUPT = -6,     /* a blob failed validation                                */
-    SD2_ERR_TIMEOUT = -7      /* reserved for bounded device-side waits                  */
+    SD2_ERR_TIMEOUT = -7      /* a bounded device-side wait ran out (sd2_stream_check)   */
 } sd2_status;
 
 /* Compressed formats.  Both are lossless; "compressed bytes" always counts every
@@ -153,7 +153,8 @@ sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, voi
  * one after another, separated by grid-wide barriers, while a producer warp keeps copying the
  * coming stages' weights into shared memory.  Such launches take every SM; two of them should
  * not be put on different streams in the hope of overlap.
- * Errors: SHAPE if the seven shapes do not chain; N must be in [0, 64]. */
+ * Errors: SHAPE if the seven shapes do not chain, or N outside [0, 65536].  Any N in that range
+ * is served: rows are independent and go through the block in panels of at most 8. */
 sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N,
                           void* workspace, void* cuda_stream);
 
@@ -169,7 +170,7 @@ sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* o
  * block's intermediates (q, k, v, hdn, g, u, t) and the grid-barrier words live in an array
  * built into the library image: 1 MiB + 256 bytes that every GPU which loads the library
  * keeps until the process exits.  Same result as sd2_block_step, same stub glue; x: device
- * bf16 [N*hidden], y: device [N*M_down] in h[6]'s y_dtype, 0 <= N <= 64.
+ * bf16 [N*hidden], y: device [N*M_down] in h[6]'s y_dtype, N >= 0.
  *  - all seven weights must be GAP4 (SD2_ERR_UNSUPPORTED otherwise), live on the current device;
  *  - sd2_block_workspace_bytes(h, N) must not exceed 1 MiB, else SD2_ERR_UNSUPPORTED and
  *    nothing is launched (e.g. a Llama-3.2-3B block fits up to N = 16);
@@ -192,7 +193,9 @@ sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, in
  * Where the shapes allow it the drafter keeps its own paired copy of every block's gate and up
  * (one stacked GAP4 matrix, gate row i and up row i side by side, as large as the two
  * together), built here on the host from the handles' decoded contents, so that a step forms
- * t = silu(g) * u where g and u are produced.
+ * t = silu(g) * u where g and u are produced.  That copy is device memory on top of the handles'
+ * (about 55 % more for a Llama-shaped block: gate and up are most of its weights);
+ * sd2_drafter_query reports what the drafter holds and what a step streams.
  * Errors: INVALID_ARG, SHAPE (shapes do not chain, L or n_max out of range), UNSUPPORTED (a
  * handle is not GAP4, or a layer is too wide for shared memory), ALLOC. */
 sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2_drafter* out);
@@ -202,6 +205,13 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
  * Asynchronous on the stream, allocates nothing.  Steps of one drafter must not overlap in
  * time (they share its buffers): keep them on one stream. */
 sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, void* cuda_stream);
+
+/* Facts about a drafter and a step of N rows (1 <= N <= n_max), out[6]:
+ *   out[0] kernel launches the step makes (one per panel of rows), out[1] rows of the widest panel,
+ *   out[2] device bytes the drafter owns (paired stacks, intermediates, tagged words, stage table),
+ *   out[3] bytes of compressed weights one launch reads (paired stacks in place of the gate and up
+ *          handles they replace), out[4] stages of a launch, out[5] kept weights of all handles. */
+sd2_status sd2_drafter_query(sd2_drafter d, int64_t N, int64_t* out);
 
 /* Device addresses of block `block`'s buffers after a step, ptrs[8] = q, k, v, hdn, g, u, t and
  * the block's bf16 output (not written for the last block, whose output goes to y).  Each is

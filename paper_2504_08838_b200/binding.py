@@ -26,7 +26,7 @@ EXPORTS = [
     "sd2_decompress", "sd2_info", "sd2_free", "sd2_spmm", "sd2_spmm_fused", "sd2_block_step",
     "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
     "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
-    "sd2_block_step_static", "sd2_selftest_timeout",
+    "sd2_block_step_static", "sd2_selftest_timeout", "sd2_drafter_query",
 ]
 
 
@@ -74,6 +74,7 @@ def lib():
             "sd2_drafter_create": [pp, i32, i64, pp],
             "sd2_drafter_step": [p, p, p, i64, p],
             "sd2_drafter_buffers": [p, i32, pp],
+            "sd2_drafter_query": [p, i64, pi64],
             "sd2_drafter_free": [p],
             "sd2_block_step_static": [pp, p, p, i64, p],
             "sd2_selftest_timeout": [p],
@@ -300,6 +301,14 @@ def sd2_drafter_buffers(d: Drafter, block: int):
     ptrs = (ctypes.c_void_p * 8)()
     _check(lib().sd2_drafter_buffers(d.raw, block, ptrs), "sd2_drafter_buffers")
     return [int(p or 0) for p in ptrs]
+
+
+def sd2_drafter_query(d: Drafter, N: int) -> dict:
+    """Launches per step of N rows, widest panel, device bytes owned, bytes streamed per launch, stages, kept weights."""
+    out = (ctypes.c_int64 * 6)()
+    _check(lib().sd2_drafter_query(d.raw, N, out), "sd2_drafter_query")
+    keys = ("launches", "panel_rows", "owned_bytes", "streamed_bytes", "stages", "kept_weights")
+    return dict(zip(keys, (int(v) for v in out)))
 
 
 def sd2_drafter_free(d: Drafter):

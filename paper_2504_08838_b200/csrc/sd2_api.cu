@@ -38,6 +38,7 @@ struct sd2_drafter_s {
     int64_t hidden, out_dim;
     std::vector<sd2_handle> handles;
     std::vector<sd2_handle> owned;      // paired gate|up stacks the drafter built for itself
+    std::vector<int> pair_block;        // the block each of them belongs to
     std::vector<int64_t> ws_off;        // per block: offsets of q,k,v,hdn,g,u,t and the block output inside d_ws
     uint8_t* d_ws;
     SStage* d_stages;
@@ -59,6 +60,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kBarrierPool = 64;             // grid-barrier word pairs handed out round-robin
 constexpr int kBarrierStrideWords = 64;      // 256 bytes apart
 constexpr int kSmemMax = 227 * 1024;         // dynamic shared memory a CTA may opt in to
+constexpr int kMaxBlockRows = 1 << 16;       // activation rows a block step accepts (taken in panels)
 constexpr int kDrafterWordsBytes = 512;      // a drafter's device words: barrier (two lines), then 64 production counts
 
 struct DeviceState {
@@ -385,10 +387,6 @@ void fill_stage(SStage& st, const sd2_handle* hs, int count, const uint16_t* x, 
     set_stage_grid(st, grid);
 }
 
-#ifdef SD2_TRACE
-long long* g_trace = nullptr;   // set through sd2_debug_set_trace (trace builds only)
-#endif
-
 long long wait_budget(int dev)
 {
     // about two seconds of SM clock; SD2_WAIT_MS overrides (tests use a short one)
@@ -454,9 +452,6 @@ sd2_status run_panels(SArgs& a, int64_t N, const int xs_need[4], int K_max, int 
         a.xs_bytes = p.xs_bytes;
         a.xlin_bytes = p.xlin_bytes;
         a.ring_bytes = p.ring_bytes;
-#ifdef SD2_TRACE
-        a.trace = g_trace;
-#endif
         sd2_status st = launch_stream(nt, a, grid, a.n_stages > 1, s);
         if (st != SD2_OK) return st;
     }
@@ -864,7 +859,7 @@ sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, voi
 sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* bytes)
 {
     if (!bytes) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -877,7 +872,7 @@ sd2_status sd2_block_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* by
 sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* offsets)
 {
     if (!offsets) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -890,7 +885,7 @@ sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* o
 sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N, void* workspace, void* cuda_stream)
 {
     if (!x || !y || !workspace) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -951,7 +946,7 @@ unsigned char* g_static_ptr[kMaxDevices];   // device address of g_static_scratc
 sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, int64_t N, void* cuda_stream)
 {
     if (!x || !y) return SD2_ERR_INVALID_ARG;
-    if (N < 0 || N > 64) return SD2_ERR_SHAPE;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
     sd2_status st = block_dims(h, &d);
     if (st != SD2_OK) return st;
@@ -988,6 +983,7 @@ sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, in
                                      (uint16_t*)(ws + off[5]), (uint16_t*)(ws + off[6]), y, false, &needs, g_dev[dev].sms);
     a.err = g_dev[dev].err_word;
     a.wait_cycles = wait_budget(dev);
+    a.free_tiles = needs.free_tiles(g_dev[dev].sms);
     a.gbar = (unsigned int*)base;
     return run_panels(a, N, needs.xs_need, needs.K_max, needs.max_tile, g_dev[dev].sms, s);
 }
@@ -1060,7 +1056,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
     if (ok && tagged) {
         for (int b = 0; b < L && st == SD2_OK; ++b) {
             st = build_gate_up_pair(h[7 * b + 4], h[7 * b + 5], &pairs[(size_t)b]);
-            if (pairs[(size_t)b]) d->owned.push_back(pairs[(size_t)b]);
+            if (pairs[(size_t)b]) { d->owned.push_back(pairs[(size_t)b]); d->pair_block.push_back(b); }
         }
         if (st != SD2_OK) {
             for (sd2_handle p : d->owned) sd2_free(p);
@@ -1156,6 +1152,38 @@ sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, vo
     return run_panels(a, N, d->xs_need, d->K_max, d->max_tile, g_dev[dev].sms, (cudaStream_t)cuda_stream);
 }
 
+sd2_status sd2_drafter_query(sd2_drafter d, int64_t N, int64_t* out)
+{
+    if (!live(d) || !out) return SD2_ERR_INVALID_ARG;
+    if (N < 1 || N > d->n_max) return SD2_ERR_SHAPE;
+    const int cap = widest_panel(d->xs_need, d->K_max, d->max_tile);
+    if (cap == 0) return SD2_ERR_UNSUPPORTED;
+    int64_t streamed = 0, owned = 0, kept = 0;
+    // what a step streams: every handle once, except that a block's gate and up are read from the
+    // drafter's own paired stack where it has one
+    std::vector<char> paired((size_t)d->L, 0);
+    for (sd2_handle p : d->owned) { streamed += p->compressed_bytes; owned += p->blob_bytes; }
+    size_t oi = 0;
+    for (int b = 0; b < d->L; ++b) {
+        // (owned stacks were built in block order, one per block that could be paired)
+        const bool has_pair = oi < d->owned.size() && d->owned[oi]->M == 2 * d->handles[(size_t)7 * b + 4]->M &&
+                              d->pair_block.size() > oi && d->pair_block[oi] == b;
+        if (has_pair) ++oi;
+        for (int i = 0; i < 7; ++i) {
+            const sd2_handle h = d->handles[(size_t)7 * b + i];
+            kept += h->nnz;
+            if (!(has_pair && (i == 4 || i == 5))) streamed += h->compressed_bytes;
+        }
+    }
+    out[0] = (N + cap - 1) / cap;                                  // launches per step of N rows
+    out[1] = cap;                                                  // rows of the widest panel
+    out[2] = owned + d->ws_off.back() + d->tags_bytes + (int64_t)sizeof(SStage) * d->n_stages + kDrafterWordsBytes;
+    out[3] = streamed;                                             // bytes of compressed weights read per launch
+    out[4] = d->n_stages;
+    out[5] = kept;
+    return SD2_OK;
+}
+
 sd2_status sd2_drafter_buffers(sd2_drafter d, int32_t block, void** ptrs)
 {
     if (!live(d) || !ptrs) return SD2_ERR_INVALID_ARG;
@@ -1182,9 +1210,5 @@ sd2_status sd2_drafter_free(sd2_drafter d)
     delete d;
     return st;
 }
-
-#ifdef SD2_TRACE
-void sd2_debug_set_trace(long long* device_buffer) { g_trace = device_buffer; }
-#endif
 
 }  // extern "C"

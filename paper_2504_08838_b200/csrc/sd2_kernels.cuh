@@ -64,10 +64,14 @@ __device__ __forceinline__ float warp_sum(float v)
 //
 // One persistent CTA per SM runs a *program* of stages.  A stage is one launch's worth of
 // work: up to four weights that read the same activations (q|k|v, gate|up, or one weight).
-// Consecutive stages depend on each other (the next one reads what this one wrote), so they
-// are separated by a grid-wide barrier; the weights, however, never depend on anything, and
-// the producer warp keeps copying the tiles of coming stages into the ring while the
-// consumer warps are still computing, waiting at the barrier or staging activations.
+// Consecutive stages depend on each other (the next one reads what this one wrote).  The hand-off
+// is either a grid-wide barrier (programs over a caller's workspace) or tagged words (drafters):
+// every intermediate activation is also written as a 32-bit word bf16 << 16 | tag, and the next
+// stage polls exactly the words it needs until they carry the tag it expects; value and tag
+// share a word, so no fence is needed.  A tag is (how often that activation row has been
+// produced & 0xFF) << 8 | (stage number + 1).  The weights never depend on anything: the
+// producer warp keeps copying the tiles of coming stages into the ring while the consumer warps
+// are still computing, waiting for the hand-off or staging activations.
 //
 // Tiles of a stage are dealt round-robin to the CTAs (tile v of the stage goes to CTA
 // v % gridDim.x) and, inside a CTA, round-robin to the consumer warps.  A warp owns whole
@@ -82,8 +86,8 @@ __device__ __forceinline__ float warp_sum(float v)
 // (row 2j in the low half, row 2j+1 in the high half of word j), W = max(1, NT / 2), groups =
 // 32 / W.  Lane l reads group l % groups, so one warp-wide gather touches every bank W times.
 //
-// Every wait (ring barriers, grid barrier) is bounded by a cycle budget: when it runs out
-// the CTA raises the error word and winds down instead of hanging.
+// Every wait (ring barriers, tag polls, grid barrier) is bounded by a cycle budget: when it runs
+// out the CTA raises the error word and winds down instead of hanging.
 
 #ifndef SD2_CONSUMER_WARPS
 #define SD2_CONSUMER_WARPS 16
@@ -154,17 +158,8 @@ struct SArgs {
                                     // words, bumped by the last CTA out)
     int free_tiles;                 // 1: a consumer warp that is done draws the next tile from a shared counter;
                                     // 0: tile k of a stage goes to warp k % 16 (see the consumer loop)
-    long long* trace;               // SD2_TRACE builds: [cta][stage][8] SM clock stamps; else unused
+    long long* reserved_ptr;
 };
-
-#ifdef SD2_TRACE
-// per-tile stamps of CTA 0 (issue, wait begin, start, end, producer waits for its release: begin, end)
-#define SD2_TILE_STAMP(q, slot) do { if (a.trace && cta == 0 && (q) < 4096u) a.trace[(size_t)gridDim.x * a.n_stages * 8 + (size_t)(q) * 8 + (slot)] = clock64(); } while (0)
-#define SD2_STAMP(slot) do { if (a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define SD2_STAMP(slot) do { } while (0)
-#define SD2_TILE_STAMP(q, slot) do { } while (0)
-#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -345,8 +340,6 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity, const 
     return true;
 }
 
-// acc[n] += w * x[n] for the NT activation rows stored side by side at `addr + OFF`;
-// w is the low (HI = 0) or high (HI = 1) bf16 of `wpair`.
 // c + w * x for bf16 w and x with an fp32 sum (the product of two bf16 values is exact in fp32,
 // so this equals an fp32 fused multiply-add of the widened values): w = half WH of wpair,
 // x = half XH of xword (0: low, 1: high)
@@ -421,11 +414,6 @@ __device__ __forceinline__ uint32_t chunk_fma(uint32_t code, const uint4& v, uin
     return byte_times_128_plus<3>(PO, xb + 1024u);
 }
 
-// Stage the activations of one stage: xs[plane][window row c][group][NT] (fp32) with
-// value = X[n][strip * B - V + c] where strip = plane * groups + group % S (for S <= groups the
-// strips repeat across the groups), zero outside the matrix, in the slack rows and for n >= N.
-// Row by row through `xlin` (bf16, linear) so that global memory is read with 128-bit loads.
-// x_src, g, u, t_out already point at the launch's first activation row.
 // One 128-bit load of four tagged words, repeated until all four carry `tag` (their producers,
 // on other SMs, have stored them) or the wait budget runs out.  Value and tag share a 32-bit
 // word, so a word that shows the tag also shows its value: no fence is needed.
@@ -534,6 +522,14 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
     }
 }
 
+// Stages the activations of one stage: xs[plane][window row c][group][W words], a word holding one
+// bf16 (NT = 1, high half) or the bf16 values of two panel rows, with the value of column
+// strip * B - V + c where strip = plane * groups + group % S (for S <= groups the strips repeat
+// across the groups), zero outside the matrix and for rows n >= N.  Row by row through `xlin` (bf16,
+// linear, zero-padded on both sides) so that global memory is read with coalesced 128-bit loads: a
+// warp that instead reads its 32 strips directly asks L2 for 32 separate sectors of lines that every
+// other SM wants at the same moment, which measured 1.7 times slower for the whole token.
+// x_src, g, u, t_out already point at the launch's first activation row.
 // `tag` != 0: x_src / g / u point at tagged 32-bit words (see stage_linear_tagged); row n's words carry
 // tag | tagb[n].
 // Panels of four and eight rows go two rows at a time: both rows are fetched into their own linear
@@ -781,7 +777,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                             const uint32_t my_head = head + incl - bytes;
                             const uint32_t my_q = q + (uint32_t)(lane - i0);
                             const uint32_t my_slot = my_q % kSlots;
-                            SD2_TILE_STAMP(my_q, 0);
                             sh->desc[my_slot] = make_int4((int)my_head, pb_cur.mi, pb_cur.ti, (int)bytes);
                             mbar_expect_tx(full0 + 8 * my_slot, bytes);
                             if (hinted) bulk_g2s(ring0 + my_head, (const void*)pb_cur.src, bytes, full0 + 8 * my_slot, weight_policy);
@@ -800,9 +795,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     }
                     // no room: wait until the oldest tile in the ring has been consumed, and take
                     // along every further tile that is already done
-                    if (lane == 0) SD2_TILE_STAMP(oldest, 4);
                     if (!wait_phase(empty0 + 8 * (oldest % kSlots), (oldest / kSlots) & 1u, wc)) { ok = false; break; }
-                    if (lane == 0) SD2_TILE_STAMP(oldest, 5);
                     ++oldest;
                     while (oldest != q) {   // each lane looks at one of the next 32 tiles; the leading run of done ones goes
                         const uint32_t t = oldest + (uint32_t)lane;
@@ -814,7 +807,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                     tail = oldest == q ? head : (uint32_t)sh->desc[oldest % kSlots].x;
                 }
             }
-            if (lane == 0) SD2_STAMP(6);
             ps_cur = ps_next;
             ps_next = ps_next2;
             pb_cur = pb_next;
@@ -859,7 +851,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
     int s = 0;
     for (; s < a.n_stages; ++s) {
         if (ctid == 0) {
-            SD2_STAMP(0);
             if (s > 0 && !a.tagged) {
                 // grid barrier: every CTA has written the previous stage's outputs
                 const unsigned int target = (unsigned int)s * (unsigned int)G;
@@ -874,7 +865,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 __threadfence();
             }
             sh->stage_dead = sh->abort_flag;
-            SD2_STAMP(1);
         }
         named_bar_sync(1, kConsumerThreads);
         if (sh->stage_dead) break;
@@ -900,7 +890,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
                         st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         }
-        if (ctid == 0) SD2_STAMP(2);
         if (warp == 1 && s + 1 < a.n_stages) {
             const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);
             for (int i = lane; i < kStageWords; i += 32) ((uint32_t*)&sh->stage[(s + 1) & 1])[i] = src[i];
@@ -916,23 +905,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         const uint32_t lt = (1u << lane) - 1u;
         const bool last_stage = s == a.n_stages - 1;
 
-#ifdef SD2_TRACE
-        long long trace_wait = 0;   // cycles this warp waited for tiles to land, stored once per stage
-#endif
         if (!a.free_tiles) q_mine = qbase + (uint32_t)warp;
         while ((int)(q_mine - (qbase + (uint32_t)n_cta)) < 0 && !failed) {
             const uint32_t q = q_mine;
             const uint32_t slot = q % kSlots;
-#ifdef SD2_TRACE
-            const long long tw0 = clock64();
-            if (lane == 0) SD2_TILE_STAMP(q, 1);
-#endif
             if (!wait_phase(full0 + 8 * slot, (q / kSlots) & 1u, wc)) { failed = true; break; }
-#ifdef SD2_TRACE
-            trace_wait += clock64() - tw0;
-#endif
-            if (ctid == 0 && q == qbase) SD2_STAMP(3);
-            if (lane == 0) SD2_TILE_STAMP(q, 2);
             const int4 d = sh->desc[slot];
             const uint32_t tb = ring0 + (uint32_t)d.x;
             const uint32_t cnt = lds_u16(tb + 2u * lane);
@@ -1052,7 +1029,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
                 }
             }
             __syncwarp();
-            if (lane == 0) SD2_TILE_STAMP(q, 3);
             uint32_t q_next = q + (uint32_t)kConsumerWarps;
             if (lane == 0) {
                 mbar_arrive(empty0 + 8 * slot);
@@ -1061,13 +1037,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             q_mine = __shfl_sync(0xFFFFFFFFu, q_next, 0);
         }
         qbase += (uint32_t)n_cta;
-        if (ctid == 0) SD2_STAMP(4);
-#ifdef SD2_TRACE
-        if (ctid == 0 && a.trace) a.trace[((size_t)cta * a.n_stages + s) * 8 + 7] = trace_wait;
-#endif
         // everything this CTA wrote in the stage is visible before it arrives at the barrier
         named_bar_sync(1, kConsumerThreads);
-        if (ctid == 0) SD2_STAMP(5);
         if (s + 1 < a.n_stages && ctid == 0 && !a.tagged) {
             __threadfence();
             atomicAdd(a.gbar, 1u);

@@ -137,6 +137,54 @@ def test_config5_sweep_shapes(M, K, sparsity):
     sd2.sd2_free(h)
 
 
+@pytest.mark.parametrize("M,K", synth.SWEEP_SHAPES)
+@pytest.mark.parametrize("N", [1, 64])
+def test_config5_sweep_shapes_narrowest_and_widest_panel(M, K, N):
+    # the rows the sweep table reports at N = 1 and N = 64, at 50 % sparsity
+    W, mask = synth.make_linear(5, 0, 1, M, K, 0.5)
+    X = synth.make_activations(5, 0, 1, N, K)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_AUTO, sd2.SD2_DTYPE_F32)
+    Y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_spmm(h, dev_bf16(X), Y)
+    sd2.sd2_stream_check()
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(Y.cpu().numpy().astype(np.float64), Yr, S, True)
+    sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("N", [1, 8])
+def test_block_step_llama_1b_block_full_size(N):
+    # sd2_block_step itself (grid barriers between the stages, caller's workspace) on one full-size
+    # block: every linear against the oracle on the input the device gave it
+    shape = synth.LLAMA_1B
+    lin = synth.make_block(2, 0, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m, sd2.SD2_FORMAT_AUTO, sd2.SD2_DTYPE_F32 if i == 6 else sd2.SD2_DTYPE_BF16)
+          for i, (W, m) in enumerate(lin)]
+    x = synth.make_activations(2, 0, 0, N, shape.hidden)
+    off = sd2.sd2_block_workspace_layout(hs, N)
+    ws = torch.full((sd2.sd2_block_workspace_bytes(hs, N) // 2,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_block_step(hs, dev_bf16(x), y, ws)
+    sd2.sd2_stream_check()
+    wsb = ws.view(torch.int16).cpu().numpy().view(np.uint16)
+    dims = [shape.hidden, shape.kv, shape.kv, shape.hidden, shape.inter, shape.inter, shape.inter]
+    q, k, v, hdn, g, u, t = [wsb[o // 2:o // 2 + N * dm].reshape(N, dm) for o, dm in zip(off, dims)]
+    for idx, xin, got in ((0, x, q), (1, x, k), (2, x, v), (3, q, hdn), (4, hdn, g), (5, hdn, u)):
+        Yr, S = oracle.masked_linear(lin[idx][0], lin[idx][1], xin)
+        check(synth.bf16_bits_to_f32(got).astype(np.float64), Yr, S, False)
+    t_ref = oracle.silu_mul(g, u)
+    t_bits = np.array([oracle.f64_to_bf16_rne(float(z)) for z in t_ref], np.uint16).reshape(N, -1)
+
+    def key(b):
+        b = b.astype(np.int32)
+        return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    assert np.abs(key(t) - key(t_bits)).max() <= 2
+    Yr, S = oracle.masked_linear(lin[6][0], lin[6][1], t)
+    check(y.cpu().numpy().astype(np.float64), Yr, S, True)
+    for h in hs:
+        sd2.sd2_free(h)
+
+
 def test_unaligned_activation_pointer():
     # X that starts on an odd element: the staging must not assume 16-byte alignment
     M, K, N = 300, 2048, 3

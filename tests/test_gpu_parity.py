@@ -493,3 +493,61 @@ def test_a_wait_that_runs_out_is_reported_and_the_library_carries_on(monkeypatch
     Yr, S = oracle.masked_linear(W, mask, X)
     check(run_spmm(h, X, True), Yr, S, True)
     sd2.sd2_free(h)
+
+
+def test_block_step_with_more_than_64_rows():
+    # 70 rows: nine panels of at most eight rows through the same block program
+    N = 70
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 1)
+    lin = synth.make_block(2, 5, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32 if i == 6 else sd2.SD2_DTYPE_BF16)
+          for i, (W, m) in enumerate(lin)]
+    x = synth.make_activations(2, 5, 0, N, shape.hidden)
+    off = sd2.sd2_block_workspace_layout(hs, N)
+    ws = torch.full((sd2.sd2_block_workspace_bytes(hs, N) // 2,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_block_step(hs, dev_bf16(x), y, ws)
+    sd2.sd2_stream_check()
+    wsb = ws.view(torch.int16).cpu().numpy().view(np.uint16)
+    t = wsb[off[6] // 2: off[6] // 2 + N * shape.inter].reshape(N, -1)
+    q = wsb[off[0] // 2: off[0] // 2 + N * shape.hidden].reshape(N, -1)
+    Yr, S = oracle.masked_linear(lin[0][0], lin[0][1], x)
+    check(synth.bf16_bits_to_f32(q).astype(np.float64), Yr, S, False)
+    Yr, S = oracle.masked_linear(lin[6][0], lin[6][1], t)
+    check(y.cpu().numpy().astype(np.float64), Yr, S, True)
+    # every row agrees with the same row pushed through alone
+    for n in (0, 63, 64, 69):
+        y1 = torch.full((1, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+        sd2.sd2_block_step(hs, dev_bf16(x[n:n + 1]), y1, ws)
+        sd2.sd2_stream_check()
+        assert np.all(np.abs((y1[0] - y[n]).cpu().numpy().astype(np.float64)) <= 1e-3 * S[n])
+    for h in hs:
+        sd2.sd2_free(h)
+
+
+def test_drafter_step_in_several_panels_with_k_8192():
+    # inter = 8192 caps a panel below 16 rows: the step runs as several launches, each a panel,
+    # and must equal the chain of block steps bit for bit
+    N = 16
+    shape, blocks, d = _tiny_drafter(2, N, dims=(256, 64, 8192))
+    facts = sd2.sd2_drafter_query(d, N)
+    assert facts["launches"] >= 2 and facts["launches"] * facts["panel_rows"] >= N
+    assert facts["stages"] > 0 and facts["kept_weights"] == sum(h.nnz for hs in blocks for h in hs)
+    x = synth.make_activations(2, 0, 0, N, shape.hidden)
+    xd = dev_bf16(x)
+    y = torch.full((N, shape.hidden), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_drafter_step(d, xd, y)
+    sd2.sd2_stream_check()
+    ref = _block_chain(blocks, shape, xd)
+    assert torch.equal(y, ref)
+    # the down projection of block 0 against the oracle on the t the device formed
+    ptrs = sd2.sd2_drafter_buffers(d, 0)
+    t = _read_u16(ptrs[6], N * shape.inter).reshape(N, -1)
+    out = _read_u16(ptrs[7], N * shape.hidden).reshape(N, -1)
+    lin = synth.make_block(2, 0, shape, 0.5)
+    Yr, S = oracle.masked_linear(lin[6][0], lin[6][1], t)
+    check(synth.bf16_bits_to_f32(out).astype(np.float64), Yr, S, False)
+    sd2.sd2_drafter_free(d)
+    for hs in blocks:
+        for h in hs:
+            sd2.sd2_free(h)
