@@ -62,11 +62,20 @@ enum {
     SD2_FORMAT_GAP4 = 2,    /* 4-bit column gaps + packed kept values in 8-entry chunks,  */
                             /* rows cut into column strips, 32 strips to a tile (the fast */
                             /* path; column strips wider than 496 are not supported)      */
-    SD2_FORMAT_GAP4_PAIRED = 3 /* as an option of sd2_pack_host / sd2_compress only: GAP4 */
+    SD2_FORMAT_GAP4_PAIRED = 3,/* as an option of sd2_pack_host / sd2_compress only: GAP4 */
                             /* whose rows 2i and 2i+1 stay next to each other in a tile   */
                             /* (for a stack that interleaves gate row i and up row i; M   */
                             /* even and at least two rows per tile, else UNSUPPORTED).    */
                             /* The blob and the handle report SD2_FORMAT_GAP4.            */
+    SD2_FORMAT_GAP4_MMA = 4 /* for panels of N >= 16 activation rows: 128 x 128 blocks    */
+                            /* whose 4-bit gaps run in the order of a tensor-core operand */
+                            /* tile; sd2_spmm expands each block in shared memory and     */
+                            /* multiplies it on the tensor cores (tcgen05.mma, fp32       */
+                            /* accumulators in tensor memory).  Any N is accepted (rows   */
+                            /* are taken 64 at a time, padded to a multiple of 16); never */
+                            /* picked by AUTO; not accepted by sd2_block_step or a        */
+                            /* drafter.  Calls on one handle must not overlap on the GPU: */
+                            /* they share the handle's partial-sum buffer.                */
 };
 
 enum { SD2_DTYPE_BF16 = 0, SD2_DTYPE_F32 = 1 };

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(HERE, "libsd2.so")
 SD2_OK = 0
 SD2_ERR_INVALID_ARG, SD2_ERR_SHAPE, SD2_ERR_ALLOC, SD2_ERR_CUDA = -1, -2, -3, -4
 SD2_ERR_UNSUPPORTED, SD2_ERR_CORRUPT, SD2_ERR_TIMEOUT = -5, -6, -7
-SD2_FORMAT_AUTO, SD2_FORMAT_BITMASK, SD2_FORMAT_GAP4, SD2_FORMAT_GAP4_PAIRED = 0, 1, 2, 3
+SD2_FORMAT_AUTO, SD2_FORMAT_BITMASK, SD2_FORMAT_GAP4, SD2_FORMAT_GAP4_PAIRED, SD2_FORMAT_GAP4_MMA = 0, 1, 2, 3, 4
 SD2_DTYPE_BF16, SD2_DTYPE_F32 = 0, 1
 
 EXPORTS = [

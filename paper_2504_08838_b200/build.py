@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsd2.so")
 SOURCES = ["sd2_api.cu"]
-DEPS = ["sd2_api.cu", "sd2_kernels.cuh", "sd2_format.hpp", os.path.join("..", "..", "include", "sd2.h")]
+DEPS = ["sd2_api.cu", "sd2_kernels.cuh", "sd2_mma_kernel.cuh", "sd2_format.hpp", "sd2_format_mma.hpp", os.path.join("..", "..", "include", "sd2.h")]
 
 
 def nvcc_path() -> str:

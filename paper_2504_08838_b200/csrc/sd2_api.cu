@@ -14,7 +14,9 @@
 
 #include "../../include/sd2.h"
 #include "sd2_format.hpp"
+#include "sd2_format_mma.hpp"
 #include "sd2_kernels.cuh"
+#include "sd2_mma_kernel.cuh"
 
 using namespace sd2;
 
@@ -28,6 +30,10 @@ struct sd2_handle_s {
     // GAP4 geometry
     int S, B, T, max_tile_bytes, V;
     int paired;   // GAP4: rows 2i, 2i+1 share a tile (header field `pairing`)
+    // GAP4_MMA: fp32 partial sums [64][rows padded to 128] followed by one arrival count per row panel,
+    // all zero between launches (the CTA that completes a panel writes Y and clears them)
+    float* d_partial;
+    int64_t partial_bytes;
 };
 
 struct sd2_drafter_s {
@@ -118,7 +124,8 @@ sd2_status ensure_device(int* dev_out)
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
         if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess ||
-            set_smem_attr<8>() != cudaSuccess) {
+            set_smem_attr<8>() != cudaSuccess ||
+            cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax) != cudaSuccess) {
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
@@ -163,6 +170,7 @@ sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K
         if (f == SD2_FORMAT_BITMASK) r = pack_bitmask(W, mask, M, K, y_dtype);
         else if (f == SD2_FORMAT_GAP4) r = pack_gap4(W, mask, M, K, y_dtype);
         else if (f == SD2_FORMAT_GAP4_PAIRED) r = pack_gap4(W, mask, M, K, y_dtype, true);
+        else if (f == SD2_FORMAT_GAP4_MMA) r = pack_gap4_mma(W, mask, M, K, y_dtype);
         else return SD2_ERR_INVALID_ARG;
     } catch (const std::bad_alloc&) {
         return SD2_ERR_ALLOC;
@@ -171,6 +179,13 @@ sd2_status pack_any(const uint16_t* W, const uint8_t* mask, int64_t M, int64_t K
     *blob = r.blob;
     *bytes = r.bytes;
     return SD2_OK;
+}
+
+int unpack_any(const BlobHeader& hd, const uint8_t* blob, uint16_t* dense)
+{
+    if (hd.format == (uint32_t)kFormatBitmask) return unpack_bitmask(hd, blob, dense);
+    if (hd.format == (uint32_t)kFormatGap4Mma) return unpack_gap4_mma(hd, blob, dense);
+    return unpack_gap4(hd, blob, dense);
 }
 
 sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_handle* out)
@@ -204,6 +219,16 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     h->max_tile_bytes = (int)hd.max_tile_bytes;
     h->V = (int)hd.overlap;
     h->paired = (int)hd.pairing;
+    h->d_partial = nullptr;
+    h->partial_bytes = 0;
+    if (h->format == SD2_FORMAT_GAP4_MMA) {
+        const int64_t panels = (hd.M + kMmaBlockRows - 1) / kMmaBlockRows;
+        h->partial_bytes = (int64_t)kMmaMaxRows * panels * kMmaBlockRows * 4 + panels * 4;
+        void* pp = nullptr;
+        if (cudaMalloc(&pp, (size_t)h->partial_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(d); delete h; return SD2_ERR_ALLOC; }
+        if (cudaMemset(pp, 0, (size_t)h->partial_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(pp); cudaFree(d); delete h; return SD2_ERR_CUDA; }
+        h->d_partial = (float*)pp;
+    }
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_live.insert(h);
@@ -473,6 +498,45 @@ sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, 
 }
 
 // Shared by sd2_spmm and sd2_spmm_fused (and by block steps that mix formats).
+// GAP4_MMA: one launch per 64 activation rows; each expands the blocks in shared memory and multiplies on the
+// tensor cores.
+sd2_status run_mma(sd2_handle h, const uint16_t* x, void* Y, int64_t N, bool y_force_bf16, int dev, cudaStream_t s)
+{
+    MmaArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.dir = h->d_sec0;
+    a.recs = (const uint8_t*)h->d_sec1;
+    a.M = (int)h->M;
+    a.K = (int)h->K;
+    a.P = (int)((h->M + kMmaBlockRows - 1) / kMmaBlockRows);
+    a.KC = (int)((h->K + kMmaBlockCols - 1) / kMmaBlockCols);
+    a.NB = (long long)a.P * a.KC;
+    a.partial = h->d_partial;
+    a.done = (unsigned int*)(h->d_partial + (size_t)kMmaMaxRows * a.P * kMmaBlockRows);
+    a.y_f32 = (!y_force_bf16 && h->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
+    a.slot_bytes = (h->max_tile_bytes + 127) & ~127;
+    a.err = g_dev[dev].err_word;
+    a.budget = wait_budget(dev);
+    const size_t esz = a.y_f32 ? 4 : 2;
+    const int grid = (int)(a.NB < g_dev[dev].sms ? a.NB : g_dev[dev].sms);
+    for (int64_t n0 = 0; n0 < N; n0 += kMmaMaxRows) {
+        a.N = (int)((N - n0) < kMmaMaxRows ? (N - n0) : kMmaMaxRows);
+        a.npad = (a.N + 15) & ~15;
+        a.X = x + n0 * h->K;
+        a.Y = (char*)Y + (size_t)n0 * (size_t)h->M * esz;
+        a.x_vec = ((h->K & 7) == 0 && (((uintptr_t)a.X) & 15) == 0) ? 1 : 0;
+        const int fixed = 1024 + kMmaGroups * kMmaTileBytes + kMmaGroups * a.npad * 256 + (int)((sizeof(MmaShared) + 127) & ~127);
+        int slots = (kSmemMax - fixed) / a.slot_bytes;
+        if (slots < 1) return SD2_ERR_UNSUPPORTED;
+        if (slots > kMmaSlots) slots = kMmaSlots;
+        a.n_slots = slots;
+        const int smem = fixed + slots * a.slot_bytes;
+        mma_kernel<<<grid, kMmaThreads, smem, s>>>(a);
+        if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
+    }
+    return SD2_OK;
+}
+
 sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const uint16_t* g, const uint16_t* u,
                      uint16_t* t_out, void* const* Y, int64_t N, bool y_force_bf16, cudaStream_t s)
 {
@@ -500,6 +564,14 @@ sd2_status run_group(const sd2_handle* hs, int count, const uint16_t* x, const u
     for (int i = 0; i < count; ++i)
         if (hs[i]->device != dev) return SD2_ERR_INVALID_ARG;
     if (hs[0]->format == SD2_FORMAT_BITMASK) return run_bitmask(hs, count, x, g, u, t_out, Y, N, y_force_bf16, dev, s);
+    if (hs[0]->format == SD2_FORMAT_GAP4_MMA) {
+        if (!x || g || u || t_out) return SD2_ERR_UNSUPPORTED;     // plain products only
+        for (int i = 0; i < count; ++i) {
+            sd2_status si = run_mma(hs[i], x, Y[i], N, y_force_bf16, dev, s);
+            if (si != SD2_OK) return si;
+        }
+        return SD2_OK;
+    }
     SArgs a;
     std::memset(&a, 0, sizeof a);
     a.n_stages = 1;
@@ -690,8 +762,7 @@ sd2_status sd2_unpack_host(const void* blob, int64_t blob_bytes, void* dense_bf1
     if (check_header((const uint8_t*)blob, blob_bytes, hd, true) != 0) return SD2_ERR_CORRUPT;
     int rc;
     try {
-        rc = hd.format == (uint32_t)kFormatBitmask ? unpack_bitmask(hd, (const uint8_t*)blob, (uint16_t*)dense_bf16_out)
-                                                   : unpack_gap4(hd, (const uint8_t*)blob, (uint16_t*)dense_bf16_out);
+        rc = unpack_any(hd, (const uint8_t*)blob, (uint16_t*)dense_bf16_out);
     } catch (const std::bad_alloc&) {
         return SD2_ERR_ALLOC;
     }
@@ -753,8 +824,7 @@ sd2_status sd2_load_blob(const void* blob, int64_t blob_bytes, sd2_handle* out)
     // full structural validation before anything reaches a kernel
     int rc;
     try {
-        rc = hd.format == (uint32_t)kFormatBitmask ? unpack_bitmask(hd, (const uint8_t*)blob, nullptr)
-                                                   : unpack_gap4(hd, (const uint8_t*)blob, nullptr);
+        rc = unpack_any(hd, (const uint8_t*)blob, nullptr);
     } catch (const std::bad_alloc&) {
         return SD2_ERR_ALLOC;
     }
@@ -801,6 +871,7 @@ sd2_status sd2_free(sd2_handle h)
     }
     sd2_status st = SD2_OK;
     if (cudaFree(h->d_blob) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
+    if (h->d_partial && cudaFree(h->d_partial) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
     delete h;
     return st;
 }
@@ -825,6 +896,8 @@ sd2_status sd2_stream_check(void* cuda_stream)
                     cudaMemset(d->d_gbar, 0, kDrafterWordsBytes);
                     if (d->d_tags) cudaMemset(d->d_tags, 0, (size_t)d->tags_bytes);
                 }
+            for (sd2_handle h : g_live)
+                if (h->device == dev && h->d_partial) cudaMemset(h->d_partial, 0, (size_t)h->partial_bytes);
         }
         cudaGetLastError();
         return SD2_ERR_TIMEOUT;

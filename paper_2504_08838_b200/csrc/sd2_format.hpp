@@ -612,7 +612,7 @@ inline int check_header(const uint8_t* blob, int64_t bytes, BlobHeader& h, bool 
     if (bytes < (int64_t)sizeof(BlobHeader)) return -6;
     std::memcpy(&h, blob, sizeof h);
     if (std::memcmp(h.magic, "SD2BLOB2", 8) != 0 || h.version != 2) return -6;
-    if (h.format != (uint32_t)kFormatBitmask && h.format != (uint32_t)kFormatGap4) return -6;
+    if (h.format != (uint32_t)kFormatBitmask && h.format != (uint32_t)kFormatGap4 && h.format != 4u /* GAP4_MMA */) return -6;
     if (h.y_dtype > 1 || h.n_sections != 3) return -6;
     if (h.M < 1 || h.K < 1 || h.nnz < 0 || h.nnz > h.M * h.K) return -6;
     if (h.total_bytes != bytes) return -6;

@@ -1,0 +1,402 @@
+// Tensor-core path of libsd2 for panels of activation rows (GAP4_MMA handles).
+//
+// Y[n, m] = sum over kept k of W[m, k] X[n, k] for N <= 64 rows per launch.  With that many rows
+// the product is worth a dense contraction: the compressed weights still cross HBM once, but
+// instead of gathering activations entry by entry, a CTA expands each 128 x 128 block of W into
+// shared memory as a dense bf16 operand tile and lets tcgen05.mma multiply it with the matching
+// 128 columns of X; the fp32 sums live in tensor memory.  One persistent CTA per SM:
+//
+//   warp 4        producer: one bulk asynchronous copy per block record, global -> ring
+//   warps 6..21   two groups of 256 threads; a group zero-fills its operand tile, fetches its
+//                 X columns (cp.async into the swizzled B layout) and scatters the block's
+//                 values: a thread walks one piece of the block, positions are running sums of
+//                 4-bit gaps and are byte offsets in the tile already (see sd2_format_mma.hpp)
+//   warp 5        one thread issues the eight K = 16 tcgen05.mma of a block and commits them to
+//                 the mbarriers that hand the tile back and, at a row panel's end, the sums over
+//   warps 0..3    read the sums out of tensor memory (tcgen05.ld, one 32-lane quarter each)
+//
+// Blocks are dealt to the CTAs in contiguous runs, so a row panel's K range is usually shared by
+// several CTAs: each adds its part into the handle's fp32 partial-sum buffer with red.add, and
+// the CTA that brings the panel's block count to KC rounds, writes Y and clears the buffer.
+// Every wait is bounded; a wait that runs out sets the error word and the CTA leaves in order
+// (copies drained, tensor memory returned).
+
+#pragma once
+
+#include "sd2_format_mma.hpp"
+#include "sd2_kernels.cuh"
+
+namespace sd2 {
+
+constexpr int kMmaMaxRows = 64;                     // activation rows of one launch
+constexpr int kMmaGroups = 2;                       // expanding groups = operand tiles in flight
+constexpr int kMmaGroupThreads = kMmaPieces;        // a thread per piece
+constexpr int kMmaEpiWarps = 4;
+constexpr int kMmaProducerWarp = 4;
+constexpr int kMmaIssueWarp = 5;
+constexpr int kMmaFirstGroupWarp = 6;
+constexpr int kMmaThreads = 32 * kMmaFirstGroupWarp + kMmaGroups * kMmaGroupThreads;   // 704
+constexpr int kMmaSlots = 8;                        // most ring slots
+constexpr int kMmaTileBytes = kMmaBlockRows * kMmaBlockCols * 2;                       // 32 KiB
+constexpr int kMmaTmemCols = 2 * kMmaMaxRows;       // two accumulator stages of up to 64 columns
+constexpr int kMmaStepBytes = 4 * kMmaPieces + 16 * kMmaPieces;                        // a full step
+
+struct MmaArgs {
+    const uint32_t* dir;     // block directory (16-byte units into recs)
+    const uint8_t* recs;     // block records
+    const uint16_t* X;       // [N, K] bf16
+    void* Y;                 // [N, M] bf16 or fp32
+    float* partial;          // [kMmaMaxRows, P * 128] fp32, zero on entry and on exit
+    unsigned int* done;      // [P] blocks of each row panel accounted for, zero on entry and on exit
+    int M, K, N, npad;       // npad: N rounded up to a multiple of 16
+    int P, KC;               // row panels, blocks per panel
+    long long NB;            // P * KC
+    int y_f32;
+    int slot_bytes, n_slots; // ring geometry
+    int x_vec;               // 1: rows of X can be fetched in 16-byte pieces (K % 8 == 0, X 16-byte aligned)
+    int* err;
+    long long budget;        // clock cycles a wait may take
+};
+
+struct MmaShared {
+    unsigned long long full[kMmaSlots];     // block record landed
+    unsigned long long empty[kMmaSlots];    // block record expanded
+    unsigned long long a_full[kMmaGroups];  // operand tile and X columns ready
+    unsigned long long a_empty[kMmaGroups]; // the MMAs that read them have completed
+    unsigned long long acc_full[2];         // a row panel's sums are complete in tensor memory
+    unsigned long long acc_empty[2];        // ... and have been read out
+    unsigned long long drain;               // exit: nothing of ours is left in the tensor pipe
+    uint32_t tmem_base;
+    int abort_flag;
+    int last_flag;
+    int never_flag;                         // stays 0: the exit waits must not be cut short by abort_flag
+};
+
+__device__ __forceinline__ void sts_u16(uint32_t a, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ void sts_zero16(uint32_t a)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+}
+// 16 bytes global -> shared, of which only the first `src_bytes` are read (the rest is zero-filled)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// writes of this thread through the generic proxy become visible to the asynchronous proxy (the tensor core)
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// c + 2 * byte K8 of p
+template <int K8>
+__device__ __forceinline__ uint32_t byte_times_2_plus(uint32_t p, uint32_t c)
+{
+    uint32_t d;
+    asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(p), "r"(0x2u << (8 * K8)), "r"(c));
+    return d;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile under the 128-byte swizzle: rows of 128
+// bytes, groups of eight rows 1024 bytes apart.  Stepping K by 16 elements inside the 64-column
+// atom adds 32 bytes to the start address.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
+{
+    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                             // leading byte offset (not used by swizzled K-major tiles)
+    d |= (uint64_t)(1024 >> 4) << 32;                   // stride byte offset: eight rows
+    d |= (uint64_t)1 << 46;                             // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                             // 128-byte swizzle
+    return d;
+}
+
+// D[128 x npad] (+)= A[128 x 16] B[npad x 16]^T, bf16 in, fp32 out, both operands K-major in shared memory
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the mbarrier gets one arrival when every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;     // swizzled tiles want 1024-byte alignment
+    const uint32_t xbytes = (uint32_t)a.npad * 256u;                 // two atoms of npad rows x 128 bytes
+    const uint32_t abuf0 = base;
+    const uint32_t xbuf0 = base + kMmaGroups * kMmaTileBytes;
+    const uint32_t ring0 = xbuf0 + kMmaGroups * xbytes;
+    MmaShared* sh = (MmaShared*)(smem_raw + (ring0 - smem_u32(smem_raw)) + (size_t)a.n_slots * a.slot_bytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long b0 = a.NB * (long long)blockIdx.x / gridDim.x;
+    const long long b1 = a.NB * (long long)(blockIdx.x + 1) / gridDim.x;
+    const int nblk = (int)(b1 - b0);
+    const WaitCtx wc = {&sh->abort_flag, a.budget};
+
+    if (tid == 0) {
+        for (int i = 0; i < kMmaSlots; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->empty[i]), kMmaGroupThreads / 32);
+        }
+        for (int g = 0; g < kMmaGroups; ++g) {
+            mbar_init(smem_u32(&sh->a_full[g]), kMmaGroupThreads / 32);
+            mbar_init(smem_u32(&sh->a_empty[g]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&sh->acc_full[s]), 1);
+            mbar_init(smem_u32(&sh->acc_empty[s]), kMmaEpiWarps);
+        }
+        mbar_init(smem_u32(&sh->drain), 1);
+        sh->abort_flag = 0;
+        sh->last_flag = 0;
+        sh->never_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows of the X tiles beyond N are never fetched: they stay zero for the whole launch
+    for (uint32_t o = (uint32_t)tid * 16u; o < kMmaGroups * xbytes; o += kMmaThreads * 16u) sts_zero16(xbuf0 + o);
+    if (warp == kMmaIssueWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(kMmaTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *(volatile uint32_t*)&sh->tmem_base;
+
+    if (warp == kMmaProducerWarp) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0) {
+            int issued = 0;
+            uint32_t o_next = nblk > 0 ? __ldg(a.dir + b0) : 0u;
+            for (int i = 0; i < nblk; ++i) {
+                const uint32_t o0 = o_next;
+                o_next = __ldg(a.dir + b0 + i + 1);
+                const uint32_t bytes = (o_next - o0) * 16u;
+                const int slot = i % a.n_slots;
+                const uint32_t round = (uint32_t)(i / a.n_slots);
+                if (!wait_phase(smem_u32(&sh->empty[slot]), (round & 1u) ^ 1u, wc)) break;
+                const uint32_t fb = smem_u32(&sh->full[slot]);
+                mbar_expect_tx(fb, bytes);
+                bulk_g2s(ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes, a.recs + (size_t)o0 * 16, bytes, fb);
+                issued = i + 1;
+            }
+            if (sh->abort_flag) {
+                // leave nothing in flight: every copy issued into a slot's latest round must have landed
+                for (int i = issued > a.n_slots ? issued - a.n_slots : 0; i < issued; ++i)
+                    wait_phase(smem_u32(&sh->full[i % a.n_slots]), (uint32_t)(i / a.n_slots) & 1u, WaitCtx{&sh->never_flag, a.budget});
+            }
+        }
+    } else if (warp == kMmaIssueWarp) {
+        // ---------------------------------------------------------------- MMA issue
+        if (lane == 0) {
+            // instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = npad, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.npad >> 3) << 17) | ((128u >> 4) << 24);
+            int seg = 0;
+            bool ok = true;
+            for (int i = 0; i < nblk && ok; ++i) {
+                const int g = i % kMmaGroups;
+                const uint32_t use = (uint32_t)(i / kMmaGroups);
+                const long long b = b0 + i;
+                const int kc = (int)(b % a.KC);
+                const bool first = i == 0 || kc == 0;
+                const bool last = i == nblk - 1 || kc == a.KC - 1;
+                const int stage = seg & 1;
+                if (first) {
+                    ok = wait_phase(smem_u32(&sh->acc_empty[stage]), (((uint32_t)seg >> 1) & 1u) ^ 1u, wc);
+                    if (!ok) break;
+                }
+                ok = wait_phase(smem_u32(&sh->a_full[g]), use & 1u, wc);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t at = abuf0 + (uint32_t)g * kMmaTileBytes, xt = xbuf0 + (uint32_t)g * xbytes;
+                const uint32_t d = tmem + (uint32_t)stage * kMmaMaxRows;
+#pragma unroll
+                for (int kk = 0; kk < kMmaBlockCols / 16; ++kk) {
+                    const uint64_t ad = umma_desc_sw128(at + (uint32_t)(kk >> 2) * (kMmaTileBytes / 2) + (uint32_t)(kk & 3) * 32u);
+                    const uint64_t bd = umma_desc_sw128(xt + (uint32_t)(kk >> 2) * (xbytes / 2) + (uint32_t)(kk & 3) * 32u);
+                    umma_bf16(d, ad, bd, idesc, (first && kk == 0) ? 0u : 1u);
+                }
+                umma_commit(smem_u32(&sh->a_empty[g]));
+                if (last) {
+                    umma_commit(smem_u32(&sh->acc_full[stage]));
+                    ++seg;
+                }
+            }
+        }
+    } else if (warp < kMmaEpiWarps) {
+        // ---------------------------------------------------------------- epilogue
+        const int et = tid;                                  // 0..127: row of the panel
+        const size_t mpad = (size_t)a.P * kMmaBlockRows;
+        int seg = 0;
+        bool dead = false;   // a wait ran out: no more work, but every named barrier below is still attended
+        for (int i = 0; i < nblk;) {
+            const long long b = b0 + i;
+            const int p = (int)(b / a.KC), kc = (int)(b % a.KC);
+            const int nseg = min(nblk - i, a.KC - kc);
+            const int stage = seg & 1;
+            const int row = p * kMmaBlockRows + et;
+            const bool whole = nseg == a.KC;                 // this CTA had the panel's whole K range
+            if (!dead && !wait_phase(smem_u32(&sh->acc_full[stage]), ((uint32_t)seg >> 1) & 1u, wc)) dead = true;
+            dead = __any_sync(0xFFFFFFFFu, dead);            // the warp stays together: tcgen05.ld is warp-wide
+            if (!dead) {
+                tc_fence_after();
+                const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)stage * kMmaMaxRows;
+                for (int c0 = 0; c0 < a.npad; c0 += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)c0, r);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int n = c0 + j;
+                        if (n < a.N && row < a.M) {
+                            const float v = __uint_as_float(r[j]);
+                            if (!whole) atomicAdd(a.partial + (size_t)n * mpad + row, v);
+                            else if (a.y_f32) ((float*)a.Y)[(size_t)n * a.M + row] = v;
+                            else ((uint16_t*)a.Y)[(size_t)n * a.M + row] = f32_to_bf16_rne(v);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[stage]));
+            }
+            if (!whole) {
+                __threadfence();
+                named_bar_sync(1, 32 * kMmaEpiWarps);
+                if (et == 0) {
+                    int lastone = 0;
+                    if (!dead) {
+                        const unsigned int old = atomicAdd(a.done + p, (unsigned int)nseg);
+                        lastone = (old + (unsigned int)nseg == (unsigned int)a.KC) ? 1 : 0;
+                    }
+                    sh->last_flag = lastone;
+                }
+                named_bar_sync(1, 32 * kMmaEpiWarps);
+                if (sh->last_flag) {
+                    __threadfence();
+                    if (row < a.M) {
+                        for (int n = 0; n < a.N; ++n) {
+                            float* ps = a.partial + (size_t)n * mpad + row;
+                            const float v = __ldcg(ps);
+                            *ps = 0.f;
+                            if (a.y_f32) ((float*)a.Y)[(size_t)n * a.M + row] = v;
+                            else ((uint16_t*)a.Y)[(size_t)n * a.M + row] = f32_to_bf16_rne(v);
+                        }
+                    }
+                    if (et == 0) a.done[p] = 0u;
+                }
+                named_bar_sync(1, 32 * kMmaEpiWarps);        // last_flag is rewritten by the next segment
+            }
+            ++seg;
+            i += nseg;
+        }
+    } else {
+        // ---------------------------------------------------------------- expanding groups
+        const int g = (warp - kMmaFirstGroupWarp) / (kMmaGroupThreads / 32);
+        const int t = tid - 32 * kMmaFirstGroupWarp - g * kMmaGroupThreads;      // the piece this thread walks
+        const uint32_t at = abuf0 + (uint32_t)g * kMmaTileBytes, xt = xbuf0 + (uint32_t)g * xbytes;
+        bool dead = false;   // a wait ran out: no more work, but the group's barrier is still attended
+        for (int i = g; i < nblk; i += kMmaGroups) {
+            const uint32_t use = (uint32_t)(i / kMmaGroups);
+            if (!dead && !wait_phase(smem_u32(&sh->a_empty[g]), (use & 1u) ^ 1u, wc)) dead = true;
+            dead = __any_sync(0xFFFFFFFFu, dead);            // the warp stays together
+            if (dead) {
+                named_bar_sync(2 + g, kMmaGroupThreads);
+                continue;
+            }
+            // the block's 128 columns of X, rows < N, into the swizzled B tile
+            const int k0 = (int)((b0 + i) % a.KC) * kMmaBlockCols;
+            if (a.x_vec) {
+                for (int q = t; q < a.N * 16; q += kMmaGroupThreads) {
+                    const int n = q >> 4, ch = q & 15;
+                    const int kcol = k0 + ch * 8;
+                    const uint32_t dst = xt + (uint32_t)(ch >> 3) * (xbytes / 2) + (uint32_t)n * 128u + (uint32_t)(((ch & 7) ^ (n & 7)) << 4);
+                    if (kcol < a.K) cp_async16(dst, a.X + (size_t)n * a.K + kcol, 16u);   // K % 8 == 0: a piece is inside or outside
+                    else sts_zero16(dst);
+                }
+            } else {
+                for (int q = t; q < a.N * kMmaBlockCols; q += kMmaGroupThreads) {
+                    const int n = q >> 7, c = q & 127;
+                    const uint32_t v = (k0 + c < a.K) ? (uint32_t)a.X[(size_t)n * a.K + k0 + c] : 0u;
+                    sts_u16(xt + (uint32_t)(c >> 6) * (xbytes / 2) + (uint32_t)n * 128u + (uint32_t)(((((c & 63) >> 3) ^ (n & 7)) << 4) | ((c & 7) << 1)), v);
+                }
+            }
+            // a clean tile: kept entries are scattered into zeros
+#pragma unroll
+            for (int j = 0; j < kMmaTileBytes / (16 * kMmaGroupThreads); ++j) sts_zero16(at + (uint32_t)(j * kMmaGroupThreads + t) * 16u);
+            named_bar_sync(2 + g, kMmaGroupThreads);
+
+            const int slot = i % a.n_slots;
+            if (!wait_phase(smem_u32(&sh->full[slot]), (uint32_t)(i / a.n_slots) & 1u, wc)) dead = true;
+            dead = __any_sync(0xFFFFFFFFu, dead);
+            if (dead) continue;
+            const uint32_t rec = ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes;
+            const int cpp = (int)lds_u32(rec + 4u), nfull = (int)lds_u32(rec + 8u);
+            const int nt = t < nfull ? cpp : cpp - 1;
+            uint32_t cur = at + 2u * lds_u16(rec + 16u + 2u * (uint32_t)t);
+            uint32_t w = rec + (uint32_t)kMmaBlockHeaderBytes;
+            for (int j = 0; j < nt; ++j) {
+                const uint32_t tj = j < cpp - 1 ? (uint32_t)kMmaPieces : (uint32_t)nfull;
+                const uint32_t code = lds_u32(w + 4u * (uint32_t)t);
+                const uint4 v = lds_v4(w + ((4u * tj + 15u) & ~15u) + 16u * (uint32_t)t);
+                const uint32_t lo = code & 0x0F0F0F0Fu, hi = (code >> 4) & 0x0F0F0F0Fu;
+                const uint32_t po = (lo + hi) * 0x01010101u;        // byte k: gaps summed through entry 2k + 1
+                const uint32_t pe = po - hi;                       // byte k: ... through entry 2k
+                const uint32_t a0 = byte_times_2_plus<0>(pe, cur), a1 = byte_times_2_plus<0>(po, cur);
+                const uint32_t a2 = byte_times_2_plus<1>(pe, cur), a3 = byte_times_2_plus<1>(po, cur);
+                const uint32_t a4 = byte_times_2_plus<2>(pe, cur), a5 = byte_times_2_plus<2>(po, cur);
+                const uint32_t a6 = byte_times_2_plus<3>(pe, cur), a7 = byte_times_2_plus<3>(po, cur);
+                sts_u16(a0, v.x); sts_u16(a1, v.x >> 16);
+                sts_u16(a2, v.y); sts_u16(a3, v.y >> 16);
+                sts_u16(a4, v.z); sts_u16(a5, v.z >> 16);
+                sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
+                cur = a7;
+                w += ((4u * tj + 15u) & ~15u) + 16u * tj;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot]));
+            cp_async_wait_all();
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->a_full[g]));
+        }
+        cp_async_wait_all();
+    }
+
+    // ---------------------------------------------------------------- exit
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaIssueWarp) {
+        if (sh->abort_flag && lane == 0) {
+            // MMAs may still be running on tiles and columns that are about to go away
+            umma_commit(smem_u32(&sh->drain));
+            wait_phase(smem_u32(&sh->drain), 0u, WaitCtx{&sh->never_flag, a.budget});
+        }
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kMmaTmemCols) : "memory");
+    }
+    if (tid == 0 && sh->abort_flag && a.err) atomicExch(a.err, 1);
+}
+
+}  // namespace sd2

@@ -200,3 +200,20 @@ def test_unaligned_activation_pointer():
     Yr, S = oracle.masked_linear(W, mask, X)
     check(Y.cpu().numpy().astype(np.float64), Yr, S, True)
     sd2.sd2_free(h)
+
+
+@pytest.mark.parametrize("M,K", synth.SWEEP_SHAPES + [(1024, 3072)])
+@pytest.mark.parametrize("N", [16, 32, 64])
+def test_mma_path_full_size_shapes(M, K, N):
+    # the tensor-core path on the sweep shapes (two of them are 3B-block matrices) and on the 3B k/v shape, 50 % sparsity
+    W, mask = synth.make_linear(5, 1, 0, M, K, 0.5)
+    X = synth.make_activations(5, 1, 0, N, K)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32)
+    Y = torch.full((N, M), float("nan"), dtype=torch.float32, device="cuda")
+    sd2.sd2_spmm(h, dev_bf16(X), Y)
+    sd2.sd2_stream_check()
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(Y.cpu().numpy().astype(np.float64), Yr, S, True)
+    if N == 16:
+        assert np.array_equal(sd2.sd2_decompress(h), oracle.roundtrip_ref(W, mask))
+    sd2.sd2_free(h)

@@ -551,3 +551,77 @@ def test_drafter_step_in_several_panels_with_k_8192():
     for hs in blocks:
         for h in hs:
             sd2.sd2_free(h)
+
+
+# ---- GAP4_MMA: blocks expanded in shared memory, multiplied on the tensor cores ------------------
+
+def _mma_case(seed, M, K, d, N, f32):
+    W, mask, X = case(seed, M, K, d, N)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32 if f32 else sd2.SD2_DTYPE_BF16)
+    assert h.format == sd2.SD2_FORMAT_GAP4_MMA and h.nnz == int(mask.sum())
+    Yr, S = oracle.masked_linear(W, mask, X)
+    y = run_spmm(h, X, f32)
+    check(y, Yr, S, f32)
+    return h, W, mask
+
+
+@pytest.mark.parametrize("M,K,d,N", [(128, 128, 0.5, 16), (128, 256, 0.5, 64), (130, 264, 0.5, 16), (300, 1000, 0.1, 17),
+                                     (256, 2048, 0.5, 32), (1000, 520, 0.9, 48), (64, 4099, 0.5, 16), (257, 129, 1.0, 5),
+                                     (2048, 512, 0.5, 1), (40, 24, 0.02, 64)])
+@pytest.mark.parametrize("f32", [True, False])
+def test_mma_path_matches_oracle(M, K, d, N, f32):
+    h, W, mask = _mma_case(9000 + M + K + N, M, K, d, N, f32)
+    assert np.array_equal(sd2.sd2_decompress(h), oracle.roundtrip_ref(W, mask))
+    sd2.sd2_free(h)
+
+
+def test_mma_path_more_than_64_rows_and_repeated_calls():
+    # 150 rows: three launches of at most 64; a second call must find the partial sums clean
+    M, K, N = 384, 1024, 150
+    W, mask, X = case(9100, M, K, 0.5, N)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    for _ in range(3):
+        check(run_spmm(h, X, True), Yr, S, True)
+    sd2.sd2_free(h)
+
+
+def test_mma_path_integer_exact():
+    # small integers: every partial sum is exact in fp32, so any summation order gives the same bits
+    M, K, N = 200, 1536, 32
+    W = synth.integer_bf16(9200, (M, K), -8, 8)
+    X = synth.integer_bf16(9201, (N, K), -8, 8)
+    mask = synth.bernoulli_mask(9202, (M, K), 0.5)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32)
+    Yr, _ = oracle.masked_linear(W, mask, X)
+    y = run_spmm(h, X, True)
+    assert np.array_equal(y, Yr)
+    sd2.sd2_free(h)
+
+
+def test_mma_path_one_hot_rows_pick_single_weights():
+    # X = rows of the identity: Y[n, m] is W[m, n] where kept, 0 elsewhere, exactly
+    M, K = 130, 160
+    W, mask, _ = case(9300, M, K, 0.5, 1)
+    N = 64
+    X = np.zeros((N, K), np.uint16)
+    cols = [(37 * n + 5) % K for n in range(N)]
+    for n, c in enumerate(cols):
+        X[n, c] = 0x3F80
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_BF16)
+    y = run_spmm(h, X, False)
+    ref = synth.bf16_bits_to_f32(oracle.roundtrip_ref(W, mask)).astype(np.float64)
+    for n, c in enumerate(cols):
+        assert np.array_equal(y[n], ref[:, c])
+    sd2.sd2_free(h)
+
+
+def test_mma_handles_are_not_block_step_material():
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 1)
+    lin = synth.make_block(2, 0, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4_MMA) for W, m in lin]
+    with pytest.raises(sd2.Sd2Error) as e:
+        sd2.sd2_drafter_create([hs], n_max=1)
+    assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
+    for h in hs:
+        sd2.sd2_free(h)
