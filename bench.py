@@ -58,6 +58,7 @@ def parse_args():
                     help="silu(g)*u of the fused dense cuBLAS arm: vllm's silu_and_mul kernel (one launch), one torch.compile'd "
                          "kernel, or two eager elementwise launches; auto = vllm's if it loads, else eager")
     ap.add_argument("--quick", action="store_true", help="sweep: first shape only")
+    ap.add_argument("--sweep-both", action="store_true", help="sweep: time both formats at every N (default: GAP4 below 16 rows, GAP4_MMA from 16)")
     ap.add_argument("--sparsity", type=float, default=0.5)
     ap.add_argument("--mask", default="bernoulli", choices=["bernoulli", "magnitude", "2:4"],
                     help="mask recipe; 2:4 keeps two of every four columns (sparsity is then 0.5)")
@@ -680,18 +681,23 @@ def run_sweep(args):
     ns = [int(v) for v in args.sweep_n.split(",")]
     shapes = synth.SWEEP_SHAPES[:1] if args.quick else synth.SWEEP_SHAPES
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    print("| M x K | N | sparsity | B / kept weight | sparse us | sparse GB/s | dense us | dense / sparse |")
-    print("|---|---|---|---|---|---|---|---|")
+    print("| M x K | N | sparsity | path | B / kept weight | sparse us | sparse GB/s | dense us | dense / sparse |")
+    print("|---|---|---|---|---|---|---|---|---|")
     summary = []
     for (M, K) in shapes:
         W = synth.normal_bf16(synth.stream_seed(5, 0, 0, synth.WHAT_W) + M, (M, K), 0.02)
         cross = {n: [] for n in ns}
         for sp in sparsities:
             mask = synth.bernoulli_mask(synth.stream_seed(5, 0, 0, synth.WHAT_MASK) + M + int(1000 * sp), (M, K), 1.0 - sp)
-            blob = sd2.sd2_pack_host(W, mask, sd2.SD2_FORMAT_AUTO, sd2.SD2_DTYPE_BF16)
-            h0 = sd2.sd2_load_blob(blob)
-            R = max(2, int(np.ceil(4.0 * l2 / h0.compressed_bytes)))
-            hs = [h0] + [sd2.sd2_load_blob(blob) for _ in range(R - 1)]
+            # two handles per matrix: GAP4 (gathers, N < 16) and GAP4_MMA (tensor cores, N >= 16)
+            loaded = {}
+            for name, fmt in (("gap4", sd2.SD2_FORMAT_AUTO), ("mma", sd2.SD2_FORMAT_GAP4_MMA)):
+                if (name == "gap4" and min(ns) >= 16 and not args.sweep_both) or (name == "mma" and max(ns) < 16 and not args.sweep_both):
+                    continue
+                blob = sd2.sd2_pack_host(W, mask, fmt, sd2.SD2_DTYPE_BF16)
+                h0 = sd2.sd2_load_blob(blob)
+                R = max(2, int(np.ceil(4.0 * l2 / h0.compressed_bytes)))
+                loaded[name] = [h0] + [sd2.sd2_load_blob(blob) for _ in range(R - 1)]
             Wd0 = torch.from_numpy(np.where(mask != 0, W, np.uint16(0)).view(np.int16)).cuda().view(torch.bfloat16)
             Rd = max(2, int(np.ceil(4.0 * l2 / (2 * M * K))))
             Wd = [Wd0] + [Wd0.clone() for _ in range(Rd - 1)]
@@ -699,21 +705,31 @@ def run_sweep(args):
                 X = torch.from_numpy(synth.make_activations(5, 0, 0, N, K).view(np.int16).copy()).cuda().view(torch.bfloat16)
                 Y = torch.zeros((N, M), dtype=torch.bfloat16, device="cuda")
 
-                def sparse_all():
-                    for h in hs:
-                        sd2.sd2_spmm(h, X, Y)
-
                 def dense_all():
                     for w in Wd:
                         torch.matmul(X, w.t(), out=Y)
 
-                us_s = time_graph_us(torch, sparse_all, 20) / R
                 us_d = time_graph_us(torch, dense_all, 20) / Rd
-                cross[N].append((sp, us_s, us_d))
-                print("| %dx%d | %d | %.2f | %.3f | %.2f | %.0f | %.2f | %.2f |" % (
-                    M, K, N, sp, h0.compressed_bytes / max(h0.nnz, 1), us_s, h0.compressed_bytes / us_s / 1e3, us_d, us_d / us_s), flush=True)
-            for h in hs:
-                sd2.sd2_free(h)
+                paths = [p for p in (("mma", "gap4") if N >= 16 else ("gap4", "mma")) if p in loaded]
+                if not args.sweep_both:
+                    paths = paths[:1]
+                best = None
+                for path in paths:
+                    hs = loaded[path]
+
+                    def sparse_all():
+                        for h in hs:
+                            sd2.sd2_spmm(h, X, Y)
+
+                    us_s = time_graph_us(torch, sparse_all, 20) / len(hs)
+                    best = us_s if best is None else min(best, us_s)
+                    print("| %dx%d | %d | %.2f | %s | %.3f | %.2f | %.0f | %.2f | %.2f |" % (
+                        M, K, N, sp, path, hs[0].compressed_bytes / max(hs[0].nnz, 1), us_s, hs[0].compressed_bytes / us_s / 1e3,
+                        us_d, us_d / us_s), flush=True)
+                cross[N].append((sp, best, us_d))
+            for hs in loaded.values():
+                for h in hs:
+                    sd2.sd2_free(h)
             del Wd, Wd0
             torch.cuda.empty_cache()
         for N in ns:

@@ -498,6 +498,42 @@ sd2_status run_program(SArgs& a, int dev, int64_t N, const ProgramNeeds& needs, 
 }
 
 // Shared by sd2_spmm and sd2_spmm_fused (and by block steps that mix formats).
+// cuTensorMapEncodeTiled through the runtime (no link against the driver library).  NULL: not available.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn()
+{
+    static std::atomic<void*> cached{nullptr};
+    static std::atomic<int> tried{0};
+    if (!tried.load()) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            fn = nullptr;
+        }
+        cached.store(fn);
+        tried.store(1);
+    }
+    return (EncodeTiledFn)cached.load();
+}
+
+// Tensor map over X [N, K] bf16 whose boxes are 64 columns x npad rows, stored with the 128-byte swizzle;
+// what a box reaches beyond N rows or K columns is filled with zeros.  false: X cannot be described
+// (unaligned base or row pitch), the kernel's groups fetch it themselves.
+bool make_x_map(CUtensorMap* map, const uint16_t* X, int64_t N, int64_t K, int npad)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc || (((uintptr_t)X) & 15) || (K & 7) || K < kMmaBlockCols) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kMmaBlockCols, (cuuint32_t)npad};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)X, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // GAP4_MMA: one launch per 64 activation rows; each expands the blocks in shared memory and multiplies on the
 // tensor cores.
 sd2_status run_mma(sd2_handle h, const uint16_t* x, void* Y, int64_t N, bool y_force_bf16, int dev, cudaStream_t s)
@@ -524,14 +560,17 @@ sd2_status run_mma(sd2_handle h, const uint16_t* x, void* Y, int64_t N, bool y_f
         a.npad = (a.N + 15) & ~15;
         a.X = x + n0 * h->K;
         a.Y = (char*)Y + (size_t)n0 * (size_t)h->M * esz;
+        CUtensorMap xmap;
+        std::memset(&xmap, 0, sizeof xmap);
+        a.x_tma = make_x_map(&xmap, a.X, a.N, h->K, a.npad) ? 1 : 0;
         a.x_vec = ((h->K & 7) == 0 && (((uintptr_t)a.X) & 15) == 0) ? 1 : 0;
-        const int fixed = 1024 + kMmaGroups * kMmaTileBytes + kMmaGroups * a.npad * 256 + (int)((sizeof(MmaShared) + 127) & ~127);
+        const int fixed = 1024 + kMmaStages * kMmaTileBytes + kMmaStages * a.npad * 128 + (int)((sizeof(MmaShared) + 127) & ~127);
         int slots = (kSmemMax - fixed) / a.slot_bytes;
         if (slots < 1) return SD2_ERR_UNSUPPORTED;
         if (slots > kMmaSlots) slots = kMmaSlots;
         a.n_slots = slots;
         const int smem = fixed + slots * a.slot_bytes;
-        mma_kernel<<<grid, kMmaThreads, smem, s>>>(a);
+        mma_kernel<<<grid, kMmaThreads, smem, s>>>(a, xmap);
         if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
     }
     return SD2_OK;

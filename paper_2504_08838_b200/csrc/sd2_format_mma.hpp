@@ -5,12 +5,12 @@
 // block of the matrix decodes straight into the shared-memory image that a tcgen05.mma
 // instruction reads as its A operand, with no address arithmetic beyond a running sum.
 //
-//   - W is cut into blocks of 128 rows x 128 columns (edge blocks are padded with absent
+//   - W is cut into blocks of 128 rows x 64 columns (edge blocks are padded with absent
 //     entries).  Blocks are numbered row panel by row panel, ascending columns inside a panel.
 //   - Inside a block an entry (r, c) has the *operand position*
-//         pos(r, c) = (c / 64) * 8192 + r * 64 + ((((c % 64) / 8) ^ (r % 8)) * 8) + c % 8
-//     which is half its byte offset in a K-major bf16 tile of two 128-row x 64-column atoms
-//     under the 128-byte swizzle (16-byte chunk index XOR row mod 8); pos < 16384.
+//         pos(r, c) = r * 64 + (((c / 8) ^ (r % 8)) * 8) + c % 8
+//     which is half its byte offset in a K-major bf16 tile of 128 rows x 64 columns (rows of
+//     128 bytes) under the 128-byte swizzle (16-byte chunk index XOR row mod 8); pos < 8192.
 //   - The block's kept entries, ascending in pos, become one list of (gap, value) entries: a
 //     cursor starts at 0; an entry at position p is coded as g = p - cursor in [0, 15] and
 //     moves the cursor to p.  When the next kept position is more than 15 ahead, a filler
@@ -19,11 +19,11 @@
 //     entry with gap 0 (the same value written twice to the same place); an empty block has
 //     no entries at all.  Eight consecutive entries form a chunk: one 32-bit code word
 //     (nibble i = gap of entry i) and 16 bytes of values.
-//   - The chunks are dealt to 256 *pieces* in order: with n chunks, cpp = ceil(n / 256), the
-//     first nfull = n - 256 (cpp - 1) pieces take cpp chunks each, the others cpp - 1.  A
+//   - The chunks are dealt to 128 *pieces* in order: with n chunks, cpp = ceil(n / 128), the
+//     first nfull = n - 128 (cpp - 1) pieces take cpp chunks each, the others cpp - 1.  A
 //     piece is what one thread expands; start[t] is the cursor before the piece's first entry.
 //   - Storage is step-major: step j holds chunk j of every piece that has more than j
-//     chunks (all 256 for j < cpp - 1, the first nfull for j = cpp - 1): their code words,
+//     chunks (all 128 for j < cpp - 1, the first nfull for j = cpp - 1): their code words,
 //     padded to 16 bytes, then their values.
 //
 //   blob    sec0  block_off  u32[NB+1]   start of each block record in sec1, in 16-byte units
@@ -31,7 +31,7 @@
 //           (sec2 is empty)
 //
 //   block record   u32 n_chunks, u32 cpp, u32 nfull, u32 n_kept (entries that are not fillers)
-//                  u16 start[256]
+//                  u16 start[128]
 //                  per step: u32 code[T_j] (pad to 16 bytes), u16 val[8 * T_j]
 //
 // Fillers and repeats are not counted in nnz; their bytes are part of "compressed bytes".
@@ -44,24 +44,23 @@ namespace sd2 {
 
 constexpr int kFormatGap4Mma = 4;
 constexpr int kMmaBlockRows = 128;
-constexpr int kMmaBlockCols = 128;
-constexpr int kMmaPieces = 256;
+constexpr int kMmaBlockCols = 64;
+constexpr int kMmaPieces = 128;
+constexpr int kMmaTilePositions = kMmaBlockRows * kMmaBlockCols;
 constexpr int kMmaBlockHeaderBytes = 16 + 2 * kMmaPieces;
 
-// Operand position of entry (r, c) of a block, r and c in [0, 128).
+// Operand position of entry (r, c) of a block, r in [0, 128), c in [0, 64).
 SD2_HD int mma_operand_pos(int r, int c)
 {
-    const int cc = c & 63;
-    return (c >> 6) * 8192 + r * 64 + ((((cc >> 3) ^ (r & 7)) << 3) | (cc & 7));
+    return r * 64 + ((((c >> 3) ^ (r & 7)) << 3) | (c & 7));
 }
 
 // Inverse of mma_operand_pos.
 SD2_HD void mma_operand_rc(int pos, int* r, int* c)
 {
-    const int atom = pos >> 13, in = pos & 8191;
-    const int row = in >> 6, chunk = ((in >> 3) & 7) ^ (row & 7);
+    const int row = pos >> 6, chunk = ((pos >> 3) & 7) ^ (row & 7);
     *r = row;
-    *c = atom * 64 + chunk * 8 + (in & 7);
+    *c = chunk * 8 + (pos & 7);
 }
 
 // Bytes of the steps of a block with n chunks.
@@ -83,8 +82,8 @@ inline PackResult pack_gap4_mma(const uint16_t* W, const uint8_t* mask, int64_t 
     if (NB > 0x3FFFFFFF) { res.status = -2; return res; }
     std::vector<uint32_t> dir((size_t)NB + 1);
     std::vector<uint8_t> recs;
-    std::vector<uint16_t> byval(16384);
-    std::vector<uint8_t> present(16384);
+    std::vector<uint16_t> byval(kMmaTilePositions);
+    std::vector<uint8_t> present(kMmaTilePositions);
     std::vector<uint8_t> gaps;
     std::vector<uint16_t> vals;
     int64_t nnz = 0, chunks_total = 0;
@@ -109,7 +108,7 @@ inline PackResult pack_gap4_mma(const uint16_t* W, const uint8_t* mask, int64_t 
             gaps.clear();
             vals.clear();
             int cursor = 0;
-            for (int pos = 0; pos < 16384; ++pos) {
+            for (int pos = 0; pos < kMmaTilePositions; ++pos) {
                 if (!present[(size_t)pos]) continue;
                 while (pos - cursor > 15) {
                     cursor += 15;
@@ -209,7 +208,7 @@ inline int unpack_gap4_mma(const BlobHeader& h, const uint8_t* blob, uint16_t* d
         uint32_t head[4];
         std::memcpy(head, rec, 16);
         const int64_t n = head[0], cpp = head[1], nfull = head[2];
-        if (n > 16384 / 8 + 16384 / 15 / 8 + 2) return -6;
+        if (n > kMmaTilePositions / 8 + kMmaTilePositions / 15 / 8 + 2) return -6;
         if (cpp != (n + kMmaPieces - 1) / kMmaPieces) return -6;
         if (nfull != (n ? n - (int64_t)kMmaPieces * (cpp - 1) : 0)) return -6;
         if (rec_bytes != kMmaBlockHeaderBytes + mma_steps_bytes(n)) return -6;
@@ -231,7 +230,7 @@ inline int unpack_gap4_mma(const BlobHeader& h, const uint8_t* blob, uint16_t* d
                 for (int i = 0; i < 8; ++i, ++entry) {
                     const int g = (int)((cw >> (4 * i)) & 15u);
                     const int pos = cursor + g;
-                    if (pos >= 16384) return -6;
+                    if (pos >= kMmaTilePositions) return -6;
                     if (g == 0 && entry > 0) {
                         if (val[i] != prev_val) return -6;  // a repeat rewrites what is already there
                     } else {

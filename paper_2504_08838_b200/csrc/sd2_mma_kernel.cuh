@@ -2,26 +2,33 @@
 //
 // Y[n, m] = sum over kept k of W[m, k] X[n, k] for N <= 64 rows per launch.  With that many rows
 // the product is worth a dense contraction: the compressed weights still cross HBM once, but
-// instead of gathering activations entry by entry, a CTA expands each 128 x 128 block of W into
+// instead of gathering activations entry by entry, a CTA expands each 128 x 64 block of W into
 // shared memory as a dense bf16 operand tile and lets tcgen05.mma multiply it with the matching
-// 128 columns of X; the fp32 sums live in tensor memory.  One persistent CTA per SM:
+// 64 columns of X; the fp32 sums live in tensor memory.  One persistent CTA per SM:
 //
-//   warp 4        producer: one bulk asynchronous copy per block record, global -> ring
-//   warps 6..21   two groups of 256 threads; a group zero-fills its operand tile, fetches its
-//                 X columns (cp.async into the swizzled B layout) and scatters the block's
-//                 values: a thread walks one piece of the block, positions are running sums of
-//                 4-bit gaps and are byte offsets in the tile already (see sd2_format_mma.hpp)
-//   warp 5        one thread issues the eight K = 16 tcgen05.mma of a block and commits them to
-//                 the mbarriers that hand the tile back and, at a row panel's end, the sums over
+//   warp 4        producer: per block one bulk asynchronous copy of its record (global -> ring)
+//                 and one tensor-map copy of its X columns, which arrive in shared memory in the
+//                 swizzled K-major layout the B operand needs (rows beyond N and columns beyond
+//                 K are filled with zeros by the copy engine)
+//   warps 6..21   four groups of 128 threads take the blocks in turn; a group zero-fills the
+//                 operand tile of the block's stage and scatters the block's values into it: a
+//                 thread walks one piece of the block, positions are running sums of 4-bit gaps
+//                 and are byte offsets in the tile already (see sd2_format_mma.hpp)
+//   warp 5        one thread issues the four K = 16 tcgen05.mma of a block, in block order, and
+//                 commits them to the mbarriers that free the stage and, at a row panel's end,
+//                 hand the sums over
 //   warps 0..3    read the sums out of tensor memory (tcgen05.ld, one 32-lane quarter each)
 //
-// Blocks are dealt to the CTAs in contiguous runs, so a row panel's K range is usually shared by
-// several CTAs: each adds its part into the handle's fp32 partial-sum buffer with red.add, and
-// the CTA that brings the panel's block count to KC rounds, writes Y and clears the buffer.
-// Every wait is bounded; a wait that runs out sets the error word and the CTA leaves in order
-// (copies drained, tensor memory returned).
+// Six stages (operand tile + X columns) are in flight, so a group never waits for the MMAs of
+// the block it has just expanded.  Blocks are dealt to the CTAs in contiguous runs, so a row
+// panel's K range is usually shared by several CTAs: each adds its part into the handle's fp32
+// partial-sum buffer with red.add, and the CTA that brings the panel's block count to KC rounds,
+// writes Y and clears the buffer.  Every wait is bounded; a wait that runs out sets the error
+// word and the CTA leaves in order (copies drained, tensor memory returned).
 
 #pragma once
+
+#include <cuda.h>
 
 #include "sd2_format_mma.hpp"
 #include "sd2_kernels.cuh"
@@ -29,17 +36,17 @@
 namespace sd2 {
 
 constexpr int kMmaMaxRows = 64;                     // activation rows of one launch
-constexpr int kMmaGroups = 2;                       // expanding groups = operand tiles in flight
+constexpr int kMmaGroups = 4;                       // expanding groups
 constexpr int kMmaGroupThreads = kMmaPieces;        // a thread per piece
+constexpr int kMmaStages = 6;                       // operand tiles (and X column sets) in flight
 constexpr int kMmaEpiWarps = 4;
 constexpr int kMmaProducerWarp = 4;
 constexpr int kMmaIssueWarp = 5;
 constexpr int kMmaFirstGroupWarp = 6;
 constexpr int kMmaThreads = 32 * kMmaFirstGroupWarp + kMmaGroups * kMmaGroupThreads;   // 704
-constexpr int kMmaSlots = 8;                        // most ring slots
-constexpr int kMmaTileBytes = kMmaBlockRows * kMmaBlockCols * 2;                       // 32 KiB
+constexpr int kMmaSlots = 12;                       // most ring slots
+constexpr int kMmaTileBytes = kMmaBlockRows * kMmaBlockCols * 2;                       // 16 KiB
 constexpr int kMmaTmemCols = 2 * kMmaMaxRows;       // two accumulator stages of up to 64 columns
-constexpr int kMmaStepBytes = 4 * kMmaPieces + 16 * kMmaPieces;                        // a full step
 
 struct MmaArgs {
     const uint32_t* dir;     // block directory (16-byte units into recs)
@@ -53,23 +60,25 @@ struct MmaArgs {
     long long NB;            // P * KC
     int y_f32;
     int slot_bytes, n_slots; // ring geometry
-    int x_vec;               // 1: rows of X can be fetched in 16-byte pieces (K % 8 == 0, X 16-byte aligned)
+    int x_tma;               // 1: the producer fetches X through the tensor map; 0: the groups fetch it
+    int x_vec;               // x_tma == 0: rows of X can be fetched in 16-byte pieces
     int* err;
     long long budget;        // clock cycles a wait may take
 };
 
 struct MmaShared {
-    unsigned long long full[kMmaSlots];     // block record landed
-    unsigned long long empty[kMmaSlots];    // block record expanded
-    unsigned long long a_full[kMmaGroups];  // operand tile and X columns ready
-    unsigned long long a_empty[kMmaGroups]; // the MMAs that read them have completed
-    unsigned long long acc_full[2];         // a row panel's sums are complete in tensor memory
-    unsigned long long acc_empty[2];        // ... and have been read out
-    unsigned long long drain;               // exit: nothing of ours is left in the tensor pipe
+    unsigned long long full[kMmaSlots];       // block record landed
+    unsigned long long empty[kMmaSlots];      // block record expanded
+    unsigned long long a_full[kMmaStages];    // operand tile ready
+    unsigned long long x_full[kMmaStages];    // X columns landed (tensor-map copies)
+    unsigned long long st_empty[kMmaStages];  // the MMAs that read the stage have completed
+    unsigned long long acc_full[2];           // a row panel's sums are complete in tensor memory
+    unsigned long long acc_empty[2];          // ... and have been read out
+    unsigned long long drain;                 // exit: nothing of ours is left in the tensor pipe
     uint32_t tmem_base;
     int abort_flag;
     int last_flag;
-    int never_flag;                         // stays 0: the exit waits must not be cut short by abort_flag
+    int never_flag;                           // stays 0: the exit waits must not be cut short by abort_flag
 };
 
 __device__ __forceinline__ void sts_u16(uint32_t a, uint32_t v)
@@ -138,14 +147,22 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
+// one box of the tensor map (64 columns x npad rows of X, swizzled) -> shared memory
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(map), "r"(bar), "r"(c0), "r"(c1)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap xmap)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;     // swizzled tiles want 1024-byte alignment
-    const uint32_t xbytes = (uint32_t)a.npad * 256u;                 // two atoms of npad rows x 128 bytes
+    const uint32_t xbytes = (uint32_t)a.npad * 128u;                 // npad rows x 128 bytes
     const uint32_t abuf0 = base;
-    const uint32_t xbuf0 = base + kMmaGroups * kMmaTileBytes;
-    const uint32_t ring0 = xbuf0 + kMmaGroups * xbytes;
+    const uint32_t xbuf0 = base + kMmaStages * kMmaTileBytes;
+    const uint32_t ring0 = xbuf0 + kMmaStages * xbytes;
     MmaShared* sh = (MmaShared*)(smem_raw + (ring0 - smem_u32(smem_raw)) + (size_t)a.n_slots * a.slot_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -159,9 +176,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
             mbar_init(smem_u32(&sh->full[i]), 1);
             mbar_init(smem_u32(&sh->empty[i]), kMmaGroupThreads / 32);
         }
-        for (int g = 0; g < kMmaGroups; ++g) {
+        for (int g = 0; g < kMmaStages; ++g) {
             mbar_init(smem_u32(&sh->a_full[g]), kMmaGroupThreads / 32);
-            mbar_init(smem_u32(&sh->a_empty[g]), 1);
+            mbar_init(smem_u32(&sh->x_full[g]), 1);
+            mbar_init(smem_u32(&sh->st_empty[g]), 1);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&sh->acc_full[s]), 1);
@@ -173,8 +191,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
         sh->never_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // rows of the X tiles beyond N are never fetched: they stay zero for the whole launch
-    for (uint32_t o = (uint32_t)tid * 16u; o < kMmaGroups * xbytes; o += kMmaThreads * 16u) sts_zero16(xbuf0 + o);
+    if (!a.x_tma)   // rows of the X tiles beyond N are never fetched by the groups: they stay zero for the whole launch
+        for (uint32_t o = (uint32_t)tid * 16u; o < kMmaStages * xbytes; o += kMmaThreads * 16u) sts_zero16(xbuf0 + o);
     if (warp == kMmaIssueWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(kMmaTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -187,7 +205,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
     if (warp == kMmaProducerWarp) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
-            int issued = 0;
+            int issued = 0, x_issued = 0;
             uint32_t o_next = nblk > 0 ? __ldg(a.dir + b0) : 0u;
             for (int i = 0; i < nblk; ++i) {
                 const uint32_t o0 = o_next;
@@ -200,11 +218,22 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
                 mbar_expect_tx(fb, bytes);
                 bulk_g2s(ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes, a.recs + (size_t)o0 * 16, bytes, fb);
                 issued = i + 1;
+                if (a.x_tma) {
+                    const int st = i % kMmaStages;
+                    if (!wait_phase(smem_u32(&sh->st_empty[st]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) break;
+                    const uint32_t xb = smem_u32(&sh->x_full[st]);
+                    mbar_expect_tx(xb, xbytes);
+                    tma_load_2d(xbuf0 + (uint32_t)st * xbytes, &xmap, (int)((b0 + i) % a.KC) * kMmaBlockCols, 0, xb);
+                    x_issued = i + 1;
+                }
             }
             if (sh->abort_flag) {
-                // leave nothing in flight: every copy issued into a slot's latest round must have landed
+                // leave nothing in flight: every copy issued into a slot's or stage's latest round must have landed
+                const WaitCtx wx = {&sh->never_flag, a.budget};
                 for (int i = issued > a.n_slots ? issued - a.n_slots : 0; i < issued; ++i)
-                    wait_phase(smem_u32(&sh->full[i % a.n_slots]), (uint32_t)(i / a.n_slots) & 1u, WaitCtx{&sh->never_flag, a.budget});
+                    wait_phase(smem_u32(&sh->full[i % a.n_slots]), (uint32_t)(i / a.n_slots) & 1u, wx);
+                for (int i = x_issued > kMmaStages ? x_issued - kMmaStages : 0; i < x_issued; ++i)
+                    wait_phase(smem_u32(&sh->x_full[i % kMmaStages]), (uint32_t)(i / kMmaStages) & 1u, wx);
             }
         }
     } else if (warp == kMmaIssueWarp) {
@@ -213,31 +242,24 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
             // instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = npad, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.npad >> 3) << 17) | ((128u >> 4) << 24);
             int seg = 0;
-            bool ok = true;
-            for (int i = 0; i < nblk && ok; ++i) {
-                const int g = i % kMmaGroups;
-                const uint32_t use = (uint32_t)(i / kMmaGroups);
-                const long long b = b0 + i;
-                const int kc = (int)(b % a.KC);
+            for (int i = 0; i < nblk; ++i) {
+                const int st = i % kMmaStages;
+                const uint32_t use = (uint32_t)(i / kMmaStages);
+                const int kc = (int)((b0 + i) % a.KC);
                 const bool first = i == 0 || kc == 0;
                 const bool last = i == nblk - 1 || kc == a.KC - 1;
                 const int stage = seg & 1;
-                if (first) {
-                    ok = wait_phase(smem_u32(&sh->acc_empty[stage]), (((uint32_t)seg >> 1) & 1u) ^ 1u, wc);
-                    if (!ok) break;
-                }
-                ok = wait_phase(smem_u32(&sh->a_full[g]), use & 1u, wc);
-                if (!ok) break;
+                if (first && !wait_phase(smem_u32(&sh->acc_empty[stage]), (((uint32_t)seg >> 1) & 1u) ^ 1u, wc)) break;
+                if (!wait_phase(smem_u32(&sh->a_full[st]), use & 1u, wc)) break;
+                if (a.x_tma && !wait_phase(smem_u32(&sh->x_full[st]), use & 1u, wc)) break;
                 tc_fence_after();
-                const uint32_t at = abuf0 + (uint32_t)g * kMmaTileBytes, xt = xbuf0 + (uint32_t)g * xbytes;
+                const uint32_t at = abuf0 + (uint32_t)st * kMmaTileBytes, xt = xbuf0 + (uint32_t)st * xbytes;
                 const uint32_t d = tmem + (uint32_t)stage * kMmaMaxRows;
 #pragma unroll
-                for (int kk = 0; kk < kMmaBlockCols / 16; ++kk) {
-                    const uint64_t ad = umma_desc_sw128(at + (uint32_t)(kk >> 2) * (kMmaTileBytes / 2) + (uint32_t)(kk & 3) * 32u);
-                    const uint64_t bd = umma_desc_sw128(xt + (uint32_t)(kk >> 2) * (xbytes / 2) + (uint32_t)(kk & 3) * 32u);
-                    umma_bf16(d, ad, bd, idesc, (first && kk == 0) ? 0u : 1u);
-                }
-                umma_commit(smem_u32(&sh->a_empty[g]));
+                for (int kk = 0; kk < kMmaBlockCols / 16; ++kk)
+                    umma_bf16(d, umma_desc_sw128(at + (uint32_t)kk * 32u), umma_desc_sw128(xt + (uint32_t)kk * 32u), idesc,
+                              (first && kk == 0) ? 0u : 1u);
+                umma_commit(smem_u32(&sh->st_empty[st]));
                 if (last) {
                     umma_commit(smem_u32(&sh->acc_full[stage]));
                     ++seg;
@@ -293,14 +315,22 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
                 }
                 named_bar_sync(1, 32 * kMmaEpiWarps);
                 if (sh->last_flag) {
+                    // every part of the panel is in: round, write Y, leave the buffer clean (loads in batches of 8)
                     __threadfence();
                     if (row < a.M) {
-                        for (int n = 0; n < a.N; ++n) {
-                            float* ps = a.partial + (size_t)n * mpad + row;
-                            const float v = __ldcg(ps);
-                            *ps = 0.f;
-                            if (a.y_f32) ((float*)a.Y)[(size_t)n * a.M + row] = v;
-                            else ((uint16_t*)a.Y)[(size_t)n * a.M + row] = f32_to_bf16_rne(v);
+                        for (int n0 = 0; n0 < a.N; n0 += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] = (n0 + j < a.N) ? __ldcg(a.partial + (size_t)(n0 + j) * mpad + row) : 0.f;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int n = n0 + j;
+                                if (n < a.N) {
+                                    a.partial[(size_t)n * mpad + row] = 0.f;
+                                    if (a.y_f32) ((float*)a.Y)[(size_t)n * a.M + row] = v[j];
+                                    else ((uint16_t*)a.Y)[(size_t)n * a.M + row] = f32_to_bf16_rne(v[j]);
+                                }
+                            }
                         }
                     }
                     if (et == 0) a.done[p] = 0u;
@@ -314,31 +344,32 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
         // ---------------------------------------------------------------- expanding groups
         const int g = (warp - kMmaFirstGroupWarp) / (kMmaGroupThreads / 32);
         const int t = tid - 32 * kMmaFirstGroupWarp - g * kMmaGroupThreads;      // the piece this thread walks
-        const uint32_t at = abuf0 + (uint32_t)g * kMmaTileBytes, xt = xbuf0 + (uint32_t)g * xbytes;
         bool dead = false;   // a wait ran out: no more work, but the group's barrier is still attended
         for (int i = g; i < nblk; i += kMmaGroups) {
-            const uint32_t use = (uint32_t)(i / kMmaGroups);
-            if (!dead && !wait_phase(smem_u32(&sh->a_empty[g]), (use & 1u) ^ 1u, wc)) dead = true;
+            const int st = i % kMmaStages;
+            const uint32_t at = abuf0 + (uint32_t)st * kMmaTileBytes, xt = xbuf0 + (uint32_t)st * xbytes;
+            if (!dead && !wait_phase(smem_u32(&sh->st_empty[st]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) dead = true;
             dead = __any_sync(0xFFFFFFFFu, dead);            // the warp stays together
             if (dead) {
                 named_bar_sync(2 + g, kMmaGroupThreads);
                 continue;
             }
-            // the block's 128 columns of X, rows < N, into the swizzled B tile
-            const int k0 = (int)((b0 + i) % a.KC) * kMmaBlockCols;
-            if (a.x_vec) {
-                for (int q = t; q < a.N * 16; q += kMmaGroupThreads) {
-                    const int n = q >> 4, ch = q & 15;
-                    const int kcol = k0 + ch * 8;
-                    const uint32_t dst = xt + (uint32_t)(ch >> 3) * (xbytes / 2) + (uint32_t)n * 128u + (uint32_t)(((ch & 7) ^ (n & 7)) << 4);
-                    if (kcol < a.K) cp_async16(dst, a.X + (size_t)n * a.K + kcol, 16u);   // K % 8 == 0: a piece is inside or outside
-                    else sts_zero16(dst);
-                }
-            } else {
-                for (int q = t; q < a.N * kMmaBlockCols; q += kMmaGroupThreads) {
-                    const int n = q >> 7, c = q & 127;
-                    const uint32_t v = (k0 + c < a.K) ? (uint32_t)a.X[(size_t)n * a.K + k0 + c] : 0u;
-                    sts_u16(xt + (uint32_t)(c >> 6) * (xbytes / 2) + (uint32_t)n * 128u + (uint32_t)(((((c & 63) >> 3) ^ (n & 7)) << 4) | ((c & 7) << 1)), v);
+            if (!a.x_tma) {
+                // the block's 64 columns of X, rows < N, into the swizzled B tile
+                const int k0 = (int)((b0 + i) % a.KC) * kMmaBlockCols;
+                if (a.x_vec) {
+                    for (int q = t; q < a.N * 8; q += kMmaGroupThreads) {
+                        const int n = q >> 3, ch = q & 7;
+                        const uint32_t dst = xt + (uint32_t)n * 128u + (uint32_t)((ch ^ (n & 7)) << 4);
+                        if (k0 + ch * 8 < a.K) cp_async16(dst, a.X + (size_t)n * a.K + k0 + ch * 8, 16u);   // K % 8 == 0
+                        else sts_zero16(dst);
+                    }
+                } else {
+                    for (int q = t; q < a.N * kMmaBlockCols; q += kMmaGroupThreads) {
+                        const int n = q >> 6, c = q & 63;
+                        const uint32_t v = (k0 + c < a.K) ? (uint32_t)a.X[(size_t)n * a.K + k0 + c] : 0u;
+                        sts_u16(xt + (uint32_t)n * 128u + (uint32_t)((((c >> 3) ^ (n & 7)) << 4) | ((c & 7) << 1)), v);
+                    }
                 }
             }
             // a clean tile: kept entries are scattered into zeros
@@ -375,10 +406,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a)
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot]));
-            cp_async_wait_all();
+            if (!a.x_tma) cp_async_wait_all();
             fence_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->a_full[g]));
+            if (lane == 0) mbar_arrive(smem_u32(&sh->a_full[st]));
         }
         cp_async_wait_all();
     }

@@ -1,7 +1,7 @@
 """GAP4_MMA on the host: lossless, and its records expand into the tensor-core operand tile.
 
 No GPU needed.  The second half walks a packed blob the way the kernel's threads do (same
-integer arithmetic, restated here on numpy scalars) and reads the resulting 32 KiB tile back
+integer arithmetic, restated here on numpy scalars) and reads the resulting 16 KiB tile back
 through the textbook description of a K-major tile under the 128-byte swizzle: if the encoder's
 position order, the gap sums or the piece starts were off, the tile would not be W.*mask.
 """
@@ -67,17 +67,17 @@ def test_corrupt_blob_is_rejected():
 
 
 def _expand_like_the_kernel(rec: bytes) -> np.ndarray:
-    """One block record -> the 32 KiB operand tile, thread by thread as mma_kernel's groups do."""
-    tile = np.zeros(32768, np.uint8)
+    """One block record -> the 16 KiB operand tile, thread by thread as mma_kernel's groups do."""
+    tile = np.zeros(16384, np.uint8)
     n, cpp, nfull, _ = struct.unpack_from("<4I", rec, 0)
-    start = np.frombuffer(rec, np.uint16, 256, 16)
+    start = np.frombuffer(rec, np.uint16, 128, 16)
     u32 = lambda v: v & 0xFFFFFFFF
-    for t in range(256):
+    for t in range(128):
         nt = cpp if t < nfull else cpp - 1
         cur = 2 * int(start[t])
-        w = 16 + 512
+        w = 16 + 256
         for j in range(nt):
-            tj = 256 if j < cpp - 1 else nfull
+            tj = 128 if j < cpp - 1 else nfull
             code = struct.unpack_from("<I", rec, w + 4 * t)[0]
             vals = struct.unpack_from("<8H", rec, w + ((4 * tj + 15) & ~15) + 16 * t)
             lo, hi = code & 0x0F0F0F0F, (code >> 4) & 0x0F0F0F0F
@@ -96,16 +96,15 @@ def _expand_like_the_kernel(rec: bytes) -> np.ndarray:
 
 
 def _read_k_major_sw128(tile: np.ndarray) -> np.ndarray:
-    """The 128 x 128 bf16 matrix a K-major, 128-byte-swizzled tile of two 64-column atoms holds:
-    row r of an atom is 128 bytes at r * 128, groups of eight rows are 1024 bytes apart, and the
-    16-byte chunk c of a row is stored at chunk index c XOR (r mod 8)."""
-    out = np.zeros((128, 128), np.uint16)
+    """The 128 x 64 bf16 matrix a K-major, 128-byte-swizzled tile holds: row r is 128 bytes at
+    r * 128 (groups of eight rows are 1024 bytes apart), and the 16-byte chunk c of a row is
+    stored at chunk index c XOR (r mod 8)."""
+    out = np.zeros((128, 64), np.uint16)
     t16 = tile.view(np.uint16)
-    for atom in range(2):
-        for r in range(128):
-            for chunk in range(8):
-                src = atom * 8192 + r * 64 + ((chunk ^ (r & 7)) * 8)
-                out[r, atom * 64 + chunk * 8: atom * 64 + chunk * 8 + 8] = t16[src:src + 8]
+    for r in range(128):
+        for chunk in range(8):
+            src = r * 64 + ((chunk ^ (r & 7)) * 8)
+            out[r, chunk * 8: chunk * 8 + 8] = t16[src:src + 8]
     return out
 
 
@@ -114,7 +113,7 @@ def test_records_expand_into_the_operand_tile(M, K, d):
     W, mask = _case(77 + M, M, K, d)
     blob = sd2.sd2_pack_host(W, mask, FMT)
     sec_off = struct.unpack_from("<4Q", blob, 64)
-    P, KC = (M + 127) // 128, (K + 127) // 128
+    P, KC = (M + 127) // 128, (K + 63) // 64
     dirv = np.frombuffer(blob, np.uint32, P * KC + 1, sec_off[0])
     ref = oracle.roundtrip_ref(W, mask)
     for p in range(P):
@@ -122,7 +121,7 @@ def test_records_expand_into_the_operand_tile(M, K, d):
             b = p * KC + kc
             rec = blob[sec_off[1] + 16 * int(dirv[b]): sec_off[1] + 16 * int(dirv[b + 1])]
             got = _read_k_major_sw128(_expand_like_the_kernel(rec))
-            want = np.zeros((128, 128), np.uint16)
-            blk = ref[p * 128:(p + 1) * 128, kc * 128:(kc + 1) * 128]
+            want = np.zeros((128, 64), np.uint16)
+            blk = ref[p * 128:(p + 1) * 128, kc * 64:(kc + 1) * 64]
             want[:blk.shape[0], :blk.shape[1]] = blk
             assert np.array_equal(got, want), (p, kc)
