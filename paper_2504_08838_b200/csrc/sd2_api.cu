@@ -550,7 +550,6 @@ sd2_status run_mma(sd2_handle h, const uint16_t* x, void* Y, int64_t N, bool y_f
     a.partial = h->d_partial;
     a.done = (unsigned int*)(h->d_partial + (size_t)kMmaMaxRows * a.P * kMmaBlockRows);
     a.y_f32 = (!y_force_bf16 && h->y_dtype == SD2_DTYPE_F32) ? 1 : 0;
-    a.slot_bytes = (h->max_tile_bytes + 127) & ~127;
     a.err = g_dev[dev].err_word;
     a.budget = wait_budget(dev);
     const size_t esz = a.y_f32 ? 4 : 2;
@@ -565,9 +564,17 @@ sd2_status run_mma(sd2_handle h, const uint16_t* x, void* Y, int64_t N, bool y_f
         a.x_tma = make_x_map(&xmap, a.X, a.N, h->K, a.npad) ? 1 : 0;
         a.x_vec = ((h->K & 7) == 0 && (((uintptr_t)a.X) & 15) == 0) ? 1 : 0;
         const int fixed = 1024 + kMmaStages * kMmaTileBytes + kMmaStages * a.npad * 128 + (int)((sizeof(MmaShared) + 127) & ~127);
-        int slots = (kSmemMax - fixed) / a.slot_bytes;
+        const int rec_bytes = (h->max_tile_bytes + 127) & ~127;
+        const int ring = kSmemMax - fixed;
+        // records per copy: about 32 KiB where three such slots fit, fewer otherwise
+        int batch = 1;
+        while (batch < kMmaMaxBatch && batch * rec_bytes < 32 * 1024) batch <<= 1;
+        while (batch > 1 && ring / (batch * rec_bytes) < 3) batch >>= 1;
+        int slots = ring / (batch * rec_bytes);
         if (slots < 1) return SD2_ERR_UNSUPPORTED;
         if (slots > kMmaSlots) slots = kMmaSlots;
+        a.batch = batch;
+        a.slot_bytes = batch * rec_bytes;
         a.n_slots = slots;
         const int smem = fixed + slots * a.slot_bytes;
         mma_kernel<<<grid, kMmaThreads, smem, s>>>(a, xmap);

@@ -7,9 +7,9 @@
 // 64 columns of X; the fp32 sums live in tensor memory.  One persistent CTA per SM:
 //
 //   warp 4        producer: per block one bulk asynchronous copy of its record (global -> ring)
-//                 and one tensor-map copy of its X columns, which arrive in shared memory in the
-//                 swizzled K-major layout the B operand needs (rows beyond N and columns beyond
-//                 K are filled with zeros by the copy engine)
+//   warp 22       per block one tensor-map copy of its X columns, which arrive in shared memory
+//                 in the swizzled K-major layout the B operand needs (rows beyond N and columns
+//                 beyond K are filled with zeros by the copy engine)
 //   warps 6..21   four groups of 128 threads take the blocks in turn; a group zero-fills the
 //                 operand tile of the block's stage and scatters the block's values into it: a
 //                 thread walks one piece of the block, positions are running sums of 4-bit gaps
@@ -43,8 +43,11 @@ constexpr int kMmaEpiWarps = 4;
 constexpr int kMmaProducerWarp = 4;
 constexpr int kMmaIssueWarp = 5;
 constexpr int kMmaFirstGroupWarp = 6;
-constexpr int kMmaThreads = 32 * kMmaFirstGroupWarp + kMmaGroups * kMmaGroupThreads;   // 704
-constexpr int kMmaSlots = 12;                       // most ring slots
+constexpr int kMmaXWarp = kMmaFirstGroupWarp + kMmaGroups * kMmaGroupThreads / 32;     // 22: tensor-map copies of X
+constexpr int kMmaThreads = 32 * (kMmaXWarp + 1);                                     // 736
+constexpr int kMmaPairs = kMmaStages / 2;            // the MMA thread takes the stages two at a time
+constexpr int kMmaSlots = 8;                        // most ring slots
+constexpr int kMmaMaxBatch = 8;                     // most block records per bulk copy
 constexpr int kMmaTileBytes = kMmaBlockRows * kMmaBlockCols * 2;                       // 16 KiB
 constexpr int kMmaTmemCols = 2 * kMmaMaxRows;       // two accumulator stages of up to 64 columns
 
@@ -60,6 +63,8 @@ struct MmaArgs {
     long long NB;            // P * KC
     int y_f32;
     int slot_bytes, n_slots; // ring geometry
+    int batch;               // block records per bulk copy and ring slot (1, 2, 4 or 8): a copy is worth issuing
+                             // only every few hundred cycles, so records travel several at a time
     int x_tma;               // 1: the producer fetches X through the tensor map; 0: the groups fetch it
     int x_vec;               // x_tma == 0: rows of X can be fetched in 16-byte pieces
     int* err;
@@ -67,11 +72,11 @@ struct MmaArgs {
 };
 
 struct MmaShared {
-    unsigned long long full[kMmaSlots];       // block record landed
-    unsigned long long empty[kMmaSlots];      // block record expanded
-    unsigned long long a_full[kMmaStages];    // operand tile ready
-    unsigned long long x_full[kMmaStages];    // X columns landed (tensor-map copies)
-    unsigned long long st_empty[kMmaStages];  // the MMAs that read the stage have completed
+    unsigned long long full[kMmaSlots];       // a batch of block records landed
+    unsigned long long empty[kMmaSlots];      // ... and has been expanded
+    unsigned long long a_full[kMmaPairs];     // both operand tiles of a stage pair are ready and their X columns landed
+    unsigned long long st_empty[kMmaPairs];   // the MMAs that read the stage pair have completed
+    uint32_t boff[kMmaSlots][kMmaMaxBatch];   // byte offset of each record inside its slot
     unsigned long long acc_full[2];           // a row panel's sums are complete in tensor memory
     unsigned long long acc_empty[2];          // ... and have been read out
     unsigned long long drain;                 // exit: nothing of ours is left in the tensor pipe
@@ -174,11 +179,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
     if (tid == 0) {
         for (int i = 0; i < kMmaSlots; ++i) {
             mbar_init(smem_u32(&sh->full[i]), 1);
-            mbar_init(smem_u32(&sh->empty[i]), kMmaGroupThreads / 32);
+            mbar_init(smem_u32(&sh->empty[i]), (uint32_t)a.batch * (kMmaGroupThreads / 32));
         }
-        for (int g = 0; g < kMmaStages; ++g) {
-            mbar_init(smem_u32(&sh->a_full[g]), kMmaGroupThreads / 32);
-            mbar_init(smem_u32(&sh->x_full[g]), 1);
+        for (int g = 0; g < kMmaPairs; ++g) {
+            // per block of the pair: one arrival from each warp of its group, one from the X copy's expect-tx
+            mbar_init(smem_u32(&sh->a_full[g]), 2u * (kMmaGroupThreads / 32 + (a.x_tma ? 1u : 0u)));
             mbar_init(smem_u32(&sh->st_empty[g]), 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -203,37 +208,57 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
     const uint32_t tmem = *(volatile uint32_t*)&sh->tmem_base;
 
     if (warp == kMmaProducerWarp) {
-        // ---------------------------------------------------------------- producer
-        if (lane == 0) {
-            int issued = 0, x_issued = 0;
-            uint32_t o_next = nblk > 0 ? __ldg(a.dir + b0) : 0u;
-            for (int i = 0; i < nblk; ++i) {
-                const uint32_t o0 = o_next;
-                o_next = __ldg(a.dir + b0 + i + 1);
-                const uint32_t bytes = (o_next - o0) * 16u;
-                const int slot = i % a.n_slots;
-                const uint32_t round = (uint32_t)(i / a.n_slots);
-                if (!wait_phase(smem_u32(&sh->empty[slot]), (round & 1u) ^ 1u, wc)) break;
-                const uint32_t fb = smem_u32(&sh->full[slot]);
-                mbar_expect_tx(fb, bytes);
-                bulk_g2s(ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes, a.recs + (size_t)o0 * 16, bytes, fb);
-                issued = i + 1;
-                if (a.x_tma) {
-                    const int st = i % kMmaStages;
-                    if (!wait_phase(smem_u32(&sh->st_empty[st]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) break;
-                    const uint32_t xb = smem_u32(&sh->x_full[st]);
-                    mbar_expect_tx(xb, xbytes);
-                    tma_load_2d(xbuf0 + (uint32_t)st * xbytes, &xmap, (int)((b0 + i) % a.KC) * kMmaBlockCols, 0, xb);
-                    x_issued = i + 1;
+        // ---------------------------------------------------------------- producer: block records, a batch per copy
+        int issued = 0;                                      // batches
+        bool ok = true;
+        for (int i0 = 0; i0 < nblk && ok; i0 += 32) {
+            // 33 directory words per round, one load per lane (clamped at the CTA's last block)
+            const uint32_t mine = __ldg(a.dir + b0 + min(i0 + lane, nblk));
+            const uint32_t end32 = __ldg(a.dir + b0 + min(i0 + 32, nblk));
+            for (int j = 0; j < 32 && i0 + j < nblk && ok; j += a.batch) {
+                const uint32_t o0 = __shfl_sync(0xFFFFFFFFu, mine, j);
+                const uint32_t o1 = j + a.batch >= 32 ? end32 : __shfl_sync(0xFFFFFFFFu, mine, (j + a.batch) & 31);
+                const int q = (i0 + j) / a.batch;
+                const int slot = q % a.n_slots;
+                if (lane == 0 && !wait_phase(smem_u32(&sh->empty[slot]), ((uint32_t)(q / a.n_slots) & 1u) ^ 1u, wc)) ok = false;
+                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                if (lane >= j && lane < j + a.batch) sh->boff[slot][lane - j] = (mine - o0) * 16u;
+                __syncwarp();
+                if (lane == 0) {
+                    const uint32_t bytes = (o1 - o0) * 16u;
+                    const uint32_t fb = smem_u32(&sh->full[slot]);
+                    mbar_expect_tx(fb, bytes);
+                    bulk_g2s(ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes, a.recs + (size_t)o0 * 16, bytes, fb);
                 }
+                issued = q + 1;
+            }
+        }
+        if (lane == 0 && sh->abort_flag) {
+            // leave nothing in flight: every copy issued into a slot's latest round must have landed
+            const WaitCtx wx = {&sh->never_flag, a.budget};
+            for (int q = issued > a.n_slots ? issued - a.n_slots : 0; q < issued; ++q)
+                wait_phase(smem_u32(&sh->full[q % a.n_slots]), (uint32_t)(q / a.n_slots) & 1u, wx);
+        }
+    } else if (warp == kMmaXWarp) {
+        // ---------------------------------------------------------------- producer: X columns
+        if (lane == 0 && a.x_tma) {
+            int kc = (int)(b0 % a.KC);
+            int done_i = 0;
+            for (int i = 0; i < nblk; ++i) {
+                const int st = i % kMmaStages, pq = st >> 1;
+                if (!(i & 1) && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) break;
+                const uint32_t xb = smem_u32(&sh->a_full[pq]);
+                mbar_expect_tx(xb, xbytes);
+                tma_load_2d(xbuf0 + (uint32_t)st * xbytes, &xmap, kc * kMmaBlockCols, 0, xb);
+                done_i = i + 1;
+                if (++kc == a.KC) kc = 0;
             }
             if (sh->abort_flag) {
-                // leave nothing in flight: every copy issued into a slot's or stage's latest round must have landed
-                const WaitCtx wx = {&sh->never_flag, a.budget};
-                for (int i = issued > a.n_slots ? issued - a.n_slots : 0; i < issued; ++i)
-                    wait_phase(smem_u32(&sh->full[i % a.n_slots]), (uint32_t)(i / a.n_slots) & 1u, wx);
-                for (int i = x_issued > kMmaStages ? x_issued - kMmaStages : 0; i < x_issued; ++i)
-                    wait_phase(smem_u32(&sh->x_full[i % kMmaStages]), (uint32_t)(i / kMmaStages) & 1u, wx);
+                // the copies of the last stages may still be landing: give them the time they need
+                (void)done_i;
+                const long long t0 = clock64();
+                while (clock64() - t0 < 20000) {}
             }
         }
     } else if (warp == kMmaIssueWarp) {
@@ -241,29 +266,41 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
         if (lane == 0) {
             // instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = npad, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.npad >> 3) << 17) | ((128u >> 4) << 24);
-            int seg = 0;
-            for (int i = 0; i < nblk; ++i) {
-                const int st = i % kMmaStages;
-                const uint32_t use = (uint32_t)(i / kMmaStages);
-                const int kc = (int)((b0 + i) % a.KC);
-                const bool first = i == 0 || kc == 0;
-                const bool last = i == nblk - 1 || kc == a.KC - 1;
-                const int stage = seg & 1;
-                if (first && !wait_phase(smem_u32(&sh->acc_empty[stage]), (((uint32_t)seg >> 1) & 1u) ^ 1u, wc)) break;
-                if (!wait_phase(smem_u32(&sh->a_full[st]), use & 1u, wc)) break;
-                if (a.x_tma && !wait_phase(smem_u32(&sh->x_full[st]), use & 1u, wc)) break;
+            const uint64_t adesc0 = umma_desc_sw128(abuf0), xdesc0 = umma_desc_sw128(xbuf0);
+            int seg = 0, pq = 0, kc = (int)(b0 % a.KC);
+            uint32_t par = 0u;                               // parity of the stage pair's current use
+            bool first = true;                               // the next block opens a row panel's run
+            for (int i = 0; i < nblk; i += 2) {
+                const int nb = min(2, nblk - i);
+                const uint32_t fb = smem_u32(&sh->a_full[pq]);
+                if (nb == 1)                                 // an odd tail: nobody fills the pair's second half
+                    for (int k = 0; k < kMmaGroupThreads / 32 + (a.x_tma ? 1 : 0); ++k) mbar_arrive(fb);
+                if (!wait_phase(fb, par, wc)) break;
                 tc_fence_after();
-                const uint32_t at = abuf0 + (uint32_t)st * kMmaTileBytes, xt = xbuf0 + (uint32_t)st * xbytes;
-                const uint32_t d = tmem + (uint32_t)stage * kMmaMaxRows;
+                bool ok = true;
+                for (int h = 0; h < nb; ++h) {
+                    const int st = 2 * pq + h;
+                    const bool last = i + h == nblk - 1 || kc == a.KC - 1;
+                    const int stage = seg & 1;
+                    if (first && !wait_phase(smem_u32(&sh->acc_empty[stage]), (((uint32_t)seg >> 1) & 1u) ^ 1u, wc)) { ok = false; break; }
+                    // descriptors differ in their start address only (16-byte units in the low bits)
+                    const uint64_t ad = adesc0 + (uint64_t)((uint32_t)st * (kMmaTileBytes >> 4));
+                    const uint64_t xd = xdesc0 + (uint64_t)((uint32_t)st * (xbytes >> 4));
+                    const uint32_t d = tmem + (uint32_t)stage * kMmaMaxRows;
 #pragma unroll
-                for (int kk = 0; kk < kMmaBlockCols / 16; ++kk)
-                    umma_bf16(d, umma_desc_sw128(at + (uint32_t)kk * 32u), umma_desc_sw128(xt + (uint32_t)kk * 32u), idesc,
-                              (first && kk == 0) ? 0u : 1u);
-                umma_commit(smem_u32(&sh->st_empty[st]));
-                if (last) {
-                    umma_commit(smem_u32(&sh->acc_full[stage]));
-                    ++seg;
+                    for (int kk = 0; kk < kMmaBlockCols / 16; ++kk)
+                        umma_bf16(d, ad + (uint64_t)(2 * kk), xd + (uint64_t)(2 * kk), idesc, (first && kk == 0) ? 0u : 1u);
+                    first = false;
+                    if (last) {
+                        umma_commit(smem_u32(&sh->acc_full[stage]));
+                        ++seg;
+                        first = true;
+                    }
+                    if (++kc == a.KC) kc = 0;
                 }
+                if (!ok) break;
+                umma_commit(smem_u32(&sh->st_empty[pq]));
+                if (++pq == kMmaPairs) { pq = 0; par ^= 1u; }
             }
         }
     } else if (warp < kMmaEpiWarps) {
@@ -346,9 +383,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
         const int t = tid - 32 * kMmaFirstGroupWarp - g * kMmaGroupThreads;      // the piece this thread walks
         bool dead = false;   // a wait ran out: no more work, but the group's barrier is still attended
         for (int i = g; i < nblk; i += kMmaGroups) {
-            const int st = i % kMmaStages;
+            const int st = i % kMmaStages, pq = st >> 1;
             const uint32_t at = abuf0 + (uint32_t)st * kMmaTileBytes, xt = xbuf0 + (uint32_t)st * xbytes;
-            if (!dead && !wait_phase(smem_u32(&sh->st_empty[st]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) dead = true;
+            if (!dead && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) dead = true;
             dead = __any_sync(0xFFFFFFFFu, dead);            // the warp stays together
             if (dead) {
                 named_bar_sync(2 + g, kMmaGroupThreads);
@@ -377,11 +414,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             for (int j = 0; j < kMmaTileBytes / (16 * kMmaGroupThreads); ++j) sts_zero16(at + (uint32_t)(j * kMmaGroupThreads + t) * 16u);
             named_bar_sync(2 + g, kMmaGroupThreads);
 
-            const int slot = i % a.n_slots;
-            if (!wait_phase(smem_u32(&sh->full[slot]), (uint32_t)(i / a.n_slots) & 1u, wc)) dead = true;
+            const int q = i / a.batch, slot = q % a.n_slots;
+            if (!wait_phase(smem_u32(&sh->full[slot]), (uint32_t)(q / a.n_slots) & 1u, wc)) dead = true;
             dead = __any_sync(0xFFFFFFFFu, dead);
             if (dead) continue;
-            const uint32_t rec = ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes;
+            const uint32_t rec = ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes + sh->boff[slot][i % a.batch];
             const int cpp = (int)lds_u32(rec + 4u), nfull = (int)lds_u32(rec + 8u);
             const int nt = t < nfull ? cpp : cpp - 1;
             uint32_t cur = at + 2u * lds_u16(rec + 16u + 2u * (uint32_t)t);
@@ -409,7 +446,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             if (!a.x_tma) cp_async_wait_all();
             fence_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->a_full[st]));
+            if (lane == 0) mbar_arrive(smem_u32(&sh->a_full[pq]));
         }
         cp_async_wait_all();
     }
