@@ -10,21 +10,22 @@
 //   warp 22       per block one tensor-map copy of its X columns, which arrive in shared memory
 //                 in the swizzled K-major layout the B operand needs (rows beyond N and columns
 //                 beyond K are filled with zeros by the copy engine)
-//   warps 6..21   four groups of 128 threads take the blocks in turn; a group zero-fills the
-//                 operand tile of the block's stage and scatters the block's values into it: a
-//                 thread walks one piece of the block, positions are running sums of 4-bit gaps
-//                 and are byte offsets in the tile already (see sd2_format_mma.hpp)
-//   warp 5        one thread issues the four K = 16 tcgen05.mma of a block, in block order, and
-//                 commits them to the mbarriers that free the stage and, at a row panel's end,
-//                 hand the sums over
+//   warps 6..21   eight teams of two warps take the blocks in turn; a team zero-fills the operand
+//                 tile of the block's stage and scatters the block's values into it: lane w of
+//                 the team's warp h walks the 16-bit half h of word column w down the rows, row
+//                 offsets are running sums of 4-bit gaps, and the 32 lanes of a store always hit
+//                 32 different banks (see sd2_format_mma.hpp)
+//   warp 5        one thread issues the four K = 16 tcgen05.mma of a block, in block order, two
+//                 blocks per barrier wait, and commits them to the mbarriers that free the
+//                 stages and, at a row panel's end, hand the sums over
 //   warps 0..3    read the sums out of tensor memory (tcgen05.ld, one 32-lane quarter each)
 //
-// Six stages (operand tile + X columns) are in flight, so a group never waits for the MMAs of
-// the block it has just expanded.  Blocks are dealt to the CTAs in contiguous runs, so a row
-// panel's K range is usually shared by several CTAs: each adds its part into the handle's fp32
-// partial-sum buffer with red.add, and the CTA that brings the panel's block count to KC rounds,
-// writes Y and clears the buffer.  Every wait is bounded; a wait that runs out sets the error
-// word and the CTA leaves in order (copies drained, tensor memory returned).
+// Six or eight stages (operand tile + X columns) are in flight, so a team never waits for the
+// MMAs of the block it has just expanded.  Blocks are dealt to the CTAs in contiguous runs, so a
+// row panel's K range is usually shared by several CTAs: each adds its part into the handle's
+// fp32 partial-sum buffer with red.add, and the CTA that brings the panel's block count to KC
+// rounds, writes Y and clears the buffer.  Every wait is bounded; a wait that runs out sets the
+// error word and the CTA leaves in order (copies drained, tensor memory returned).
 
 #pragma once
 
@@ -36,14 +37,13 @@
 namespace sd2 {
 
 constexpr int kMmaMaxRows = 64;                     // activation rows of one launch
-constexpr int kMmaGroups = 4;                       // expanding groups
-constexpr int kMmaGroupThreads = kMmaPieces;        // a thread per piece
-constexpr int kMmaStages = 6;                       // operand tiles (and X column sets) in flight
+constexpr int kMmaTeams = 8;                        // expanding teams of two warps (one per 16-bit side of the words)
+constexpr int kMmaStages = 8;                       // most operand tiles (and X column sets) in flight
 constexpr int kMmaEpiWarps = 4;
 constexpr int kMmaProducerWarp = 4;
 constexpr int kMmaIssueWarp = 5;
 constexpr int kMmaFirstGroupWarp = 6;
-constexpr int kMmaXWarp = kMmaFirstGroupWarp + kMmaGroups * kMmaGroupThreads / 32;     // 22: tensor-map copies of X
+constexpr int kMmaXWarp = kMmaFirstGroupWarp + kMmaTeams * kMmaSides;                 // 22: tensor-map copies of X
 constexpr int kMmaThreads = 32 * (kMmaXWarp + 1);                                     // 736
 constexpr int kMmaPairs = kMmaStages / 2;            // the MMA thread takes the stages two at a time
 constexpr int kMmaSlots = 8;                        // most ring slots
@@ -62,6 +62,7 @@ struct MmaArgs {
     int P, KC;               // row panels, blocks per panel
     long long NB;            // P * KC
     int y_f32;
+    int stages;              // operand tiles in flight: 6 or 8 (what shared memory allows)
     int slot_bytes, n_slots; // ring geometry
     int batch;               // block records per bulk copy and ring slot (1, 2, 4 or 8): a copy is worth issuing
                              // only every few hundred cycles, so records travel several at a time
@@ -81,6 +82,8 @@ struct MmaShared {
     unsigned long long acc_empty[2];          // ... and have been read out
     unsigned long long drain;                 // exit: nothing of ours is left in the tensor pipe
     uint32_t tmem_base;
+    uint32_t issued;                          // batches whose copy has been issued: a team looks at a slot's barrier only
+                                              // once its batch is on the way, so that a parity always means one phase
     int abort_flag;
     int last_flag;
     int never_flag;                           // stays 0: the exit waits must not be cut short by abort_flag
@@ -166,8 +169,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;     // swizzled tiles want 1024-byte alignment
     const uint32_t xbytes = (uint32_t)a.npad * 128u;                 // npad rows x 128 bytes
     const uint32_t abuf0 = base;
-    const uint32_t xbuf0 = base + kMmaStages * kMmaTileBytes;
-    const uint32_t ring0 = xbuf0 + kMmaStages * xbytes;
+    const uint32_t xbuf0 = base + (uint32_t)a.stages * kMmaTileBytes;
+    const uint32_t ring0 = xbuf0 + (uint32_t)a.stages * xbytes;
     MmaShared* sh = (MmaShared*)(smem_raw + (ring0 - smem_u32(smem_raw)) + (size_t)a.n_slots * a.slot_bytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -179,11 +182,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
     if (tid == 0) {
         for (int i = 0; i < kMmaSlots; ++i) {
             mbar_init(smem_u32(&sh->full[i]), 1);
-            mbar_init(smem_u32(&sh->empty[i]), (uint32_t)a.batch * (kMmaGroupThreads / 32));
+            mbar_init(smem_u32(&sh->empty[i]), (uint32_t)a.batch * kMmaSides);
         }
         for (int g = 0; g < kMmaPairs; ++g) {
-            // per block of the pair: one arrival from each warp of its group, one from the X copy's expect-tx
-            mbar_init(smem_u32(&sh->a_full[g]), 2u * (kMmaGroupThreads / 32 + (a.x_tma ? 1u : 0u)));
+            // per block of the pair: one arrival from each warp of its team, one from the X copy's expect-tx
+            mbar_init(smem_u32(&sh->a_full[g]), 2u * (kMmaSides + (a.x_tma ? 1u : 0u)));
             mbar_init(smem_u32(&sh->st_empty[g]), 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -192,12 +195,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
         }
         mbar_init(smem_u32(&sh->drain), 1);
         sh->abort_flag = 0;
+        sh->issued = 0u;
         sh->last_flag = 0;
         sh->never_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (!a.x_tma)   // rows of the X tiles beyond N are never fetched by the groups: they stay zero for the whole launch
-        for (uint32_t o = (uint32_t)tid * 16u; o < kMmaStages * xbytes; o += kMmaThreads * 16u) sts_zero16(xbuf0 + o);
+        for (uint32_t o = (uint32_t)tid * 16u; o < (uint32_t)a.stages * xbytes; o += kMmaThreads * 16u) sts_zero16(xbuf0 + o);
     if (warp == kMmaIssueWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(kMmaTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -230,6 +234,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
                     const uint32_t fb = smem_u32(&sh->full[slot]);
                     mbar_expect_tx(fb, bytes);
                     bulk_g2s(ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes, a.recs + (size_t)o0 * 16, bytes, fb);
+                    *(volatile uint32_t*)&sh->issued = (uint32_t)q + 1u;
                 }
                 issued = q + 1;
             }
@@ -246,8 +251,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             int kc = (int)(b0 % a.KC);
             int done_i = 0;
             for (int i = 0; i < nblk; ++i) {
-                const int st = i % kMmaStages, pq = st >> 1;
-                if (!(i & 1) && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) break;
+                const int st = i % a.stages, pq = st >> 1;
+                if (!(i & 1) && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / a.stages) & 1u) ^ 1u, wc)) break;
                 const uint32_t xb = smem_u32(&sh->a_full[pq]);
                 mbar_expect_tx(xb, xbytes);
                 tma_load_2d(xbuf0 + (uint32_t)st * xbytes, &xmap, kc * kMmaBlockCols, 0, xb);
@@ -274,7 +279,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
                 const int nb = min(2, nblk - i);
                 const uint32_t fb = smem_u32(&sh->a_full[pq]);
                 if (nb == 1)                                 // an odd tail: nobody fills the pair's second half
-                    for (int k = 0; k < kMmaGroupThreads / 32 + (a.x_tma ? 1 : 0); ++k) mbar_arrive(fb);
+                    for (int k = 0; k < kMmaSides + (a.x_tma ? 1 : 0); ++k) mbar_arrive(fb);
                 if (!wait_phase(fb, par, wc)) break;
                 tc_fence_after();
                 bool ok = true;
@@ -300,7 +305,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
                 }
                 if (!ok) break;
                 umma_commit(smem_u32(&sh->st_empty[pq]));
-                if (++pq == kMmaPairs) { pq = 0; par ^= 1u; }
+                if (++pq == (a.stages >> 1)) { pq = 0; par ^= 1u; }
             }
         }
     } else if (warp < kMmaEpiWarps) {
@@ -378,68 +383,89 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             i += nseg;
         }
     } else {
-        // ---------------------------------------------------------------- expanding groups
-        const int g = (warp - kMmaFirstGroupWarp) / (kMmaGroupThreads / 32);
-        const int t = tid - 32 * kMmaFirstGroupWarp - g * kMmaGroupThreads;      // the piece this thread walks
-        bool dead = false;   // a wait ran out: no more work, but the group's barrier is still attended
-        for (int i = g; i < nblk; i += kMmaGroups) {
-            const int st = i % kMmaStages, pq = st >> 1;
+        // ---------------------------------------------------------------- expanding teams
+        const int tm = (warp - kMmaFirstGroupWarp) >> 1, side = (warp - kMmaFirstGroupWarp) & 1;
+        const int tt = side * 32 + lane;                     // thread of the team
+        const uint32_t lt = (1u << lane) - 1u;
+        bool dead = false;   // a wait ran out: no more work, but the team's barrier is still attended
+        // block i goes to team i % stages and to stage i % stages: a stage is always refilled by the team that
+        // filled it before, so its barrier is never looked at more than one phase early (teams beyond the stage
+        // count stay idle)
+        for (int i = tm; tm < a.stages && i < nblk; i += a.stages) {
+            const int st = i % a.stages, pq = st >> 1;
             const uint32_t at = abuf0 + (uint32_t)st * kMmaTileBytes, xt = xbuf0 + (uint32_t)st * xbytes;
-            if (!dead && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / kMmaStages) & 1u) ^ 1u, wc)) dead = true;
+            if (!dead && !wait_phase(smem_u32(&sh->st_empty[pq]), ((uint32_t)(i / a.stages) & 1u) ^ 1u, wc)) dead = true;
             dead = __any_sync(0xFFFFFFFFu, dead);            // the warp stays together
             if (dead) {
-                named_bar_sync(2 + g, kMmaGroupThreads);
+                named_bar_sync(2 + tm, 64);
                 continue;
             }
             if (!a.x_tma) {
                 // the block's 64 columns of X, rows < N, into the swizzled B tile
                 const int k0 = (int)((b0 + i) % a.KC) * kMmaBlockCols;
                 if (a.x_vec) {
-                    for (int q = t; q < a.N * 8; q += kMmaGroupThreads) {
+                    for (int q = tt; q < a.N * 8; q += 64) {
                         const int n = q >> 3, ch = q & 7;
                         const uint32_t dst = xt + (uint32_t)n * 128u + (uint32_t)((ch ^ (n & 7)) << 4);
                         if (k0 + ch * 8 < a.K) cp_async16(dst, a.X + (size_t)n * a.K + k0 + ch * 8, 16u);   // K % 8 == 0
                         else sts_zero16(dst);
                     }
                 } else {
-                    for (int q = t; q < a.N * kMmaBlockCols; q += kMmaGroupThreads) {
+                    for (int q = tt; q < a.N * kMmaBlockCols; q += 64) {
                         const int n = q >> 6, c = q & 63;
                         const uint32_t v = (k0 + c < a.K) ? (uint32_t)a.X[(size_t)n * a.K + k0 + c] : 0u;
                         sts_u16(xt + (uint32_t)n * 128u + (uint32_t)((((c >> 3) ^ (n & 7)) << 4) | ((c & 7) << 1)), v);
                     }
                 }
             }
-            // a clean tile: kept entries are scattered into zeros
+            // a clean tile: kept entries are scattered into zeros (each warp clears half of the rows)
 #pragma unroll
-            for (int j = 0; j < kMmaTileBytes / (16 * kMmaGroupThreads); ++j) sts_zero16(at + (uint32_t)(j * kMmaGroupThreads + t) * 16u);
-            named_bar_sync(2 + g, kMmaGroupThreads);
+            for (int j = 0; j < kMmaTileBytes / (16 * 64); ++j) sts_zero16(at + (uint32_t)(j * 64 + tt) * 16u);
+            named_bar_sync(2 + tm, 64);
 
             const int q = i / a.batch, slot = q % a.n_slots;
-            if (!wait_phase(smem_u32(&sh->full[slot]), (uint32_t)(q / a.n_slots) & 1u, wc)) dead = true;
+            {
+                // not before the batch's copy is on its way (the slot's earlier phases are then over)
+                const long long t0 = clock64();
+                uint32_t it = 0;
+                while (*(volatile uint32_t*)&sh->issued <= (uint32_t)q) {
+                    if ((++it & 63u) == 0u && (sh->abort_flag || clock64() - t0 > a.budget)) {
+                        sh->abort_flag = 1;
+                        dead = true;
+                        break;
+                    }
+                }
+            }
+            if (!dead && !wait_phase(smem_u32(&sh->full[slot]), (uint32_t)(q / a.n_slots) & 1u, wc)) dead = true;
             dead = __any_sync(0xFFFFFFFFu, dead);
             if (dead) continue;
             const uint32_t rec = ring0 + (uint32_t)slot * (uint32_t)a.slot_bytes + sh->boff[slot][i % a.batch];
-            const int cpp = (int)lds_u32(rec + 4u), nfull = (int)lds_u32(rec + 8u);
-            const int nt = t < nfull ? cpp : cpp - 1;
-            uint32_t cur = at + 2u * lds_u16(rec + 16u + 2u * (uint32_t)t);
-            uint32_t w = rec + (uint32_t)kMmaBlockHeaderBytes;
-            for (int j = 0; j < nt; ++j) {
-                const uint32_t tj = j < cpp - 1 ? (uint32_t)kMmaPieces : (uint32_t)nfull;
-                const uint32_t code = lds_u32(w + 4u * (uint32_t)t);
-                const uint4 v = lds_v4(w + ((4u * tj + 15u) & ~15u) + 16u * (uint32_t)t);
-                const uint32_t lo = code & 0x0F0F0F0Fu, hi = (code >> 4) & 0x0F0F0F0Fu;
-                const uint32_t po = (lo + hi) * 0x01010101u;        // byte k: gaps summed through entry 2k + 1
-                const uint32_t pe = po - hi;                       // byte k: ... through entry 2k
-                const uint32_t a0 = byte_times_2_plus<0>(pe, cur), a1 = byte_times_2_plus<0>(po, cur);
-                const uint32_t a2 = byte_times_2_plus<1>(pe, cur), a3 = byte_times_2_plus<1>(po, cur);
-                const uint32_t a4 = byte_times_2_plus<2>(pe, cur), a5 = byte_times_2_plus<2>(po, cur);
-                const uint32_t a6 = byte_times_2_plus<3>(pe, cur), a7 = byte_times_2_plus<3>(po, cur);
-                sts_u16(a0, v.x); sts_u16(a1, v.x >> 16);
-                sts_u16(a2, v.y); sts_u16(a3, v.y >> 16);
-                sts_u16(a4, v.z); sts_u16(a5, v.z >> 16);
-                sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
-                cur = a7;
-                w += ((4u * tj + 15u) & ~15u) + 16u * tj;
+            const int steps = (int)lds_u16(rec + 8u + 2u * (uint32_t)side);
+            const int cnt = (int)((lds_u32(rec + 16u + 32u * (uint32_t)side + ((uint32_t)lane & ~3u)) >> (8 * (lane & 3))) & 0xFFu);
+            uint32_t w = rec + (side ? lds_u32(rec + 12u) : (uint32_t)kMmaBlockHeaderBytes);
+            uint32_t cur = at + 4u * (uint32_t)lane + 2u * (uint32_t)side;       // row 0 of this lane's piece
+            for (int j = 0; j < steps; ++j) {
+                const bool active = cnt > j;
+                const uint32_t m = __ballot_sync(0xFFFFFFFFu, active);
+                const uint32_t nj = (uint32_t)__popc(m);
+                if (active) {
+                    const uint32_t idx = (uint32_t)__popc(m & lt);
+                    const uint32_t code = lds_u32(w + 4u * idx);
+                    const uint4 v = lds_v4(w + ((4u * nj + 15u) & ~15u) + 16u * idx);
+                    const uint32_t lo = code & 0x0F0F0F0Fu, hi = (code >> 4) & 0x0F0F0F0Fu;
+                    const uint32_t po = (lo + hi) * 0x01010101u;        // byte k: gaps summed through entry 2k + 1
+                    const uint32_t pe = po - hi;                       // byte k: ... through entry 2k
+                    const uint32_t a0 = byte_times_128_plus<0>(pe, cur), a1 = byte_times_128_plus<0>(po, cur);
+                    const uint32_t a2 = byte_times_128_plus<1>(pe, cur), a3 = byte_times_128_plus<1>(po, cur);
+                    const uint32_t a4 = byte_times_128_plus<2>(pe, cur), a5 = byte_times_128_plus<2>(po, cur);
+                    const uint32_t a6 = byte_times_128_plus<3>(pe, cur), a7 = byte_times_128_plus<3>(po, cur);
+                    sts_u16(a0, v.x); sts_u16(a1, v.x >> 16);
+                    sts_u16(a2, v.y); sts_u16(a3, v.y >> 16);
+                    sts_u16(a4, v.z); sts_u16(a5, v.z >> 16);
+                    sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
+                    cur = a7;
+                }
+                w += ((4u * nj + 15u) & ~15u) + 16u * nj;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot]));

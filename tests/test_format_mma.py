@@ -54,7 +54,7 @@ def test_bytes_per_kept_weight():
     W, mask = _case(21, 512, 1024, 0.5)
     blob = sd2.sd2_pack_host(W, mask, FMT)
     _, info = sd2.sd2_unpack_host(blob, want_dense=False)
-    assert info["compressed_bytes"] / info["nnz"] < 2.60      # 2.5 + piece starts + directory + a few repeats
+    assert info["compressed_bytes"] / info["nnz"] < 2.70      # 2.5 + repeats that fill each piece's last chunk + headers
 
 
 def test_corrupt_blob_is_rejected():
@@ -67,31 +67,33 @@ def test_corrupt_blob_is_rejected():
 
 
 def _expand_like_the_kernel(rec: bytes) -> np.ndarray:
-    """One block record -> the 16 KiB operand tile, thread by thread as mma_kernel's groups do."""
+    """One block record -> the 16 KiB operand tile, lane by lane as mma_kernel's teams do."""
     tile = np.zeros(16384, np.uint8)
-    n, cpp, nfull, _ = struct.unpack_from("<4I", rec, 0)
-    start = np.frombuffer(rec, np.uint16, 128, 16)
+    n, kept, steps_packed, side1_off = struct.unpack_from("<4I", rec, 0)
+    steps = (steps_packed & 0xFFFF, steps_packed >> 16)
+    cnt = np.frombuffer(rec, np.uint8, 64, 16).reshape(2, 32)
     u32 = lambda v: v & 0xFFFFFFFF
-    for t in range(128):
-        nt = cpp if t < nfull else cpp - 1
-        cur = 2 * int(start[t])
-        w = 16 + 256
-        for j in range(nt):
-            tj = 128 if j < cpp - 1 else nfull
-            code = struct.unpack_from("<I", rec, w + 4 * t)[0]
-            vals = struct.unpack_from("<8H", rec, w + ((4 * tj + 15) & ~15) + 16 * t)
-            lo, hi = code & 0x0F0F0F0F, (code >> 4) & 0x0F0F0F0F
-            po = u32((lo + hi) * 0x01010101)
-            pe = u32(po - hi)
-            addr = []
-            for k in range(4):
-                addr.append(cur + 2 * ((pe >> (8 * k)) & 0xFF))
-                addr.append(cur + 2 * ((po >> (8 * k)) & 0xFF))
-            for i in range(8):
-                tile[addr[i]] = vals[i] & 0xFF
-                tile[addr[i] + 1] = vals[i] >> 8
-            cur = addr[7]
-            w += ((4 * tj + 15) & ~15) + 16 * tj
+    for side in range(2):
+        w = 16 + 64 if side == 0 else side1_off
+        cur = [4 * lane + 2 * side for lane in range(32)]
+        for j in range(steps[side]):
+            lanes = [lane for lane in range(32) if cnt[side, lane] > j]
+            nj = len(lanes)
+            for idx, lane in enumerate(lanes):
+                code = struct.unpack_from("<I", rec, w + 4 * idx)[0]
+                vals = struct.unpack_from("<8H", rec, w + ((4 * nj + 15) & ~15) + 16 * idx)
+                lo, hi = code & 0x0F0F0F0F, (code >> 4) & 0x0F0F0F0F
+                po = u32((lo + hi) * 0x01010101)
+                pe = u32(po - hi)
+                addr = []
+                for k in range(4):
+                    addr.append(cur[lane] + 128 * ((pe >> (8 * k)) & 0xFF))
+                    addr.append(cur[lane] + 128 * ((po >> (8 * k)) & 0xFF))
+                for i in range(8):
+                    tile[addr[i]] = vals[i] & 0xFF
+                    tile[addr[i] + 1] = vals[i] >> 8
+                cur[lane] = addr[7]
+            w += ((4 * nj + 15) & ~15) + 16 * nj
     return tile
 
 

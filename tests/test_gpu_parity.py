@@ -567,7 +567,9 @@ def _mma_case(seed, M, K, d, N, f32):
 
 @pytest.mark.parametrize("M,K,d,N", [(128, 128, 0.5, 16), (128, 256, 0.5, 64), (130, 264, 0.5, 16), (300, 1000, 0.1, 17),
                                      (256, 2048, 0.5, 32), (1000, 520, 0.9, 48), (64, 4099, 0.5, 16), (257, 129, 1.0, 5),
-                                     (2048, 512, 0.5, 1), (40, 24, 0.02, 64)])
+                                     (2048, 512, 0.5, 1), (40, 24, 0.02, 64),
+                                     # many blocks per CTA: every stage, ring slot and accumulator is reused several times
+                                     (2048, 8192, 0.5, 16), (1024, 16384, 0.7, 64), (3072, 4160, 0.3, 33)])
 @pytest.mark.parametrize("f32", [True, False])
 def test_mma_path_matches_oracle(M, K, d, N, f32):
     h, W, mask = _mma_case(9000 + M + K + N, M, K, d, N, f32)
