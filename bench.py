@@ -548,7 +548,7 @@ def run_ours(args):
                 xin = torch.zeros((N, K_), **bf).normal_()
                 yo = torch.zeros((N, M_), **bf)
                 hs_same = [handles[j // 7][j % 7] for j in same]
-                reps = max(1, 200 // len(same))
+                reps = max(5, 200 // len(same))
 
                 def ours():
                     for h in hs_same:
@@ -557,16 +557,7 @@ def run_ours(args):
                 def theirs():
                     for j in same:
                         torch.matmul(xin, dense[j].t(), out=yo)
-                out_t = []
-                for fn in (ours, theirs):
-                    fn()
-                    stream.synchronize()
-                    e0.record(stream)
-                    for _ in range(reps):
-                        fn()
-                    e1.record(stream)
-                    stream.synchronize()
-                    out_t.append(e0.elapsed_time(e1) / (reps * len(same)) * 1e3)
+                out_t = [time_graph_us(torch, fn, reps, stream) / len(same) for fn in (ours, theirs)]   # CUDA-graph replays
                 per_shape.append({"M": int(M_), "K": int(K_), "copies_cycled": len(same), "sd2_spmm_us": out_t[0],
                                   "cublas_dense_us": out_t[1], "ratio": out_t[1] / out_t[0]})
             dense_res["per_shape_single_launch"] = per_shape

@@ -20,8 +20,8 @@
 //                 stages and, at a row panel's end, hand the sums over
 //   warps 0..3    read the sums out of tensor memory (tcgen05.ld, one 32-lane quarter each)
 //
-// Six or eight stages (operand tile + X columns) are in flight, so a team never waits for the
-// MMAs of the block it has just expanded.  Blocks are dealt to the CTAs in contiguous runs, so a
+// Six stages (operand tile + X columns) are in flight, one per working team, so a team never
+// waits for the MMAs of the block it has just expanded.  Blocks are dealt to the CTAs in contiguous runs, so a
 // row panel's K range is usually shared by several CTAs: each adds its part into the handle's
 // fp32 partial-sum buffer with red.add, and the CTA that brings the panel's block count to KC
 // rounds, writes Y and clears the buffer.  Every wait is bounded; a wait that runs out sets the
