@@ -67,6 +67,9 @@ def parse_args():
     ap.add_argument("--blocks", type=int, default=0, help="override the block count (0 = the drafter's)")
     ap.add_argument("--no-dense", action="store_true", help="skip the cuBLAS dense comparison")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
+    ap.add_argument("--full-step", action="store_true",
+                    help="also time the whole decode step (glue + dense LM head around the sparse linears)")
+    ap.add_argument("--context", type=int, default=300, help="--full-step: cached positions the new token attends over")
     args = ap.parse_args()
     if args.mask == "2:4":
         args.sparsity = 0.5
@@ -323,6 +326,46 @@ def check_block0(sd2, drafter, shape, cfg_id, density, mask_kind, N, x_bits, thr
             "silu_mul_max_bf16_ulps": int(np.abs(key(t) - key(t_bits)).max()), "against": "oracle, teacher-forced"}
 
 
+ATTENTION_HEADS = {"llama-3.2-1b": (32, 8, 128256), "qwen-2.5-1.5b": (12, 2, 151936), "llama-3.2-3b": (24, 8, 128256)}
+
+
+def time_full_step(torch, sd2, args, shape, handles, harr, N, stream):
+    """Microseconds per token of a whole drafter forward pass for one new token per row (the numerator of c in
+    Eq. 3): sd2_embedding, one sd2_decoder_block_step per block, a final sd2_rmsnorm, sd2_lm_head with the greedy
+    token; captured in one CUDA graph.  Weights of the glue are seeded and dense (norm gains, embedding table
+    = LM head matrix, as in the tied Llama-3.2 models); the cache holds --context random positions."""
+    heads_q, heads_kv, vocab = ATTENTION_HEADS[shape.name]
+    blocks = len(handles)
+    hid, d = shape.hidden, shape.hidden // heads_q
+    T_max = args.context + 8
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    gains = [torch.ones(hid, **bf) for _ in range(2 * blocks + 1)]
+    table = torch.empty((vocab, hid), **bf).normal_(0.0, 0.02)
+    kcs = [torch.empty((N, T_max, heads_kv * d), **bf).normal_() for _ in range(blocks)]
+    vcs = [torch.empty((N, T_max, heads_kv * d), **bf).normal_() for _ in range(blocks)]
+    ws = torch.zeros(sd2.sd2_decoder_workspace_bytes(handles[0], N) // 2, **bf)
+    xs = [torch.zeros((N, hid), **bf) for _ in range(blocks + 2)]
+    tokens_in = torch.arange(N, dtype=torch.int32, device="cuda")
+    tokens_out = torch.zeros(N, dtype=torch.int32, device="cuda")
+    logits = torch.zeros((N, vocab), dtype=torch.float32, device="cuda")
+
+    def step():
+        sd2.sd2_embedding(tokens_in, table, xs[0])
+        for b in range(blocks):
+            sd2.sd2_decoder_block_step(handles[b], gains[2 * b], gains[2 * b + 1], xs[b], xs[b + 1], kcs[b], vcs[b], heads_q,
+                                       heads_kv, args.context, 1e-5, 500000.0, ws, handle_array=harr[b])
+        sd2.sd2_rmsnorm(xs[blocks], gains[2 * blocks], xs[blocks + 1], 1e-5)
+        sd2.sd2_lm_head(xs[blocks + 1], table, logits, tokens_out)
+
+    us = time_graph_us(torch, step, max(20, args.steps // 20), stream)
+    sd2.sd2_stream_check()
+    head_bytes = 2.0 * vocab * hid
+    return {"us_per_token": us, "launches_per_step": 10 * blocks + 4, "context": args.context, "vocab": vocab,
+            "heads": [heads_q, heads_kv, d], "lm_head_bytes": head_bytes,
+            "note": "one launch per group of linears that share an input (4 per block) and per glue operation (6 per block); "
+                    "the linears here are single-stage launches, not the one-launch drafter step timed above"}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -452,6 +495,12 @@ def run_ours(args):
         e1.record(stream)
         stream.synchronize()
         ms_stream = e0.elapsed_time(e1) / 50
+
+        # ---- the whole decode step: embedding, L decoder blocks (norms, rotary embedding, attention over a cache
+        # of --context positions, residuals around the same sparse linears), final norm, dense LM head, greedy token
+        full_step = None
+        if args.full_step and N <= 8:
+            full_step = time_full_step(torch, sd2, args, shape, handles, harr, N, stream)
 
         # ---- cuBLAS dense bf16 on the same masked weights, same chaining, same graph treatment.
         # Two arms: "fused" is what a tuned dense decoder does (q|k|v as one GEMM, gate|up as one GEMM,
@@ -626,6 +675,7 @@ def run_ours(args):
             "cpu_baseline": cpu,
             "parity": parity,
             "block_step_launches_us_per_token": ms_stream * 1e3,
+            "full_decode_step": full_step,
             "cublas_dense": dense_res,
             "cublas_dense_bf16_us_per_token": dense_res["fused_us_per_token"] if dense_res else None,
             "speedup_vs_cublas_dense": (dense_res["fused_us_per_token"] / (ms_step * 1e3)) if dense_res else None,

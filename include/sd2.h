@@ -241,6 +241,59 @@ sd2_status sd2_stream_check(void* cuda_stream);
  * kernel ends normally and the next sd2_stream_check returns SD2_ERR_TIMEOUT once.  Asynchronous. */
 sd2_status sd2_selftest_timeout(void* cuda_stream);
 
+/* ---- glue of a whole decode step (the parts of a drafter forward pass that are not sparse linears) ----
+ *
+ * The paper prunes the decoder blocks and leaves the embedding and the LM head dense (Section
+ * "Results"); a block is a self-attention module and a feed-forward module (Section "Layer
+ * pruning").  What those compute is not restated there: the calls below follow the published
+ * definitions of the Llama / Qwen family.  All tensors are device memory, bf16 bit patterns unless
+ * said otherwise, row-major; fp32 arithmetic, one rounding per output.  Asynchronous on the stream,
+ * no allocation.  Errors: INVALID_ARG (NULL pointer), SHAPE (non-positive or inconsistent sizes),
+ * UNSUPPORTED (limits named per call), CUDA. */
+
+/* y[n, :] = x[n, :] / sqrt(mean(x[n, :]^2) + eps) * w.   x, y [N*H]; w [H].  y may be x. */
+sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t H, float eps, void* cuda_stream);
+
+/* Rotary embedding of one new token per row at position `pos` (pairs (i, i + head_dim/2) of a head
+ * turn by pos * theta^(-2i/head_dim)), and the cache append: q [N, heads_q, head_dim] is rotated in
+ * place; the rotated k and the plain v ([N, heads_kv, head_dim]) are written to position `pos` of
+ * row n's cache, k_cache / v_cache [N, T_max, heads_kv, head_dim].  head_dim even, pos < T_max. */
+sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, void* v_cache, int64_t N, int64_t heads_q,
+                          int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta, void* cuda_stream);
+
+/* Grouped-query attention of one new token per row over the first T cached positions (its own
+ * included): query head h reads key/value head h / (heads_q / heads_kv); scores q.k / sqrt(head_dim),
+ * softmax over the T positions, out = sum of weights times values.  q, out [N, heads_q, head_dim].
+ * UNSUPPORTED: head_dim > 128 or T > 8192. */
+sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* v_cache, void* out, int64_t N, int64_t heads_q,
+                                int64_t heads_kv, int64_t head_dim, int64_t T, int64_t T_max, void* cuda_stream);
+
+/* y = a + b over `count` elements (residual connection).  y may be a or b. */
+sd2_status sd2_add(const void* a, const void* b, void* y, int64_t count, void* cuda_stream);
+
+/* x[n, :] = table[tokens[n], :].  tokens: device int32 [N]; table [V*H]; a token outside [0, V) gives a zero row. */
+sd2_status sd2_embedding(const int32_t* tokens, const void* table, void* x, int64_t N, int64_t V, int64_t H, void* cuda_stream);
+
+/* Dense LM head: logits[n, v] = sum over h of w_out[v, h] * x[n, h] (fp32 out, device [N*V]), and, if
+ * tokens is not NULL (device int32 [N]), the greedy token of each row: the index of the largest logit,
+ * the lowest index among equals.  w_out [V*H] bf16, 16-byte aligned.  UNSUPPORTED: H not a multiple of 8. */
+sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t* tokens, int64_t N, int64_t V, int64_t H,
+                       void* cuda_stream);
+
+/* One whole decoder block for one new token per row:
+ *     x1 = x  + Wo attention(rope(Wq n), cache + rope(Wk n), cache + Wv n),   n = rmsnorm(x,  norm_attn)
+ *     y  = x1 + Wd (silu(Wg m) * Wu m),                                        m = rmsnorm(x1, norm_ffn)
+ * h[7] = q, k, v, o, gate, up, down handles (GAP4 or BITMASK; one launch per group of linears that share
+ * an input); every intermediate is rounded to bf16.  x, y [N*hidden]; caches as in sd2_rope_cache; the
+ * block writes position `pos` of them and attends over positions 0..pos.  workspace: device, 256-byte
+ * aligned, sd2_decoder_workspace_bytes(h, N) bytes; it holds, in this order, q, k, v, o-projection,
+ * gate, up, t (offsets of sd2_block_workspace_layout), then n/m, x1, the attention output and the down
+ * projection (each rounded up to 256 bytes), which tests read back. */
+sd2_status sd2_decoder_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* bytes);
+sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, const void* norm_ffn, const void* x, void* y,
+                                  void* k_cache, void* v_cache, int64_t N, int64_t heads_q, int64_t heads_kv, int64_t pos,
+                                  int64_t T_max, float eps, double theta, void* workspace, void* cuda_stream);
+
 /* Static string for a status code. */
 const char* sd2_status_string(sd2_status s);
 

@@ -27,6 +27,8 @@ EXPORTS = [
     "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
     "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
     "sd2_block_step_static", "sd2_selftest_timeout", "sd2_drafter_query",
+    "sd2_rmsnorm", "sd2_rope_cache", "sd2_attention_decode", "sd2_add", "sd2_embedding", "sd2_lm_head",
+    "sd2_decoder_workspace_bytes", "sd2_decoder_block_step",
 ]
 
 
@@ -78,6 +80,14 @@ def lib():
             "sd2_drafter_free": [p],
             "sd2_block_step_static": [pp, p, p, i64, p],
             "sd2_selftest_timeout": [p],
+            "sd2_rmsnorm": [p, p, p, i64, i64, ctypes.c_float, p],
+            "sd2_rope_cache": [p, p, p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p],
+            "sd2_attention_decode": [p, p, p, p, i64, i64, i64, i64, i64, i64, p],
+            "sd2_add": [p, p, p, i64, p],
+            "sd2_embedding": [p, p, p, i64, i64, i64, p],
+            "sd2_lm_head": [p, p, p, p, i64, i64, i64, p],
+            "sd2_decoder_workspace_bytes": [pp, i64, pi64],
+            "sd2_decoder_block_step": [pp, p, p, p, p, p, p, i64, i64, i64, i64, i64, ctypes.c_float, ctypes.c_double, p, p],
         }
         for name, argtypes in sig.items():
             fn = getattr(L, name)
@@ -325,3 +335,56 @@ def sd2_block_step_static(hs, x, y, stream=None):
 def sd2_selftest_timeout(stream=None):
     """Launch the diagnostic whose device-side wait must run out (see ``sd2_stream_check``)."""
     _check(lib().sd2_selftest_timeout(_stream(stream)), "sd2_selftest_timeout")
+
+
+# ---- glue of a whole decode step -----------------------------------------------------------
+
+def sd2_rmsnorm(x, w, y, eps: float, stream=None):
+    N, H = x.shape
+    _check(lib().sd2_rmsnorm(_ptr(x), _ptr(w), _ptr(y), N, H, eps, _stream(stream)), "sd2_rmsnorm")
+
+
+def sd2_rope_cache(q, k, v, k_cache, v_cache, heads_q: int, heads_kv: int, pos: int, theta: float, stream=None):
+    """q [N, heads_q*d] rotated in place; rope(k), v appended at ``pos`` of the caches [N, T_max, heads_kv*d]."""
+    N = q.shape[0]
+    d = q.shape[1] // heads_q
+    _check(lib().sd2_rope_cache(_ptr(q), _ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), N, heads_q, heads_kv, d, pos,
+                                k_cache.shape[1], theta, _stream(stream)), "sd2_rope_cache")
+
+
+def sd2_attention_decode(q, k_cache, v_cache, out, heads_q: int, heads_kv: int, T: int, stream=None):
+    N = q.shape[0]
+    d = q.shape[1] // heads_q
+    _check(lib().sd2_attention_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), N, heads_q, heads_kv, d, T,
+                                      k_cache.shape[1], _stream(stream)), "sd2_attention_decode")
+
+
+def sd2_add(a, b, y, stream=None):
+    _check(lib().sd2_add(_ptr(a), _ptr(b), _ptr(y), a.numel(), _stream(stream)), "sd2_add")
+
+
+def sd2_embedding(tokens, table, x, stream=None):
+    V, H = table.shape
+    _check(lib().sd2_embedding(_ptr(tokens), _ptr(table), _ptr(x), tokens.numel(), V, H, _stream(stream)), "sd2_embedding")
+
+
+def sd2_lm_head(x, w_out, logits, tokens=None, stream=None):
+    N, H = x.shape
+    V = w_out.shape[0]
+    _check(lib().sd2_lm_head(_ptr(x), _ptr(w_out), _ptr(logits), _ptr(tokens) if tokens is not None else None, N, V, H,
+                             _stream(stream)), "sd2_lm_head")
+
+
+def sd2_decoder_workspace_bytes(hs, N: int) -> int:
+    out = ctypes.c_int64()
+    _check(lib().sd2_decoder_workspace_bytes(_handle_array(hs), N, ctypes.byref(out)), "sd2_decoder_workspace_bytes")
+    return out.value
+
+
+def sd2_decoder_block_step(hs, norm_attn, norm_ffn, x, y, k_cache, v_cache, heads_q: int, heads_kv: int, pos: int,
+                           eps: float, theta: float, workspace, stream=None, handle_array=None):
+    N = x.shape[0]
+    arr = handle_array if handle_array is not None else _handle_array(hs)
+    _check(lib().sd2_decoder_block_step(arr, _ptr(norm_attn), _ptr(norm_ffn), _ptr(x), _ptr(y), _ptr(k_cache), _ptr(v_cache), N,
+                                        heads_q, heads_kv, pos, k_cache.shape[1], eps, theta, _ptr(workspace), _stream(stream)),
+           "sd2_decoder_block_step")

@@ -17,6 +17,7 @@
 #include "sd2_format_mma.hpp"
 #include "sd2_kernels.cuh"
 #include "sd2_mma_kernel.cuh"
+#include "sd2_glue.cuh"
 
 using namespace sd2;
 
@@ -957,6 +958,151 @@ sd2_status sd2_stream_check(void* cuda_stream)
         return SD2_ERR_TIMEOUT;
     }
     return SD2_OK;
+}
+
+// ------------------------------------------------------------------ decode-step glue
+
+sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t H, float eps, void* cuda_stream)
+{
+    if (!x || !w || !y) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || H < 1 || N > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    rmsnorm_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)x, (const uint16_t*)w, (uint16_t*)y, (int)H, eps);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, void* v_cache, int64_t N, int64_t heads_q,
+                          int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta, void* cuda_stream)
+{
+    if (!q || !k || !v || !k_cache || !v_cache) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || heads_q < 1 || heads_kv < 1 || head_dim < 2 || (head_dim & 1) || pos < 0 || pos >= T_max || T_max > 0x7FFFFFFF ||
+        heads_q > 65536 || heads_kv > 65536 || head_dim > 65536 || N > 0x7FFFFFFF || !(theta > 0.0))
+        return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    rope_cache_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v,
+                                                                                    (uint16_t*)k_cache, (uint16_t*)v_cache, (int)heads_q,
+                                                                                    (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, theta);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* v_cache, void* out, int64_t N, int64_t heads_q,
+                                int64_t heads_kv, int64_t head_dim, int64_t T, int64_t T_max, void* cuda_stream)
+{
+    if (!q || !k_cache || !v_cache || !out) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || heads_q < 1 || heads_kv < 1 || heads_q % heads_kv || head_dim < 1 || T < 1 || T > T_max || T_max > 0x7FFFFFFF ||
+        N * heads_q > 0x7FFFFFFF)
+        return SD2_ERR_SHAPE;
+    if (head_dim > kAttnThreads || T > kAttnMaxT) return SD2_ERR_UNSUPPORTED;
+    if (N == 0) return SD2_OK;
+    attention_decode_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)T * 4, (cudaStream_t)cuda_stream>>>(
+        (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, (uint16_t*)out, (int)heads_q, (int)heads_kv, (int)head_dim,
+        (int)T, (int)T_max);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_add(const void* a, const void* b, void* y, int64_t count, void* cuda_stream)
+{
+    if (!a || !b || !y) return SD2_ERR_INVALID_ARG;
+    if (count < 0) return SD2_ERR_SHAPE;
+    if (count == 0) return SD2_OK;
+    int64_t grid = (count + kGlueThreads - 1) / kGlueThreads;
+    if (grid > 148 * 8) grid = 148 * 8;
+    add_kernel<<<(unsigned)grid, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)a, (const uint16_t*)b, (uint16_t*)y, (long long)count);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_embedding(const int32_t* tokens, const void* table, void* x, int64_t N, int64_t V, int64_t H, void* cuda_stream)
+{
+    if (!tokens || !table || !x) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || V < 1 || H < 1 || N > 0x7FFFFFFF || V > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    embedding_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>(tokens, (const uint16_t*)table, (uint16_t*)x, (int)H, (int)V);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t* tokens, int64_t N, int64_t V, int64_t H,
+                       void* cuda_stream)
+{
+    if (!x || !w_out || !logits) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || V < 1 || H < 1 || V > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
+    if ((H & 7) || (((uintptr_t)w_out) & 15)) return SD2_ERR_UNSUPPORTED;
+    if ((size_t)kHeadMaxRows * (size_t)H * 4 > (size_t)kSmemMax) return SD2_ERR_UNSUPPORTED;
+    int dev = 0;
+    sd2_status st = ensure_device(&dev);
+    if (st != SD2_OK) return st;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    for (int64_t n0 = 0; n0 < N; n0 += kHeadMaxRows) {
+        const int n = (int)((N - n0) < kHeadMaxRows ? (N - n0) : kHeadMaxRows);
+        const size_t smem = (size_t)n * (size_t)H * 4;
+        int64_t grid = (V + kGlueThreads / 32 - 1) / (kGlueThreads / 32);
+        const int64_t cap = (int64_t)g_dev[dev].sms * (smem > 100 * 1024 ? 1 : 2);
+        if (grid > cap) grid = cap;
+        lm_head_kernel<<<(unsigned)grid, kGlueThreads, smem, s>>>((const uint16_t*)x + n0 * H, (const uint16_t*)w_out, logits + n0 * V, n, (int)V, (int)H);
+        if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
+    }
+    if (tokens && N > 0) {
+        argmax_kernel<<<(unsigned)N, 1024, 0, s>>>(logits, tokens, (int)V);
+        if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
+    }
+    return SD2_OK;
+}
+
+sd2_status sd2_decoder_workspace_bytes(const sd2_handle* h, int64_t N, int64_t* bytes)
+{
+    if (!bytes) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    BlockDims d;
+    sd2_status st = block_dims(h, &d);
+    if (st != SD2_OK) return st;
+    int64_t off[8];
+    block_layout(h, d, N, off);
+    // the linears' intermediates, then xn (normalised input), att (attention output), x1 (after the first residual), down
+    *bytes = off[7] + 2 * a256(2 * N * d.hidden) + a256(2 * N * d.q_out) + a256(2 * N * d.out);
+    return SD2_OK;
+}
+
+sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, const void* norm_ffn, const void* x, void* y,
+                                  void* k_cache, void* v_cache, int64_t N, int64_t heads_q, int64_t heads_kv, int64_t pos,
+                                  int64_t T_max, float eps, double theta, void* workspace, void* cuda_stream)
+{
+    if (!norm_attn || !norm_ffn || !x || !y || !k_cache || !v_cache || !workspace) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
+    BlockDims d;
+    sd2_status st = block_dims(h, &d);
+    if (st != SD2_OK) return st;
+    if (heads_q < 1 || heads_kv < 1 || d.q_out % heads_q || d.kv % heads_kv || d.q_out / heads_q != d.kv / heads_kv ||
+        d.out != d.hidden || h[3]->M != d.hidden)
+        return SD2_ERR_SHAPE;
+    if (((uintptr_t)workspace) & 255) return SD2_ERR_INVALID_ARG;
+    if (N == 0) return SD2_OK;
+    const int64_t hd = d.q_out / heads_q;
+    int64_t off[8];
+    block_layout(h, d, N, off);
+    char* ws = (char*)workspace;
+    uint16_t *q = (uint16_t*)(ws + off[0]), *k = (uint16_t*)(ws + off[1]), *v = (uint16_t*)(ws + off[2]);
+    uint16_t *hdn = (uint16_t*)(ws + off[3]), *g = (uint16_t*)(ws + off[4]), *u = (uint16_t*)(ws + off[5]), *t = (uint16_t*)(ws + off[6]);
+    int64_t o = off[7];
+    uint16_t* xn = (uint16_t*)(ws + o); o += a256(2 * N * d.hidden);
+    uint16_t* x1 = (uint16_t*)(ws + o); o += a256(2 * N * d.hidden);
+    uint16_t* att = (uint16_t*)(ws + o); o += a256(2 * N * d.q_out);
+    uint16_t* dn = (uint16_t*)(ws + o);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // attention module: x1 = x + Wo attention(rope(Wq n), cache + rope(Wk n), cache + Wv n), n = rmsnorm(x)
+    if ((st = sd2_rmsnorm(x, norm_attn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
+    void* yqkv[3] = {q, k, v};
+    if ((st = run_group(h, 3, xn, nullptr, nullptr, nullptr, yqkv, N, true, s)) != SD2_OK) return st;
+    if ((st = sd2_rope_cache(q, k, v, k_cache, v_cache, N, heads_q, heads_kv, hd, pos, T_max, theta, s)) != SD2_OK) return st;
+    if ((st = sd2_attention_decode(q, k_cache, v_cache, att, N, heads_q, heads_kv, hd, pos + 1, T_max, s)) != SD2_OK) return st;
+    void* yo[1] = {hdn};
+    if ((st = run_group(h + 3, 1, att, nullptr, nullptr, nullptr, yo, N, true, s)) != SD2_OK) return st;
+    if ((st = sd2_add(x, hdn, x1, N * d.hidden, s)) != SD2_OK) return st;
+    // feed-forward module: y = x1 + Wd (silu(Wg m) * Wu m), m = rmsnorm(x1)
+    if ((st = sd2_rmsnorm(x1, norm_ffn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
+    void* ygu[2] = {g, u};
+    if ((st = run_group(h + 4, 2, xn, nullptr, nullptr, nullptr, ygu, N, true, s)) != SD2_OK) return st;
+    void* yd[1] = {dn};
+    if ((st = run_group(h + 6, 1, nullptr, g, u, t, yd, N, true, s)) != SD2_OK) return st;
+    return sd2_add(x1, dn, y, N * d.hidden, s);
 }
 
 sd2_status sd2_selftest_timeout(void* cuda_stream)

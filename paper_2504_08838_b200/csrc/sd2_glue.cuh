@@ -1,0 +1,215 @@
+// Glue of one drafter decode step around the sparse linears: RMSNorm, rotary embedding with the
+// key/value cache append, grouped-query attention of one new token over the cache, residual add,
+// embedding look-up, dense LM head with greedy token.  The paper leaves the embedding and the LM
+// head dense (Section "Results") and says a block is an attention module and a feed-forward module
+// (Section "Layer pruning"); what those compute is the published definition of the Llama / Qwen
+// family.  All of it is small beside the linears (activations of a few KB per row), except the LM
+// head, which streams vocab x hidden bf16 weights from HBM once per step.
+//
+// bf16 in and out, fp32 arithmetic (rotary angles in fp64), one rounding per output.
+
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sd2_kernels.cuh"
+
+namespace sd2 {
+
+constexpr int kGlueThreads = 256;
+constexpr int kAttnThreads = 128;
+constexpr int kAttnMaxT = 8192;            // cached positions whose scores fit the kernel's shared memory
+constexpr int kHeadMaxRows = 8;            // activation rows one LM-head launch keeps in shared memory
+
+__device__ __forceinline__ float block_sum(float v, float* red)
+{
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (l == 0) red[w] = v;
+    __syncthreads();
+    float t = l < nw ? red[l] : 0.f;
+    for (int d = 16; d > 0; d >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, d);
+    return t;
+}
+
+__device__ __forceinline__ float block_max(float v, float* red)
+{
+    for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, d));
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+    __syncthreads();
+    if (l == 0) red[w] = v;
+    __syncthreads();
+    float t = l < nw ? red[l] : -INFINITY;
+    for (int d = 16; d > 0; d >>= 1) t = fmaxf(t, __shfl_xor_sync(0xFFFFFFFFu, t, d));
+    return t;
+}
+
+// y[n, :] = x[n, :] / sqrt(mean(x[n, :]^2) + eps) * w;  one CTA per row
+__global__ void __launch_bounds__(kGlueThreads) rmsnorm_kernel(const uint16_t* x, const uint16_t* w, uint16_t* y, int H, float eps)
+{
+    __shared__ float red[32];
+    const uint16_t* xr = x + (size_t)blockIdx.x * H;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < H; i += blockDim.x) {
+        const float v = bf16_to_f32(xr[i]);
+        ss += v * v;
+    }
+    const float r = rsqrtf(block_sum(ss, red) / (float)H + eps);
+    for (int i = threadIdx.x; i < H; i += blockDim.x)
+        y[(size_t)blockIdx.x * H + i] = f32_to_bf16_rne(bf16_to_f32(xr[i]) * r * bf16_to_f32(w[i]));
+}
+
+// Rotates q in place and writes the rotated k and the plain v of row n into position `pos` of row n's cache.
+// Caches are [N, T_max, Hkv * d].  One CTA per row.
+__global__ void __launch_bounds__(kGlueThreads) rope_cache_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
+                                                                 uint16_t* vc, int Hq, int Hkv, int d, int pos, int T_max, double theta)
+{
+    const int n = blockIdx.x, half = d / 2;
+    uint16_t* qr = q + (size_t)n * Hq * d;
+    const uint16_t* kr = k + (size_t)n * Hkv * d;
+    uint16_t* kdst = kc + ((size_t)n * T_max + pos) * Hkv * d;
+    uint16_t* vdst = vc + ((size_t)n * T_max + pos) * Hkv * d;
+    for (int p = threadIdx.x; p < (Hq + Hkv) * half; p += blockDim.x) {
+        const int h = p / half, i = p % half;
+        double sn, cs;
+        sincos((double)pos * pow(theta, -2.0 * (double)i / (double)d), &sn, &cs);
+        const float c = (float)cs, s = (float)sn;
+        if (h < Hq) {
+            const float a = bf16_to_f32(qr[h * d + i]), b = bf16_to_f32(qr[h * d + i + half]);
+            qr[h * d + i] = f32_to_bf16_rne(a * c - b * s);
+            qr[h * d + i + half] = f32_to_bf16_rne(b * c + a * s);
+        } else {
+            const int hk = h - Hq;
+            const float a = bf16_to_f32(kr[hk * d + i]), b = bf16_to_f32(kr[hk * d + i + half]);
+            kdst[hk * d + i] = f32_to_bf16_rne(a * c - b * s);
+            kdst[hk * d + i + half] = f32_to_bf16_rne(b * c + a * s);
+        }
+    }
+    for (int i = threadIdx.x; i < Hkv * d; i += blockDim.x) vdst[i] = v[(size_t)n * Hkv * d + i];
+}
+
+// One new token per row over T cached positions; one CTA per (row, query head); d <= 128.
+__global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const uint16_t* q, const uint16_t* kc, const uint16_t* vc,
+                                                                       uint16_t* out, int Hq, int Hkv, int d, int T, int T_max)
+{
+    extern __shared__ float sc[];            // T scores, then the weights
+    __shared__ float red[32];
+    __shared__ float qs[128];
+    const int n = blockIdx.x / Hq, h = blockIdx.x % Hq, g = h / (Hq / Hkv);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    if (threadIdx.x < d) qs[threadIdx.x] = bf16_to_f32(q[((size_t)n * Hq + h) * d + threadIdx.x]);
+    __syncthreads();
+    const uint16_t* kb = kc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
+    const uint16_t* vb = vc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
+    const float scale = rsqrtf((float)d);
+    for (int t = warp; t < T; t += nw) {
+        float s = 0.f;
+        for (int i = lane; i < d; i += 32) s += qs[i] * bf16_to_f32(kb[(size_t)t * Hkv * d + i]);
+        for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+        if (lane == 0) sc[t] = s * scale;
+    }
+    __syncthreads();
+    float m = -INFINITY;
+    for (int t = threadIdx.x; t < T; t += blockDim.x) m = fmaxf(m, sc[t]);
+    m = block_max(m, red);
+    float z = 0.f;
+    for (int t = threadIdx.x; t < T; t += blockDim.x) {
+        const float e = expf(sc[t] - m);
+        sc[t] = e;
+        z += e;
+    }
+    z = block_sum(z, red);
+    __syncthreads();
+    if (threadIdx.x < d) {
+        float acc = 0.f;
+        for (int t = 0; t < T; ++t) acc += sc[t] * bf16_to_f32(vb[(size_t)t * Hkv * d + threadIdx.x]);
+        out[((size_t)n * Hq + h) * d + threadIdx.x] = f32_to_bf16_rne(acc / z);
+    }
+}
+
+// y = a + b, element by element
+__global__ void __launch_bounds__(kGlueThreads) add_kernel(const uint16_t* a, const uint16_t* b, uint16_t* y, long long count)
+{
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x)
+        y[i] = f32_to_bf16_rne(bf16_to_f32(a[i]) + bf16_to_f32(b[i]));
+}
+
+// x[n, :] = table[token[n], :]
+__global__ void __launch_bounds__(kGlueThreads) embedding_kernel(const int32_t* tokens, const uint16_t* table, uint16_t* x, int H, int V)
+{
+    const int tok = tokens[blockIdx.x];
+    for (int i = threadIdx.x; i < H; i += blockDim.x)
+        x[(size_t)blockIdx.x * H + i] = (tok >= 0 && tok < V) ? table[(size_t)tok * H + i] : (uint16_t)0;
+}
+
+// logits[n, v] = sum_h W[v, h] x[n, h]: a warp per vocabulary row, 128-bit loads of the row, the
+// N <= 8 activation rows in shared memory as fp32.  H a multiple of 8.
+__global__ void __launch_bounds__(kGlueThreads) lm_head_kernel(const uint16_t* x, const uint16_t* W, float* logits, int N, int V, int H)
+{
+    extern __shared__ float xs[];            // [N][H]
+    for (int i = threadIdx.x; i < N * H; i += blockDim.x) xs[i] = bf16_to_f32(x[i]);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int v = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; v < V; v += warps) {
+        const uint4* wr = (const uint4*)(W + (size_t)v * H);
+        float acc[kHeadMaxRows];
+#pragma unroll
+        for (int n = 0; n < kHeadMaxRows; ++n) acc[n] = 0.f;
+        for (int c = lane; c < H / 8; c += 32) {
+            const uint4 w4 = __ldg(wr + c);
+            const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+            for (int n = 0; n < kHeadMaxRows; ++n) {
+                if (n < N) {
+                    const float* xr = xs + n * H + c * 8;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[n] += bf16_lo(ww[j]) * xr[2 * j] + bf16_hi(ww[j]) * xr[2 * j + 1];
+                }
+            }
+        }
+#pragma unroll
+        for (int n = 0; n < kHeadMaxRows; ++n) {
+            if (n < N) {
+                float s = acc[n];
+                for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+                if (lane == 0) logits[(size_t)n * V + v] = s;
+            }
+        }
+    }
+}
+
+// token[n] = index of the largest logit of row n, the lowest index among equals; one CTA per row
+__global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int32_t* token, int V)
+{
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    const float* r = logits + (size_t)blockIdx.x * V;
+    float best = -INFINITY;
+    int at = 0x7FFFFFFF;
+    for (int i = threadIdx.x; i < V; i += blockDim.x) {
+        const float v = r[i];
+        if (v > best || (v == best && i < at)) { best = v; at = i; }
+    }
+    for (int d = 16; d > 0; d >>= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, d);
+        const int oi = __shfl_xor_sync(0xFFFFFFFFu, at, d);
+        if (ov > best || (ov == best && oi < at)) { best = ov; at = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { bv[threadIdx.x >> 5] = best; bi[threadIdx.x >> 5] = at; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        best = threadIdx.x < (blockDim.x >> 5) ? bv[threadIdx.x] : -INFINITY;
+        at = threadIdx.x < (blockDim.x >> 5) ? bi[threadIdx.x] : 0x7FFFFFFF;
+        for (int d = 16; d > 0; d >>= 1) {
+            const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, d);
+            const int oi = __shfl_xor_sync(0xFFFFFFFFu, at, d);
+            if (ov > best || (ov == best && oi < at)) { best = ov; at = oi; }
+        }
+        if (threadIdx.x == 0) token[blockIdx.x] = at == 0x7FFFFFFF ? 0 : at;
+    }
+}
+
+}  // namespace sd2
