@@ -359,9 +359,14 @@ def time_full_step(torch, sd2, args, shape, handles, harr, N, stream):
 
     us = time_graph_us(torch, step, max(20, args.steps // 20), stream)
     sd2.sd2_stream_check()
+    us_head = time_graph_us(torch, lambda: sd2.sd2_lm_head(xs[blocks + 1], table, logits, tokens_out), 50, stream)
+    us_block = time_graph_us(torch, lambda: sd2.sd2_decoder_block_step(
+        handles[0], gains[0], gains[1], xs[0], xs[1], kcs[0], vcs[0], heads_q, heads_kv, args.context, 1e-5, 500000.0, ws,
+        handle_array=harr[0]), 50, stream)
     head_bytes = 2.0 * vocab * hid
     return {"us_per_token": us, "launches_per_step": 10 * blocks + 4, "context": args.context, "vocab": vocab,
-            "heads": [heads_q, heads_kv, d], "lm_head_bytes": head_bytes,
+            "heads": [heads_q, heads_kv, d], "lm_head_bytes": head_bytes, "lm_head_us": us_head,
+            "lm_head_gbs": head_bytes / us_head / 1e3, "block0_alone_us_l2_warm": us_block,
             "note": "one launch per group of linears that share an input (4 per block) and per glue operation (6 per block); "
                     "the linears here are single-stage launches, not the one-launch drafter step timed above"}
 

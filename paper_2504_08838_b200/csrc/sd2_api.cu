@@ -126,7 +126,8 @@ sd2_status ensure_device(int* dev_out)
             cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
         if (set_smem_attr<1>() != cudaSuccess || set_smem_attr<2>() != cudaSuccess || set_smem_attr<4>() != cudaSuccess ||
             set_smem_attr<8>() != cudaSuccess ||
-            cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax) != cudaSuccess) {
+            cudaFuncSetAttribute(mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax) != cudaSuccess ||
+            cudaFuncSetAttribute(lm_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax) != cudaSuccess) {
             cudaGetLastError();
             return SD2_ERR_CUDA;
         }
@@ -976,10 +977,10 @@ sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, 
 {
     if (!q || !k || !v || !k_cache || !v_cache) return SD2_ERR_INVALID_ARG;
     if (N < 0 || heads_q < 1 || heads_kv < 1 || head_dim < 2 || (head_dim & 1) || pos < 0 || pos >= T_max || T_max > 0x7FFFFFFF ||
-        heads_q > 65536 || heads_kv > 65536 || head_dim > 65536 || N > 0x7FFFFFFF || !(theta > 0.0))
+        heads_q > 65536 || heads_kv > 65536 || head_dim > 8192 || N > 0x7FFFFFFF || !(theta > 0.0))
         return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;
-    rope_cache_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v,
+    rope_cache_kernel<<<(unsigned)N, kGlueThreads, (size_t)head_dim * 4, (cudaStream_t)cuda_stream>>>((uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v,
                                                                                     (uint16_t*)k_cache, (uint16_t*)v_cache, (int)heads_q,
                                                                                     (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, theta);
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
@@ -992,7 +993,7 @@ sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* 
     if (N < 0 || heads_q < 1 || heads_kv < 1 || heads_q % heads_kv || head_dim < 1 || T < 1 || T > T_max || T_max > 0x7FFFFFFF ||
         N * heads_q > 0x7FFFFFFF)
         return SD2_ERR_SHAPE;
-    if (head_dim > kAttnThreads || T > kAttnMaxT) return SD2_ERR_UNSUPPORTED;
+    if (head_dim > 128 || T > kAttnMaxT) return SD2_ERR_UNSUPPORTED;
     if (N == 0) return SD2_OK;
     attention_decode_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)T * 4, (cudaStream_t)cuda_stream>>>(
         (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, (uint16_t*)out, (int)heads_q, (int)heads_kv, (int)head_dim,
@@ -1035,7 +1036,10 @@ sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t*
         const int n = (int)((N - n0) < kHeadMaxRows ? (N - n0) : kHeadMaxRows);
         const size_t smem = (size_t)n * (size_t)H * 4;
         int64_t grid = (V + kGlueThreads / 32 - 1) / (kGlueThreads / 32);
-        const int64_t cap = (int64_t)g_dev[dev].sms * (smem > 100 * 1024 ? 1 : 2);
+        // as many CTAs per SM as the staged rows allow (8 x 256 threads fill an SM): the stream needs many loads in flight
+        int per_sm = smem ? (int)((200 * 1024) / smem) : 8;
+        per_sm = per_sm < 1 ? 1 : per_sm > 8 ? 8 : per_sm;
+        const int64_t cap = (int64_t)g_dev[dev].sms * per_sm;
         if (grid > cap) grid = cap;
         lm_head_kernel<<<(unsigned)grid, kGlueThreads, smem, s>>>((const uint16_t*)x + n0 * H, (const uint16_t*)w_out, logits + n0 * V, n, (int)V, (int)H);
         if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;

@@ -18,7 +18,7 @@
 namespace sd2 {
 
 constexpr int kGlueThreads = 256;
-constexpr int kAttnThreads = 128;
+constexpr int kAttnThreads = 256;
 constexpr int kAttnMaxT = 8192;            // cached positions whose scores fit the kernel's shared memory
 constexpr int kHeadMaxRows = 8;            // activation rows one LM-head launch keeps in shared memory
 
@@ -66,16 +66,22 @@ __global__ void __launch_bounds__(kGlueThreads) rmsnorm_kernel(const uint16_t* x
 __global__ void __launch_bounds__(kGlueThreads) rope_cache_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
                                                                  uint16_t* vc, int Hq, int Hkv, int d, int pos, int T_max, double theta)
 {
+    extern __shared__ float cs_tab[];        // cos and sin of the d / 2 angles of this position
     const int n = blockIdx.x, half = d / 2;
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        double sn, cs;
+        sincos((double)pos * pow(theta, -2.0 * (double)i / (double)d), &sn, &cs);
+        cs_tab[i] = (float)cs;
+        cs_tab[half + i] = (float)sn;
+    }
+    __syncthreads();
     uint16_t* qr = q + (size_t)n * Hq * d;
     const uint16_t* kr = k + (size_t)n * Hkv * d;
     uint16_t* kdst = kc + ((size_t)n * T_max + pos) * Hkv * d;
     uint16_t* vdst = vc + ((size_t)n * T_max + pos) * Hkv * d;
     for (int p = threadIdx.x; p < (Hq + Hkv) * half; p += blockDim.x) {
         const int h = p / half, i = p % half;
-        double sn, cs;
-        sincos((double)pos * pow(theta, -2.0 * (double)i / (double)d), &sn, &cs);
-        const float c = (float)cs, s = (float)sn;
+        const float c = cs_tab[i], s = cs_tab[half + i];
         if (h < Hq) {
             const float a = bf16_to_f32(qr[h * d + i]), b = bf16_to_f32(qr[h * d + i + half]);
             qr[h * d + i] = f32_to_bf16_rne(a * c - b * s);
@@ -97,6 +103,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     extern __shared__ float sc[];            // T scores, then the weights
     __shared__ float red[32];
     __shared__ float qs[128];
+    __shared__ float part[(kAttnThreads / 32) * 128];
     const int n = blockIdx.x / Hq, h = blockIdx.x % Hq, g = h / (Hq / Hkv);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     if (threadIdx.x < d) qs[threadIdx.x] = bf16_to_f32(q[((size_t)n * Hq + h) * d + threadIdx.x]);
@@ -104,6 +111,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     const uint16_t* kb = kc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
     const uint16_t* vb = vc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
     const float scale = rsqrtf((float)d);
+#pragma unroll 4
     for (int t = warp; t < T; t += nw) {
         float s = 0.f;
         for (int i = lane; i < d; i += 32) s += qs[i] * bf16_to_f32(kb[(size_t)t * Hkv * d + i]);
@@ -122,10 +130,26 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     }
     z = block_sum(z, red);
     __syncthreads();
+    // weights times values: every warp takes every nw-th position, a lane the dimensions lane, lane + 32, ...;
+    // the warps' partial sums meet in shared memory
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+    for (int t = warp; t < T; t += nw) {
+        const float p = sc[t];
+        const uint16_t* vr = vb + (size_t)t * Hkv * d;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (lane + 32 * j < d) acc[j] += p * bf16_to_f32(vr[lane + 32 * j]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (lane + 32 * j < d) part[warp * 128 + lane + 32 * j] = acc[j];
+    __syncthreads();
     if (threadIdx.x < d) {
-        float acc = 0.f;
-        for (int t = 0; t < T; ++t) acc += sc[t] * bf16_to_f32(vb[(size_t)t * Hkv * d + threadIdx.x]);
-        out[((size_t)n * Hq + h) * d + threadIdx.x] = f32_to_bf16_rne(acc / z);
+        float a = 0.f;
+        for (int w = 0; w < nw; ++w) a += part[w * 128 + threadIdx.x];
+        out[((size_t)n * Hq + h) * d + threadIdx.x] = f32_to_bf16_rne(a / z);
     }
 }
 
@@ -158,6 +182,7 @@ __global__ void __launch_bounds__(kGlueThreads) lm_head_kernel(const uint16_t* x
         float acc[kHeadMaxRows];
 #pragma unroll
         for (int n = 0; n < kHeadMaxRows; ++n) acc[n] = 0.f;
+#pragma unroll 4
         for (int c = lane; c < H / 8; c += 32) {
             const uint4 w4 = __ldg(wr + c);
             const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};

@@ -444,37 +444,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             const int cnt = (int)((lds_u32(rec + 16u + 32u * (uint32_t)side + ((uint32_t)lane & ~3u)) >> (8 * (lane & 3))) & 0xFFu);
             uint32_t w = rec + (side ? lds_u32(rec + 12u) : (uint32_t)kMmaBlockHeaderBytes);
             uint32_t cur = at + 4u * (uint32_t)lane + 2u * (uint32_t)side;       // row 0 of this lane's piece
-            // the loads of step j + 1 are issued before step j is expanded: a step is a dependent chain
-            // (load, prefix sums, addresses, stores) and a lane has nothing else to overlap it with
-            bool act_n = cnt > 0;
-            uint32_t code_n = 0u;
-            uint4 v_n = make_uint4(0u, 0u, 0u, 0u);
-            {
-                const uint32_t m = __ballot_sync(0xFFFFFFFFu, act_n);
-                const uint32_t nj = (uint32_t)__popc(m);
-                if (act_n) {
-                    const uint32_t idx = (uint32_t)__popc(m & lt);
-                    code_n = lds_u32(w + 4u * idx);
-                    v_n = lds_v4(w + ((4u * nj + 15u) & ~15u) + 16u * idx);
-                }
-                w += ((4u * nj + 15u) & ~15u) + 16u * nj;
-            }
             for (int j = 0; j < steps; ++j) {
-                const bool active = act_n;
-                const uint32_t code = code_n;
-                const uint4 v = v_n;
-                if (j + 1 < steps) {
-                    act_n = cnt > j + 1;
-                    const uint32_t m = __ballot_sync(0xFFFFFFFFu, act_n);
-                    const uint32_t nj = (uint32_t)__popc(m);
-                    if (act_n) {
-                        const uint32_t idx = (uint32_t)__popc(m & lt);
-                        code_n = lds_u32(w + 4u * idx);
-                        v_n = lds_v4(w + ((4u * nj + 15u) & ~15u) + 16u * idx);
-                    }
-                    w += ((4u * nj + 15u) & ~15u) + 16u * nj;
-                }
+                const bool active = cnt > j;
+                const uint32_t m = __ballot_sync(0xFFFFFFFFu, active);
+                const uint32_t nj = (uint32_t)__popc(m);
                 if (active) {
+                    const uint32_t idx = (uint32_t)__popc(m & lt);
+                    const uint32_t code = lds_u32(w + 4u * idx);
+                    const uint4 v = lds_v4(w + ((4u * nj + 15u) & ~15u) + 16u * idx);
                     const uint32_t lo = code & 0x0F0F0F0Fu, hi = (code >> 4) & 0x0F0F0F0Fu;
                     const uint32_t po = (lo + hi) * 0x01010101u;        // byte k: gaps summed through entry 2k + 1
                     const uint32_t pe = po - hi;                       // byte k: ... through entry 2k
@@ -488,6 +465,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
                     sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
                     cur = a7;
                 }
+                w += ((4u * nj + 15u) & ~15u) + 16u * nj;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->empty[slot]));

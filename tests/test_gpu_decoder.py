@@ -104,7 +104,7 @@ def test_add_embedding():
     assert np.array_equal(got[:4], do.embedding(toks[:4], table)) and np.all(got[4] == 0)
 
 
-@pytest.mark.parametrize("N,V,H", [(1, 4099, 2048), (3, 1000, 1536), (9, 257, 64)])
+@pytest.mark.parametrize("N,V,H", [(1, 4099, 2048), (3, 1000, 1536), (9, 257, 64), (8, 300, 3072)])
 def test_lm_head_and_greedy_token(N, V, H):
     W = synth.normal_bf16(500 + V, (V, H), 0.02)
     x = synth.normal_bf16(501 + V, (N, H), 1.0)
