@@ -968,7 +968,8 @@ sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t
     if (!x || !w || !y) return SD2_ERR_INVALID_ARG;
     if (N < 0 || H < 1 || N > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;
-    rmsnorm_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)x, (const uint16_t*)w, (uint16_t*)y, (int)H, eps);
+    const int vec = ((H & 7) == 0 && ((((uintptr_t)x) | ((uintptr_t)w) | ((uintptr_t)y)) & 15) == 0) ? 1 : 0;
+    rmsnorm_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)x, (const uint16_t*)w, (uint16_t*)y, (int)H, eps, vec);
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
@@ -995,9 +996,11 @@ sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* 
         return SD2_ERR_SHAPE;
     if (head_dim > 128 || T > kAttnMaxT) return SD2_ERR_UNSUPPORTED;
     if (N == 0) return SD2_OK;
+    const bool pow2 = (head_dim & (head_dim - 1)) == 0;
+    const int vec = (pow2 && head_dim >= 8 && ((((uintptr_t)k_cache) | ((uintptr_t)v_cache)) & 15) == 0) ? 1 : 0;
     attention_decode_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)T * 4, (cudaStream_t)cuda_stream>>>(
         (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, (uint16_t*)out, (int)heads_q, (int)heads_kv, (int)head_dim,
-        (int)T, (int)T_max);
+        (int)T, (int)T_max, vec);
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
@@ -1045,7 +1048,8 @@ sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t*
         if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
     }
     if (tokens && N > 0) {
-        argmax_kernel<<<(unsigned)N, 1024, 0, s>>>(logits, tokens, (int)V);
+        const int vec = ((V & 3) == 0 && (((uintptr_t)logits) & 15) == 0) ? 1 : 0;
+        argmax_kernel<<<(unsigned)N, 1024, 0, s>>>(logits, tokens, (int)V, vec);
         if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
     }
     return SD2_OK;

@@ -46,19 +46,44 @@ __device__ __forceinline__ float block_max(float v, float* red)
     return t;
 }
 
-// y[n, :] = x[n, :] / sqrt(mean(x[n, :]^2) + eps) * w;  one CTA per row
-__global__ void __launch_bounds__(kGlueThreads) rmsnorm_kernel(const uint16_t* x, const uint16_t* w, uint16_t* y, int H, float eps)
+// y[n, :] = x[n, :] / sqrt(mean(x[n, :]^2) + eps) * w;  one CTA per row.  vec: H is a multiple of 8 and x, w, y are
+// 16-byte aligned, so a thread moves eight values per load (the second pass finds the row in L1)
+__global__ void __launch_bounds__(kGlueThreads) rmsnorm_kernel(const uint16_t* x, const uint16_t* w, uint16_t* y, int H, float eps, int vec)
 {
     __shared__ float red[32];
     const uint16_t* xr = x + (size_t)blockIdx.x * H;
+    uint16_t* yr = y + (size_t)blockIdx.x * H;
     float ss = 0.f;
-    for (int i = threadIdx.x; i < H; i += blockDim.x) {
-        const float v = bf16_to_f32(xr[i]);
-        ss += v * v;
+    if (vec) {
+        const uint4* x4 = (const uint4*)xr;
+        for (int i = threadIdx.x; i < H / 8; i += blockDim.x) {
+            const uint4 v = x4[i];
+            const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ss += bf16_lo(u[j]) * bf16_lo(u[j]) + bf16_hi(u[j]) * bf16_hi(u[j]);
+        }
+    } else {
+        for (int i = threadIdx.x; i < H; i += blockDim.x) {
+            const float v = bf16_to_f32(xr[i]);
+            ss += v * v;
+        }
     }
     const float r = rsqrtf(block_sum(ss, red) / (float)H + eps);
-    for (int i = threadIdx.x; i < H; i += blockDim.x)
-        y[(size_t)blockIdx.x * H + i] = f32_to_bf16_rne(bf16_to_f32(xr[i]) * r * bf16_to_f32(w[i]));
+    if (vec) {
+        const uint4* x4 = (const uint4*)xr;
+        const uint4* w4 = (const uint4*)w;
+        for (int i = threadIdx.x; i < H / 8; i += blockDim.x) {
+            const uint4 v = x4[i], g = w4[i];
+            const uint32_t u[4] = {v.x, v.y, v.z, v.w}, q[4] = {g.x, g.y, g.z, g.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                o[j] = (uint32_t)f32_to_bf16_rne(bf16_lo(u[j]) * r * bf16_lo(q[j])) | ((uint32_t)f32_to_bf16_rne(bf16_hi(u[j]) * r * bf16_hi(q[j])) << 16);
+            ((uint4*)yr)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    } else {
+        for (int i = threadIdx.x; i < H; i += blockDim.x) yr[i] = f32_to_bf16_rne(bf16_to_f32(xr[i]) * r * bf16_to_f32(w[i]));
+    }
 }
 
 // Rotates q in place and writes the rotated k and the plain v of row n into position `pos` of row n's cache.
@@ -97,8 +122,10 @@ __global__ void __launch_bounds__(kGlueThreads) rope_cache_kernel(uint16_t* q, c
 }
 
 // One new token per row over T cached positions; one CTA per (row, query head); d <= 128.
+// vec: d is 8, 16, 32, 64 or 128 and the caches are 16-byte aligned: d / 8 lanes share a position, a lane holds eight
+// dimensions (one 128-bit load), so a warp takes 256 / d positions per step and all its loads are independent.
 __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const uint16_t* q, const uint16_t* kc, const uint16_t* vc,
-                                                                       uint16_t* out, int Hq, int Hkv, int d, int T, int T_max)
+                                                                       uint16_t* out, int Hq, int Hkv, int d, int T, int T_max, int vec)
 {
     extern __shared__ float sc[];            // T scores, then the weights
     __shared__ float red[32];
@@ -110,13 +137,36 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     __syncthreads();
     const uint16_t* kb = kc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
     const uint16_t* vb = vc + (size_t)n * T_max * Hkv * d + (size_t)g * d;
+    const size_t pitch = (size_t)Hkv * d;
     const float scale = rsqrtf((float)d);
+    const int lpp = d >> 3;                  // lanes per position (vec)
+    const int ppw = vec ? 32 / lpp : 1;      // positions per warp step
+    const int sub = vec ? lane / lpp : 0, dl = vec ? (lane % lpp) * 8 : 0;
+    if (vec) {
+        float qv[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) qv[j] = qs[dl + j];
 #pragma unroll 4
-    for (int t = warp; t < T; t += nw) {
-        float s = 0.f;
-        for (int i = lane; i < d; i += 32) s += qs[i] * bf16_to_f32(kb[(size_t)t * Hkv * d + i]);
-        for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
-        if (lane == 0) sc[t] = s * scale;
+        for (int t0 = warp * ppw; t0 < T; t0 += nw * ppw) {
+            const int t = t0 + sub;
+            float s = 0.f;
+            if (t < T) {
+                const uint4 kv = *(const uint4*)(kb + (size_t)t * pitch + dl);
+                const uint32_t u[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s += qv[2 * j] * bf16_lo(u[j]) + qv[2 * j + 1] * bf16_hi(u[j]);
+            }
+            for (int dd = 1; dd < lpp; dd <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+            if (t < T && (lane % lpp) == 0) sc[t] = s * scale;
+        }
+    } else {
+#pragma unroll 4
+        for (int t = warp; t < T; t += nw) {
+            float s = 0.f;
+            for (int i = lane; i < d; i += 32) s += qs[i] * bf16_to_f32(kb[(size_t)t * pitch + i]);
+            for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+            if (lane == 0) sc[t] = s * scale;
+        }
     }
     __syncthreads();
     float m = -INFINITY;
@@ -130,21 +180,44 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     }
     z = block_sum(z, red);
     __syncthreads();
-    // weights times values: every warp takes every nw-th position, a lane the dimensions lane, lane + 32, ...;
-    // the warps' partial sums meet in shared memory
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    // weights times values; the warps' partial sums meet in shared memory
+    if (vec) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 4
-    for (int t = warp; t < T; t += nw) {
-        const float p = sc[t];
-        const uint16_t* vr = vb + (size_t)t * Hkv * d;
+        for (int t0 = warp * ppw; t0 < T; t0 += nw * ppw) {
+            const int t = t0 + sub;
+            if (t < T) {
+                const float p = sc[t];
+                const uint4 vv = *(const uint4*)(vb + (size_t)t * pitch + dl);
+                const uint32_t u[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc[2 * j] += p * bf16_lo(u[j]);
+                    acc[2 * j + 1] += p * bf16_hi(u[j]);
+                }
+            }
+        }
+        // the 32 / lpp position groups of the warp add up
+        for (int dd = lpp; dd < 32; dd <<= 1)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], dd);
+        if (lane < lpp)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) part[warp * 128 + dl + j] = acc[j];
+    } else {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int t = warp; t < T; t += nw) {
+            const float p = sc[t];
+            const uint16_t* vr = vb + (size_t)t * pitch;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (lane + 32 * j < d) acc[j] += p * bf16_to_f32(vr[lane + 32 * j]);
+        }
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (lane + 32 * j < d) acc[j] += p * bf16_to_f32(vr[lane + 32 * j]);
+            if (lane + 32 * j < d) part[warp * 128 + lane + 32 * j] = acc[j];
     }
-    __syncthreads();
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-        if (lane + 32 * j < d) part[warp * 128 + lane + 32 * j] = acc[j];
     __syncthreads();
     if (threadIdx.x < d) {
         float a = 0.f;
@@ -206,17 +279,30 @@ __global__ void __launch_bounds__(kGlueThreads) lm_head_kernel(const uint16_t* x
     }
 }
 
-// token[n] = index of the largest logit of row n, the lowest index among equals; one CTA per row
-__global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int32_t* token, int V)
+// token[n] = index of the largest logit of row n, the lowest index among equals; one CTA per row.
+// vec: V is a multiple of 4 and the row is 16-byte aligned (four logits per load, eight loads in flight).
+__global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int32_t* token, int V, int vec)
 {
     __shared__ float bv[32];
     __shared__ int bi[32];
     const float* r = logits + (size_t)blockIdx.x * V;
     float best = -INFINITY;
     int at = 0x7FFFFFFF;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
-        const float v = r[i];
-        if (v > best || (v == best && i < at)) { best = v; at = i; }
+    if (vec) {
+        const float4* r4 = (const float4*)r;
+#pragma unroll 8
+        for (int i = threadIdx.x; i < V / 4; i += blockDim.x) {
+            const float4 v = r4[i];
+            const float c[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (c[j] > best) { best = c[j]; at = 4 * i + j; }      // a thread meets its indices in ascending order
+        }
+    } else {
+        for (int i = threadIdx.x; i < V; i += blockDim.x) {
+            const float v = r[i];
+            if (v > best) { best = v; at = i; }
+        }
     }
     for (int d = 16; d > 0; d >>= 1) {
         const float ov = __shfl_xor_sync(0xFFFFFFFFu, best, d);

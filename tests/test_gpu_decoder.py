@@ -71,7 +71,8 @@ def test_rope_and_cache_append(pos):
         assert np.array_equal(bits_of(qd), q)                           # position 0 is the identity
 
 
-@pytest.mark.parametrize("N,Hq,Hkv,d,T", [(1, 32, 8, 64, 300), (2, 12, 2, 128, 1), (3, 8, 8, 64, 1000), (1, 24, 8, 128, 77)])
+@pytest.mark.parametrize("N,Hq,Hkv,d,T", [(1, 32, 8, 64, 300), (2, 12, 2, 128, 1), (3, 8, 8, 64, 1000), (1, 24, 8, 128, 77),
+                                         (2, 4, 2, 24, 50), (1, 6, 3, 8, 133), (1, 2, 1, 16, 4097)])
 def test_attention_decode(N, Hq, Hkv, d, T):
     T_max = T + 5
     q = synth.normal_bf16(300 + T, (N, Hq * d), 1.0)
