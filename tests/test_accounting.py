@@ -57,8 +57,8 @@ def test_hand_counted_rounds():
     target = _table_model({i: i + 1 for i in range(20)}, 0)
     draft = _table_model({**{i: i + 1 for i in range(20)}, 3: 9}, 0)
     out, rounds = acc.speculative_decode(draft, target, [1], k=3, max_new_tokens=6)
-    # round 1: drafts 2, 3, 9 -> 2 and 3 accepted, 9 rejected and replaced by the target's 4: 3 tokens
-    # round 2: context ends in 4: drafts 5, 6, 7 all accepted, the target adds 8: 4 tokens (cut at 6 in total)
+    # first draft-verify cycle: drafts 2, 3, 9 -> 2 and 3 accepted, 9 rejected and replaced by the target's 4: 3 tokens
+    # second cycle: context ends in 4: drafts 5, 6, 7 all accepted, the target adds 8: 4 tokens (cut at 6 in total)
     assert out == [2, 3, 4, 5, 6, 7]
     assert rounds == [3, 3]
     out, rounds = acc.speculative_decode(draft, target, [1], k=3, max_new_tokens=7)
