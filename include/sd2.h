@@ -254,6 +254,11 @@ sd2_status sd2_selftest_timeout(void* cuda_stream);
 /* y[n, :] = x[n, :] / sqrt(mean(x[n, :]^2) + eps) * w.   x, y [N*H]; w [H].  y may be x. */
 sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t H, float eps, void* cuda_stream);
 
+/* The residual connection and the norm that follows it, in one launch: sum = a + b (rounded to bf16), y = the
+ * sd2_rmsnorm of sum with gain w.  a, b, sum, y [N*H]; sum may be a or b; y must not overlap sum. */
+sd2_status sd2_add_rmsnorm(const void* a, const void* b, void* sum, const void* w, void* y, int64_t N, int64_t H, float eps,
+                           void* cuda_stream);
+
 /* Rotary embedding of one new token per row at position `pos` (pairs (i, i + head_dim/2) of a head
  * turn by pos * theta^(-2i/head_dim)), and the cache append: q [N, heads_q, head_dim] is rotated in
  * place; the rotated k and the plain v ([N, heads_kv, head_dim]) are written to position `pos` of
@@ -267,6 +272,12 @@ sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, 
  * UNSUPPORTED: head_dim > 128 or T > 8192. */
 sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* v_cache, void* out, int64_t N, int64_t heads_q,
                                 int64_t heads_kv, int64_t head_dim, int64_t T, int64_t T_max, void* cuda_stream);
+
+/* sd2_rope_cache followed by sd2_attention_decode over positions 0..pos, in one launch: q is rotated in place, the
+ * rotated k and v are appended at `pos`, out [N, heads_q, head_dim] is the attention output.  Same limits as the two. */
+sd2_status sd2_rope_attention(void* q, const void* k, const void* v, void* k_cache, void* v_cache, void* out, int64_t N,
+                              int64_t heads_q, int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta,
+                              void* cuda_stream);
 
 /* y = a + b over `count` elements (residual connection).  y may be a or b. */
 sd2_status sd2_add(const void* a, const void* b, void* y, int64_t count, void* cuda_stream);

@@ -27,7 +27,7 @@ EXPORTS = [
     "sd2_block_workspace_bytes", "sd2_block_workspace_layout", "sd2_status_string", "sd2_stream_check",
     "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
     "sd2_block_step_static", "sd2_selftest_timeout", "sd2_drafter_query",
-    "sd2_rmsnorm", "sd2_rope_cache", "sd2_attention_decode", "sd2_add", "sd2_embedding", "sd2_lm_head",
+    "sd2_rmsnorm", "sd2_add_rmsnorm", "sd2_rope_cache", "sd2_attention_decode", "sd2_rope_attention", "sd2_add", "sd2_embedding", "sd2_lm_head",
     "sd2_decoder_workspace_bytes", "sd2_decoder_block_step",
 ]
 
@@ -81,8 +81,10 @@ def lib():
             "sd2_block_step_static": [pp, p, p, i64, p],
             "sd2_selftest_timeout": [p],
             "sd2_rmsnorm": [p, p, p, i64, i64, ctypes.c_float, p],
+            "sd2_add_rmsnorm": [p, p, p, p, p, i64, i64, ctypes.c_float, p],
             "sd2_rope_cache": [p, p, p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p],
             "sd2_attention_decode": [p, p, p, p, i64, i64, i64, i64, i64, i64, p],
+            "sd2_rope_attention": [p, p, p, p, p, p, i64, i64, i64, i64, i64, i64, ctypes.c_double, p],
             "sd2_add": [p, p, p, i64, p],
             "sd2_embedding": [p, p, p, i64, i64, i64, p],
             "sd2_lm_head": [p, p, p, p, i64, i64, i64, p],
@@ -344,6 +346,11 @@ def sd2_rmsnorm(x, w, y, eps: float, stream=None):
     _check(lib().sd2_rmsnorm(_ptr(x), _ptr(w), _ptr(y), N, H, eps, _stream(stream)), "sd2_rmsnorm")
 
 
+def sd2_add_rmsnorm(a, b, total, w, y, eps: float, stream=None):
+    N, H = a.shape
+    _check(lib().sd2_add_rmsnorm(_ptr(a), _ptr(b), _ptr(total), _ptr(w), _ptr(y), N, H, eps, _stream(stream)), "sd2_add_rmsnorm")
+
+
 def sd2_rope_cache(q, k, v, k_cache, v_cache, heads_q: int, heads_kv: int, pos: int, theta: float, stream=None):
     """q [N, heads_q*d] rotated in place; rope(k), v appended at ``pos`` of the caches [N, T_max, heads_kv*d]."""
     N = q.shape[0]
@@ -357,6 +364,13 @@ def sd2_attention_decode(q, k_cache, v_cache, out, heads_q: int, heads_kv: int, 
     d = q.shape[1] // heads_q
     _check(lib().sd2_attention_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), N, heads_q, heads_kv, d, T,
                                       k_cache.shape[1], _stream(stream)), "sd2_attention_decode")
+
+
+def sd2_rope_attention(q, k, v, k_cache, v_cache, out, heads_q: int, heads_kv: int, pos: int, theta: float, stream=None):
+    N = q.shape[0]
+    d = q.shape[1] // heads_q
+    _check(lib().sd2_rope_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), _ptr(out), N, heads_q, heads_kv, d,
+                                    pos, k_cache.shape[1], theta, _stream(stream)), "sd2_rope_attention")
 
 
 def sd2_add(a, b, y, stream=None):

@@ -973,6 +973,17 @@ sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
+sd2_status sd2_add_rmsnorm(const void* a, const void* b, void* sum, const void* w, void* y, int64_t N, int64_t H, float eps,
+                           void* cuda_stream)
+{
+    if (!a || !b || !sum || !w || !y) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || H < 1 || N > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
+    if (N == 0) return SD2_OK;
+    add_rmsnorm_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((const uint16_t*)a, (const uint16_t*)b, (uint16_t*)sum,
+                                                                                     (const uint16_t*)w, (uint16_t*)y, (int)H, eps);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
 sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, void* v_cache, int64_t N, int64_t heads_q,
                           int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta, void* cuda_stream)
 {
@@ -1001,6 +1012,24 @@ sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* 
     attention_decode_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)T * 4, (cudaStream_t)cuda_stream>>>(
         (const uint16_t*)q, (const uint16_t*)k_cache, (const uint16_t*)v_cache, (uint16_t*)out, (int)heads_q, (int)heads_kv, (int)head_dim,
         (int)T, (int)T_max, vec);
+    return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
+}
+
+sd2_status sd2_rope_attention(void* q, const void* k, const void* v, void* k_cache, void* v_cache, void* out, int64_t N,
+                              int64_t heads_q, int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta,
+                              void* cuda_stream)
+{
+    if (!q || !k || !v || !k_cache || !v_cache || !out) return SD2_ERR_INVALID_ARG;
+    if (N < 0 || heads_q < 1 || heads_kv < 1 || heads_q % heads_kv || head_dim < 2 || (head_dim & 1) || pos < 0 || pos >= T_max ||
+        T_max > 0x7FFFFFFF || N * heads_q > 0x7FFFFFFF || !(theta > 0.0))
+        return SD2_ERR_SHAPE;
+    if (head_dim > 128 || pos + 1 > kAttnMaxT) return SD2_ERR_UNSUPPORTED;
+    if (N == 0) return SD2_OK;
+    const bool pow2 = (head_dim & (head_dim - 1)) == 0;
+    const int vec = (pow2 && head_dim >= 8 && ((((uintptr_t)k_cache) | ((uintptr_t)v_cache)) & 15) == 0) ? 1 : 0;
+    rope_attention_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)(pos + 1) * 4, (cudaStream_t)cuda_stream>>>(
+        (uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, (uint16_t*)k_cache, (uint16_t*)v_cache, (uint16_t*)out, (int)heads_q,
+        (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, theta, vec);
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
@@ -1099,13 +1128,11 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
     if ((st = sd2_rmsnorm(x, norm_attn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
     void* yqkv[3] = {q, k, v};
     if ((st = run_group(h, 3, xn, nullptr, nullptr, nullptr, yqkv, N, true, s)) != SD2_OK) return st;
-    if ((st = sd2_rope_cache(q, k, v, k_cache, v_cache, N, heads_q, heads_kv, hd, pos, T_max, theta, s)) != SD2_OK) return st;
-    if ((st = sd2_attention_decode(q, k_cache, v_cache, att, N, heads_q, heads_kv, hd, pos + 1, T_max, s)) != SD2_OK) return st;
+    if ((st = sd2_rope_attention(q, k, v, k_cache, v_cache, att, N, heads_q, heads_kv, hd, pos, T_max, theta, s)) != SD2_OK) return st;
     void* yo[1] = {hdn};
     if ((st = run_group(h + 3, 1, att, nullptr, nullptr, nullptr, yo, N, true, s)) != SD2_OK) return st;
-    if ((st = sd2_add(x, hdn, x1, N * d.hidden, s)) != SD2_OK) return st;
-    // feed-forward module: y = x1 + Wd (silu(Wg m) * Wu m), m = rmsnorm(x1)
-    if ((st = sd2_rmsnorm(x1, norm_ffn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
+    // feed-forward module: y = x1 + Wd (silu(Wg m) * Wu m), m = rmsnorm(x1); the residual and the norm in one launch
+    if ((st = sd2_add_rmsnorm(x, hdn, x1, norm_ffn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
     void* ygu[2] = {g, u};
     if ((st = run_group(h + 4, 2, xn, nullptr, nullptr, nullptr, ygu, N, true, s)) != SD2_OK) return st;
     void* yd[1] = {dn};

@@ -86,6 +86,24 @@ __global__ void __launch_bounds__(kGlueThreads) rmsnorm_kernel(const uint16_t* x
     }
 }
 
+// s = a + b (rounded to bf16 and stored), y = rmsnorm(s) * w: the residual connection and the norm that follows it in
+// one pass over the row.  One CTA per row; the second pass re-reads what the same thread stored.
+__global__ void __launch_bounds__(kGlueThreads) add_rmsnorm_kernel(const uint16_t* a, const uint16_t* b, uint16_t* sum, const uint16_t* w,
+                                                                  uint16_t* y, int H, float eps)
+{
+    __shared__ float red[32];
+    const size_t r0 = (size_t)blockIdx.x * H;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < H; i += blockDim.x) {
+        const uint16_t sb = f32_to_bf16_rne(bf16_to_f32(a[r0 + i]) + bf16_to_f32(b[r0 + i]));
+        sum[r0 + i] = sb;
+        const float v = bf16_to_f32(sb);
+        ss += v * v;
+    }
+    const float r = rsqrtf(block_sum(ss, red) / (float)H + eps);
+    for (int i = threadIdx.x; i < H; i += blockDim.x) y[r0 + i] = f32_to_bf16_rne(bf16_to_f32(sum[r0 + i]) * r * bf16_to_f32(w[i]));
+}
+
 // Rotates q in place and writes the rotated k and the plain v of row n into position `pos` of row n's cache.
 // Caches are [N, T_max, Hkv * d].  One CTA per row.
 __global__ void __launch_bounds__(kGlueThreads) rope_cache_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
@@ -221,6 +239,149 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
     __syncthreads();
     if (threadIdx.x < d) {
         float a = 0.f;
+        for (int w = 0; w < nw; ++w) a += part[w * 128 + threadIdx.x];
+        out[((size_t)n * Hq + h) * d + threadIdx.x] = f32_to_bf16_rne(a / z);
+    }
+}
+
+// sd2_rope_cache and sd2_attention_decode in one launch, one CTA per (row, query head): the CTA rotates its query head
+// (and writes it back), rotates the key head of its group for itself, and attends over the cached positions 0..pos-1
+// plus the new token, whose key and value it takes from its own shared memory and from `v`, not from the cache; the
+// first head of every group also appends the rotated key and the value to the caches.  No CTA reads what another writes.
+__global__ void __launch_bounds__(kAttnThreads) rope_attention_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
+                                                                     uint16_t* vc, uint16_t* out, int Hq, int Hkv, int d, int pos,
+                                                                     int T_max, double theta, int vec)
+{
+    extern __shared__ float sc[];            // pos + 1 scores, then the weights
+    __shared__ float red[32];
+    __shared__ float qs[128], ks[128], cs_tab[128];
+    __shared__ float part[(kAttnThreads / 32) * 128];
+    const int n = blockIdx.x / Hq, h = blockIdx.x % Hq, group = Hq / Hkv, g = h / group;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    const int half = d / 2, T = pos;         // cached positions; the new token is handled apart
+    if (threadIdx.x < half) {
+        double sn, cs;
+        sincos((double)pos * pow(theta, -2.0 * (double)threadIdx.x / (double)d), &sn, &cs);
+        cs_tab[threadIdx.x] = (float)cs;
+        cs_tab[half + threadIdx.x] = (float)sn;
+    }
+    __syncthreads();
+    uint16_t* qr = q + ((size_t)n * Hq + h) * d;
+    const uint16_t* kr = k + ((size_t)n * Hkv + g) * d;
+    const size_t pitch = (size_t)Hkv * d;
+    uint16_t* kdst = kc + ((size_t)n * T_max + pos) * pitch + (size_t)g * d;
+    uint16_t* vdst = vc + ((size_t)n * T_max + pos) * pitch + (size_t)g * d;
+    const uint16_t* vnew = v + ((size_t)n * Hkv + g) * d;
+    const bool writer = (h % group) == 0;
+    if (threadIdx.x < half) {
+        const int i = threadIdx.x;
+        const float c = cs_tab[i], sn = cs_tab[half + i];
+        const float a = bf16_to_f32(qr[i]), b = bf16_to_f32(qr[i + half]);
+        const uint16_t q0 = f32_to_bf16_rne(a * c - b * sn), q1 = f32_to_bf16_rne(b * c + a * sn);
+        qr[i] = q0;
+        qr[i + half] = q1;
+        qs[i] = bf16_to_f32(q0);
+        qs[i + half] = bf16_to_f32(q1);
+        const float ka = bf16_to_f32(kr[i]), kb2 = bf16_to_f32(kr[i + half]);
+        const uint16_t k0 = f32_to_bf16_rne(ka * c - kb2 * sn), k1 = f32_to_bf16_rne(kb2 * c + ka * sn);
+        ks[i] = bf16_to_f32(k0);
+        ks[i + half] = bf16_to_f32(k1);
+        if (writer) {
+            kdst[i] = k0;
+            kdst[i + half] = k1;
+        }
+    }
+    if (writer && threadIdx.x < d) vdst[threadIdx.x] = vnew[threadIdx.x];
+    __syncthreads();
+    const uint16_t* kb = kc + (size_t)n * T_max * pitch + (size_t)g * d;
+    const uint16_t* vb = vc + (size_t)n * T_max * pitch + (size_t)g * d;
+    const float scale = rsqrtf((float)d);
+    const int lpp = d >> 3;
+    const int ppw = vec ? 32 / lpp : 1;
+    const int sub = vec ? lane / lpp : 0, dl = vec ? (lane % lpp) * 8 : 0;
+    if (vec) {
+        float qv[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) qv[j] = qs[dl + j];
+#pragma unroll 4
+        for (int t0 = warp * ppw; t0 < T; t0 += nw * ppw) {
+            const int t = t0 + sub;
+            float s = 0.f;
+            if (t < T) {
+                const uint4 kv = *(const uint4*)(kb + (size_t)t * pitch + dl);
+                const uint32_t u[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s += qv[2 * j] * bf16_lo(u[j]) + qv[2 * j + 1] * bf16_hi(u[j]);
+            }
+            for (int dd = 1; dd < lpp; dd <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+            if (t < T && (lane % lpp) == 0) sc[t] = s * scale;
+        }
+    } else {
+#pragma unroll 4
+        for (int t = warp; t < T; t += nw) {
+            float s = 0.f;
+            for (int i = lane; i < d; i += 32) s += qs[i] * bf16_to_f32(kb[(size_t)t * pitch + i]);
+            for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+            if (lane == 0) sc[t] = s * scale;
+        }
+    }
+    if (warp == 0) {                         // the new token's own score
+        float s = 0.f;
+        for (int i = lane; i < d; i += 32) s += qs[i] * ks[i];
+        for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+        if (lane == 0) sc[T] = s * scale;
+    }
+    __syncthreads();
+    float m = -INFINITY;
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) m = fmaxf(m, sc[t]);
+    m = block_max(m, red);
+    float z = 0.f;
+    for (int t = threadIdx.x; t <= T; t += blockDim.x) {
+        const float e = expf(sc[t] - m);
+        sc[t] = e;
+        z += e;
+    }
+    z = block_sum(z, red);
+    __syncthreads();
+    if (vec) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int t0 = warp * ppw; t0 < T; t0 += nw * ppw) {
+            const int t = t0 + sub;
+            if (t < T) {
+                const float p = sc[t];
+                const uint4 vv = *(const uint4*)(vb + (size_t)t * pitch + dl);
+                const uint32_t u[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    acc[2 * j] += p * bf16_lo(u[j]);
+                    acc[2 * j + 1] += p * bf16_hi(u[j]);
+                }
+            }
+        }
+        for (int dd = lpp; dd < 32; dd <<= 1)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], dd);
+        if (lane < lpp)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) part[warp * 128 + dl + j] = acc[j];
+    } else {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int t = warp; t < T; t += nw) {
+            const float p = sc[t];
+            const uint16_t* vr = vb + (size_t)t * pitch;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (lane + 32 * j < d) acc[j] += p * bf16_to_f32(vr[lane + 32 * j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (lane + 32 * j < d) part[warp * 128 + lane + 32 * j] = acc[j];
+    }
+    __syncthreads();
+    if (threadIdx.x < d) {
+        float a = sc[T] * bf16_to_f32(vnew[threadIdx.x]);
         for (int w = 0; w < nw; ++w) a += part[w * 128 + threadIdx.x];
         out[((size_t)n * Hq + h) * d + threadIdx.x] = f32_to_bf16_rne(a / z);
     }

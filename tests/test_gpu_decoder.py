@@ -48,6 +48,21 @@ def test_rmsnorm(N, H):
     close_bf16(bits_of(y), do.rmsnorm(f64(x), f64(w), EPS), 1e-5)
 
 
+def test_add_rmsnorm_is_the_two_operations_in_a_row():
+    N, H = 4, 2048
+    a = synth.normal_bf16(150, (N, H), 1.0)
+    b = synth.normal_bf16(151, (N, H), 0.3)
+    w = synth.normal_bf16(152, (H,), 0.5)
+    total = torch.zeros((N, H), dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros((N, H), dtype=torch.bfloat16, device="cuda")
+    sd2.sd2_add_rmsnorm(dev(a), dev(b), total, dev(w), y, EPS)
+    torch.cuda.synchronize()
+    ref = f64(a) + f64(b)
+    want = np.array([oracle.f64_to_bf16_rne(float(z)) for z in ref.ravel()], np.uint16).reshape(ref.shape)
+    assert np.array_equal(bits_of(total), want)
+    close_bf16(bits_of(y), do.rmsnorm(f64(want), f64(w), EPS), 1e-5)
+
+
 @pytest.mark.parametrize("pos", [0, 1, 77, 4000])
 def test_rope_and_cache_append(pos):
     N, Hq, Hkv, d, T_max = 3, 8, 2, 64, 4096 + 8
@@ -85,6 +100,31 @@ def test_attention_decode(N, Hq, Hkv, d, T):
     for n in range(N):
         ref = do.attention_decode(f64(q[n]).reshape(Hq, d), f64(kc[n, :T]).reshape(T, Hkv, d), f64(vc[n, :T]).reshape(T, Hkv, d))
         close_bf16(got[n], ref, 2e-4 * float(np.abs(f64(vc[n, :T])).max()))
+
+
+@pytest.mark.parametrize("N,Hq,Hkv,d,pos", [(1, 32, 8, 64, 300), (2, 12, 2, 128, 0), (2, 4, 2, 24, 37), (3, 8, 8, 64, 1)])
+def test_rope_attention_in_one_launch_equals_the_two_calls(N, Hq, Hkv, d, pos):
+    T_max = pos + 4
+    q = synth.normal_bf16(350 + pos, (N, Hq * d), 1.0)
+    k = synth.normal_bf16(351 + pos, (N, Hkv * d), 1.0)
+    v = synth.normal_bf16(352 + pos, (N, Hkv * d), 1.0)
+    kc = synth.normal_bf16(353 + pos, (N, T_max, Hkv * d), 1.0)
+    vc = synth.normal_bf16(354 + pos, (N, T_max, Hkv * d), 1.0)
+    q1, kc1, vc1 = dev(q), dev(kc), dev(vc)
+    out1 = torch.zeros((N, Hq * d), dtype=torch.bfloat16, device="cuda")
+    sd2.sd2_rope_cache(q1, dev(k), dev(v), kc1, vc1, Hq, Hkv, pos, THETA)
+    sd2.sd2_attention_decode(q1, kc1, vc1, out1, Hq, Hkv, pos + 1)
+    q2, kc2, vc2 = dev(q), dev(kc), dev(vc)
+    out2 = torch.zeros((N, Hq * d), dtype=torch.bfloat16, device="cuda")
+    sd2.sd2_rope_attention(q2, dev(k), dev(v), kc2, vc2, out2, Hq, Hkv, pos, THETA)
+    torch.cuda.synchronize()
+    assert torch.equal(q1, q2) and torch.equal(kc1, kc2) and torch.equal(vc1, vc2)       # same rotation, same append
+    got = bits_of(out2).reshape(N, Hq, d)
+    kcb, vcb = bits_of(kc2), bits_of(vc2)
+    for n in range(N):
+        ref = do.attention_decode(f64(bits_of(q2)[n]).reshape(Hq, d), f64(kcb[n, :pos + 1]).reshape(pos + 1, Hkv, d),
+                                  f64(vcb[n, :pos + 1]).reshape(pos + 1, Hkv, d))
+        close_bf16(got[n], ref, 2e-4 * float(np.abs(f64(vcb[n, :pos + 1])).max()))
 
 
 def test_add_embedding():
