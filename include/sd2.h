@@ -305,6 +305,12 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
                                   void* k_cache, void* v_cache, int64_t N, int64_t heads_q, int64_t heads_kv, int64_t pos,
                                   int64_t T_max, float eps, double theta, void* workspace, void* cuda_stream);
 
+/* Failure injection for tests (the paper has no counterpart): the next `skip` allocations the library makes
+ * for itself (host blobs and staging copies, handle and drafter objects, device memory) succeed, the `fail`
+ * after them fail as if memory had run out; (0, 0) switches it off.  A call that meets a failed allocation
+ * returns SD2_ERR_ALLOC and releases what it had taken.  Process-wide, not meant for concurrent use. */
+sd2_status sd2_debug_fail_allocations(int64_t skip, int64_t fail);
+
 /* Static string for a status code. */
 const char* sd2_status_string(sd2_status s);
 

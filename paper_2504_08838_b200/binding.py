@@ -28,7 +28,7 @@ EXPORTS = [
     "sd2_drafter_create", "sd2_drafter_step", "sd2_drafter_buffers", "sd2_drafter_free",
     "sd2_block_step_static", "sd2_selftest_timeout", "sd2_drafter_query",
     "sd2_rmsnorm", "sd2_add_rmsnorm", "sd2_rope_cache", "sd2_attention_decode", "sd2_rope_attention", "sd2_add", "sd2_embedding", "sd2_lm_head",
-    "sd2_decoder_workspace_bytes", "sd2_decoder_block_step",
+    "sd2_decoder_workspace_bytes", "sd2_decoder_block_step", "sd2_debug_fail_allocations",
 ]
 
 
@@ -88,6 +88,7 @@ def lib():
             "sd2_add": [p, p, p, i64, p],
             "sd2_embedding": [p, p, p, i64, i64, i64, p],
             "sd2_lm_head": [p, p, p, p, i64, i64, i64, p],
+            "sd2_debug_fail_allocations": [i64, i64],
             "sd2_decoder_workspace_bytes": [pp, i64, pi64],
             "sd2_decoder_block_step": [pp, p, p, p, p, p, p, i64, i64, i64, i64, i64, ctypes.c_float, ctypes.c_double, p, p],
         }
@@ -402,3 +403,8 @@ def sd2_decoder_block_step(hs, norm_attn, norm_ffn, x, y, k_cache, v_cache, head
     _check(lib().sd2_decoder_block_step(arr, _ptr(norm_attn), _ptr(norm_ffn), _ptr(x), _ptr(y), _ptr(k_cache), _ptr(v_cache), N,
                                         heads_q, heads_kv, pos, k_cache.shape[1], eps, theta, _ptr(workspace), _stream(stream)),
            "sd2_decoder_block_step")
+
+
+def sd2_debug_fail_allocations(skip: int, fail: int):
+    """Let the library's next ``skip`` allocations through and fail the ``fail`` after them; (0, 0) = off."""
+    _check(lib().sd2_debug_fail_allocations(skip, fail), "sd2_debug_fail_allocations")

@@ -2,6 +2,7 @@
 // points, kernel dispatch.  No torch types, no exceptions across the boundary.
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <atomic>
 #include <cstdio>
@@ -58,6 +59,22 @@ struct sd2_drafter_s {
 };
 
 namespace {
+
+// cudaMalloc behind the same failure plan as the host allocations (see lib_alloc_fails)
+cudaError_t dev_malloc(void** p, size_t n)
+{
+    if (lib_alloc_fails()) { *p = nullptr; return cudaErrorMemoryAllocation; }
+    return cudaMalloc(p, n);
+}
+template <class T>
+cudaError_t dev_malloc(T** p, size_t n) { return dev_malloc((void**)p, n); }
+
+// NVTX range over a call (a profiler's timeline then shows the library's calls by name; without a profiler
+// attached the push and pop are a pointer test each)
+struct Range {
+    explicit Range(const char* name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
 
 std::mutex g_mu;
 std::unordered_set<sd2_handle> g_live;
@@ -134,8 +151,8 @@ sd2_status ensure_device(int* dev_out)
         int* err = nullptr;
         unsigned int* bars = nullptr;
         const size_t bar_bytes = (size_t)kBarrierPool * kBarrierStrideWords * 4;
-        if (cudaMalloc((void**)&err, 256) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_ALLOC; }
-        if (cudaMalloc((void**)&bars, bar_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(err); return SD2_ERR_ALLOC; }
+        if (dev_malloc((void**)&err, 256) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_ALLOC; }
+        if (dev_malloc((void**)&bars, bar_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(err); return SD2_ERR_ALLOC; }
         if (cudaMemset(err, 0, 256) != cudaSuccess || cudaMemset(bars, 0, bar_bytes) != cudaSuccess) {
             cudaGetLastError();
             cudaFree(err);
@@ -195,10 +212,10 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
     int dev = 0;
     sd2_status st = ensure_device(&dev);
     if (st != SD2_OK) return st;
-    sd2_handle h = new (std::nothrow) sd2_handle_s();
+    sd2_handle h = lib_alloc_fails() ? nullptr : new (std::nothrow) sd2_handle_s();
     if (!h) return SD2_ERR_ALLOC;
     void* d = nullptr;
-    if (cudaMalloc(&d, (size_t)bytes) != cudaSuccess) { cudaGetLastError(); delete h; return SD2_ERR_ALLOC; }
+    if (dev_malloc(&d, (size_t)bytes) != cudaSuccess) { cudaGetLastError(); delete h; return SD2_ERR_ALLOC; }
     if (cudaMemcpy(d, blob, (size_t)bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(d);
@@ -227,7 +244,7 @@ sd2_status upload(const uint8_t* blob, int64_t bytes, const BlobHeader& hd, sd2_
         const int64_t panels = (hd.M + kMmaBlockRows - 1) / kMmaBlockRows;
         h->partial_bytes = (int64_t)kMmaMaxRows * panels * kMmaBlockRows * 4 + panels * 4;
         void* pp = nullptr;
-        if (cudaMalloc(&pp, (size_t)h->partial_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(d); delete h; return SD2_ERR_ALLOC; }
+        if (dev_malloc(&pp, (size_t)h->partial_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(d); delete h; return SD2_ERR_ALLOC; }
         if (cudaMemset(pp, 0, (size_t)h->partial_bytes) != cudaSuccess) { cudaGetLastError(); cudaFree(pp); cudaFree(d); delete h; return SD2_ERR_CUDA; }
         h->d_partial = (float*)pp;
     }
@@ -753,8 +770,8 @@ sd2_status build_gate_up_pair(sd2_handle gate, sd2_handle up, sd2_handle* out)
     if (up->M != I || up->K != K) return SD2_OK;
     const Gap4Geom g = gap4_geometry(2 * I, K, true);
     if (g.S == 0 || g.R < 2) return SD2_OK;
-    uint16_t* dense = (uint16_t*)std::malloc((size_t)(2 * I * K) * 2);
-    uint16_t* one = (uint16_t*)std::malloc((size_t)(I * K) * 2);
+    uint16_t* dense = (uint16_t*)lib_malloc((size_t)(2 * I * K) * 2);
+    uint16_t* one = (uint16_t*)lib_malloc((size_t)(I * K) * 2);
     sd2_status st = (dense && one) ? SD2_OK : SD2_ERR_ALLOC;
     for (int w = 0; w < 2 && st == SD2_OK; ++w) {
         st = sd2_decompress(w == 0 ? gate : up, one);
@@ -841,6 +858,7 @@ sd2_status sd2_blob_free(void* blob)
 sd2_status sd2_compress(const void* weight_bf16, const uint8_t* mask, int64_t M, int64_t K, const sd2_options* opt,
                         sd2_handle* out)
 {
+    Range range_("sd2_compress");
     if (!weight_bf16 || !out) return SD2_ERR_INVALID_ARG;
     if (M < 1 || K < 1 || M * K > (1ll << 40)) return SD2_ERR_SHAPE;
     const uint16_t* W = (const uint16_t*)weight_bf16;
@@ -848,13 +866,13 @@ sd2_status sd2_compress(const void* weight_bf16, const uint8_t* mask, int64_t M,
     uint8_t* m_tmp = nullptr;
     sd2_status st = SD2_OK;
     if (is_device_ptr(weight_bf16)) {
-        w_tmp = (uint16_t*)std::malloc((size_t)(M * K) * 2);
+        w_tmp = (uint16_t*)lib_malloc((size_t)(M * K) * 2);
         if (!w_tmp) return SD2_ERR_ALLOC;
         if (cudaMemcpy(w_tmp, weight_bf16, (size_t)(M * K) * 2, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
         W = w_tmp;
     }
     if (st == SD2_OK && mask && is_device_ptr(mask)) {
-        m_tmp = (uint8_t*)std::malloc((size_t)(M * K));
+        m_tmp = (uint8_t*)lib_malloc((size_t)(M * K));
         if (!m_tmp) st = SD2_ERR_ALLOC;
         else if (cudaMemcpy(m_tmp, mask, (size_t)(M * K), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
         mask = m_tmp;
@@ -891,13 +909,13 @@ sd2_status sd2_load_blob(const void* blob, int64_t blob_bytes, sd2_handle* out)
 sd2_status sd2_decompress(sd2_handle h, void* dense_bf16_out)
 {
     if (!live(h) || !dense_bf16_out) return SD2_ERR_INVALID_ARG;
-    uint8_t* blob = (uint8_t*)std::malloc((size_t)h->blob_bytes);
+    uint8_t* blob = (uint8_t*)lib_malloc((size_t)h->blob_bytes);
     if (!blob) return SD2_ERR_ALLOC;
     sd2_status st = SD2_OK;
     if (cudaMemcpy(blob, h->d_blob, (size_t)h->blob_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); st = SD2_ERR_CUDA; }
     const size_t dense_bytes = (size_t)(h->M * h->K) * 2;
     const bool to_dev = is_device_ptr(dense_bf16_out);
-    uint16_t* host_out = to_dev ? (uint16_t*)std::malloc(dense_bytes) : (uint16_t*)dense_bf16_out;
+    uint16_t* host_out = to_dev ? (uint16_t*)lib_malloc(dense_bytes) : (uint16_t*)dense_bf16_out;
     if (!host_out) st = SD2_ERR_ALLOC;
     if (st == SD2_OK) st = sd2_unpack_host(blob, h->blob_bytes, host_out, nullptr, nullptr, nullptr, nullptr, nullptr);
     if (st == SD2_OK && to_dev &&
@@ -956,7 +974,7 @@ sd2_status sd2_stream_check(void* cuda_stream)
                 if (h->device == dev && h->d_partial) cudaMemset(h->d_partial, 0, (size_t)h->partial_bytes);
         }
         cudaGetLastError();
-        return SD2_ERR_TIMEOUT;
+        return flag == 2 ? SD2_ERR_CORRUPT : SD2_ERR_TIMEOUT;      // 2: an index check of a checked build failed
     }
     return SD2_OK;
 }
@@ -965,6 +983,7 @@ sd2_status sd2_stream_check(void* cuda_stream)
 
 sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t H, float eps, void* cuda_stream)
 {
+    Range range_("sd2_rmsnorm");
     if (!x || !w || !y) return SD2_ERR_INVALID_ARG;
     if (N < 0 || H < 1 || N > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;
@@ -976,6 +995,7 @@ sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t
 sd2_status sd2_add_rmsnorm(const void* a, const void* b, void* sum, const void* w, void* y, int64_t N, int64_t H, float eps,
                            void* cuda_stream)
 {
+    Range range_("sd2_add_rmsnorm");
     if (!a || !b || !sum || !w || !y) return SD2_ERR_INVALID_ARG;
     if (N < 0 || H < 1 || N > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;
@@ -1001,6 +1021,7 @@ sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, 
 sd2_status sd2_attention_decode(const void* q, const void* k_cache, const void* v_cache, void* out, int64_t N, int64_t heads_q,
                                 int64_t heads_kv, int64_t head_dim, int64_t T, int64_t T_max, void* cuda_stream)
 {
+    Range range_("sd2_attention_decode");
     if (!q || !k_cache || !v_cache || !out) return SD2_ERR_INVALID_ARG;
     if (N < 0 || heads_q < 1 || heads_kv < 1 || heads_q % heads_kv || head_dim < 1 || T < 1 || T > T_max || T_max > 0x7FFFFFFF ||
         N * heads_q > 0x7FFFFFFF)
@@ -1019,6 +1040,7 @@ sd2_status sd2_rope_attention(void* q, const void* k, const void* v, void* k_cac
                               int64_t heads_q, int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta,
                               void* cuda_stream)
 {
+    Range range_("sd2_rope_attention");
     if (!q || !k || !v || !k_cache || !v_cache || !out) return SD2_ERR_INVALID_ARG;
     if (N < 0 || heads_q < 1 || heads_kv < 1 || heads_q % heads_kv || head_dim < 2 || (head_dim & 1) || pos < 0 || pos >= T_max ||
         T_max > 0x7FFFFFFF || N * heads_q > 0x7FFFFFFF || !(theta > 0.0))
@@ -1056,6 +1078,7 @@ sd2_status sd2_embedding(const int32_t* tokens, const void* table, void* x, int6
 sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t* tokens, int64_t N, int64_t V, int64_t H,
                        void* cuda_stream)
 {
+    Range range_("sd2_lm_head");
     if (!x || !w_out || !logits) return SD2_ERR_INVALID_ARG;
     if (N < 0 || V < 1 || H < 1 || V > 0x7FFFFFFF || H > 0x7FFFFFFF) return SD2_ERR_SHAPE;
     if ((H & 7) || (((uintptr_t)w_out) & 15)) return SD2_ERR_UNSUPPORTED;
@@ -1102,6 +1125,7 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
                                   void* k_cache, void* v_cache, int64_t N, int64_t heads_q, int64_t heads_kv, int64_t pos,
                                   int64_t T_max, float eps, double theta, void* workspace, void* cuda_stream)
 {
+    Range range_("sd2_decoder_block_step");
     if (!norm_attn || !norm_ffn || !x || !y || !k_cache || !v_cache || !workspace) return SD2_ERR_INVALID_ARG;
     if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
@@ -1127,17 +1151,38 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
     // attention module: x1 = x + Wo attention(rope(Wq n), cache + rope(Wk n), cache + Wv n), n = rmsnorm(x)
     if ((st = sd2_rmsnorm(x, norm_attn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
     void* yqkv[3] = {q, k, v};
-    if ((st = run_group(h, 3, xn, nullptr, nullptr, nullptr, yqkv, N, true, s)) != SD2_OK) return st;
+    nvtxRangePushA("q|k|v");
+    st = run_group(h, 3, xn, nullptr, nullptr, nullptr, yqkv, N, true, s);
+    nvtxRangePop();
+    if (st != SD2_OK) return st;
     if ((st = sd2_rope_attention(q, k, v, k_cache, v_cache, att, N, heads_q, heads_kv, hd, pos, T_max, theta, s)) != SD2_OK) return st;
     void* yo[1] = {hdn};
-    if ((st = run_group(h + 3, 1, att, nullptr, nullptr, nullptr, yo, N, true, s)) != SD2_OK) return st;
+    nvtxRangePushA("o");
+    st = run_group(h + 3, 1, att, nullptr, nullptr, nullptr, yo, N, true, s);
+    nvtxRangePop();
+    if (st != SD2_OK) return st;
     // feed-forward module: y = x1 + Wd (silu(Wg m) * Wu m), m = rmsnorm(x1); the residual and the norm in one launch
     if ((st = sd2_add_rmsnorm(x, hdn, x1, norm_ffn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
     void* ygu[2] = {g, u};
-    if ((st = run_group(h + 4, 2, xn, nullptr, nullptr, nullptr, ygu, N, true, s)) != SD2_OK) return st;
+    nvtxRangePushA("gate|up");
+    st = run_group(h + 4, 2, xn, nullptr, nullptr, nullptr, ygu, N, true, s);
+    nvtxRangePop();
+    if (st != SD2_OK) return st;
     void* yd[1] = {dn};
-    if ((st = run_group(h + 6, 1, nullptr, g, u, t, yd, N, true, s)) != SD2_OK) return st;
+    nvtxRangePushA("down");
+    st = run_group(h + 6, 1, nullptr, g, u, t, yd, N, true, s);
+    nvtxRangePop();
+    if (st != SD2_OK) return st;
     return sd2_add(x1, dn, y, N * d.hidden, s);
+}
+
+sd2_status sd2_debug_fail_allocations(int64_t skip, int64_t fail)
+{
+    if (skip < 0 || fail < 0) return SD2_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_mu);
+    alloc_plan().skip_left = skip;
+    alloc_plan().fail_left = fail;
+    return SD2_OK;
 }
 
 sd2_status sd2_selftest_timeout(void* cuda_stream)
@@ -1152,6 +1197,7 @@ sd2_status sd2_selftest_timeout(void* cuda_stream)
 
 sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_stream)
 {
+    Range range_("sd2_spmm");
     if (!X || !Y) return SD2_ERR_INVALID_ARG;
     void* ys[1] = {Y};
     return run_group(&h, 1, (const uint16_t*)X, nullptr, nullptr, nullptr, ys, N, false, (cudaStream_t)cuda_stream);
@@ -1160,6 +1206,7 @@ sd2_status sd2_spmm(sd2_handle h, const void* X, void* Y, int64_t N, void* cuda_
 sd2_status sd2_spmm_fused(const sd2_handle* h, int32_t count, const void* X, void* const* Y, int64_t N,
                           void* cuda_stream)
 {
+    Range range_("sd2_spmm_fused");
     if (!h || !X || !Y) return SD2_ERR_INVALID_ARG;
     return run_group(h, count, (const uint16_t*)X, nullptr, nullptr, nullptr, Y, N, false, (cudaStream_t)cuda_stream);
 }
@@ -1192,6 +1239,7 @@ sd2_status sd2_block_workspace_layout(const sd2_handle* h, int64_t N, int64_t* o
 
 sd2_status sd2_block_step(const sd2_handle* h, const void* x, void* y, int64_t N, void* workspace, void* cuda_stream)
 {
+    Range range_("sd2_block_step");
     if (!x || !y || !workspace) return SD2_ERR_INVALID_ARG;
     if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
@@ -1253,6 +1301,7 @@ unsigned char* g_static_ptr[kMaxDevices];   // device address of g_static_scratc
 
 sd2_status sd2_block_step_static(const sd2_handle* h, const void* x, void* y, int64_t N, void* cuda_stream)
 {
+    Range range_("sd2_block_step_static");
     if (!x || !y) return SD2_ERR_INVALID_ARG;
     if (N < 0 || N > kMaxBlockRows) return SD2_ERR_SHAPE;
     BlockDims d;
@@ -1315,7 +1364,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
         }
         if (b > 0 && dims[(size_t)b].hidden != dims[(size_t)b - 1].out) return SD2_ERR_SHAPE;
     }
-    sd2_drafter d = new (std::nothrow) sd2_drafter_s();
+    sd2_drafter d = lib_alloc_fails() ? nullptr : new (std::nothrow) sd2_drafter_s();
     if (!d) return SD2_ERR_ALLOC;
     d->L = L;
     d->device = dev;
@@ -1340,7 +1389,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
     d->ws_off[(size_t)L * 8] = o;
     std::vector<SStage> stages((size_t)L * 7);
     ProgramNeeds needs;
-    bool ok = cudaMalloc((void**)&d->d_ws, (size_t)o) == cudaSuccess && cudaMemset(d->d_ws, 0, (size_t)o) == cudaSuccess;
+    bool ok = dev_malloc((void**)&d->d_ws, (size_t)o) == cudaSuccess && cudaMemset(d->d_ws, 0, (size_t)o) == cudaSuccess;
     // Tagged hand-off (stage tags are 8 bits wide): per block q, hdn, g, u, out as 32-bit words
     const bool tagged = 7 * L <= 254;
     std::vector<int64_t> tag_off((size_t)L * 6 + 1, 0);
@@ -1357,7 +1406,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
             }
         }
         d->tags_bytes = to;
-        ok = ok && cudaMalloc((void**)&d->d_tags, (size_t)to) == cudaSuccess && cudaMemset(d->d_tags, 0, (size_t)to) == cudaSuccess;
+        ok = ok && dev_malloc((void**)&d->d_tags, (size_t)to) == cudaSuccess && cudaMemset(d->d_tags, 0, (size_t)to) == cudaSuccess;
     }
     int n = 0;
     std::vector<sd2_handle> pairs((size_t)L, nullptr);
@@ -1398,9 +1447,9 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
                                      tagged ? &tg : nullptr, pairs[(size_t)b]);
         }
         d->n_stages = n;
-        ok = cudaMalloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
+        ok = dev_malloc((void**)&d->d_stages, sizeof(SStage) * (size_t)n) == cudaSuccess &&
              cudaMemcpy(d->d_stages, stages.data(), sizeof(SStage) * (size_t)n, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMalloc((void**)&d->d_gbar, kDrafterWordsBytes) == cudaSuccess && cudaMemset(d->d_gbar, 0, kDrafterWordsBytes) == cudaSuccess;
+             dev_malloc((void**)&d->d_gbar, kDrafterWordsBytes) == cudaSuccess && cudaMemset(d->d_gbar, 0, kDrafterWordsBytes) == cudaSuccess;
     }
     if (ok && widest_panel(needs.xs_need, needs.K_max, needs.max_tile) == 0) {
         for (sd2_handle p : d->owned) sd2_free(p);
@@ -1430,6 +1479,7 @@ sd2_status sd2_drafter_create(const sd2_handle* h, int32_t L, int64_t n_max, sd2
 
 sd2_status sd2_drafter_step(sd2_drafter d, const void* x, void* y, int64_t N, void* cuda_stream)
 {
+    Range range_("sd2_drafter_step");
     if (!live(d) || !x || !y) return SD2_ERR_INVALID_ARG;
     if (N < 0 || N > d->n_max) return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;

@@ -157,6 +157,27 @@ inline uint64_t fnv1a(const uint8_t* p, size_t n)
     return r;
 }
 
+// Failure injection for tests: the library's own host and device allocations go through lib_alloc_fails(), which says
+// "fail" for `fail_left` calls after letting `skip_left` calls through (both 0: never).  Set by sd2_debug_fail_allocations.
+struct AllocPlan {
+    long long skip_left = 0, fail_left = 0;
+};
+inline AllocPlan& alloc_plan()
+{
+    static AllocPlan p;
+    return p;
+}
+inline bool lib_alloc_fails()
+{
+    AllocPlan& p = alloc_plan();
+    if (p.fail_left <= 0) return false;
+    if (p.skip_left > 0) { --p.skip_left; return false; }
+    --p.fail_left;
+    return true;
+}
+inline void* lib_malloc(size_t n) { return lib_alloc_fails() ? nullptr : std::malloc(n); }
+inline void* lib_calloc(size_t n) { return lib_alloc_fails() ? nullptr : std::calloc(n, 1); }
+
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
 
@@ -221,7 +242,7 @@ inline PackResult pack_bitmask(const uint16_t* W, const uint8_t* mask, int64_t M
     size_t sec[3] = {(size_t)(M + 1) * 4, (size_t)(M * K32) * 4, (size_t)nnz * 2};
     BlobHeader h;
     fill_header(h, kFormatBitmask, y_dtype, M, K, nnz, sec, 0);
-    uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
+    uint8_t* blob = (uint8_t*)lib_calloc((size_t)h.total_bytes);
     if (!blob) { r.status = -3; return r; }
     std::memcpy(blob + h.sec_off[0], rvp.data(), sec[0]);
     uint32_t* words = (uint32_t*)(blob + h.sec_off[1]);
@@ -406,7 +427,7 @@ inline PackResult pack_gap4(const uint16_t* W, const uint8_t* mask, int64_t M, i
     h.max_tile_bytes = max_tile;
     h.overlap = (uint32_t)V;
     h.pairing = pair_rows ? 1u : 0u;
-    uint8_t* blob = (uint8_t*)std::calloc((size_t)h.total_bytes, 1);
+    uint8_t* blob = (uint8_t*)lib_calloc((size_t)h.total_bytes);
     if (!blob) { r.status = -3; return r; }
     std::memcpy(blob + h.sec_off[0], toff.data(), sec[0]);
     uint8_t* tiles = blob + h.sec_off[1];

@@ -152,7 +152,7 @@ inline PackResult pack_gap4_mma(const uint16_t* W, const uint8_t* mask, int64_t 
     fill_header(h, kFormatGap4Mma, y_dtype, M, K, nnz, sec_bytes, (uint64_t)chunks_total);
     h.n_tiles = (uint32_t)NB;
     h.max_tile_bytes = max_rec;
-    uint8_t* blob = (uint8_t*)std::calloc(1, (size_t)h.total_bytes);
+    uint8_t* blob = (uint8_t*)lib_calloc((size_t)h.total_bytes);
     if (!blob) { res.status = -3; return res; }
     std::memcpy(blob + h.sec_off[0], dir.data(), sec_bytes[0]);
     if (sec_bytes[1]) std::memcpy(blob + h.sec_off[1], recs.data(), sec_bytes[1]);

@@ -444,10 +444,24 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
             const int cnt = (int)((lds_u32(rec + 16u + 32u * (uint32_t)side + ((uint32_t)lane & ~3u)) >> (8 * (lane & 3))) & 0xFFu);
             uint32_t w = rec + (side ? lds_u32(rec + 12u) : (uint32_t)kMmaBlockHeaderBytes);
             uint32_t cur = at + 4u * (uint32_t)lane + 2u * (uint32_t)side;       // row 0 of this lane's piece
+#ifdef SD2_CHECKED
+            // checked build: what the record says must stay inside its ring slot, and every store inside the tile;
+            // a violation is recorded in the error word (value 2) and the access is skipped
+            const uint32_t slot_end = ring0 + (uint32_t)(slot + 1) * (uint32_t)a.slot_bytes;
+            bool bad = steps > 2 * kMmaBlockRows / 8 || cnt > steps || w < rec || w > slot_end;
+#endif
             for (int j = 0; j < steps; ++j) {
                 const bool active = cnt > j;
                 const uint32_t m = __ballot_sync(0xFFFFFFFFu, active);
                 const uint32_t nj = (uint32_t)__popc(m);
+#ifdef SD2_CHECKED
+                bad = bad || w + ((4u * nj + 15u) & ~15u) + 16u * nj > slot_end;
+                bad = __any_sync(0xFFFFFFFFu, bad);
+                if (bad) {
+                    if (lane == 0 && a.err) atomicExch(a.err, 2);
+                    break;
+                }
+#endif
                 if (active) {
                     const uint32_t idx = (uint32_t)__popc(m & lt);
                     const uint32_t code = lds_u32(w + 4u * idx);
@@ -459,11 +473,18 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_kernel(const MmaArgs a, co
                     const uint32_t a2 = byte_times_128_plus<1>(pe, cur), a3 = byte_times_128_plus<1>(po, cur);
                     const uint32_t a4 = byte_times_128_plus<2>(pe, cur), a5 = byte_times_128_plus<2>(po, cur);
                     const uint32_t a6 = byte_times_128_plus<3>(pe, cur), a7 = byte_times_128_plus<3>(po, cur);
-                    sts_u16(a0, v.x); sts_u16(a1, v.x >> 16);
-                    sts_u16(a2, v.y); sts_u16(a3, v.y >> 16);
-                    sts_u16(a4, v.z); sts_u16(a5, v.z >> 16);
-                    sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
-                    cur = a7;
+#ifdef SD2_CHECKED
+                    if (a0 < at || a7 >= at + (uint32_t)kMmaTileBytes) {
+                        if (a.err) atomicExch(a.err, 2);
+                    } else
+#endif
+                    {
+                        sts_u16(a0, v.x); sts_u16(a1, v.x >> 16);
+                        sts_u16(a2, v.y); sts_u16(a3, v.y >> 16);
+                        sts_u16(a4, v.z); sts_u16(a5, v.z >> 16);
+                        sts_u16(a6, v.w); sts_u16(a7, v.w >> 16);
+                        cur = a7;
+                    }
                 }
                 w += ((4u * nj + 15u) & ~15u) + 16u * nj;
             }

@@ -299,3 +299,17 @@ def test_bad_arguments():
     with pytest.raises(sd2.Sd2Error) as e:
         sd2.sd2_pack_host(W, mask, y_dtype=5)
     assert e.value.status == sd2.SD2_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("fmt", FORMATS + [sd2.SD2_FORMAT_GAP4_MMA])
+def test_a_failed_blob_allocation_is_reported_not_fatal(fmt):
+    W, mask = _case(4242, 40, 300, 0.5)
+    try:
+        sd2.sd2_debug_fail_allocations(0, 1)
+        with pytest.raises(sd2.Sd2Error) as e:
+            sd2.sd2_pack_host(W, mask, fmt)
+        assert e.value.status == sd2.SD2_ERR_ALLOC
+    finally:
+        sd2.sd2_debug_fail_allocations(0, 0)
+    dense, _ = sd2.sd2_unpack_host(sd2.sd2_pack_host(W, mask, fmt))      # and the next call works
+    assert np.array_equal(dense, oracle.roundtrip_ref(W, mask))

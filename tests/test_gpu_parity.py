@@ -627,3 +627,45 @@ def test_mma_handles_are_not_block_step_material():
     assert e.value.status == sd2.SD2_ERR_UNSUPPORTED
     for h in hs:
         sd2.sd2_free(h)
+
+
+def test_failed_allocations_are_reported_and_leak_nothing():
+    # every allocation on the way to a handle and to a drafter is made to fail in turn: the call says ALLOC,
+    # the device memory in use is what it was before, and the same call then succeeds
+    W, mask, X = case(9400, 300, 1024, 0.5, 2)
+    torch.cuda.synchronize()
+    sd2.sd2_free(sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA))      # device set-up is done before counting
+    free0 = torch.cuda.mem_get_info()[0]
+    for fmt, n_allocs in ((sd2.SD2_FORMAT_GAP4, 3), (sd2.SD2_FORMAT_GAP4_MMA, 4)):
+        for skip in range(n_allocs):
+            sd2.sd2_debug_fail_allocations(skip, 1)
+            try:
+                with pytest.raises(sd2.Sd2Error) as e:
+                    sd2.sd2_compress(W, mask, fmt)
+                assert e.value.status == sd2.SD2_ERR_ALLOC
+            finally:
+                sd2.sd2_debug_fail_allocations(0, 0)
+            assert torch.cuda.mem_get_info()[0] == free0
+    shape, blocks, d = _tiny_drafter(1, 2)
+    sd2.sd2_drafter_free(d)
+    free1 = torch.cuda.mem_get_info()[0]
+    failed = 0
+    for skip in range(12):
+        sd2.sd2_debug_fail_allocations(skip, 1)
+        try:
+            d = sd2.sd2_drafter_create(blocks, n_max=2)
+            sd2.sd2_drafter_free(d)                                      # the plan ran past the call's allocations
+        except sd2.Sd2Error as e:
+            assert e.status == sd2.SD2_ERR_ALLOC
+            failed += 1
+        finally:
+            sd2.sd2_debug_fail_allocations(0, 0)
+        assert torch.cuda.mem_get_info()[0] == free1
+    assert failed >= 4
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4, sd2.SD2_DTYPE_F32)
+    Yr, S = oracle.masked_linear(W, mask, X)
+    check(run_spmm(h, X, True), Yr, S, True)
+    sd2.sd2_free(h)
+    for hs in blocks:
+        for hh in hs:
+            sd2.sd2_free(hh)
