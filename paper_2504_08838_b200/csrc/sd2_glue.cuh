@@ -402,8 +402,9 @@ __global__ void __launch_bounds__(kGlueThreads) embedding_kernel(const int32_t* 
         x[(size_t)blockIdx.x * H + i] = (tok >= 0 && tok < V) ? table[(size_t)tok * H + i] : (uint16_t)0;
 }
 
-// logits[n, v] = sum_h W[v, h] x[n, h]: a warp per vocabulary row, 128-bit loads of the row, the
-// N <= 8 activation rows in shared memory as fp32.  H a multiple of 8.
+// logits[n, v] = sum_h W[v, h] x[n, h]: a warp takes kHeadRowsPerWarp vocabulary rows at a time (as many independent
+// 128-bit loads in flight per lane), the N <= 8 activation rows sit in shared memory as fp32.  H a multiple of 8.
+constexpr int kHeadRowsPerWarp = 4;
 __global__ void __launch_bounds__(kGlueThreads) lm_head_kernel(const uint16_t* x, const uint16_t* W, float* logits, int N, int V, int H)
 {
     extern __shared__ float xs[];            // [N][H]
@@ -411,7 +412,34 @@ __global__ void __launch_bounds__(kGlueThreads) lm_head_kernel(const uint16_t* x
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
-    for (int v = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; v < V; v += warps) {
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (N == 1) {
+        // the draft-token case: four rows per warp step
+        for (int v0 = gw * kHeadRowsPerWarp; v0 < V; v0 += warps * kHeadRowsPerWarp) {
+            float acc[kHeadRowsPerWarp] = {0.f, 0.f, 0.f, 0.f};
+            for (int c = lane; c < H / 8; c += 32) {
+                uint4 w4[kHeadRowsPerWarp];
+#pragma unroll
+                for (int r = 0; r < kHeadRowsPerWarp; ++r)
+                    w4[r] = v0 + r < V ? __ldg((const uint4*)(W + (size_t)(v0 + r) * H) + c) : make_uint4(0u, 0u, 0u, 0u);
+                const float* xr = xs + c * 8;
+#pragma unroll
+                for (int r = 0; r < kHeadRowsPerWarp; ++r) {
+                    const uint32_t ww[4] = {w4[r].x, w4[r].y, w4[r].z, w4[r].w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[r] += bf16_lo(ww[j]) * xr[2 * j] + bf16_hi(ww[j]) * xr[2 * j + 1];
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < kHeadRowsPerWarp; ++r) {
+                float s = acc[r];
+                for (int dd = 16; dd > 0; dd >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, dd);
+                if (lane == 0 && v0 + r < V) logits[v0 + r] = s;
+            }
+        }
+        return;
+    }
+    for (int v = gw; v < V; v += warps) {
         const uint4* wr = (const uint4*)(W + (size_t)v * H);
         float acc[kHeadMaxRows];
 #pragma unroll

@@ -256,3 +256,50 @@ def test_decoder_block_step_operation_by_operation(shape, Hq, Hkv, N, pos):
     assert np.array_equal(kc_after[:, keep], kc[:, keep]) and np.array_equal(vc_after[:, keep], vc[:, keep])
     for h in hs:
         sd2.sd2_free(h)
+
+
+def test_argument_checks_of_the_glue_calls():
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    x = torch.zeros((2, 64), **bf)
+    w = torch.zeros((64,), **bf)
+    L = sd2.lib()
+    # NULL pointers
+    assert L.sd2_rmsnorm(None, sd2._ptr(w), sd2._ptr(x), 2, 64, 1e-5, None) == sd2.SD2_ERR_INVALID_ARG
+    assert L.sd2_add(sd2._ptr(x), None, sd2._ptr(x), 128, None) == sd2.SD2_ERR_INVALID_ARG
+    # sizes
+    assert L.sd2_rmsnorm(sd2._ptr(x), sd2._ptr(w), sd2._ptr(x), 2, 0, 1e-5, None) == sd2.SD2_ERR_SHAPE
+    assert L.sd2_rmsnorm(sd2._ptr(x), sd2._ptr(w), sd2._ptr(x), 0, 64, 1e-5, None) == sd2.SD2_OK          # no rows: nothing to do
+    kc = torch.zeros((2, 8, 64), **bf)
+    q = torch.zeros((2, 128), **bf)
+    k = torch.zeros((2, 64), **bf)
+    out = torch.zeros((2, 128), **bf)
+    args = (sd2._ptr(q), sd2._ptr(k), sd2._ptr(k), sd2._ptr(kc), sd2._ptr(kc))
+    assert L.sd2_rope_cache(*args, 2, 4, 2, 32, 8, 8, 10000.0, None) == sd2.SD2_ERR_SHAPE                # pos == T_max
+    assert L.sd2_rope_cache(*args, 2, 4, 2, 31, 0, 8, 10000.0, None) == sd2.SD2_ERR_SHAPE                # odd head width
+    assert L.sd2_attention_decode(sd2._ptr(q), sd2._ptr(kc), sd2._ptr(kc), sd2._ptr(out), 2, 4, 3, 32, 1, 8, None) == sd2.SD2_ERR_SHAPE  # 4 % 3
+    assert L.sd2_attention_decode(sd2._ptr(q), sd2._ptr(kc), sd2._ptr(kc), sd2._ptr(out), 2, 4, 2, 32, 9, 8, None) == sd2.SD2_ERR_SHAPE  # T > T_max
+    assert L.sd2_attention_decode(sd2._ptr(q), sd2._ptr(kc), sd2._ptr(kc), sd2._ptr(out), 1, 1, 1, 256, 1, 8, None) == sd2.SD2_ERR_UNSUPPORTED
+    logits = torch.zeros((2, 10), dtype=torch.float32, device="cuda")
+    W = torch.zeros((10, 60), **bf)
+    xx = torch.zeros((2, 60), **bf)
+    assert L.sd2_lm_head(sd2._ptr(xx), sd2._ptr(W), sd2._ptr(logits), None, 2, 10, 60, None) == sd2.SD2_ERR_UNSUPPORTED   # H % 8
+    torch.cuda.synchronize()
+
+
+def test_decoder_block_step_rejects_inconsistent_heads():
+    shape = synth.DrafterShape("tiny", 256, 64, 1024, 1)
+    lin = synth.make_block(2, 0, shape, 0.5)
+    hs = [sd2.sd2_compress(W, m) for W, m in lin]
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    x = torch.zeros((1, 256), **bf)
+    w = torch.ones((256,), **bf)
+    kc = torch.zeros((1, 4, 64), **bf)
+    ws = torch.zeros(sd2.sd2_decoder_workspace_bytes(hs, 1) // 2, **bf)
+    with pytest.raises(sd2.Sd2Error) as e:          # 8 query heads of 32 against 4 key heads of 16
+        sd2.sd2_decoder_block_step(hs, w, w, x, x.clone(), kc, kc.clone(), 8, 4, 0, EPS, THETA, ws)
+    assert e.value.status == sd2.SD2_ERR_SHAPE
+    with pytest.raises(sd2.Sd2Error) as e:          # the cache has 4 positions
+        sd2.sd2_decoder_block_step(hs, w, w, x, x.clone(), kc, kc.clone(), 8, 2, 4, EPS, THETA, ws)
+    assert e.value.status == sd2.SD2_ERR_SHAPE
+    for h in hs:
+        sd2.sd2_free(h)

@@ -669,3 +669,23 @@ def test_failed_allocations_are_reported_and_leak_nothing():
     for hs in blocks:
         for hh in hs:
             sd2.sd2_free(hh)
+
+
+def test_mma_handles_edge_calls():
+    W, mask, X = case(9500, 130, 264, 0.5, 4)
+    h = sd2.sd2_compress(W, mask, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32)
+    Y = torch.full((4, 130), 7.0, dtype=torch.float32, device="cuda")
+    L = sd2.lib()
+    assert L.sd2_spmm(h.raw, sd2._ptr(dev_bf16(X)), sd2._ptr(Y), 0, None) == sd2.SD2_OK          # no rows: Y untouched
+    torch.cuda.synchronize()
+    assert bool((Y == 7.0).all())
+    assert L.sd2_spmm(h.raw, sd2._ptr(dev_bf16(X)), sd2._ptr(Y), -1, None) == sd2.SD2_ERR_SHAPE
+    assert L.sd2_spmm(h.raw, None, sd2._ptr(Y), 4, None) == sd2.SD2_ERR_INVALID_ARG
+    # an all-zero mask and a full mask
+    for m in (np.zeros_like(mask), np.ones_like(mask)):
+        hh = sd2.sd2_compress(W, m, sd2.SD2_FORMAT_GAP4_MMA, sd2.SD2_DTYPE_F32)
+        Yr, S = oracle.masked_linear(W, m, X)
+        y = run_spmm(hh, X, True)
+        check(y, Yr, S, True)
+        sd2.sd2_free(hh)
+    sd2.sd2_free(h)
