@@ -364,11 +364,12 @@ def time_full_step(torch, sd2, args, shape, handles, harr, N, stream):
         handles[0], gains[0], gains[1], xs[0], xs[1], kcs[0], vcs[0], heads_q, heads_kv, args.context, 1e-5, 500000.0, ws,
         handle_array=harr[0]), 50, stream)
     head_bytes = 2.0 * vocab * hid
-    return {"us_per_token": us, "launches_per_step": 8 * blocks + 4, "context": args.context, "vocab": vocab,
+    return {"us_per_token": us, "launches_per_step": 4 * blocks + 4, "context": args.context, "vocab": vocab,
             "heads": [heads_q, heads_kv, d], "lm_head_bytes": head_bytes, "lm_head_us": us_head,
             "lm_head_gbs": head_bytes / us_head / 1e3, "block0_alone_us_l2_warm": us_block,
-            "note": "one launch per group of linears that share an input (4 per block) and per glue operation (4 per block); "
-                    "the linears here are single-stage launches, not the one-launch drafter step timed above"}
+            "note": "four launches per block: q|k|v with the first norm folded into their staging pass; rotation + cache append + "
+                    "attention; o, gate|up and down as one persistent launch (grid barriers between the stages, residual and "
+                    "second norm folded into gate|up's staging pass); the last residual"}
 
 
 def run_ours(args):

@@ -294,8 +294,10 @@ sd2_status sd2_lm_head(const void* x, const void* w_out, float* logits, int32_t*
 /* One whole decoder block for one new token per row:
  *     x1 = x  + Wo attention(rope(Wq n), cache + rope(Wk n), cache + Wv n),   n = rmsnorm(x,  norm_attn)
  *     y  = x1 + Wd (silu(Wg m) * Wu m),                                        m = rmsnorm(x1, norm_ffn)
- * h[7] = q, k, v, o, gate, up, down handles (GAP4 or BITMASK; one launch per group of linears that share
- * an input); every intermediate is rounded to bf16.  x, y [N*hidden]; caches as in sd2_rope_cache; the
+ * h[7] = q, k, v, o, gate, up, down handles.  With seven GAP4 handles the block is four launches: q|k|v with
+ * the first norm folded into their activation staging; rotation, cache append and attention; o, gate|up and
+ * down as one persistent launch with the residual and the second norm folded into gate|up's staging; the last
+ * residual.  Other formats take one launch per operation (8 per block).  Every intermediate is rounded to bf16.  x, y [N*hidden]; caches as in sd2_rope_cache; the
  * block writes position `pos` of them and attends over positions 0..pos.  workspace: device, 256-byte
  * aligned, sd2_decoder_workspace_bytes(h, N) bytes; it holds, in this order, q, k, v, o-projection,
  * gate, up, t (offsets of sd2_block_workspace_layout), then n/m, x1, the attention output and the down

@@ -699,6 +699,26 @@ struct BlockTags {
     uint32_t* t_t;                               // tagged t = silu(g) * u, one slice per CTA
 };
 
+// Appends one group of linears that share an input to `stages` (plain hand-off): one stage if they share a strip
+// geometry, else a stage each.  Returns the new stage count.
+int append_group(SStage* stages, int n, ProgramNeeds* needs, const sd2_handle* hs, int count, const uint16_t* xin,
+                 const uint16_t* gg, const uint16_t* uu, uint16_t* tt, void* const* Y, bool force_bf16, int grid)
+{
+    bool same = true;
+    for (int i = 1; i < count; ++i)
+        if (hs[i]->S != hs[0]->S) same = false;
+    if (same) {
+        fill_stage(stages[n++], hs, count, xin, gg, uu, tt, Y, force_bf16, grid);
+        needs->add(hs, count);
+    } else {
+        for (int i = 0; i < count; ++i) {
+            fill_stage(stages[n++], hs + i, 1, xin, gg, uu, i == 0 ? tt : nullptr, Y + i, force_bf16, grid);
+            needs->add(hs + i, 1);
+        }
+    }
+    return n;
+}
+
 // Appends the stages of one block (h[0..6] = q,k,v,o,gate,up,down) to `stages`.  Weights of a
 // group that do not share a strip geometry get a stage each.  Returns the number appended.
 int append_block_stages(SStage* stages, const sd2_handle* h, const uint16_t* x, uint16_t* q, uint16_t* k, uint16_t* v,
@@ -1148,6 +1168,57 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
     uint16_t* att = (uint16_t*)(ws + o); o += a256(2 * N * d.q_out);
     uint16_t* dn = (uint16_t*)(ws + o);
     cudaStream_t s = (cudaStream_t)cuda_stream;
+    bool all_gap4 = true;
+    for (int i = 0; i < 7; ++i)
+        if (h[i]->format != SD2_FORMAT_GAP4) all_gap4 = false;
+    if (all_gap4) {
+        // Four launches: (1) q|k|v with the first norm folded into their staging pass, (2) rotation + cache append +
+        // attention, (3) one persistent launch for o, gate|up and down, the residual and the second norm folded into
+        // the staging pass of gate|up (CTA 0 stores x1 and the normalised row for whoever wants to look), (4) the
+        // last residual.
+        int dev = 0;
+        if ((st = ensure_device(&dev)) != SD2_OK) return st;
+        for (int i = 0; i < 7; ++i)
+            if (h[i]->device != dev) return SD2_ERR_INVALID_ARG;
+        const int grid = g_dev[dev].sms;
+        {
+            SArgs a;
+            std::memset(&a, 0, sizeof a);
+            ProgramNeeds needs;
+            void* yqkv[3] = {q, k, v};
+            a.n_stages = append_group(a.inl, 0, &needs, h, 3, (const uint16_t*)x, nullptr, nullptr, nullptr, yqkv, true, grid);
+            for (int i = 0; i < a.n_stages; ++i) {
+                a.inl[i].norm_w = (const uint16_t*)norm_attn;
+                a.inl[i].eps = eps;
+            }
+            Range r_("q|k|v");
+            if ((st = run_program(a, dev, N, needs, s)) != SD2_OK) return st;
+        }
+        if ((st = sd2_rope_attention(q, k, v, k_cache, v_cache, att, N, heads_q, heads_kv, hd, pos, T_max, theta, s)) != SD2_OK) return st;
+        {
+            SArgs a;
+            std::memset(&a, 0, sizeof a);
+            ProgramNeeds needs;
+            void* yo[1] = {hdn};
+            void* ygu[2] = {g, u};
+            void* yd[1] = {dn};
+            int n = append_group(a.inl, 0, &needs, h + 3, 1, att, nullptr, nullptr, nullptr, yo, true, grid);
+            const int first_gu = n;
+            n = append_group(a.inl, n, &needs, h + 4, 2, hdn, nullptr, nullptr, nullptr, ygu, true, grid);
+            for (int i = first_gu; i < n; ++i) {
+                a.inl[i].res = (const uint16_t*)x;
+                a.inl[i].norm_w = (const uint16_t*)norm_ffn;
+                a.inl[i].eps = eps;
+                a.inl[i].sum_out = x1;
+                a.inl[i].norm_out = xn;
+            }
+            n = append_group(a.inl, n, &needs, h + 6, 1, nullptr, g, u, t, yd, true, grid);
+            a.n_stages = n;
+            Range r_("o, gate|up, down");
+            if ((st = run_program(a, dev, N, needs, s)) != SD2_OK) return st;
+        }
+        return sd2_add(x1, dn, y, N * d.hidden, s);
+    }
     // attention module: x1 = x + Wo attention(rope(Wq n), cache + rope(Wk n), cache + Wv n), n = rmsnorm(x)
     if ((st = sd2_rmsnorm(x, norm_attn, xn, N, d.hidden, eps, s)) != SD2_OK) return st;
     void* yqkv[3] = {q, k, v};

@@ -136,6 +136,16 @@ struct SStage {
     int paired;            // mat[0] stacks gate row i (row 2i) and up row i (row 2i+1), pairs share a tile:
                            // the stage stores g, u, t_out (plain bf16, each may be NULL) and tt (tagged t)
     int reserved[2];
+    // Decoder glue folded into the staging pass (all NULL / 0 for a plain linear).  With norm_w set, every CTA turns
+    // the activation row it has just fetched into  rmsnorm(row [+ res]) * norm_w  before scattering it into the
+    // lane windows: the residual connection and the norm in front of a block's linears cost no launch and no
+    // hand-off of their own.  CTA 0 also stores the bf16 sum (sum_out) and the normalised row (norm_out).
+    const uint16_t* res;       // [N * K] added to the row first (rounded to bf16), or NULL
+    const uint16_t* norm_w;    // [K] gains of the norm, or NULL: no norm
+    uint16_t* sum_out;         // [N * K] or NULL
+    uint16_t* norm_out;        // [N * K] or NULL
+    float eps;
+    int reserved2[3];
 };
 static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
@@ -315,6 +325,7 @@ struct StreamShared {
     int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
     unsigned int tag_base[8];          // tagged programs: (production count of activation row n0 + n & 0xFF) << 8
     unsigned int next_q;               // next tile (sequence number) no consumer warp has taken yet
+    float red[2][kConsumerWarps];      // per-warp partial sums of squares of the rows being normalised
 };
 
 struct WaitCtx {
@@ -539,7 +550,8 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
 template <int NT>
 __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
                                         const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int xlin_row, int ctid,
-                                        uint32_t tag, const unsigned int* tagb, const WaitCtx& wc)
+                                        uint32_t tag, const unsigned int* tagb, const WaitCtx& wc, int row0 = 0,
+                                        float (*red)[kConsumerWarps] = nullptr)
 {
     constexpr int W = xs_words(NT);
     constexpr int kGroups = 32 / W;
@@ -594,6 +606,48 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                         if (pub) t_out[(size_t)n * K + i] = v;
                     }
                     xl[i] = v;
+                }
+            }
+        }
+        if (st.norm_w && red) {
+            // residual and norm on the linear row(s), each thread on the elements it revisits in the second loop
+            named_bar_sync(1, kConsumerThreads);
+            const bool pubn = blockIdx.x == 0;
+#pragma unroll
+            for (int r = 0; r < kRowsPerPass; ++r) {
+                const int n = n0 + r;
+                if (n >= N) continue;
+                uint16_t* xl = xlin + (size_t)r * xlin_row + st.V;
+                const size_t go = (size_t)(row0 + n) * K;
+                float ss = 0.f;
+                for (int i = ctid; i < K; i += kConsumerThreads) {
+                    float v = bf16_to_f32(xl[i]);
+                    if (st.res) {
+                        const uint16_t sb = f32_to_bf16_rne(v + bf16_to_f32(__ldcg(st.res + go + i)));
+                        xl[i] = sb;
+                        if (pubn && st.sum_out) st.sum_out[go + i] = sb;
+                        v = bf16_to_f32(sb);
+                    }
+                    ss += v * v;
+                }
+                for (int dd = 16; dd > 0; dd >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, dd);
+                if ((ctid & 31) == 0) red[r][ctid >> 5] = ss;
+            }
+            named_bar_sync(1, kConsumerThreads);
+#pragma unroll
+            for (int r = 0; r < kRowsPerPass; ++r) {
+                const int n = n0 + r;
+                if (n >= N) continue;
+                uint16_t* xl = xlin + (size_t)r * xlin_row + st.V;
+                const size_t go = (size_t)(row0 + n) * K;
+                float tot = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) tot += red[r][w];
+                const float rs = rsqrtf(tot / (float)K + st.eps);
+                for (int i = ctid; i < K; i += kConsumerThreads) {
+                    const uint16_t o = f32_to_bf16_rne(bf16_to_f32(xl[i]) * rs * bf16_to_f32(__ldg(st.norm_w + i)));
+                    xl[i] = o;
+                    if (pubn && st.norm_out) st.norm_out[go + i] = o;
                 }
             }
         }
@@ -888,7 +942,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
             stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         } else {
             stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
-                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
+                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc, a.n0, sh->red);
         }
         if (warp == 1 && s + 1 < a.n_stages) {
             const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);

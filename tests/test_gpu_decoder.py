@@ -189,10 +189,13 @@ def _block(shape, Hq, Hkv, N, pos, fmt):
     return d, lin, hs, wn1, wn2, x, T_max, kc, vc
 
 
-@pytest.mark.parametrize("shape,Hq,Hkv,N,pos", [(synth.DrafterShape("tiny", 256, 64, 1024, 1), 8, 2, 3, 9),
-                                                 (synth.LLAMA_1B, 32, 8, 1, 40)])
-def test_decoder_block_step_operation_by_operation(shape, Hq, Hkv, N, pos):
-    d, lin, hs, wn1, wn2, x, T_max, kc, vc = _block(shape, Hq, Hkv, N, pos, sd2.SD2_FORMAT_AUTO)
+@pytest.mark.parametrize("shape,Hq,Hkv,N,pos,fmt", [
+    (synth.DrafterShape("tiny", 256, 64, 1024, 1), 8, 2, 3, 9, sd2.SD2_FORMAT_AUTO),
+    (synth.DrafterShape("tiny", 256, 64, 1024, 1), 8, 2, 11, 0, sd2.SD2_FORMAT_AUTO),       # two panels of rows, an empty cache
+    (synth.DrafterShape("tiny", 256, 64, 1024, 1), 8, 2, 2, 5, sd2.SD2_FORMAT_BITMASK),     # the launch-per-operation path
+    (synth.LLAMA_1B, 32, 8, 1, 40, sd2.SD2_FORMAT_AUTO)])
+def test_decoder_block_step_operation_by_operation(shape, Hq, Hkv, N, pos, fmt):
+    d, lin, hs, wn1, wn2, x, T_max, kc, vc = _block(shape, Hq, Hkv, N, pos, fmt)
     kcd, vcd = dev(kc), dev(vc)
     ws = torch.full((sd2.sd2_decoder_workspace_bytes(hs, N) // 2,), float("nan"), dtype=torch.bfloat16, device="cuda")
     y = torch.full((N, shape.hidden), float("nan"), dtype=torch.bfloat16, device="cuda")
