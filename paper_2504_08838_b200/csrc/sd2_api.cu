@@ -123,10 +123,14 @@ sd2_status from_pack(int s)
     }
 }
 
+constexpr int kFoldStaticBytes = 256;   // static shared memory of the kernel instances that fold a norm into staging
+
 template <int NT>
 cudaError_t set_smem_attr()
 {
-    return cudaFuncSetAttribute(stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    cudaError_t e = cudaFuncSetAttribute(stream_kernel<NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(stream_kernel<NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax - kFoldStaticBytes);
 }
 
 // Once per device: SM count, shared-memory opt-in, the error word and the barrier pool.
@@ -374,13 +378,15 @@ sd2_status launch_stream_nt(const SArgs& a, int grid, int smem, bool cooperative
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = cooperative ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, stream_kernel<NT>, a) != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
+    const cudaError_t e = a.fold_any ? cudaLaunchKernelEx(&cfg, stream_kernel<NT, true>, a) : cudaLaunchKernelEx(&cfg, stream_kernel<NT, false>, a);
+    if (e != cudaSuccess) { cudaGetLastError(); return SD2_ERR_CUDA; }
     if (cudaGetLastError() != cudaSuccess) return SD2_ERR_CUDA;
     return SD2_OK;
 }
 
-sd2_status launch_stream(int nt, const SArgs& a, int grid, bool cooperative, cudaStream_t s)
+sd2_status launch_stream(int nt, SArgs& a, int grid, bool cooperative, cudaStream_t s)
 {
+    if (a.fold_any) a.ring_bytes -= kFoldStaticBytes;   // those instances keep a little static shared memory (the ring still holds two tiles)
     const int smem = a.xs_bytes + a.xlin_bytes + (int)((sizeof(StreamShared) + 127) & ~127) + a.ring_bytes;
     switch (nt) {
         case 1: return launch_stream_nt<1>(a, grid, smem, cooperative, s);
@@ -1188,9 +1194,10 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
             void* yqkv[3] = {q, k, v};
             a.n_stages = append_group(a.inl, 0, &needs, h, 3, (const uint16_t*)x, nullptr, nullptr, nullptr, yqkv, true, grid);
             for (int i = 0; i < a.n_stages; ++i) {
-                a.inl[i].norm_w = (const uint16_t*)norm_attn;
-                a.inl[i].eps = eps;
+                a.fold[i].norm_w = (const uint16_t*)norm_attn;
+                a.fold[i].eps = eps;
             }
+            a.fold_any = 1;
             Range r_("q|k|v");
             if ((st = run_program(a, dev, N, needs, s)) != SD2_OK) return st;
         }
@@ -1206,12 +1213,13 @@ sd2_status sd2_decoder_block_step(const sd2_handle* h, const void* norm_attn, co
             const int first_gu = n;
             n = append_group(a.inl, n, &needs, h + 4, 2, hdn, nullptr, nullptr, nullptr, ygu, true, grid);
             for (int i = first_gu; i < n; ++i) {
-                a.inl[i].res = (const uint16_t*)x;
-                a.inl[i].norm_w = (const uint16_t*)norm_ffn;
-                a.inl[i].eps = eps;
-                a.inl[i].sum_out = x1;
-                a.inl[i].norm_out = xn;
+                a.fold[i].res = (const uint16_t*)x;
+                a.fold[i].norm_w = (const uint16_t*)norm_ffn;
+                a.fold[i].eps = eps;
+                a.fold[i].sum_out = x1;
+                a.fold[i].norm_out = xn;
             }
+            a.fold_any = 1;
             n = append_group(a.inl, n, &needs, h + 6, 1, nullptr, g, u, t, yd, true, grid);
             a.n_stages = n;
             Range r_("o, gate|up, down");

@@ -136,18 +136,23 @@ struct SStage {
     int paired;            // mat[0] stacks gate row i (row 2i) and up row i (row 2i+1), pairs share a tile:
                            // the stage stores g, u, t_out (plain bf16, each may be NULL) and tt (tagged t)
     int reserved[2];
-    // Decoder glue folded into the staging pass (all NULL / 0 for a plain linear).  With norm_w set, every CTA turns
-    // the activation row it has just fetched into  rmsnorm(row [+ res]) * norm_w  before scattering it into the
-    // lane windows: the residual connection and the norm in front of a block's linears cost no launch and no
-    // hand-off of their own.  CTA 0 also stores the bf16 sum (sum_out) and the normalised row (norm_out).
+};
+static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
+
+// Decoder glue folded into a stage's staging pass (kernel instances with FOLD only; all NULL / 0: a plain linear).
+// With norm_w set, every CTA turns the activation row it has just fetched into  rmsnorm(row [+ res]) * norm_w
+// before scattering it into the lane windows: the residual connection and the norm in front of a block's linears
+// cost no launch and no hand-off of their own.  CTA 0 also stores the bf16 sum (sum_out) and the normalised row
+// (norm_out).  Kept out of SStage and out of the plain kernel instances: the drafter step's time is sensitive to
+// the size of the stage descriptors and of the CTA's bookkeeping (1.3 % when these fields sat in SStage).
+struct SFold {
     const uint16_t* res;       // [N * K] added to the row first (rounded to bf16), or NULL
     const uint16_t* norm_w;    // [K] gains of the norm, or NULL: no norm
     uint16_t* sum_out;         // [N * K] or NULL
     uint16_t* norm_out;        // [N * K] or NULL
     float eps;
-    int reserved2[3];
+    int reserved;
 };
-static_assert(sizeof(SStage) % 16 == 0, "stage descriptors are copied in 16-byte pieces");
 
 struct SArgs {
     SStage inl[kMaxStagesInline];   // used when ext == NULL
@@ -169,6 +174,8 @@ struct SArgs {
     int free_tiles;                 // 1: a consumer warp that is done draws the next tile from a shared counter;
                                     // 0: tile k of a stage goes to warp k % 16 (see the consumer loop)
     long long* reserved_ptr;
+    SFold fold[kMaxStagesInline];   // per inline stage; read by FOLD instances only
+    int fold_any;                   // host side: launch the FOLD instance
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -325,7 +332,6 @@ struct StreamShared {
     int stage_dead;                    // thread 0 only: copy of abort_flag taken before a barrier
     unsigned int tag_base[8];          // tagged programs: (production count of activation row n0 + n & 0xFF) << 8
     unsigned int next_q;               // next tile (sequence number) no consumer warp has taken yet
-    float red[2][kConsumerWarps];      // per-warp partial sums of squares of the rows being normalised
 };
 
 struct WaitCtx {
@@ -547,11 +553,11 @@ __device__ __forceinline__ void publish_t_slice(int K, int N, const uint32_t* g,
 // buffer (xlin holds two, `xlin_row` elements apart), then one scatter writes the packed words.
 // (Panels of two keep one buffer and take a pass per row: the second buffer would come out of the
 // weight ring, which costs them more than the extra pass.)
-template <int NT>
+template <int NT, bool FOLD = false>
 __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t* x_src, const uint16_t* g,
                                         const uint16_t* u, uint16_t* t_out, float* xs, uint16_t* xlin, int xlin_row, int ctid,
                                         uint32_t tag, const unsigned int* tagb, const WaitCtx& wc, int row0 = 0,
-                                        float (*red)[kConsumerWarps] = nullptr)
+                                        float (*red)[kConsumerWarps] = nullptr, const SFold* fold = nullptr)
 {
     constexpr int W = xs_words(NT);
     constexpr int kGroups = 32 / W;
@@ -609,7 +615,8 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                 }
             }
         }
-        if (st.norm_w && red) {
+        if (FOLD && fold && fold->norm_w) {
+            const SFold& f = *fold;
             // residual and norm on the linear row(s), each thread on the elements it revisits in the second loop
             named_bar_sync(1, kConsumerThreads);
             const bool pubn = blockIdx.x == 0;
@@ -622,10 +629,10 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                 float ss = 0.f;
                 for (int i = ctid; i < K; i += kConsumerThreads) {
                     float v = bf16_to_f32(xl[i]);
-                    if (st.res) {
-                        const uint16_t sb = f32_to_bf16_rne(v + bf16_to_f32(__ldcg(st.res + go + i)));
+                    if (f.res) {
+                        const uint16_t sb = f32_to_bf16_rne(v + bf16_to_f32(__ldcg(f.res + go + i)));
                         xl[i] = sb;
-                        if (pubn && st.sum_out) st.sum_out[go + i] = sb;
+                        if (pubn && f.sum_out) f.sum_out[go + i] = sb;
                         v = bf16_to_f32(sb);
                     }
                     ss += v * v;
@@ -643,11 +650,11 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
                 float tot = 0.f;
 #pragma unroll
                 for (int w = 0; w < kConsumerWarps; ++w) tot += red[r][w];
-                const float rs = rsqrtf(tot / (float)K + st.eps);
+                const float rs = rsqrtf(tot / (float)K + f.eps);
                 for (int i = ctid; i < K; i += kConsumerThreads) {
-                    const uint16_t o = f32_to_bf16_rne(bf16_to_f32(xl[i]) * rs * bf16_to_f32(__ldg(st.norm_w + i)));
+                    const uint16_t o = f32_to_bf16_rne(bf16_to_f32(xl[i]) * rs * bf16_to_f32(__ldg(f.norm_w + i)));
                     xl[i] = o;
-                    if (pubn && st.norm_out) st.norm_out[go + i] = o;
+                    if (pubn && f.norm_out) f.norm_out[go + i] = o;
                 }
             }
         }
@@ -697,7 +704,7 @@ __device__ __forceinline__ void stage_x(const SStage& st, int N, const uint16_t*
     }
 }
 
-template <int NT>
+template <int NT, bool FOLD = false>
 __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_constant__ SArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -941,8 +948,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) stream_kernel(const __grid_
         } else if (st.paired) {   // g, u, t_out are this stage's outputs
             stage_x<NT>(st, N, x_src + xw, nullptr, nullptr, nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
         } else {
-            stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
-                        st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc, a.n0, sh->red);
+            if constexpr (FOLD) {
+                __shared__ float fold_red[2][kConsumerWarps];   // per-warp partial sums of squares of the rows being normalised
+                stage_x<NT, true>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
+                                  st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc, a.n0, fold_red,
+                                  (!a.ext && s < kMaxStagesInline) ? &a.fold[s] : nullptr);
+            } else {
+                stage_x<NT>(st, N, x_src ? x_src + xw : nullptr, st.g ? st.g + xw : nullptr, st.u ? st.u + xw : nullptr,
+                            st.t_out ? st.t_out + xoff : nullptr, xs, xlin, xlin_row, ctid, tag_in, tagb, wc);
+            }
         }
         if (warp == 1 && s + 1 < a.n_stages) {
             const uint32_t* src = (const uint32_t*)(a.ext ? a.ext + (s + 1) : &a.inl[s + 1]);
