@@ -67,8 +67,9 @@ def parse_args():
     ap.add_argument("--blocks", type=int, default=0, help="override the block count (0 = the drafter's)")
     ap.add_argument("--no-dense", action="store_true", help="skip the cuBLAS dense comparison")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle")
-    ap.add_argument("--full-step", action="store_true",
-                    help="also time the whole decode step (glue + dense LM head around the sparse linears)")
+    ap.add_argument("--no-full-step", dest="full_step", action="store_false",
+                    help="skip the timing of the whole decode step (glue + dense LM head around the sparse linears)")
+    ap.add_argument("--full-step", dest="full_step", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--context", type=int, default=300, help="--full-step: cached positions the new token attends over")
     args = ap.parse_args()
     if args.mask == "2:4":
@@ -505,7 +506,7 @@ def run_ours(args):
         # ---- the whole decode step: embedding, L decoder blocks (norms, rotary embedding, attention over a cache
         # of --context positions, residuals around the same sparse linears), final norm, dense LM head, greedy token
         full_step = None
-        if args.full_step and N <= 8:
+        if args.full_step and N <= 8 and rank == 0:
             full_step = time_full_step(torch, sd2, args, shape, handles, harr, N, stream)
 
         # ---- cuBLAS dense bf16 on the same masked weights, same chaining, same graph treatment.

@@ -262,7 +262,8 @@ sd2_status sd2_add_rmsnorm(const void* a, const void* b, void* sum, const void* 
 /* Rotary embedding of one new token per row at position `pos` (pairs (i, i + head_dim/2) of a head
  * turn by pos * theta^(-2i/head_dim)), and the cache append: q [N, heads_q, head_dim] is rotated in
  * place; the rotated k and the plain v ([N, heads_kv, head_dim]) are written to position `pos` of
- * row n's cache, k_cache / v_cache [N, T_max, heads_kv, head_dim].  head_dim even, pos < T_max. */
+ * row n's cache, k_cache / v_cache [N, T_max, heads_kv, head_dim].  head_dim even, pos < T_max.
+ * UNSUPPORTED: head_dim > 128.  The angles are computed on the host (fp64) at the call. */
 sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, void* v_cache, int64_t N, int64_t heads_q,
                           int64_t heads_kv, int64_t head_dim, int64_t pos, int64_t T_max, double theta, void* cuda_stream);
 

@@ -5,6 +5,7 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include <atomic>
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -1018,6 +1019,20 @@ sd2_status sd2_rmsnorm(const void* x, const void* w, void* y, int64_t N, int64_t
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
+namespace {
+RopeTable rope_table(int64_t head_dim, int64_t pos, double theta)
+{
+    RopeTable t;
+    std::memset(&t, 0, sizeof t);
+    for (int64_t i = 0; i < head_dim / 2 && i < kRopeMaxHalf; ++i) {
+        const double ang = (double)pos * std::pow(theta, -2.0 * (double)i / (double)head_dim);
+        t.c[i] = (float)std::cos(ang);
+        t.s[i] = (float)std::sin(ang);
+    }
+    return t;
+}
+}  // namespace
+
 sd2_status sd2_add_rmsnorm(const void* a, const void* b, void* sum, const void* w, void* y, int64_t N, int64_t H, float eps,
                            void* cuda_stream)
 {
@@ -1038,9 +1053,11 @@ sd2_status sd2_rope_cache(void* q, const void* k, const void* v, void* k_cache, 
         heads_q > 65536 || heads_kv > 65536 || head_dim > 8192 || N > 0x7FFFFFFF || !(theta > 0.0))
         return SD2_ERR_SHAPE;
     if (N == 0) return SD2_OK;
-    rope_cache_kernel<<<(unsigned)N, kGlueThreads, (size_t)head_dim * 4, (cudaStream_t)cuda_stream>>>((uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v,
+    if (head_dim > 2 * kRopeMaxHalf) return SD2_ERR_UNSUPPORTED;
+    rope_cache_kernel<<<(unsigned)N, kGlueThreads, 0, (cudaStream_t)cuda_stream>>>((uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v,
                                                                                     (uint16_t*)k_cache, (uint16_t*)v_cache, (int)heads_q,
-                                                                                    (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, theta);
+                                                                                    (int)heads_kv, (int)head_dim, (int)pos, (int)T_max,
+                                                                                    rope_table(head_dim, pos, theta));
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 
@@ -1077,7 +1094,7 @@ sd2_status sd2_rope_attention(void* q, const void* k, const void* v, void* k_cac
     const int vec = (pow2 && head_dim >= 8 && ((((uintptr_t)k_cache) | ((uintptr_t)v_cache)) & 15) == 0) ? 1 : 0;
     rope_attention_kernel<<<(unsigned)(N * heads_q), kAttnThreads, (size_t)(pos + 1) * 4, (cudaStream_t)cuda_stream>>>(
         (uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, (uint16_t*)k_cache, (uint16_t*)v_cache, (uint16_t*)out, (int)heads_q,
-        (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, theta, vec);
+        (int)heads_kv, (int)head_dim, (int)pos, (int)T_max, rope_table(head_dim, pos, theta), vec);
     return cudaGetLastError() == cudaSuccess ? SD2_OK : SD2_ERR_CUDA;
 }
 

@@ -21,6 +21,14 @@ constexpr int kGlueThreads = 256;
 constexpr int kAttnThreads = 256;
 constexpr int kAttnMaxT = 8192;            // cached positions whose scores fit the kernel's shared memory
 constexpr int kHeadMaxRows = 8;            // activation rows one LM-head launch keeps in shared memory
+constexpr int kRopeMaxHalf = 64;           // head widths up to 128
+
+// cos and sin of the head_dim / 2 rotary angles of one position, computed on the host in fp64 (pos * theta^(-2i/d))
+// and handed to the kernels by value: no double-precision transcendental on the device
+struct RopeTable {
+    float c[kRopeMaxHalf];
+    float s[kRopeMaxHalf];
+};
 
 __device__ __forceinline__ float block_sum(float v, float* red)
 {
@@ -107,24 +115,17 @@ __global__ void __launch_bounds__(kGlueThreads) add_rmsnorm_kernel(const uint16_
 // Rotates q in place and writes the rotated k and the plain v of row n into position `pos` of row n's cache.
 // Caches are [N, T_max, Hkv * d].  One CTA per row.
 __global__ void __launch_bounds__(kGlueThreads) rope_cache_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
-                                                                 uint16_t* vc, int Hq, int Hkv, int d, int pos, int T_max, double theta)
+                                                                 uint16_t* vc, int Hq, int Hkv, int d, int pos, int T_max,
+                                                                 const RopeTable tab)
 {
-    extern __shared__ float cs_tab[];        // cos and sin of the d / 2 angles of this position
     const int n = blockIdx.x, half = d / 2;
-    for (int i = threadIdx.x; i < half; i += blockDim.x) {
-        double sn, cs;
-        sincos((double)pos * pow(theta, -2.0 * (double)i / (double)d), &sn, &cs);
-        cs_tab[i] = (float)cs;
-        cs_tab[half + i] = (float)sn;
-    }
-    __syncthreads();
     uint16_t* qr = q + (size_t)n * Hq * d;
     const uint16_t* kr = k + (size_t)n * Hkv * d;
     uint16_t* kdst = kc + ((size_t)n * T_max + pos) * Hkv * d;
     uint16_t* vdst = vc + ((size_t)n * T_max + pos) * Hkv * d;
     for (int p = threadIdx.x; p < (Hq + Hkv) * half; p += blockDim.x) {
         const int h = p / half, i = p % half;
-        const float c = cs_tab[i], s = cs_tab[half + i];
+        const float c = tab.c[i], s = tab.s[i];
         if (h < Hq) {
             const float a = bf16_to_f32(qr[h * d + i]), b = bf16_to_f32(qr[h * d + i + half]);
             qr[h * d + i] = f32_to_bf16_rne(a * c - b * s);
@@ -250,22 +251,15 @@ __global__ void __launch_bounds__(kAttnThreads) attention_decode_kernel(const ui
 // first head of every group also appends the rotated key and the value to the caches.  No CTA reads what another writes.
 __global__ void __launch_bounds__(kAttnThreads) rope_attention_kernel(uint16_t* q, const uint16_t* k, const uint16_t* v, uint16_t* kc,
                                                                      uint16_t* vc, uint16_t* out, int Hq, int Hkv, int d, int pos,
-                                                                     int T_max, double theta, int vec)
+                                                                     int T_max, const RopeTable tab, int vec)
 {
     extern __shared__ float sc[];            // pos + 1 scores, then the weights
     __shared__ float red[32];
-    __shared__ float qs[128], ks[128], cs_tab[128];
+    __shared__ float qs[128], ks[128];
     __shared__ float part[(kAttnThreads / 32) * 128];
     const int n = blockIdx.x / Hq, h = blockIdx.x % Hq, group = Hq / Hkv, g = h / group;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     const int half = d / 2, T = pos;         // cached positions; the new token is handled apart
-    if (threadIdx.x < half) {
-        double sn, cs;
-        sincos((double)pos * pow(theta, -2.0 * (double)threadIdx.x / (double)d), &sn, &cs);
-        cs_tab[threadIdx.x] = (float)cs;
-        cs_tab[half + threadIdx.x] = (float)sn;
-    }
-    __syncthreads();
     uint16_t* qr = q + ((size_t)n * Hq + h) * d;
     const uint16_t* kr = k + ((size_t)n * Hkv + g) * d;
     const size_t pitch = (size_t)Hkv * d;
@@ -275,7 +269,7 @@ __global__ void __launch_bounds__(kAttnThreads) rope_attention_kernel(uint16_t* 
     const bool writer = (h % group) == 0;
     if (threadIdx.x < half) {
         const int i = threadIdx.x;
-        const float c = cs_tab[i], sn = cs_tab[half + i];
+        const float c = tab.c[i], sn = tab.s[i];
         const float a = bf16_to_f32(qr[i]), b = bf16_to_f32(qr[i + half]);
         const uint16_t q0 = f32_to_bf16_rne(a * c - b * sn), q1 = f32_to_bf16_rne(b * c + a * sn);
         qr[i] = q0;
