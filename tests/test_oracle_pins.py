@@ -298,3 +298,22 @@ def test_printed_mal_identities():
     assert abs(g["mal_llama3b_sd2_50"] / g["mal_llama3b_layer_pruned_50"] - g["mal_ratio_sd2_over_layer_pruned"]) < 0.005
     loss = 100 * (g["mal_llama3b_dense"] - g["mal_llama3b_sd2_50"]) / g["mal_llama3b_dense"]
     assert abs(loss - g["mal_loss_percent_vs_dense"]) < 0.02   # printed MALs are rounded
+
+
+def test_bf16_rounding_in_the_subnormal_range():
+    # below 2^-126 bf16 values are multiples of 2^-133: the spacing stops shrinking.  Pinned against the
+    # definition of the format (bit pattern k for k * 2^-133, k < 128), with ties going to the even pattern
+    step = 2.0 ** -133
+    assert oracle.f64_to_bf16_rne(step) == 0x0001
+    assert oracle.f64_to_bf16_rne(5 * step) == 0x0005
+    assert oracle.f64_to_bf16_rne(127 * step) == 0x007F
+    assert oracle.f64_to_bf16_rne(128 * step) == 0x0080                 # 2^-126, the smallest normal value
+    assert oracle.f64_to_bf16_rne(0.5 * step) == 0x0000                 # tie between 0 and 1: even
+    assert oracle.f64_to_bf16_rne(1.5 * step) == 0x0002                 # tie between 1 and 2: even
+    assert oracle.f64_to_bf16_rne(2.5 * step) == 0x0002
+    assert oracle.f64_to_bf16_rne(2.5000001 * step) == 0x0003
+    assert oracle.f64_to_bf16_rne(0.49 * step) == 0x0000
+    assert oracle.f64_to_bf16_rne(-3 * step) == 0x8003
+    assert oracle.f64_to_bf16_rne(127.5 * step) == 0x0080               # rounds up into the normal range
+    # and the widening of those patterns gives the values back
+    assert float(synth.bf16_bits_to_f32(np.array([0x0005], np.uint16))[0]) == 5 * step
